@@ -1,0 +1,177 @@
+/*
+ * maxdnn.h — C ABI of the B200-native FPROP direct convolution library.
+ *
+ * The operation (paper Section 2, "Convolution"): a minibatch of Nb maps of
+ * Wi x Hi x Nc is convolved with a bank of No filters of Sk x Sk x Nc; products
+ * are taken channel by channel and summed over channels; the filter moves with
+ * a stride; the origin is offset by a padding parameter and the map is wrapped
+ * in an apron of zeros; the result is scaled by alpha:
+ *
+ *   out[o,y,x,n] = alpha * sum_{c,kh,kw} filt[c,kh,kw,o]
+ *                                        * in0[c, y*stride-pad+kh, x*stride-pad+kw, n]
+ *
+ * in0 is `in` inside the map and zero outside.  The filter is not flipped
+ * (Section 3 multiplies the unrolled patch by the filter matrix as stored).
+ * Ho = floor((Hi + 2*pad - Sk)/stride) + 1, Wo likewise.
+ *
+ * Layout (Section 3: batch / filter index innermost), all row-major:
+ *   in   [Nc][Hi][Wi][Nb]
+ *   filt [Nc][Sk][Sk][No]      = the (Sk^2 Nc) x No filter matrix of Section 3
+ *   out  [No][Ho][Wo][Nb]
+ *
+ * Every fprop entry point computes this as the implicit GEMM of Section 3
+ * (per output coordinate: unrolled patch Nb x Sk^2 Nc times filter matrix
+ * Sk^2 Nc x No), with the patch gathered on the fly.
+ *
+ * Conventions for all entry points
+ *   - Pointers named d_* (and in/filt/out of the device entry points) are
+ *     DEVICE pointers of the current CUDA device, owned by the caller, at least
+ *     16-byte aligned, non-overlapping.  h_* are HOST pointers.
+ *   - `out` is overwritten in full (there is no accumulate mode; the paper has
+ *     alpha only).
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work and return; they never synchronise the stream.
+ *   - Errors are return codes; nothing throws or aborts.  A call that returns
+ *     an error other than MAXDNN_CUDA_ERROR has launched nothing.
+ *   - The library keeps one small per-device status word (device memory,
+ *     allocated on the first fprop call on that device — make that first call
+ *     outside any stream capture).  Kernels give every internal wait an
+ *     iteration limit; a wait that runs out records a code there instead of
+ *     hanging.  maxdnn_last_device_status() reads it.
+ *   - There is no CPU fallback: without an sm_100 device the fprop calls fail
+ *     with MAXDNN_NOT_SUPPORTED / MAXDNN_CUDA_ERROR.
+ */
+#ifndef MAXDNN_H_
+#define MAXDNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Section 2's symbols.  Sk is the (square) filter size; one stride and one
+ * padding for both axes. */
+typedef struct maxdnn_conv_desc {
+  int32_t Nb, Wi, Hi, Nc, No, Sk, stride, pad;
+  float alpha;
+} maxdnn_conv_desc;
+
+typedef enum maxdnn_status {
+  MAXDNN_OK = 0,
+  MAXDNN_INVALID_VALUE = 1,  /* null pointer, non-positive size, empty output, non-finite alpha */
+  MAXDNN_NOT_SUPPORTED = 2,  /* valid problem this build cannot run (see each entry point) */
+  MAXDNN_CUDA_ERROR = 3,     /* a CUDA runtime / driver call failed */
+  MAXDNN_DEVICE_TIMEOUT = 4  /* a kernel's bounded wait ran out (reported by last_device_status) */
+} maxdnn_status;
+
+/* Arithmetic of the inner product (Section 3.2's inner loop). */
+typedef enum maxdnn_kernel_kind {
+  MAXDNN_KERNEL_FP32 = 0, /* exact fp32 fused multiply-add on the CUDA cores */
+  MAXDNN_KERNEL_TF32 = 1, /* tensor cores, fp32 storage read as TF32, fp32 accumulate */
+  MAXDNN_KERNEL_BF16 = 2  /* tensor cores, bf16 storage, fp32 accumulate */
+} maxdnn_kernel_kind;
+
+const char* maxdnn_status_string(maxdnn_status s);
+
+/* Output map size (Section 2: the stride "yields the desired output map
+ * size"; floor division, consistent with every row of Table 1).
+ * INVALID_VALUE if desc is null, a size is <= 0, pad < 0, alpha is not finite
+ * or the padded map is smaller than the filter.  Ho / Wo may be null. */
+maxdnn_status maxdnn_conv_out_dims(const maxdnn_conv_desc* desc, int32_t* Ho, int32_t* Wo);
+
+/* Section 2's complexity C = 2 Nb Wo Ho (Nc Sk^2 + 1) No, one multiply-
+ * accumulate = 2 FLOPs.  0 for an invalid descriptor. */
+uint64_t maxdnn_conv_flops(const maxdnn_conv_desc* desc);
+
+/* Number of elements of in / filt / out for a descriptor (0 if invalid). */
+uint64_t maxdnn_conv_in_elems(const maxdnn_conv_desc* desc);
+uint64_t maxdnn_conv_filt_elems(const maxdnn_conv_desc* desc);
+uint64_t maxdnn_conv_out_elems(const maxdnn_conv_desc* desc);
+
+/*
+ * The address-generation stage (Section 3.2: pixel / channel offsets of the
+ * patch are precomputed so that the three nested loops over channels, rows
+ * and columns of a patch become one loop over a table).  Here one table entry
+ * ("K step") names a box of patch rows that one TMA transfer stages into
+ * shared memory, and the matching box of filter-matrix rows.
+ */
+typedef struct maxdnn_kstep {
+  int16_t c0;   /* first channel of the box */
+  int8_t kh;    /* filter row of the box */
+  int8_t kw0;   /* first filter column of the box */
+} maxdnn_kstep;
+
+typedef struct maxdnn_plan_info {
+  int32_t Ho, Wo;
+  int32_t tile_m;      /* filters per tile (rows of the GEMM block) */
+  int32_t tile_px;     /* adjacent output pixels (along x) per tile */
+  int32_t tile_n;      /* images per tile */
+  int32_t kc;          /* channels per K step */
+  int32_t kwc;         /* filter columns per K step (1 or Sk) */
+  int32_t n_ksteps;    /* length of the K-step table */
+  int32_t stages;      /* depth of the shared-memory ring */
+  int32_t n_tiles;     /* tiles in the whole problem */
+  int32_t grid;        /* persistent CTAs launched */
+  int32_t smem_bytes;  /* dynamic shared memory per CTA */
+} maxdnn_plan_info;
+
+/* Host-only: fills *info and, if steps != NULL, up to max_steps table entries
+ * (HOST memory, caller-owned).  Needs no GPU when sm_count > 0 is given
+ * (sm_count <= 0 asks the current device).  NOT_SUPPORTED as for the matching
+ * fprop call. */
+maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     int32_t sm_count, maxdnn_plan_info* info,
+                                     maxdnn_kstep* steps, int32_t max_steps);
+
+/*
+ * FPROP with exact fp32 arithmetic (Sections 3.1-3.2: register-blocked
+ * multiply-accumulate inner loop over the staged patch, alpha scaling and
+ * coalesced store).  in / filt / out: device fp32 buffers in the layout above.
+ * NOT_SUPPORTED: Nb or No not a multiple of 4 (16-byte row rule of the bulk
+ * tensor copies), Sk > 127, Nc > 32767, a map dimension that does not fit the
+ * tensor-copy descriptor (>= 2^31 bytes in one row pitch), or a device that is
+ * not sm_100.
+ */
+maxdnn_status maxdnn_conv_fprop(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                                float* out, void* cuda_stream);
+
+/*
+ * FPROP on the tensor cores, fp32 accumulate.  _tf32 reads the same fp32
+ * buffers as maxdnn_conv_fprop (the tensor core ignores the low 13 mantissa
+ * bits of each operand).  _bf16 reads bfloat16 `in` and `filt` (same layout,
+ * 2-byte elements, supplied by the caller) and writes fp32 `out`.
+ * NOT_SUPPORTED: as above, and No not a multiple of 32, or Nb not a multiple
+ * of 32 (tf32) / 64 (bf16).
+ */
+maxdnn_status maxdnn_conv_fprop_tf32(const maxdnn_conv_desc* desc, const float* in,
+                                     const float* filt, float* out, void* cuda_stream);
+maxdnn_status maxdnn_conv_fprop_bf16(const maxdnn_conv_desc* desc, const void* in,
+                                     const void* filt, float* out, void* cuda_stream);
+
+/*
+ * The same operation from HOST buffers, for callers that keep their data on
+ * the host: enqueues on `cuda_stream` the host->device copies of h_in and
+ * h_filt into the caller's device staging buffers d_in / d_filt, the chosen
+ * kernel, and the device->host copy of d_out into h_out.  Element types as for
+ * the matching device entry point.  Pinned host memory makes the copies
+ * asynchronous; the caller synchronises the stream before reading h_out.
+ * Allocates nothing.
+ */
+maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     const void* h_in, const void* h_filt, float* h_out,
+                                     void* d_in, void* d_filt, float* d_out, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then reads and clears the current device's
+ * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside a
+ * kernel ran out; its output is not valid) or MAXDNN_CUDA_ERROR. */
+maxdnn_status maxdnn_last_device_status(void* cuda_stream);
+
+/* How many kernels this library has launched in this process (all devices). */
+uint64_t maxdnn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAXDNN_H_ */

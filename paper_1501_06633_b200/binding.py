@@ -1,0 +1,219 @@
+"""ctypes binding of ``libmaxdnn.so``: same names as ``include/maxdnn.h``,
+argument marshalling only.  Tensors are torch CUDA tensors (device memory and
+streams are all torch is used for); every step of the computation runs in the
+library's kernels.  A missing library or a failing call raises — nothing here
+falls back to another implementation."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+__all__ = [
+    "MaxdnnError", "ConvDesc", "PlanInfo", "KStep", "KERNEL_FP32", "KERNEL_TF32", "KERNEL_BF16",
+    "OK", "INVALID_VALUE", "NOT_SUPPORTED", "CUDA_ERROR", "DEVICE_TIMEOUT",
+    "library_path", "load_library", "status_string", "conv_out_dims", "conv_flops",
+    "conv_in_elems", "conv_filt_elems", "conv_out_elems", "conv_plan_query", "conv_fprop",
+    "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "last_device_status",
+    "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
+]
+
+OK, INVALID_VALUE, NOT_SUPPORTED, CUDA_ERROR, DEVICE_TIMEOUT = 0, 1, 2, 3, 4
+KERNEL_FP32, KERNEL_TF32, KERNEL_BF16 = 0, 1, 2
+
+EXPORTED_SYMBOLS = [
+    "maxdnn_status_string", "maxdnn_conv_out_dims", "maxdnn_conv_flops", "maxdnn_conv_in_elems",
+    "maxdnn_conv_filt_elems", "maxdnn_conv_out_elems", "maxdnn_conv_plan_query",
+    "maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16",
+    "maxdnn_conv_fprop_host", "maxdnn_last_device_status", "maxdnn_launch_count",
+]
+
+
+class MaxdnnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s failed: %s" % (where, status_string(status)))
+
+
+class ConvDesc(ctypes.Structure):
+    """maxdnn_conv_desc: Section 2's symbols."""
+
+    _fields_ = [
+        ("Nb", ctypes.c_int32), ("Wi", ctypes.c_int32), ("Hi", ctypes.c_int32),
+        ("Nc", ctypes.c_int32), ("No", ctypes.c_int32), ("Sk", ctypes.c_int32),
+        ("stride", ctypes.c_int32), ("pad", ctypes.c_int32), ("alpha", ctypes.c_float),
+    ]
+
+    @classmethod
+    def make(cls, Nb, Wi, Hi, Nc, No, Sk, stride=1, pad=0, alpha=1.0) -> "ConvDesc":
+        return cls(int(Nb), int(Wi), int(Hi), int(Nc), int(No), int(Sk), int(stride), int(pad),
+                   float(alpha))
+
+
+class KStep(ctypes.Structure):
+    _fields_ = [("c0", ctypes.c_int16), ("kh", ctypes.c_int8), ("kw0", ctypes.c_int8)]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "Ho", "Wo", "tile_m", "tile_px", "tile_n", "kc", "kwc", "n_ksteps", "stages", "n_tiles",
+        "grid", "smem_bytes")]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmaxdnn.so")
+
+
+def load_library():
+    """Load ``libmaxdnn.so`` (built in-tree by ``paper_1501_06633_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(
+            "%s is missing: build it with `python -m paper_1501_06633_b200.build` "
+            "(there is no fallback implementation)" % path)
+    lib = ctypes.CDLL(path)
+    P = ctypes.POINTER
+    vp = ctypes.c_void_p
+    lib.maxdnn_status_string.restype = ctypes.c_char_p
+    lib.maxdnn_status_string.argtypes = [ctypes.c_int]
+    lib.maxdnn_conv_out_dims.restype = ctypes.c_int
+    lib.maxdnn_conv_out_dims.argtypes = [P(ConvDesc), P(ctypes.c_int32), P(ctypes.c_int32)]
+    for name in ("maxdnn_conv_flops", "maxdnn_conv_in_elems", "maxdnn_conv_filt_elems",
+                 "maxdnn_conv_out_elems"):
+        getattr(lib, name).restype = ctypes.c_uint64
+        getattr(lib, name).argtypes = [P(ConvDesc)]
+    lib.maxdnn_conv_plan_query.restype = ctypes.c_int
+    lib.maxdnn_conv_plan_query.argtypes = [P(ConvDesc), ctypes.c_int, ctypes.c_int32, P(PlanInfo),
+                                           P(KStep), ctypes.c_int32]
+    for name in ("maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16"):
+        getattr(lib, name).restype = ctypes.c_int
+        getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
+    lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
+    lib.maxdnn_conv_fprop_host.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.maxdnn_last_device_status.restype = ctypes.c_int
+    lib.maxdnn_last_device_status.argtypes = [vp]
+    lib.maxdnn_launch_count.restype = ctypes.c_uint64
+    lib.maxdnn_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().maxdnn_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise MaxdnnError(status, where)
+
+
+def conv_out_dims(desc: ConvDesc):
+    ho, wo = ctypes.c_int32(), ctypes.c_int32()
+    _check(load_library().maxdnn_conv_out_dims(ctypes.byref(desc), ctypes.byref(ho),
+                                               ctypes.byref(wo)), "maxdnn_conv_out_dims")
+    return ho.value, wo.value
+
+
+def conv_flops(desc: ConvDesc) -> int:
+    return int(load_library().maxdnn_conv_flops(ctypes.byref(desc)))
+
+
+def conv_in_elems(desc: ConvDesc) -> int:
+    return int(load_library().maxdnn_conv_in_elems(ctypes.byref(desc)))
+
+
+def conv_filt_elems(desc: ConvDesc) -> int:
+    return int(load_library().maxdnn_conv_filt_elems(ctypes.byref(desc)))
+
+
+def conv_out_elems(desc: ConvDesc) -> int:
+    return int(load_library().maxdnn_conv_out_elems(ctypes.byref(desc)))
+
+
+def conv_plan_query(desc: ConvDesc, kind: int = KERNEL_FP32, sm_count: int = 148):
+    """(PlanInfo, [KStep...]) — host-only; needs no GPU when sm_count > 0."""
+    info = PlanInfo()
+    steps = (KStep * 1024)()
+    _check(load_library().maxdnn_conv_plan_query(ctypes.byref(desc), int(kind), int(sm_count),
+                                                 ctypes.byref(info), steps, 1024),
+           "maxdnn_conv_plan_query")
+    return info, [steps[i] for i in range(info.n_ksteps)]
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(int(stream.cuda_stream))
+
+
+def _dev_ptr(t, dtype_names, n_elems, what):
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor" % what)
+    if str(t.dtype).replace("torch.", "") not in dtype_names:
+        raise TypeError("%s has dtype %s, expected one of %s" % (what, t.dtype, dtype_names))
+    if t.numel() != n_elems:
+        raise ValueError("%s has %d elements, expected %d" % (what, t.numel(), n_elems))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def fprop_status(desc: ConvDesc, inp, filt, out, kind: int = KERNEL_FP32, stream=None) -> int:
+    """Enqueue one FPROP on torch tensors and return the raw status code."""
+    lib = load_library()
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pin = _dev_ptr(inp, in_types, conv_in_elems(desc), "in")
+    pf = _dev_ptr(filt, in_types, conv_filt_elems(desc), "filt")
+    po = _dev_ptr(out, ("float32",), conv_out_elems(desc), "out")
+    fn = {KERNEL_FP32: lib.maxdnn_conv_fprop, KERNEL_TF32: lib.maxdnn_conv_fprop_tf32,
+          KERNEL_BF16: lib.maxdnn_conv_fprop_bf16}[kind]
+    return int(fn(ctypes.byref(desc), pin, pf, po, _stream_ptr(stream)))
+
+
+def conv_fprop(desc: ConvDesc, inp, filt, out, stream=None) -> None:
+    """maxdnn_conv_fprop: exact fp32 FPROP on device tensors (asynchronous)."""
+    _check(fprop_status(desc, inp, filt, out, KERNEL_FP32, stream), "maxdnn_conv_fprop")
+
+
+def conv_fprop_tf32(desc: ConvDesc, inp, filt, out, stream=None) -> None:
+    _check(fprop_status(desc, inp, filt, out, KERNEL_TF32, stream), "maxdnn_conv_fprop_tf32")
+
+
+def conv_fprop_bf16(desc: ConvDesc, inp, filt, out, stream=None) -> None:
+    _check(fprop_status(desc, inp, filt, out, KERNEL_BF16, stream), "maxdnn_conv_fprop_bf16")
+
+
+def conv_fprop_host(desc: ConvDesc, kind: int, h_in, h_filt, h_out, d_in, d_filt, d_out,
+                    stream=None) -> None:
+    """maxdnn_conv_fprop_host: h_* are CPU (ideally pinned) tensors, d_* device
+    staging tensors of the same sizes; copies and kernel are enqueued on the stream."""
+    import torch
+    for t, what in ((h_in, "h_in"), (h_filt, "h_filt"), (h_out, "h_out")):
+        if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.is_contiguous()):
+            raise TypeError("%s must be a contiguous CPU tensor" % what)
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pin = _dev_ptr(d_in, in_types, conv_in_elems(desc), "d_in")
+    pf = _dev_ptr(d_filt, in_types, conv_filt_elems(desc), "d_filt")
+    po = _dev_ptr(d_out, ("float32",), conv_out_elems(desc), "d_out")
+    if h_in.numel() != d_in.numel() or h_filt.numel() != d_filt.numel() or \
+            h_out.numel() != d_out.numel() or h_in.element_size() != d_in.element_size() or \
+            h_filt.element_size() != d_filt.element_size() or h_out.dtype != torch.float32:
+        raise ValueError("host and device buffers do not match")
+    _check(load_library().maxdnn_conv_fprop_host(
+        ctypes.byref(desc), int(kind), ctypes.c_void_p(h_in.data_ptr()),
+        ctypes.c_void_p(h_filt.data_ptr()), ctypes.c_void_p(h_out.data_ptr()), pin, pf, po,
+        _stream_ptr(stream)), "maxdnn_conv_fprop_host")
+
+
+def last_device_status(stream=None) -> int:
+    return int(load_library().maxdnn_last_device_status(_stream_ptr(stream)))
+
+
+def launch_count() -> int:
+    return int(load_library().maxdnn_launch_count())

@@ -1,0 +1,310 @@
+// C ABI of the library (see include/maxdnn.h): descriptor checks, per-device
+// state, tensor-copy descriptor encoding and kernel launches.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/maxdnn.h"
+#include "ffma_conv.cuh"
+#include "plan.h"
+#include "umma_conv.cuh"
+
+namespace maxdnn {
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceState {
+  bool ready = false;
+  bool sm100 = false;
+  int sm_count = 0;
+  uint32_t* status = nullptr;   // one word of device memory
+  bool ffma_attr[5] = {false, false, false, false, false};
+  bool umma_attr[2] = {false, false};
+};
+
+std::mutex g_mu;
+DeviceState g_dev[kMaxDevices];
+std::atomic<uint64_t> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+maxdnn_status device_state(DeviceState** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+  if (dev < 0 || dev >= kMaxDevices) return MAXDNN_NOT_SUPPORTED;
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceState& s = g_dev[dev];
+  if (!s.ready) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    s.sm100 = (prop.major == 10);
+    s.sm_count = prop.multiProcessorCount;
+    if (s.sm100) {
+      if (cudaMalloc(&s.status, 256) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+      if (cudaMemset(s.status, 0, 256) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+    }
+    s.ready = true;
+  }
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) !=
+            cudaSuccess || !fn) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = &s;
+  return MAXDNN_OK;
+}
+
+// dims[0] is the contiguous dimension; strides[i] is the byte pitch of dims[i+1].
+maxdnn_status encode_map(CUtensorMap* m, CUtensorMapDataType dt, int rank, const void* base,
+                         const uint64_t* dims, const uint64_t* strides, const uint32_t* box,
+                         CUtensorMapSwizzle swz) {
+  cuuint64_t gd[5];
+  cuuint64_t gs[4];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gs[i] = strides[i];
+  CUresult r = g_encode(m, dt, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MAXDNN_OK : MAXDNN_CUDA_ERROR;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int env_int(const char* name) {
+  const char* v = getenv(name);
+  return v ? atoi(v) : 0;
+}
+
+template <int MR>
+maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
+                          const FfmaArgs& args, cudaStream_t stream) {
+  auto kern = ffma_conv_kernel<MR>;
+  if (!ds->ffma_attr[slot]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->ffma_attr[slot] = true;
+  }
+  kern<<<args.g.grid, kFfmaThreads, args.g.smem_bytes, stream>>>(mf, mi, args);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
+maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                         float* out, cudaStream_t stream) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+
+  static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
+  st = plan_ffma(*desc, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), &args.g, &args.table);
+  if (st != MAXDNN_OK) return st;
+  args.out = out;
+  args.status = ds->status;
+  const ConvGeom& g = args.g;
+
+  CUtensorMap mf, mi;
+  {
+    // filter bank as (o, kw, kh, c)
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Sk, (uint64_t)g.Sk, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Sk * g.No * 4,
+                             (uint64_t)g.Sk * g.Sk * g.No * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    // maps as (n, w, h, c)
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
+                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st != MAXDNN_OK) return st;
+  }
+  switch (g.tile_m) {
+    case 128: return launch_ffma<8>(ds, 4, mf, mi, args, stream);
+    case 96: return launch_ffma<6>(ds, 3, mf, mi, args, stream);
+    case 64: return launch_ffma<4>(ds, 2, mf, mi, args, stream);
+    case 32: return launch_ffma<2>(ds, 1, mf, mi, args, stream);
+    default: return MAXDNN_NOT_SUPPORTED;
+  }
+}
+
+maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const void* in,
+                         const void* filt, float* out, cudaStream_t stream) {
+  (void)desc; (void)elem_bytes; (void)in; (void)filt; (void)out; (void)stream;
+  return MAXDNN_NOT_SUPPORTED;
+}
+
+}  // namespace
+}  // namespace maxdnn
+
+using namespace maxdnn;
+
+extern "C" {
+
+const char* maxdnn_status_string(maxdnn_status s) {
+  switch (s) {
+    case MAXDNN_OK: return "MAXDNN_OK";
+    case MAXDNN_INVALID_VALUE: return "MAXDNN_INVALID_VALUE";
+    case MAXDNN_NOT_SUPPORTED: return "MAXDNN_NOT_SUPPORTED";
+    case MAXDNN_CUDA_ERROR: return "MAXDNN_CUDA_ERROR";
+    case MAXDNN_DEVICE_TIMEOUT: return "MAXDNN_DEVICE_TIMEOUT";
+    default: return "MAXDNN_UNKNOWN_STATUS";
+  }
+}
+
+maxdnn_status maxdnn_conv_out_dims(const maxdnn_conv_desc* desc, int32_t* Ho, int32_t* Wo) {
+  return check_desc(desc, Ho, Wo);
+}
+
+uint64_t maxdnn_conv_flops(const maxdnn_conv_desc* d) {
+  int32_t Ho, Wo;
+  if (check_desc(d, &Ho, &Wo) != MAXDNN_OK) return 0;
+  return 2ull * (uint64_t)d->Nb * (uint64_t)Wo * (uint64_t)Ho *
+         ((uint64_t)d->Nc * (uint64_t)d->Sk * (uint64_t)d->Sk + 1ull) * (uint64_t)d->No;
+}
+
+uint64_t maxdnn_conv_in_elems(const maxdnn_conv_desc* d) {
+  if (check_desc(d, nullptr, nullptr) != MAXDNN_OK) return 0;
+  return (uint64_t)d->Nc * d->Hi * d->Wi * d->Nb;
+}
+
+uint64_t maxdnn_conv_filt_elems(const maxdnn_conv_desc* d) {
+  if (check_desc(d, nullptr, nullptr) != MAXDNN_OK) return 0;
+  return (uint64_t)d->Nc * d->Sk * d->Sk * d->No;
+}
+
+uint64_t maxdnn_conv_out_elems(const maxdnn_conv_desc* d) {
+  int32_t Ho, Wo;
+  if (check_desc(d, &Ho, &Wo) != MAXDNN_OK) return 0;
+  return (uint64_t)d->No * Ho * Wo * d->Nb;
+}
+
+maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     int32_t sm_count, maxdnn_plan_info* info,
+                                     maxdnn_kstep* steps, int32_t max_steps) {
+  if (!desc || !info) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  if (sm_count <= 0) {
+    DeviceState* ds = nullptr;
+    st = device_state(&ds);
+    if (st != MAXDNN_OK) return st;
+    sm_count = ds->sm_count;
+  }
+  static thread_local ConvGeom g;
+  static thread_local KStepTable t;
+  switch (kind) {
+    case MAXDNN_KERNEL_FP32:
+      st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), &g, &t);
+      break;
+    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, &g, &t); break;
+    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, &g, &t); break;
+    default: return MAXDNN_INVALID_VALUE;
+  }
+  if (st != MAXDNN_OK) return st;
+  info->Ho = g.Ho; info->Wo = g.Wo;
+  info->tile_m = g.tile_m; info->tile_px = g.tile_px; info->tile_n = g.tile_n;
+  info->kc = g.kc; info->kwc = g.kwc; info->n_ksteps = g.n_ksteps; info->stages = g.stages;
+  info->n_tiles = g.n_tiles; info->grid = g.grid; info->smem_bytes = g.smem_bytes;
+  if (steps)
+    for (int i = 0; i < g.n_ksteps && i < max_steps; ++i) steps[i] = t.s[i];
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_fprop(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                                float* out, void* cuda_stream) {
+  return fprop_fp32(desc, in, filt, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_fprop_tf32(const maxdnn_conv_desc* desc, const float* in,
+                                     const float* filt, float* out, void* cuda_stream) {
+  return fprop_umma(desc, 4, in, filt, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_fprop_bf16(const maxdnn_conv_desc* desc, const void* in,
+                                     const void* filt, float* out, void* cuda_stream) {
+  return fprop_umma(desc, 2, in, filt, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     const void* h_in, const void* h_filt, float* h_out,
+                                     void* d_in, void* d_filt, float* d_out, void* cuda_stream) {
+  if (!h_in || !h_filt || !h_out || !d_in || !d_filt || !d_out) return MAXDNN_INVALID_VALUE;
+  if (check_desc(desc, nullptr, nullptr) != MAXDNN_OK) return MAXDNN_INVALID_VALUE;
+  if (kind != MAXDNN_KERNEL_FP32 && kind != MAXDNN_KERNEL_TF32 && kind != MAXDNN_KERNEL_BF16)
+    return MAXDNN_INVALID_VALUE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t eb = (kind == MAXDNN_KERNEL_BF16) ? 2 : 4;
+  if (cudaMemcpyAsync(d_in, h_in, maxdnn_conv_in_elems(desc) * eb, cudaMemcpyHostToDevice,
+                      stream) != cudaSuccess ||
+      cudaMemcpyAsync(d_filt, h_filt, maxdnn_conv_filt_elems(desc) * eb, cudaMemcpyHostToDevice,
+                      stream) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  maxdnn_status st;
+  if (kind == MAXDNN_KERNEL_FP32)
+    st = fprop_fp32(desc, static_cast<const float*>(d_in), static_cast<const float*>(d_filt),
+                    d_out, stream);
+  else
+    st = fprop_umma(desc, (int)eb, d_in, d_filt, d_out, stream);
+  if (st != MAXDNN_OK) return st;
+  if (cudaMemcpyAsync(h_out, d_out, maxdnn_conv_out_elems(desc) * 4, cudaMemcpyDeviceToHost,
+                      stream) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_last_device_status(void* cuda_stream) {
+  DeviceState* ds = nullptr;
+  maxdnn_status st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->status) return MAXDNN_NOT_SUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  if (cudaStreamSynchronize(stream) != cudaSuccess ||
+      cudaMemcpy(&word, ds->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  if (word != 0) {
+    cudaMemset(ds->status, 0, 4);
+    return MAXDNN_DEVICE_TIMEOUT;
+  }
+  return MAXDNN_OK;
+}
+
+uint64_t maxdnn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,152 @@
+#include "plan.h"
+
+#include <math.h>
+#include <string.h>
+
+namespace maxdnn {
+
+maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo) {
+  if (!d) return MAXDNN_INVALID_VALUE;
+  if (d->Nb <= 0 || d->Wi <= 0 || d->Hi <= 0 || d->Nc <= 0 || d->No <= 0 || d->Sk <= 0 ||
+      d->stride <= 0 || d->pad < 0)
+    return MAXDNN_INVALID_VALUE;
+  if (!isfinite(d->alpha)) return MAXDNN_INVALID_VALUE;
+  const int64_t span_h = (int64_t)d->Hi + 2 * (int64_t)d->pad - d->Sk;
+  const int64_t span_w = (int64_t)d->Wi + 2 * (int64_t)d->pad - d->Sk;
+  if (span_h < 0 || span_w < 0) return MAXDNN_INVALID_VALUE;
+  if (Ho) *Ho = (int32_t)(span_h / d->stride + 1);
+  if (Wo) *Wo = (int32_t)(span_w / d->stride + 1);
+  return MAXDNN_OK;
+}
+
+static maxdnn_status common_limits(const maxdnn_conv_desc& d, int elem_bytes) {
+  if (d.Sk > 127 || d.Nc > 32767) return MAXDNN_NOT_SUPPORTED;
+  // Row pitches of the tensor-copy descriptors are 32-bit-safe byte counts here.
+  const int64_t plane = (int64_t)d.Hi * d.Wi * d.Nb * elem_bytes;
+  const int64_t frow = (int64_t)d.Sk * d.Sk * d.No * elem_bytes;
+  if (plane >= ((int64_t)1 << 40) || frow >= ((int64_t)1 << 40)) return MAXDNN_NOT_SUPPORTED;
+  const int64_t out_elems = (int64_t)d.No * d.Nb;
+  if (out_elems <= 0) return MAXDNN_INVALID_VALUE;
+  return MAXDNN_OK;
+}
+
+// Relative cost per multiply-accumulate of a filter tile of height m (smaller
+// register blocks spend a larger share of issue slots on operand loads).
+static double tile_m_cost(int m) {
+  switch (m) {
+    case 128: return 1.00;
+    case 96: return 1.02;
+    case 64: return 1.06;
+    default: return 1.30;
+  }
+}
+
+static void build_table(const maxdnn_conv_desc& d, int kc, int kwc, KStepTable* t, int* n) {
+  int k = 0;
+  for (int kh = 0; kh < d.Sk; ++kh)
+    for (int kw0 = 0; kw0 < d.Sk; kw0 += kwc)
+      for (int c0 = 0; c0 < d.Nc; c0 += kc) {
+        if (k < kMaxKSteps) {
+          t->s[k].c0 = (int16_t)c0;
+          t->s[k].kh = (int8_t)kh;
+          t->s[k].kw0 = (int8_t)kw0;
+        }
+        ++k;
+      }
+  *n = k;
+}
+
+maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, ConvGeom* g,
+                        KStepTable* t) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  st = common_limits(d, 4);
+  if (st != MAXDNN_OK) return st;
+  if (d.Nb % 4 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+  if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
+  memset(g, 0, sizeof(*g));
+  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
+  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+
+  // Columns of a tile: tile_px adjacent output pixels x tile_n images <= 128.
+  int best_nn = 4, best_T = 1;
+  double best_eff = -1.0;
+  for (int nn = (d.Nb < kTileCols ? d.Nb : kTileCols); nn >= 4; nn -= 4) {
+    int T = kTileCols / nn;
+    if (T > Wo) T = Wo;
+    const double eff = ((double)d.Nb * Wo) /
+                       ((double)ceil_div(d.Nb, nn) * ceil_div(Wo, T) * (double)kTileCols);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best_nn = nn; best_T = T; }
+  }
+  g->tile_n = best_nn;
+  g->tile_px = best_T;
+  g->n_chunks = ceil_div(d.Nb, best_nn);
+  g->x_runs = ceil_div(Wo, best_T);
+
+  // Filter-tile height: fewest SM-time units over whole waves of persistent CTAs.
+  const int cand[4] = {128, 96, 64, 32};
+  int best_m = 32;
+  double best_t = 1e300;
+  for (int i = 0; i < 4; ++i) {
+    const int m = cand[i];
+    if (force_tile_m > 0 && m != force_tile_m) continue;
+    if (m > align_up(d.No, 32) && m != 32) continue;
+    const int64_t tiles = (int64_t)ceil_div(d.No, m) * g->x_runs * Ho * g->n_chunks;
+    const int64_t waves = (tiles + sm_count - 1) / sm_count;
+    const double tm = (double)waves * m * tile_m_cost(m);
+    if (tm < best_t - 1e-9) { best_t = tm; best_m = m; }
+  }
+  g->tile_m = best_m;
+  g->o_blocks = ceil_div(d.No, best_m);
+  const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
+  if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
+  g->n_tiles = (int32_t)tiles;
+
+  // K step: kc channels of one filter tap, or (few channels) kc channels of a
+  // whole filter row of Sk taps.
+  int kc, kwc;
+  if (d.Nc >= 8) {
+    kwc = 1;
+    kc = 32;
+    int best_pad = 1 << 30;
+    for (int c = 32; c >= 8; c -= 4) {
+      const int padded = ceil_div(d.Nc, c) * c;
+      if (padded < best_pad) { best_pad = padded; kc = c; }
+    }
+  } else {
+    kwc = d.Sk;
+    kc = 40 / d.Sk;
+    if (kc < 1) kc = 1;
+    if (kc > d.Nc) kc = d.Nc;
+  }
+  int n = 0;
+  build_table(d, kc, kwc, t, &n);
+  while (n > kMaxKSteps && kwc == 1 && kc < 256) {   // very deep filters: larger boxes
+    kc *= 2;
+    build_table(d, kc, kwc, t, &n);
+  }
+  if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
+  g->kc = kc; g->kwc = kwc; g->rows = kc * kwc; g->n_ksteps = n;
+
+  g->a_stage_bytes = g->rows * g->tile_m * 4;
+  g->b_slot_bytes = align_up(g->rows * g->tile_n * 4, 128);
+  g->b_stage_bytes = g->b_slot_bytes * g->tile_px;
+  const int stage = g->a_stage_bytes + g->b_stage_bytes;
+  const int budget = 200 * 1024;
+  int stages = budget / stage;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return MAXDNN_NOT_SUPPORTED;
+  g->stages = stages;
+  g->smem_bytes = stages * stage + 1024;   // + barriers, + slack for 1024-byte alignment
+  g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  return MAXDNN_OK;
+}
+
+maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, ConvGeom* g,
+                        KStepTable* t) {
+  (void)d; (void)elem_bytes; (void)sm_count; (void)g; (void)t;
+  return MAXDNN_NOT_SUPPORTED;
+}
+
+}  // namespace maxdnn

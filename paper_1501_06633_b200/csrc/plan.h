@@ -1,0 +1,54 @@
+// Host-side planning: descriptor checks, tile choice and the K-step table
+// (the address-generation stage, Section 3.2: patch offsets are precomputed so
+// one flat loop replaces the nested loops over channels, rows and columns).
+// Plain C++ — no CUDA calls — so it can be exercised without a GPU.
+#pragma once
+#include <stdint.h>
+
+#include "../../include/maxdnn.h"
+
+namespace maxdnn {
+
+constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel parameters
+constexpr int kTileCols = 128;     // GEMM-block columns (pixels x images) of the FFMA kernel
+
+// What a kernel needs to know about the problem and its tiling.  Passed by
+// value in kernel parameter space together with the K-step table.
+struct ConvGeom {
+  int32_t Nb, Wi, Hi, Nc, No, Sk, stride, pad;
+  int32_t Ho, Wo;
+  float alpha;
+  int32_t tile_m;     // filters per tile
+  int32_t tile_px;    // adjacent output pixels (x) per tile
+  int32_t tile_n;     // images per tile
+  int32_t kc, kwc;    // channels / filter columns per K step
+  int32_t rows;       // patch rows per K step = kc * kwc
+  int32_t n_ksteps;
+  int32_t stages;
+  int32_t o_blocks, n_chunks, x_runs;
+  int32_t n_tiles;
+  int32_t a_stage_bytes;   // filter box bytes per stage
+  int32_t b_slot_bytes;    // patch box bytes per pixel per stage (128-byte multiple)
+  int32_t b_stage_bytes;   // tile_px * b_slot_bytes
+  int32_t grid;
+  int32_t smem_bytes;
+};
+
+struct KStepTable {
+  maxdnn_kstep s[kMaxKSteps];
+};
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int align_up(int a, int b) { return ceil_div(a, b) * b; }
+
+maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo);
+
+// FFMA kernel plan.  force_tile_m > 0 pins the filter-tile height (ablations).
+maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, ConvGeom* g,
+                        KStepTable* t);
+
+// Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
+maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, ConvGeom* g,
+                        KStepTable* t);
+
+}  // namespace maxdnn
