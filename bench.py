@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the FPROP convolution hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--kernel fp32|tf32|bf16]
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+One step = one FPROP convolution of the named workload (patch gather, inner
+product, alpha scaling and store — one kernel launch) on synthetic seeded
+inputs.  Prints ONE JSON line on rank 0.  Throughput is the paper's FLOP count
+C = 2 Nb Wo Ho (Nc Sk^2 + 1) No (Section 2) divided by time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_1501_06633_b200 import workloads as wl  # noqa: E402
+
+METRIC = "conv FPROP TFLOPS (paper's FLOP formula)"
+UNIT = "TFLOP/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+                  "sm_max_mhz": 1965.0}
+# dram bytes per launch from the committed ncu summaries under profiles/ (None = not captured)
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=300)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER)
+    p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16"])
+    p.add_argument("--e2e-steps", type=int, default=10)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--cpu-seconds", type=float, default=12.0,
+                   help="target wall time of the CPU-baseline sample")
+    return p.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload_bytes(w, kernel):
+    """Algorithmic HBM bytes of one step: every map and filter element read
+    once, every output written once."""
+    eb = 2 if kernel == "bf16" else 4
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
+    return (w.Nc * w.Hi * w.Wi * w.Nb * eb + w.Nc * w.Sk * w.Sk * w.No * eb
+            + w.No * Ho * Wo * w.Nb * 4), Ho, Wo
+
+
+def flops(w, Ho, Wo):
+    return 2 * w.Nb * Wo * Ho * (w.Nc * w.Sk * w.Sk + 1) * w.No
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of our arm, and the whole --impl reference arm)
+# ----------------------------------------------------------------------------
+def oracle_sample(w, target_seconds, repeats=1):
+    """Time the oracle, as it stands, on a band of output rows of the workload
+    sized to take about `target_seconds`.  Returns (tflops, seconds, rows, threads)."""
+    import oracle
+    inp, filt = wl.make_inputs(w)
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
+    y_mid = Ho // 2
+    t0 = time.perf_counter()
+    oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y_mid, y_mid + 1))
+    t_row = max(time.perf_counter() - t0, 1e-6)
+    rows = int(max(1, min(Ho, target_seconds / t_row)))
+    y0 = max(0, min(Ho - rows, y_mid - rows // 2))
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y0, y0 + rows))
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    fl = flops(w, rows, Wo)
+    return fl / best / 1e12, best, rows, Ho, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = wl.WORKLOADS[args.workload]
+    inp, filt = wl.make_inputs(w)
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
+    y_mid = Ho // 2
+    t0 = time.perf_counter()
+    oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y_mid, y_mid + 1))
+    t_row = max(time.perf_counter() - t0, 1e-6)
+    total = max(1, args.steps + args.warmup)
+    budget = 150.0 / total                      # whole run within a few minutes
+    rows = int(max(1, min(Ho, budget / t_row)))
+    y0 = max(0, min(Ho - rows, y_mid - rows // 2))
+    for _ in range(args.warmup):
+        oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y0, y0 + rows))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y0, y0 + rows))
+    dt = time.perf_counter() - t0
+    value = flops(w, rows, Wo) * args.steps / dt / 1e12
+    sample = "%d of %d output rows of %s per step" % (rows, Ho, w.name)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "kernel": "cpu oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a
+    timed region runs."""
+
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+        0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+        0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            self._nv = pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {
+            "sm_mhz": float(np.median(self.samples)) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_1501_06633_b200 as mx
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    peaks, peaks_kind = load_peaks()
+    w = wl.WORKLOADS[args.workload]
+    kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}[args.kernel]
+    d = mx.ConvDesc.make(*w.dims)
+    nbytes, Ho, Wo = workload_bytes(w, args.kernel)
+    C = mx.conv_flops(d)
+    assert C == flops(w, Ho, Wo)
+
+    # Each rank holds its own batch shard (same recipe, its own seed); FPROP needs
+    # no exchange between shards.  Buffer sets are rotated so that no step finds
+    # its inputs in L2.
+    inp, filt = wl.make_inputs(w, seed_offset=rank)
+    n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / nbytes)))
+    if args.kernel == "bf16":
+        to_dev = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        to_dev = lambda a: torch.from_numpy(a).cuda()
+    d_filt = to_dev(filt).reshape(-1)
+    base_in = to_dev(inp).reshape(-1)
+    d_ins = [base_in] + [base_in.clone() for _ in range(n_sets - 1)]
+    d_outs = [torch.empty(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+              for _ in range(n_sets)]
+    fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
+             mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        fprop(d, d_ins[i % n_sets], d_filt, d_outs[i % n_sets])
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    launches0 = mx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        fprop(d, d_ins[i % n_sets], d_filt, d_outs[i % n_sets])
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = mx.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    if mx.last_device_status() != mx.OK:
+        raise SystemExit("a kernel reported a timed-out wait; results are not valid")
+
+    # end to end: pinned host buffers through maxdnn_conv_fprop_host
+    h_in = torch.from_numpy(wl.to_bf16_bits(inp).view(np.int16) if args.kernel == "bf16" else inp
+                            ).reshape(-1).pin_memory()
+    h_f = torch.from_numpy(wl.to_bf16_bits(filt).view(np.int16) if args.kernel == "bf16" else filt
+                           ).reshape(-1).pin_memory()
+    h_out = torch.empty(mx.conv_out_elems(d), dtype=torch.float32).pin_memory()
+    s_in = d_ins[0].view(torch.int16) if args.kernel == "bf16" else d_ins[0]
+    s_f = d_filt.view(torch.int16) if args.kernel == "bf16" else d_filt
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    for _ in range(2):
+        mx.conv_fprop_host(d, kind, h_in, h_f, h_out, s_in, s_f, d_outs[0])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        mx.conv_fprop_host(d, kind, h_in, h_f, h_out, s_in, s_f, d_outs[0])
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    value = world * C / (ms_step * 1e-3) / 1e12
+    e2e_value = world * C / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    if rank == 0:
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        sm_max = float(peaks.get("sm_max_mhz") or clocks.get("sm_max_mhz") or 1965.0)
+        per_gpu = C / (ms_step * 1e-3) / 1e12
+        if args.kernel == "fp32":
+            # FP32 CUDA-core peak, Section 3.3's form: 2 FLOPs x 128 cores x SMs x clock
+            peak, bound = 2.0 * 128 * sm_count * sm_max * 1e6 / 1e12, "alu"
+            peak_note = "2*128*%d SMs*%.0f MHz (max SM clock, %s)" % (sm_count, sm_max, peaks_kind)
+        else:
+            bf16 = float(peaks["bf16_tflops"])
+            peak = bf16 if args.kernel == "bf16" else bf16 * (1.1 / 2.25)
+            bound = "tensor"
+            peak_note = ("cuBLAS bf16 burst (%s)" % peaks_kind) if args.kernel == "bf16" else \
+                ("cuBLAS bf16 burst (%s) x nominal tf32/bf16 ratio 1.1/2.25" % peaks_kind)
+        t_compute = C / (peak * 1e12)
+        t_hbm = nbytes / (float(peaks["hbm_gbs"]) * 1e9)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[args.kernel],
+            "data": "synthetic",
+            "config": {
+                "workload": w.name, "kernel": args.kernel, "Nb": w.Nb, "Wi": w.Wi, "Hi": w.Hi,
+                "Nc": w.Nc, "No": w.No, "Sk": w.Sk, "stride": w.stride, "pad": w.pad,
+                "alpha": w.alpha, "flops_per_step": C, "algorithmic_bytes_per_step": nbytes,
+                "l2": "rotating %d buffer sets (%.0f MB) > L2 (126 MB)" % (n_sets, n_sets * nbytes / 1e6),
+                "parallelism": "batch shards, no collective" if world > 1 else "single GPU",
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
+                    "h2d_bytes_per_step": int(h_in.numel() * h_in.element_size()
+                                              + h_f.numel() * h_f.element_size()),
+                    "d2h_bytes_per_step": int(h_out.numel() * 4)},
+            "gpu_launches": int(launches),
+            "roofline": {
+                "bound": bound, "achieved": per_gpu, "peak": peak, "unit": "TFLOP/s",
+                "frac": per_gpu / peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.kernel)),
+                "peak_source": peak_note,
+                "roofline_time_us": max(t_compute, t_hbm) * 1e6,
+                "frac_of_roofline_time": max(t_compute, t_hbm) / (ms_step * 1e-3),
+                "achieved_hbm_gbs": nbytes / (ms_step * 1e-3) / 1e9,
+            },
+        }
+        if clocks.get("sm_mhz"):
+            # the paper's clock-independent efficiency: C / (2*128*SMs*elapsed SM cycles)
+            cycles = ms_step * 1e-3 * clocks["sm_mhz"] * 1e6
+            line["roofline"]["ce_at_sampled_clock"] = C / (2.0 * 128 * sm_count * cycles)
+        if world == 1 and not args.no_cpu_baseline:
+            tf, secs, rows, Ho_, threads = oracle_sample(w, args.cpu_seconds)
+            line["cpu_baseline"] = {
+                "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
+                "sample": "%d of %d output rows of %s, %.1f s" % (rows, Ho_, w.name, secs)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -17,7 +17,8 @@
 namespace maxdnn {
 
 constexpr int kFfmaConsumerWarps = 8;
-constexpr int kFfmaThreads = (kFfmaConsumerWarps + 1) * 32;
+// Eight consumer warps plus the producer warp.
+constexpr int ffma_threads(int) { return (kFfmaConsumerWarps + 1) * 32; }
 
 struct FfmaArgs {
   ConvGeom g;
@@ -73,8 +74,12 @@ __device__ __forceinline__ void fma_block(const Frag<MR>& f, float2 (&P)[MR / 2]
   }
 }
 
-template <int MR>
-__global__ void __launch_bounds__(kFfmaThreads, 1)
+// One row of the flat loop: operand loads for the row after next are issued
+// before the multiply-adds of the current row (register double buffering).
+#define MAXDNN_ROW_PTRS(R) a_ptr + (R) * Mt, b0_ptr + (R) * b_pitch, b1_ptr + (R) * b_pitch
+
+template <int MR, bool FIXED>
+__global__ void __launch_bounds__(ffma_threads(MR), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
                  const __grid_constant__ FfmaArgs args) {
@@ -108,12 +113,13 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int n_ksteps = g.n_ksteps;
   const int rows = g.rows;
 
-  if (warp == kFfmaConsumerWarps) {
+  if (warp >= kFfmaConsumerWarps) {
     // ------------------------------------------------------------ producer
-    if (lane == 0) {
+    if (warp == kFfmaConsumerWarps && lane == 0) {
       prefetch_tensormap(&map_filt);
       prefetch_tensormap(&map_in);
-      const uint32_t tx_bytes = (uint32_t)(rows * Mt * 4 + g.tile_px * rows * g.tile_n * 4);
+      const uint32_t tx_bytes = (uint32_t)(g.a_box_bytes + g.b_boxes * g.b_box_bytes);
+      const int w_step = g.stride;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -128,7 +134,8 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int h0 = y * g.stride - g.pad;
         const int w0 = xr * g.tile_px * g.stride - g.pad;
         for (int s = 0; s < n_ksteps; ++s) {
-          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+          if (!mbar_wait_backoff(empty_bar + 8u * stage, phase ^ 1u, args.status,
+                                 kDevTimeoutEmpty)) {
             ok = false;
             break;
           }
@@ -139,10 +146,10 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                       ks.kh, ks.c0);
           uint32_t dst = base + b_off + (uint32_t)stage * g.b_stage_bytes;
           int w = w0 + ks.kw0;
-          for (int t = 0; t < g.tile_px; ++t) {
+          for (int t = 0; t < g.b_boxes; ++t) {
             tma_load_4d(dst, &map_in, fb, n0, w, h0 + ks.kh, ks.c0);
             dst += g.b_slot_bytes;
-            w += g.stride;
+            w += w_step;
           }
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
@@ -175,9 +182,12 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     const bool live = col < used_cols;
     col_px[h] = live ? col / g.tile_n : -1;
     col_n[h] = live ? col % g.tile_n : 0;
-    b_elem[h] = live ? (uint32_t)(col_px[h] * (g.b_slot_bytes >> 2) + col_n[h]) : 0u;
+    if (FIXED)
+      b_elem[h] = (uint32_t)col;
+    else
+      b_elem[h] = live ? (uint32_t)(col_px[h] * (g.b_slot_bytes >> 2) + col_n[h]) : 0u;
   }
-  const int b_pitch = g.tile_n;   // floats between patch rows
+  const int b_pitch = FIXED ? kTileCols : g.tile_n;   // floats between patch rows
 
   int stage = 0;
   uint32_t phase = 0;
@@ -202,28 +212,43 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         reinterpret_cast<const float*>(base_ptr + b_off + (size_t)stage * g.b_stage_bytes);
     const float* b0_ptr = bs_ptr + b_elem[0];
     const float* b1_ptr = bs_ptr + b_elem[1];
-    load_frag<MR>(f0, a_ptr, b0_ptr, b1_ptr);
+    load_frag<MR>(f0, MAXDNN_ROW_PTRS(0));
 
     for (int s = 0; s < n_ksteps; ++s) {
-      // Rows 0 .. rows-2 of this stage, two per iteration, next row prefetched.
+      // f0 holds row 0 of this stage.  Four rows per iteration while the row
+      // after the block is still inside the stage.
       int r = 0;
 #pragma unroll 1
-      for (; r + 2 < rows; r += 2) {
-        load_frag<MR>(f1, a_ptr + Mt, b0_ptr + b_pitch, b1_ptr + b_pitch);
+      for (; r + 4 < rows; r += 4) {
+        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
         fma_block<MR>(f0, P, Q);
-        a_ptr += 2 * Mt; b0_ptr += 2 * b_pitch; b1_ptr += 2 * b_pitch;
-        load_frag<MR>(f0, a_ptr, b0_ptr, b1_ptr);
+        load_frag<MR>(f0, MAXDNN_ROW_PTRS(2));
         fma_block<MR>(f1, P, Q);
-      }
-      if (r + 2 == rows) {   // even row count: one more in-stage prefetch
-        load_frag<MR>(f1, a_ptr + Mt, b0_ptr + b_pitch, b1_ptr + b_pitch);
+        load_frag<MR>(f1, MAXDNN_ROW_PTRS(3));
         fma_block<MR>(f0, P, Q);
-        f0 = f1;
+        load_frag<MR>(f0, MAXDNN_ROW_PTRS(4));
+        fma_block<MR>(f1, P, Q);
+        a_ptr += 4 * Mt; b0_ptr += 4 * b_pitch; b1_ptr += 4 * b_pitch;
       }
-      // f0 now holds the last row of this stage.  Prefetch row 0 of the next one.
+#pragma unroll 1
+      for (; rows - r > 2; r += 2) {   // 3 or 4 rows left: two of them here
+        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
+        fma_block<MR>(f0, P, Q);
+        load_frag<MR>(f0, MAXDNN_ROW_PTRS(2));
+        fma_block<MR>(f1, P, Q);
+        a_ptr += 2 * Mt; b0_ptr += 2 * b_pitch; b1_ptr += 2 * b_pitch;
+      }
+      const bool two_left = (rows - r == 2);
+      if (two_left) {
+        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
+        fma_block<MR>(f0, P, Q);
+      }
+      // The last row of this stage is in f1 (two_left) or f0.  Prefetch row 0 of
+      // the next stage into the other buffer before computing it.
       const int cur_stage = stage;
       if (++stage == stages) { stage = 0; phase ^= 1u; }
-      if (s + 1 < n_ksteps) {
+      const bool more = s + 1 < n_ksteps;
+      if (more) {
         ok = mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull);
         if (!ok) break;
         a_ptr = reinterpret_cast<const float*>(base_ptr + a_off + (size_t)stage * g.a_stage_bytes) +
@@ -231,10 +256,15 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         bs_ptr = reinterpret_cast<const float*>(base_ptr + b_off + (size_t)stage * g.b_stage_bytes);
         b0_ptr = bs_ptr + b_elem[0];
         b1_ptr = bs_ptr + b_elem[1];
-        load_frag<MR>(f1, a_ptr, b0_ptr, b1_ptr);
       }
-      fma_block<MR>(f0, P, Q);
-      f0 = f1;
+      if (two_left) {
+        if (more) load_frag<MR>(f0, MAXDNN_ROW_PTRS(0));
+        fma_block<MR>(f1, P, Q);
+      } else {
+        if (more) load_frag<MR>(f1, MAXDNN_ROW_PTRS(0));
+        fma_block<MR>(f0, P, Q);
+        f0 = f1;
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar + 8u * cur_stage);
     }
@@ -279,5 +309,6 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     }
   }
 }
+#undef MAXDNN_ROW_PTRS
 
 }  // namespace maxdnn

@@ -20,7 +20,7 @@ struct DeviceState {
   bool sm100 = false;
   int sm_count = 0;
   uint32_t* status = nullptr;   // one word of device memory
-  bool ffma_attr[5] = {false, false, false, false, false};
+  bool ffma_attr[16] = {};
   bool umma_attr[2] = {false, false};
 };
 
@@ -90,10 +90,10 @@ int env_int(const char* name) {
   return v ? atoi(v) : 0;
 }
 
-template <int MR>
+template <int MR, bool FIXED>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
-  auto kern = ffma_conv_kernel<MR>;
+  auto kern = ffma_conv_kernel<MR, FIXED>;
   if (!ds->ffma_attr[slot]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
         cudaSuccess) {
@@ -102,7 +102,7 @@ maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, cons
     }
     ds->ffma_attr[slot] = true;
   }
-  kern<<<args.g.grid, kFfmaThreads, args.g.smem_bytes, stream>>>(mf, mi, args);
+  kern<<<args.g.grid, ffma_threads(MR), args.g.smem_bytes, stream>>>(mf, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return MAXDNN_OK;
@@ -143,16 +143,21 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
     const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
                              (uint64_t)g.Hi * g.Wi * g.Nb * 4};
-    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
+  const bool fx = g.fixed_pitch != 0;
   switch (g.tile_m) {
-    case 128: return launch_ffma<8>(ds, 4, mf, mi, args, stream);
-    case 96: return launch_ffma<6>(ds, 3, mf, mi, args, stream);
-    case 64: return launch_ffma<4>(ds, 2, mf, mi, args, stream);
-    case 32: return launch_ffma<2>(ds, 1, mf, mi, args, stream);
+    case 128: return fx ? launch_ffma<8, true>(ds, 2, mf, mi, args, stream)
+                        : launch_ffma<8, false>(ds, 3, mf, mi, args, stream);
+    case 96: return fx ? launch_ffma<6, true>(ds, 4, mf, mi, args, stream)
+                       : launch_ffma<6, false>(ds, 5, mf, mi, args, stream);
+    case 64: return fx ? launch_ffma<4, true>(ds, 6, mf, mi, args, stream)
+                       : launch_ffma<4, false>(ds, 7, mf, mi, args, stream);
+    case 32: return fx ? launch_ffma<2, true>(ds, 8, mf, mi, args, stream)
+                       : launch_ffma<2, false>(ds, 9, mf, mi, args, stream);
     default: return MAXDNN_NOT_SUPPORTED;
   }
 }

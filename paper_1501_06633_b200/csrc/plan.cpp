@@ -35,9 +35,9 @@ static maxdnn_status common_limits(const maxdnn_conv_desc& d, int elem_bytes) {
 static double tile_m_cost(int m) {
   switch (m) {
     case 128: return 1.00;
-    case 96: return 1.02;
-    case 64: return 1.06;
-    default: return 1.30;
+    case 96: return 1.03;
+    case 64: return 1.10;
+    default: return 1.35;
   }
 }
 
@@ -129,9 +129,25 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
   g->kc = kc; g->kwc = kwc; g->rows = kc * kwc; g->n_ksteps = n;
 
-  g->a_stage_bytes = g->rows * g->tile_m * 4;
-  g->b_slot_bytes = align_up(g->rows * g->tile_n * 4, 128);
-  g->b_stage_bytes = g->b_slot_bytes * g->tile_px;
+  g->a_box_bytes = g->rows * g->tile_m * 4;
+  g->a_stage_bytes = g->a_box_bytes;
+  // One box per stage whenever the 128 columns are one contiguous run of the map
+  // (one pixel, or adjacent pixels of a stride-1 layer); else one box per pixel.
+  g->fixed_pitch = (g->tile_px * g->tile_n == kTileCols &&
+                    (g->tile_px == 1 || (d.stride == 1 && kwc == 1))) ? 1 : 0;
+  if (g->fixed_pitch) {
+    g->b_boxes = 1;
+    g->b_box_w = g->tile_px > 1 ? g->tile_px : kwc;
+    g->b_box_bytes = g->rows * kTileCols * 4;
+    g->b_slot_bytes = g->b_box_bytes;
+    g->b_stage_bytes = g->b_box_bytes;
+  } else {
+    g->b_boxes = g->tile_px;
+    g->b_box_w = kwc;
+    g->b_box_bytes = g->rows * g->tile_n * 4;
+    g->b_slot_bytes = align_up(g->b_box_bytes, 128);
+    g->b_stage_bytes = g->b_slot_bytes * g->tile_px;
+  }
   const int stage = g->a_stage_bytes + g->b_stage_bytes;
   const int budget = 200 * 1024;
   int stages = budget / stage;

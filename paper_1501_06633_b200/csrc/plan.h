@@ -28,8 +28,13 @@ struct ConvGeom {
   int32_t o_blocks, n_chunks, x_runs;
   int32_t n_tiles;
   int32_t a_stage_bytes;   // filter box bytes per stage
-  int32_t b_slot_bytes;    // patch box bytes per pixel per stage (128-byte multiple)
-  int32_t b_stage_bytes;   // tile_px * b_slot_bytes
+  int32_t a_box_bytes;
+  int32_t fixed_pitch;     // 1: one patch box per stage, rows 128 floats apart
+  int32_t b_boxes;         // patch boxes per K step (1, or tile_px)
+  int32_t b_box_w;         // extent of a patch box along w
+  int32_t b_box_bytes;
+  int32_t b_slot_bytes;    // distance between patch boxes of one stage (128-byte multiple)
+  int32_t b_stage_bytes;   // patch bytes per stage
   int32_t grid;
   int32_t smem_bytes;
 };

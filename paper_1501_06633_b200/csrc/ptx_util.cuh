@@ -85,6 +85,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return mbar_wait_slow(bar, parity, status, code);
 }
 
+// Producer-side wait: sleeps between polls so that a warp waiting for a ring
+// slot does not take issue slots from the arithmetic warps of its scheduler.
+__device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, uint32_t* status,
+                                                  uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i) {
+    __nanosleep(200);
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return mbar_wait_slow(bar, parity, status, code);
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }

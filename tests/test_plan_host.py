@@ -1,0 +1,154 @@
+"""Host-side logic without a GPU: the library loads and exports what the
+header declares, descriptors are validated, and the K-step table plus box
+geometry of the address-generation stage reproduce the oracle's patch gather
+when the copy engine's semantics (boxes, zero fill outside the tensor) are
+emulated in numpy."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_1501_06633_b200 as mx
+from paper_1501_06633_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "maxdnn.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(maxdnn_[a-z0-9_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    lib = mx.load_library()
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert declared == set(mx.EXPORTED_SYMBOLS)
+
+
+def test_descriptor_validation_without_gpu():
+    lib = mx.load_library()
+    good = mx.ConvDesc.make(32, 16, 16, 16, 32, 3, 1, 1)
+    assert mx.conv_out_dims(good) == (16, 16)
+    assert mx.conv_flops(good) == 76021760
+    assert mx.conv_in_elems(good) == 16 * 16 * 16 * 32
+    assert mx.conv_filt_elems(good) == 16 * 9 * 32
+    assert mx.conv_out_elems(good) == 32 * 16 * 16 * 32
+    for bad in [mx.ConvDesc.make(0, 16, 16, 16, 32, 3), mx.ConvDesc.make(32, 16, 16, 16, 32, 3, 0),
+                mx.ConvDesc.make(32, 2, 2, 16, 32, 3, 1, 0), mx.ConvDesc.make(32, 16, 16, 16, 32, 3, 1, -1),
+                mx.ConvDesc.make(32, 16, 16, 16, 32, 3, 1, 1, float("nan")),
+                mx.ConvDesc.make(32, 16, 16, 16, 32, 3, 1, 1, float("inf"))]:
+        assert lib.maxdnn_conv_out_dims(ctypes.byref(bad), None, None) == mx.INVALID_VALUE
+        assert mx.conv_flops(bad) == 0
+        # an invalid descriptor is rejected before any CUDA call is made
+        assert lib.maxdnn_conv_fprop(ctypes.byref(bad), None, None, None, None) == mx.INVALID_VALUE
+    assert lib.maxdnn_conv_out_dims(None, None, None) == mx.INVALID_VALUE
+    assert lib.maxdnn_conv_fprop(ctypes.byref(good), None, None, None, None) == mx.INVALID_VALUE
+    assert mx.status_string(mx.NOT_SUPPORTED) == "MAXDNN_NOT_SUPPORTED"
+    with pytest.raises(mx.MaxdnnError):
+        mx.conv_plan_query(mx.ConvDesc.make(30, 16, 16, 16, 32, 3), mx.KERNEL_FP32, 148)
+    with pytest.raises(mx.MaxdnnError):
+        mx.conv_plan_query(mx.ConvDesc.make(32, 16, 16, 16, 30, 3), mx.KERNEL_FP32, 148)
+
+
+def test_flops_match_golden_table():
+    for line in open(os.path.join(ROOT, "tests", "golden", "flop_counts.txt")):
+        line = line.split("#")[0].split()
+        if not line:
+            continue
+        Nb, Wi, Hi, Nc, No, Sk, s, p, Ho, Wo, C = map(int, line[1:])
+        d = mx.ConvDesc.make(Nb, Wi, Hi, Nc, No, Sk, s, p)
+        assert mx.conv_out_dims(d) == (Ho, Wo)
+        assert mx.conv_flops(d) == C
+
+
+def box(arr, starts, sizes):
+    """A tiled bulk-tensor load: the box [start, start+size) per axis, zeros
+    where it leaves the tensor."""
+    out = np.zeros(sizes, dtype=np.float64)
+    src, dst = [], []
+    for st, sz, ext in zip(starts, sizes, arr.shape):
+        lo, hi = max(st, 0), min(st + sz, ext)
+        if lo >= hi:
+            return out
+        src.append(slice(lo, hi))
+        dst.append(slice(lo - st, hi - st))
+    out[tuple(dst)] = arr[tuple(src)]
+    return out
+
+
+def emulate_fp32_plan(w, inp, filt, sm_count=148):
+    d = mx.ConvDesc.make(*w.dims)
+    info, steps = mx.conv_plan_query(d, mx.KERNEL_FP32, sm_count)
+    Ho, Wo = info.Ho, info.Wo
+    Mt, T, Nn, kc, kwc = info.tile_m, info.tile_px, info.tile_n, info.kc, info.kwc
+    o_blocks = -(-w.No // Mt)
+    n_chunks = -(-w.Nb // Nn)
+    x_runs = -(-Wo // T)
+    assert info.n_tiles == o_blocks * n_chunks * x_runs * Ho
+    assert T * Nn <= 128 and Nn % 4 == 0 and Mt in (32, 64, 96, 128)
+    assert info.grid == min(info.n_tiles, sm_count)
+    # every (c, kh, kw) is covered by exactly one table entry
+    seen = np.zeros((w.Nc, w.Sk, w.Sk), dtype=np.int32)
+    for s in steps:
+        seen[s.c0:s.c0 + kc, s.kh, s.kw0:s.kw0 + kwc] += 1
+        assert s.kw0 + kwc <= w.Sk, "a box must not run past the filter row"
+    assert np.all(seen == 1)
+    out = np.full((w.No, Ho, Wo, w.Nb), np.nan)
+    for tile in range(info.n_tiles):
+        r = tile
+        ob, r = r % o_blocks, r // o_blocks
+        nch, r = r % n_chunks, r // n_chunks
+        xr, y = r % x_runs, r // x_runs
+        o0, n0, x0 = ob * Mt, nch * Nn, xr * T
+        acc = np.zeros((Mt, T, Nn))
+        for s in steps:
+            A = box(filt, (s.c0, s.kh, s.kw0, o0), (kc, 1, kwc, Mt))           # [c][1][kw][o]
+            for t in range(T):
+                Bx = box(inp, (s.c0, y * w.stride - w.pad + s.kh,
+                               (x0 + t) * w.stride - w.pad + s.kw0, n0), (kc, 1, kwc, Nn))
+                acc[:, t, :] += np.einsum("ckwo,ckwn->on", A, Bx)
+        for t in range(T):
+            if x0 + t >= Wo:
+                continue
+            o1, n1 = min(w.No, o0 + Mt), min(w.Nb, n0 + Nn)
+            assert np.all(np.isnan(out[o0:o1, y, x0 + t, n0:n1])), "an output is written twice"
+            out[o0:o1, y, x0 + t, n0:n1] = w.alpha * acc[:o1 - o0, t, :n1 - n0]
+    assert not np.isnan(out).any(), "an output is never written"
+    return out
+
+
+SHAPES = [
+    # Nb  Wi  Hi  Nc  No  Sk st pad alpha
+    (8, 7, 6, 3, 8, 3, 1, 1, 1.0),
+    (132, 5, 4, 9, 100, 3, 1, 1, 0.5),
+    (16, 23, 19, 3, 12, 11, 4, 0, 1.0),
+    (36, 10, 7, 17, 36, 3, 3, 1, -1.0),
+    (20, 13, 4, 33, 68, 2, 1, 0, 1.0),
+    (32, 8, 8, 16, 32, 3, 1, 3, 1.0),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_address_generation_reproduces_patch_gather(shape):
+    Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha = shape
+    w = wl.Workload("plan", Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), 77 + Nb)
+    inp, filt = wl.make_inputs(w)
+    ref = oracle.conv_fprop(inp, filt, stride=st, pad=pad, alpha=alpha)
+    got = emulate_fp32_plan(w, inp.astype(np.float64), filt.astype(np.float64))
+    assert np.max(np.abs(got - ref)) <= 2.0 ** -22 * max(1.0, np.max(np.abs(ref)))
+
+
+def test_benchmark_plans_fit_the_device():
+    for name in wl.ORDER:
+        w = wl.WORKLOADS[name]
+        info, steps = mx.conv_plan_query(mx.ConvDesc.make(*w.dims), mx.KERNEL_FP32, 148)
+        assert info.smem_bytes <= 227 * 1024 and info.stages >= 2
+        assert len(steps) == info.n_ksteps <= 1024
+        assert info.grid <= 148
+    # the 96-filter first layer gets a 96-high tile (no padded filter rows), the
+    # 13x13 layer a tile height that fills whole waves
+    assert mx.conv_plan_query(mx.ConvDesc.make(*wl.WORKLOADS["first11x11s4"].dims))[0].tile_m == 96
