@@ -162,10 +162,100 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   }
 }
 
+template <bool BF16>
+maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                          const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
+  auto kern = umma_conv_kernel<BF16>;
+  const int slot = BF16 ? 1 : 0;
+  if (!ds->umma_attr[slot]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->umma_attr[slot] = true;
+  }
+  kern<<<args.g.grid, kUmmaThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
 maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const void* in,
                          const void* filt, float* out, cudaStream_t stream) {
-  (void)desc; (void)elem_bytes; (void)in; (void)filt; (void)out; (void)stream;
-  return MAXDNN_NOT_SUPPORTED;
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+
+  static thread_local UmmaArgs args;
+  st = plan_umma(*desc, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"), &args.g, &args.table);
+  if (st != MAXDNN_OK) return st;
+  const ConvGeom& g = args.g;
+  const uint64_t eb = (uint64_t)elem_bytes;
+  const uint32_t atom = 128u / (uint32_t)elem_bytes;
+  const bool bf16 = elem_bytes == 2;
+  args.status = ds->status;
+  args.atom = atom;
+  args.umma_k = 32u / (uint32_t)elem_bytes;
+  args.is_bf16 = bf16 ? 1u : 0u;
+  args.lbo_bytes = (uint32_t)g.kc * 128u;     // next group of 32 / 64 filters or images
+  // next group of channel rows: 8 rows for the 16-byte-chunk swizzle, 4 rows for the
+  // 32-byte-chunk swizzle of 4-byte operands
+  args.sbo_bytes = bf16 ? 1024u : 512u;
+  args.kstep_bytes = args.umma_k * 128u;      // next MMA along K inside a stage
+  const uint32_t n_cols = (uint32_t)(g.tile_px * g.tile_n);
+  const uint32_t fmt = bf16 ? 1u : 2u;        // operand format: bf16 / tf32
+  args.idesc = (1u << 4)                      // fp32 accumulator
+               | (fmt << 7) | (fmt << 10)     // A and B formats
+               | (1u << 15) | (1u << 16)      // both operands contiguous along M / N, not K
+               | ((n_cols >> 3) << 17) | ((uint32_t)(kUmmaM >> 4) << 24);
+  const CUtensorMapDataType dt =
+      bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+
+  // 4-byte operands use the 128-byte swizzle with 32-byte chunks, 2-byte operands the
+  // one with 16-byte chunks (the patterns the MMA descriptors of each kind read).
+  const CUtensorMapSwizzle op_swz =
+      bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B;
+  CUtensorMap mf, mi, mo;
+  {
+    // filter bank as (o, c, kw, kh); one box = 128 bytes of filters x kc channels of a tap
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Nc, (uint64_t)g.Sk, (uint64_t)g.Sk};
+    const uint64_t str[3] = {(uint64_t)g.Sk * g.Sk * g.No * eb, (uint64_t)g.No * eb,
+                             (uint64_t)g.Sk * g.No * eb};
+    const uint32_t box[4] = {atom, (uint32_t)g.kc, 1u, 1u};
+    st = encode_map(&mf, dt, 4, filt, dims, str, box, op_swz);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    // maps as (n within group, c, n group, w, h): shared memory receives
+    // [pixel][image group][channel][128 bytes of images]
+    const uint64_t dims[5] = {atom, (uint64_t)g.Nc, (uint64_t)g.Nb / atom, (uint64_t)g.Wi,
+                              (uint64_t)g.Hi};
+    const uint64_t str[4] = {(uint64_t)g.Hi * g.Wi * g.Nb * eb, 128u, (uint64_t)g.Nb * eb,
+                             (uint64_t)g.Wi * g.Nb * eb};
+    const uint32_t box[5] = {atom, (uint32_t)g.kc, (uint32_t)g.tile_n / atom, (uint32_t)g.b_box_w,
+                             1u};
+    st = encode_map(&mi, dt, 5, in, dims, str, box, op_swz);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    // output as (n, x, y, o): one store = 32 filters x 32 images
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
+                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
+    const uint32_t box[4] = {32u, 1u, 1u, 32u};
+    st = encode_map(&mo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != MAXDNN_OK) return st;
+  }
+  return bf16 ? launch_umma<true>(ds, mf, mi, mo, args, stream)
+              : launch_umma<false>(ds, mf, mi, mo, args, stream);
 }
 
 }  // namespace
@@ -231,8 +321,8 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
     case MAXDNN_KERNEL_FP32:
       st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), &g, &t);
       break;
-    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, &g, &t); break;
-    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, &g, &t); break;
+    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;
+    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;
     default: return MAXDNN_INVALID_VALUE;
   }
   if (st != MAXDNN_OK) return st;

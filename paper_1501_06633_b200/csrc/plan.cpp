@@ -159,10 +159,81 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   return MAXDNN_OK;
 }
 
-maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, ConvGeom* g,
-                        KStepTable* t) {
-  (void)d; (void)elem_bytes; (void)sm_count; (void)g; (void)t;
-  return MAXDNN_NOT_SUPPORTED;
+maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
+                        ConvGeom* g, KStepTable* t) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  st = common_limits(d, elem_bytes);
+  if (st != MAXDNN_OK) return st;
+  if (elem_bytes != 4 && elem_bytes != 2) return MAXDNN_INVALID_VALUE;
+  const int atom = 128 / elem_bytes;          // elements per 128-byte swizzled row
+  if (d.Nb % atom != 0) return MAXDNN_NOT_SUPPORTED;
+  if (d.No % 32 != 0) return MAXDNN_NOT_SUPPORTED;
+  if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
+  memset(g, 0, sizeof(*g));
+  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
+  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+
+  // Columns of a tile: tile_px adjacent pixels x tile_n images <= 256 (the MMA's N).
+  const int max_cols = 256;
+  int best_nn = atom, best_T = 1;
+  double best_eff = -1.0;
+  for (int nn = (d.Nb < max_cols ? d.Nb : max_cols) / atom * atom; nn >= atom; nn -= atom) {
+    int T = max_cols / nn;
+    if (T > Wo) T = Wo;
+    const double eff = ((double)d.Nb * Wo) /
+                       ((double)ceil_div(d.Nb, nn) * ceil_div(Wo, T) * (double)max_cols);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best_nn = nn; best_T = T; }
+  }
+  g->tile_n = best_nn;
+  g->tile_px = best_T;
+  g->n_chunks = ceil_div(d.Nb, best_nn);
+  g->x_runs = ceil_div(Wo, best_T);
+  g->tile_m = 128;
+  g->o_blocks = ceil_div(d.No, 128);
+  const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
+  if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
+  g->n_tiles = (int32_t)tiles;
+
+  // K step: kc channels of one filter tap; kc a multiple of the MMA's K
+  // (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
+  const int umma_k = 32 / elem_bytes;
+  const int kc_max = 128 / elem_bytes;        // 32 (tf32) / 64 (bf16): 16 KB of filters per stage
+  int kc = kc_max, best_pad = 1 << 30;
+  for (int c = kc_max; c >= umma_k; c -= umma_k) {
+    const int padded = ceil_div(d.Nc, c) * c;
+    if (padded < best_pad) { best_pad = padded; kc = c; }
+  }
+  if (force_kc > 0 && force_kc % umma_k == 0 && force_kc <= 256) kc = force_kc;
+  int n = 0;
+  build_table(d, kc, 1, t, &n);
+  if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
+  g->kc = kc; g->kwc = 1; g->rows = kc; g->n_ksteps = n;
+
+  const int cols = g->tile_px * g->tile_n;
+  g->a_box_bytes = atom * kc * elem_bytes;              // one group of filters: kc rows x 128 B
+  g->a_stage_bytes = 128 * kc * elem_bytes;
+  if (g->tile_px == 1 || d.stride == 1) {
+    g->b_boxes = 1;
+    g->b_box_w = g->tile_px;
+    g->b_box_bytes = cols * kc * elem_bytes;
+  } else {
+    g->b_boxes = g->tile_px;
+    g->b_box_w = 1;
+    g->b_box_bytes = g->tile_n * kc * elem_bytes;
+  }
+  g->b_slot_bytes = g->b_box_bytes;
+  g->b_stage_bytes = cols * kc * elem_bytes;
+  const int stage = g->a_stage_bytes + g->b_stage_bytes;
+  const int fixed = 8 * 4096 + 1024 + 512;    // epilogue staging, alignment slack, barriers
+  int stages = (227 * 1024 - fixed) / stage;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return MAXDNN_NOT_SUPPORTED;
+  g->stages = stages;
+  g->smem_bytes = stages * stage + fixed;
+  g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  return MAXDNN_OK;
 }
 
 }  // namespace maxdnn

@@ -53,7 +53,7 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
                         KStepTable* t);
 
 // Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
-maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, ConvGeom* g,
-                        KStepTable* t);
+maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
+                        ConvGeom* g, KStepTable* t);
 
 }  // namespace maxdnn
