@@ -163,6 +163,41 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
                                      const void* h_in, const void* h_filt, float* h_out,
                                      void* d_in, void* d_filt, float* d_out, void* cuda_stream);
 
+/*
+ * maxdnn_conv_fprop for callers that must not allocate.  (The paper has no
+ * counterpart; this is a deployment variant of the entry point above.)
+ *
+ * Who needs it: code that runs where a cudaMalloc is off limits — a serving or
+ * control loop with a latency bound (cudaMalloc may synchronise the whole device
+ * and takes the driver's allocation lock), a process that handed all device
+ * memory to its own pool at start-up so that a late driver allocation can fail,
+ * or a plug-in whose host application forbids allocation calls after
+ * initialisation.  maxdnn_conv_fprop allocates its per-device status block with
+ * cudaMalloc on first use; this entry point never calls cudaMalloc, cudaFree or
+ * any allocating library routine.  The status block its kernel reports into is a
+ * 256-byte device array compiled into the library (every GPU that loads the
+ * library holds those 256 bytes until the process exits).
+ *
+ * Same arguments, layouts, result and NOT_SUPPORTED cases as maxdnn_conv_fprop
+ * (the same kernel runs; the result is bitwise the same).  In addition:
+ *   - A problem whose kernel would need more than the 256 bytes of built-in
+ *     scratch is refused with MAXDNN_NOT_SUPPORTED and nothing is launched.
+ *     (The fp32 kernel needs 4 bytes for every descriptor it supports today.)
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and sets kernel
+ *     attributes; make that first call before any stream capture begins.
+ *   - All calls on a device share the one block, and each call clears the word
+ *     it uses (a memset enqueued on `cuda_stream` ahead of the kernel).  Two
+ *     calls whose work overlaps on the GPU — different streams, no ordering
+ *     between them — therefore race on it; order them, or use
+ *     maxdnn_conv_fprop for one of them.
+ *   - A bounded wait that runs out still ends the kernel instead of hanging it,
+ *     but this entry point has no way to hand that code back:
+ *     maxdnn_last_device_status() reports on maxdnn_conv_fprop's block only.
+ */
+maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const float* in,
+                                        const float* filt, float* out, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reads and clears the current device's
  * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside a
  * kernel ran out; its output is not valid) or MAXDNN_CUDA_ERROR. */

@@ -14,7 +14,8 @@ __all__ = [
     "OK", "INVALID_VALUE", "NOT_SUPPORTED", "CUDA_ERROR", "DEVICE_TIMEOUT",
     "library_path", "load_library", "status_string", "conv_out_dims", "conv_flops",
     "conv_in_elems", "conv_filt_elems", "conv_out_elems", "conv_plan_query", "conv_fprop",
-    "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "last_device_status",
+    "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
+    "last_device_status",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
 ]
 
@@ -25,7 +26,8 @@ EXPORTED_SYMBOLS = [
     "maxdnn_status_string", "maxdnn_conv_out_dims", "maxdnn_conv_flops", "maxdnn_conv_in_elems",
     "maxdnn_conv_filt_elems", "maxdnn_conv_out_elems", "maxdnn_conv_plan_query",
     "maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16",
-    "maxdnn_conv_fprop_host", "maxdnn_last_device_status", "maxdnn_launch_count",
+    "maxdnn_conv_fprop_host", "maxdnn_conv_fprop_noalloc", "maxdnn_last_device_status",
+    "maxdnn_launch_count",
 ]
 
 
@@ -91,7 +93,8 @@ def load_library():
     lib.maxdnn_conv_plan_query.restype = ctypes.c_int
     lib.maxdnn_conv_plan_query.argtypes = [P(ConvDesc), ctypes.c_int, ctypes.c_int32, P(PlanInfo),
                                            P(KStep), ctypes.c_int32]
-    for name in ("maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16"):
+    for name in ("maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16",
+                 "maxdnn_conv_fprop_noalloc"):
         getattr(lib, name).restype = ctypes.c_int
         getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
@@ -179,6 +182,20 @@ def fprop_status(desc: ConvDesc, inp, filt, out, kind: int = KERNEL_FP32, stream
 def conv_fprop(desc: ConvDesc, inp, filt, out, stream=None) -> None:
     """maxdnn_conv_fprop: exact fp32 FPROP on device tensors (asynchronous)."""
     _check(fprop_status(desc, inp, filt, out, KERNEL_FP32, stream), "maxdnn_conv_fprop")
+
+
+def conv_fprop_noalloc(desc: ConvDesc, inp, filt, out, stream=None) -> None:
+    """maxdnn_conv_fprop_noalloc: the fp32 FPROP for callers that must not
+    allocate — the library itself makes no allocation call on this path (its
+    status block is a device array built into the library).  Tensors are the
+    caller's, as for conv_fprop; calls that overlap on the GPU race on the
+    shared block."""
+    lib = load_library()
+    pin = _dev_ptr(inp, ("float32",), conv_in_elems(desc), "in")
+    pf = _dev_ptr(filt, ("float32",), conv_filt_elems(desc), "filt")
+    po = _dev_ptr(out, ("float32",), conv_out_elems(desc), "out")
+    _check(int(lib.maxdnn_conv_fprop_noalloc(ctypes.byref(desc), pin, pf, po, _stream_ptr(stream))),
+           "maxdnn_conv_fprop_noalloc")
 
 
 def conv_fprop_tf32(desc: ConvDesc, inp, filt, out, stream=None) -> None:

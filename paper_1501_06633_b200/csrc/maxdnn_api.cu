@@ -258,6 +258,119 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
               : launch_umma<false>(ds, mf, mi, mo, args, stream);
 }
 
+// ---------------------------------------------------------------------------
+// Allocation-free fp32 entry point.  The status block its kernel reports into
+// lives in this file-scope device array instead of cudaMalloc'd memory.  Every
+// device that loads the library carries these 256 bytes until the process ends.
+// In host code the array's name is only a handle for the runtime: the device
+// address is obtained once per device with cudaGetSymbolAddress and passed on.
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 256;
+static __device__ __align__(256) uint32_t g_static_scratch[kStaticScratchBytes / sizeof(uint32_t)];
+
+// Scratch the fp32 kernel needs for a plan: one status word today.
+size_t ffma_scratch_bytes(const ConvGeom&) { return sizeof(uint32_t); }
+
+DeviceState g_static_dev[kMaxDevices];   // `status` points into g_static_scratch of that device
+
+maxdnn_status static_state(DeviceState** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+  if (dev < 0 || dev >= kMaxDevices) return MAXDNN_NOT_SUPPORTED;
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceState& s = g_static_dev[dev];
+  if (!s.ready) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    s.sm100 = (prop.major == 10);
+    s.sm_count = prop.multiProcessorCount;
+    if (s.sm100) {
+      void* p = nullptr;
+      // device `dev` is current: this is the address of ITS copy of the array
+      if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+        cudaGetLastError();
+        return MAXDNN_CUDA_ERROR;
+      }
+      s.status = static_cast<uint32_t*>(p);
+    }
+    s.ready = true;
+  }
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) !=
+            cudaSuccess || !fn) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = &s;
+  return MAXDNN_OK;
+}
+
+maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                                 float* out, cudaStream_t stream) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = static_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+
+  static thread_local FfmaArgs args;
+  st = plan_ffma(*desc, ds->sm_count, 0, &args.g, &args.table);
+  if (st != MAXDNN_OK) return st;
+  if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
+  args.out = out;
+  args.status = ds->status;
+  const ConvGeom& g = args.g;
+
+  CUtensorMap mf, mi;
+  {
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Sk, (uint64_t)g.Sk, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Sk * g.No * 4,
+                             (uint64_t)g.Sk * g.Sk * g.No * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
+                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
+    st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (st != MAXDNN_OK) return st;
+  }
+  // The block is shared by every call and keeps what the last call left: the word
+  // the kernel tests must read zero when it starts.
+  if (cudaMemsetAsync(ds->status, 0, ffma_scratch_bytes(g), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  const bool fx = g.fixed_pitch != 0;
+  switch (g.tile_m) {
+    case 128: return fx ? launch_ffma<8, true>(ds, 2, mf, mi, args, stream)
+                        : launch_ffma<8, false>(ds, 3, mf, mi, args, stream);
+    case 96: return fx ? launch_ffma<6, true>(ds, 4, mf, mi, args, stream)
+                       : launch_ffma<6, false>(ds, 5, mf, mi, args, stream);
+    case 64: return fx ? launch_ffma<4, true>(ds, 6, mf, mi, args, stream)
+                       : launch_ffma<4, false>(ds, 7, mf, mi, args, stream);
+    case 32: return fx ? launch_ffma<2, true>(ds, 8, mf, mi, args, stream)
+                       : launch_ffma<2, false>(ds, 9, mf, mi, args, stream);
+    default: return MAXDNN_NOT_SUPPORTED;
+  }
+}
+
 }  // namespace
 }  // namespace maxdnn
 
@@ -398,6 +511,11 @@ maxdnn_status maxdnn_last_device_status(void* cuda_stream) {
     return MAXDNN_DEVICE_TIMEOUT;
   }
   return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const float* in,
+                                        const float* filt, float* out, void* cuda_stream) {
+  return fprop_fp32_noalloc(desc, in, filt, out, static_cast<cudaStream_t>(cuda_stream));
 }
 
 uint64_t maxdnn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,0 +1,59 @@
+"""The allocation-free fp32 entry point (collected last on purpose: a run that
+stops at the first failure has then already run every other test).
+
+It serves callers that cannot let the library call cudaMalloc — latency-bound
+loops, processes whose device memory is fully pre-reserved, hosts that forbid
+allocation after start-up.  Its kernel is the one behind maxdnn_conv_fprop with
+the status block in a device array built into the library, so the two entry
+points must agree; the block is shared by all calls and keeps the last call's
+contents, so the check is made on two calls in a row with different inputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1501_06633_b200 as mx
+from paper_1501_06633_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5   # the tolerance of the fp32 parity tests (max error / max |reference|)
+
+
+def both_entry_points(w, seed_offset):
+    inp, filt = wl.make_inputs(w, seed_offset=seed_offset)
+    d = mx.ConvDesc.make(*w.dims)
+    d_in, d_f = torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda()
+    n_out = mx.conv_out_elems(d)
+    ref = torch.full((n_out,), -1.0, dtype=torch.float32, device="cuda")
+    got = torch.full((n_out,), -2.0, dtype=torch.float32, device="cuda")
+    mx.conv_fprop(d, d_in, d_f, ref)
+    assert mx.last_device_status() == mx.OK
+    mx.conv_fprop_noalloc(d, d_in, d_f, got)
+    torch.cuda.synchronize()
+    return got.cpu().numpy(), ref.cpu().numpy()
+
+
+def test_noalloc_entry_point_matches_fprop_twice_in_a_row():
+    shapes = [wl.WORKLOADS["tiny3x3"],
+              wl.WORKLOADS["mid5x5"].scaled(Nb=128, Wi=9, Hi=7, Nc=40, No=160)]
+    for call, w in enumerate(shapes):
+        got, ref = both_entry_points(w, seed_offset=call)
+        scale = float(np.max(np.abs(ref)))
+        assert scale > 0
+        err = float(np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64)))) / scale
+        assert err <= TOL_FP32, "call %d: E_inf = %.3e" % (call, err)
+    # and once more on the first shape: the shared block carries nothing over
+    got, ref = both_entry_points(shapes[0], seed_offset=7)
+    np.testing.assert_allclose(got, ref, rtol=0, atol=TOL_FP32 * float(np.max(np.abs(ref))))
+
+
+def test_noalloc_entry_point_rejects_what_fprop_rejects():
+    bad = mx.ConvDesc.make(30, 8, 8, 4, 32, 3, 1, 1)      # Nb not a multiple of 4
+    x = torch.zeros(mx.conv_in_elems(bad), device="cuda")
+    f = torch.zeros(mx.conv_filt_elems(bad), device="cuda")
+    o = torch.zeros(mx.conv_out_elems(bad), device="cuda")
+    before = mx.launch_count()
+    with pytest.raises(mx.MaxdnnError) as e:
+        mx.conv_fprop_noalloc(bad, x, f, o)
+    assert e.value.status == mx.NOT_SUPPORTED
+    assert mx.launch_count() == before
