@@ -76,9 +76,10 @@ def flops(w, Ho, Wo):
 # ----------------------------------------------------------------------------
 # CPU oracle legs (cpu_baseline of our arm, and the whole --impl reference arm)
 # ----------------------------------------------------------------------------
-def oracle_sample(w, target_seconds, repeats=1):
+def oracle_sample(w, target_seconds):
     """Time the oracle, as it stands, on a band of output rows of the workload
-    sized to take about `target_seconds`.  Returns (tflops, seconds, rows, threads)."""
+    sized to take about `target_seconds` (the whole workload, repeated, if that is
+    shorter).  Returns (tflops, seconds, rows, Ho, repeats, threads)."""
     import oracle
     inp, filt = wl.make_inputs(w)
     Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
@@ -89,14 +90,13 @@ def oracle_sample(w, target_seconds, repeats=1):
     t_row = max(time.perf_counter() - t0, 1e-6)
     rows = int(max(1, min(Ho, target_seconds / t_row)))
     y0 = max(0, min(Ho - rows, y_mid - rows // 2))
-    best = None
+    repeats = int(max(1, min(50, round(target_seconds / (t_row * rows)))))
+    t0 = time.perf_counter()
     for _ in range(repeats):
-        t0 = time.perf_counter()
         oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, rows=(y0, y0 + rows))
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    fl = flops(w, rows, Wo)
-    return fl / best / 1e12, best, rows, Ho, oracle.num_threads()
+    dt = time.perf_counter() - t0
+    fl = flops(w, rows, Wo) * repeats
+    return fl / dt / 1e12, dt, rows, Ho, repeats, oracle.num_threads()
 
 
 def run_reference(args):
@@ -202,6 +202,34 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------
+# multi-rank plumbing (also exercised on CPU with gloo by the tests)
+# ----------------------------------------------------------------------------
+def rank_env():
+    """(rank, local_rank, world) from the launcher's environment."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of floats over all ranks."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def shard_inputs(w, rank):
+    """Rank `rank`'s batch shard: same recipe, its own independent draw."""
+    return wl.make_inputs(w, seed_offset=rank)
+
+
+def whole_job_tflops(flops_per_rank, world, ms_step):
+    return world * flops_per_rank / (ms_step * 1e-3) / 1e12
+
+
+# ----------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------
 def run_ours(args):
@@ -210,9 +238,7 @@ def run_ours(args):
 
     import paper_1501_06633_b200 as mx
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local_rank, world = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -230,7 +256,7 @@ def run_ours(args):
     # Each rank holds its own batch shard (same recipe, its own seed); FPROP needs
     # no exchange between shards.  Buffer sets are rotated so that no step finds
     # its inputs in L2.
-    inp, filt = wl.make_inputs(w, seed_offset=rank)
+    inp, filt = shard_inputs(w, rank)
     n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / nbytes)))
     if args.kernel == "bf16":
         to_dev = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
@@ -289,13 +315,10 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], "cuda", world)
     ms_step = ms_total / args.steps
-    value = world * C / (ms_step * 1e-3) / 1e12
-    e2e_value = world * C / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    value = whole_job_tflops(C, world, ms_step)
+    e2e_value = whole_job_tflops(C, world, e2e_ms / e2e_steps)
 
     if rank == 0:
         sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
@@ -346,10 +369,11 @@ def run_ours(args):
             cycles = ms_step * 1e-3 * clocks["sm_mhz"] * 1e6
             line["roofline"]["ce_at_sampled_clock"] = C / (2.0 * 128 * sm_count * cycles)
         if world == 1 and not args.no_cpu_baseline:
-            tf, secs, rows, Ho_, threads = oracle_sample(w, args.cpu_seconds)
+            tf, secs, rows, Ho_, reps, threads = oracle_sample(w, args.cpu_seconds)
             line["cpu_baseline"] = {
                 "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
-                "sample": "%d of %d output rows of %s, %.1f s" % (rows, Ho_, w.name, secs)}
+                "sample": "%d of %d output rows of %s x %d passes, %.1f s" % (rows, Ho_, w.name,
+                                                                            reps, secs)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
