@@ -33,7 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "nvcc")
         tmp = LIB + ".tmp.%d" % os.getpid()
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + \
+        extra = os.environ.get("MAXDNN_NVCC_EXTRA", "").split()
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + \
               [os.path.join(CSRC, s) for s in SOURCES]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if verbose:

@@ -1,15 +1,20 @@
 // Exact-fp32 FPROP convolution kernel for sm_100a.
 //
 // One persistent CTA per SM walks a list of tiles.  A tile is the GEMM block of
-// Section 3.2: tile_m filters x (tile_px adjacent output pixels x tile_n images),
-// 128 columns wide.  Warp 8 is the producer: one elected lane walks the K-step
-// table (Section 3.2's precomputed offsets) and issues, per step, one bulk tensor
-// copy of filter-matrix rows and tile_px copies of patch rows into a ring of
-// shared-memory stages; the copy engine zero-fills the apron, so the consumers
-// never test a bound.  Warps 0-7 are consumers: each thread owns an MR x 8
-// register block (Section 3.1's 8 x 8 register blocking) and runs a flat loop
-// of shared loads and packed fp32 multiply-adds, operands double-buffered in
-// registers (Section 3.1, "double buffering of shared memory loads").
+// Section 3.2: tile_m filters x (tile_px adjacent output pixels x tile_n images).
+// The producer — one lane — walks the K-step table (Section 3.2's precomputed
+// offsets) and issues, per step, one bulk tensor copy of filter-matrix rows and one
+// (or tile_px) copies of patch rows into a ring of shared-memory stages; the copy
+// engine zero-fills the apron, so the consumers never test a bound.  Eight consumer
+// warps: each thread owns an MR x NR register block (Section 3.1's register
+// blocking) and runs a flat loop of shared loads and packed fp32 multiply-adds,
+// operands double-buffered in registers (Section 3.1, "double buffering of shared
+// memory loads").
+//
+// The producer is a ninth warp when the register block leaves room for it
+// (registers are allocated per four warps, so nine warps cap a thread at 168).
+// Larger blocks (MR*NR >= 96) run with eight warps and 255 registers; there the
+// first consumer warp issues the copies itself, one K step per step it consumes.
 #pragma once
 #include "plan.h"
 #include "ptx_util.cuh"
@@ -17,8 +22,10 @@
 namespace maxdnn {
 
 constexpr int kFfmaConsumerWarps = 8;
-// Eight consumer warps plus the producer warp.
-constexpr int ffma_threads(int) { return (kFfmaConsumerWarps + 1) * 32; }
+__host__ __device__ constexpr bool ffma_inline_producer(int mr, int nr) { return mr * nr >= 96; }
+__host__ __device__ constexpr int ffma_threads(int mr, int nr) {
+  return (kFfmaConsumerWarps + (ffma_inline_producer(mr, nr) ? 0 : 1)) * 32;
+}
 
 struct FfmaArgs {
   ConvGeom g;
@@ -27,15 +34,18 @@ struct FfmaArgs {
   KStepTable table;
 };
 
-template <int MR>
+template <int MR, int NR>
 struct Frag {
   float2 a[MR / 2];
-  float4 b[2];
+  float4 b[NR / 4];
 };
 
-template <int MR>
-__device__ __forceinline__ void load_frag(Frag<MR>& f, const float* a_row, const float* b0,
-                                          const float* b1) {
+// Thread (to, tn) of the 16 x 16 consumer grid reads, from row `a_row` of the staged
+// filter box, MR values (float4 groups 64 filters apart, or float2 groups 32 apart)
+// and, from the staged patch row, NR values (float4 groups 64 columns apart).
+template <int MR, int NR, bool FIXED>
+__device__ __forceinline__ void load_frag(Frag<MR, NR>& f, const float* a_row,
+                                          const float* const (&b_row)[NR / 4], int b_off) {
   if constexpr (MR % 4 == 0) {
 #pragma unroll
     for (int q = 0; q < MR / 4; ++q) {
@@ -47,43 +57,117 @@ __device__ __forceinline__ void load_frag(Frag<MR>& f, const float* a_row, const
 #pragma unroll
     for (int p = 0; p < MR / 2; ++p) f.a[p] = *reinterpret_cast<const float2*>(a_row + p * 32);
   }
-  f.b[0] = *reinterpret_cast<const float4*>(b0);
-  f.b[1] = *reinterpret_cast<const float4*>(b1);
+#pragma unroll
+  for (int h = 0; h < NR / 4; ++h) {
+    if constexpr (FIXED)
+      f.b[h] = *reinterpret_cast<const float4*>(b_row[0] + b_off + 64 * h);
+    else
+      f.b[h] = *reinterpret_cast<const float4*>(b_row[h] + b_off);
+  }
 }
 
 // acc pairs: P[i][j] = {acc(2i,2j), acc(2i+1,2j+1)}, Q[i][j] = {acc(2i,2j+1), acc(2i+1,2j)}.
 // Both products of a 2 x 2 sub-block come from one packed multiply-add each: the
 // filter pair times the patch pair, and the filter pair times the swapped patch pair.
-template <int MR>
-__device__ __forceinline__ void fma_block(const Frag<MR>& f, float2 (&P)[MR / 2][4],
-                                          float2 (&Q)[MR / 2][4]) {
-  float2 bn[4], bs[4];
-  bn[0] = make_float2(f.b[0].x, f.b[0].y);
-  bn[1] = make_float2(f.b[0].z, f.b[0].w);
-  bn[2] = make_float2(f.b[1].x, f.b[1].y);
-  bn[3] = make_float2(f.b[1].z, f.b[1].w);
+template <int MR, int NR>
+__device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR / 2][NR / 2],
+                                          float2 (&Q)[MR / 2][NR / 2]) {
+  float2 bn[NR / 2], bs[NR / 2];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) bs[j] = make_float2(bn[j].y, bn[j].x);
+  for (int h = 0; h < NR / 4; ++h) {
+    bn[2 * h] = make_float2(f.b[h].x, f.b[h].y);
+    bn[2 * h + 1] = make_float2(f.b[h].z, f.b[h].w);
+  }
+#pragma unroll
+  for (int j = 0; j < NR / 2; ++j) bs[j] = make_float2(bn[j].y, bn[j].x);
 #pragma unroll
   for (int i = 0; i < MR / 2; ++i) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NR / 2; ++j) {
       P[i][j] = __ffma2_rn(f.a[i], bn[j], P[i][j]);
       Q[i][j] = __ffma2_rn(f.a[i], bs[j], Q[i][j]);
     }
   }
 }
 
-// One row of the flat loop: operand loads for the row after next are issued
-// before the multiply-adds of the current row (register double buffering).
-#define MAXDNN_ROW_PTRS(R) a_ptr + (R) * Mt, b0_ptr + (R) * b_pitch, b1_ptr + (R) * b_pitch
+// Producer state: which (tile, K step) is loaded next, into which ring stage.
+struct FfmaProducer {
+  int tile, step, stage;
+  uint32_t phase;
+  int o0, n0, h0, w0;
 
-template <int MR, bool FIXED>
-__global__ void __launch_bounds__(ffma_threads(MR), 1)
+  __device__ __forceinline__ void set_tile(const ConvGeom& g, int mt) {
+    int r = tile;
+    const int ob = r % g.o_blocks; r /= g.o_blocks;
+    const int nch = r % g.n_chunks; r /= g.n_chunks;
+    const int xr = r % g.x_runs;
+    const int y = r / g.x_runs;
+    o0 = ob * mt;
+    n0 = nch * g.tile_n;
+    h0 = y * g.stride - g.pad;
+    w0 = xr * g.tile_px * g.stride - g.pad;
+  }
+
+  __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
+    tile = g.tile_begin + blockIdx.x;
+    step = 0; stage = 0; phase = 0;
+    o0 = n0 = h0 = w0 = 0;
+    if (tile < g.tile_end) set_tile(g, mt);
+  }
+
+  __device__ __forceinline__ bool has_work(const ConvGeom& g) const { return tile < g.tile_end; }
+
+  // Waits for the ring slot, issues the copies of one K step, advances.
+  template <bool BACKOFF>
+  __device__ __forceinline__ bool issue(const FfmaArgs& args, const CUtensorMap* map_filt,
+                                        const CUtensorMap* map_in, uint32_t a_base, uint32_t b_base,
+                                        uint32_t full_bar, uint32_t empty_bar, int mt) {
+    const ConvGeom& g = args.g;
+    const uint32_t eb = empty_bar + 8u * stage;
+    const bool ok = BACKOFF ? mbar_wait_backoff(eb, phase ^ 1u, args.status, kDevTimeoutEmpty)
+                            : mbar_wait(eb, phase ^ 1u, args.status, kDevTimeoutEmpty);
+    if (!ok) return false;
+    const maxdnn_kstep ks = args.table.s[step];
+    const uint32_t fb = full_bar + 8u * stage;
+    mbar_arrive_expect_tx(fb, (uint32_t)(g.a_box_bytes + g.b_boxes * g.b_box_bytes));
+    tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, o0, ks.kw0, ks.kh, ks.c0);
+    uint32_t dst = b_base + (uint32_t)stage * g.b_stage_bytes;
+    int w = w0 + ks.kw0;
+    for (int t = 0; t < g.b_boxes; ++t) {
+      tma_load_4d(dst, map_in, fb, n0, w, h0 + ks.kh, ks.c0);
+      dst += g.b_slot_bytes;
+      w += g.stride;
+    }
+    if (++stage == g.stages) { stage = 0; phase ^= 1u; }
+    if (++step == g.n_ksteps) {
+      step = 0;
+      tile += gridDim.x;
+      if (tile < g.tile_end) set_tile(g, mt);
+    }
+    return true;
+  }
+
+  // After a failed wait: let every copy already issued land before the CTA's shared
+  // memory is released.
+  __device__ __forceinline__ void drain(const ConvGeom& g, uint32_t full_bar) {
+    for (int s = 0; s < g.stages; ++s) {
+      const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+      mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
+    }
+  }
+};
+
+#define MAXDNN_ROW(R) a_ptr + (R) * Mt, b_ptr, (R) * b_pitch
+
+template <int MR, int NR, bool FIXED>
+__global__ void __launch_bounds__(ffma_threads(MR, NR), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
                  const __grid_constant__ FfmaArgs args) {
-  constexpr int Mt = 16 * MR;
+  constexpr int Mt = 16 * MR;           // filters per tile
+  constexpr int Nt = 16 * NR;           // columns per tile
+  constexpr int NH = NR / 4;            // float4 column groups per thread
+  constexpr bool INLINE = ffma_inline_producer(MR, NR);
   extern __shared__ uint8_t smem_raw[];
   const ConvGeom& g = args.g;
 
@@ -113,71 +197,52 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int n_ksteps = g.n_ksteps;
   const int rows = g.rows;
 
-  if (warp >= kFfmaConsumerWarps) {
-    // ------------------------------------------------------------ producer
-    if (warp == kFfmaConsumerWarps && lane == 0) {
-      prefetch_tensormap(&map_filt);
-      prefetch_tensormap(&map_in);
-      const uint32_t tx_bytes = (uint32_t)(g.a_box_bytes + g.b_boxes * g.b_box_bytes);
-      const int w_step = g.stride;
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
-        int r = tile;
-        const int ob = r % g.o_blocks; r /= g.o_blocks;
-        const int nch = r % g.n_chunks; r /= g.n_chunks;
-        const int xr = r % g.x_runs;
-        const int y = r / g.x_runs;
-        const int o0 = ob * Mt;
-        const int n0 = nch * g.tile_n;
-        const int h0 = y * g.stride - g.pad;
-        const int w0 = xr * g.tile_px * g.stride - g.pad;
-        for (int s = 0; s < n_ksteps; ++s) {
-          if (!mbar_wait_backoff(empty_bar + 8u * stage, phase ^ 1u, args.status,
-                                 kDevTimeoutEmpty)) {
-            ok = false;
-            break;
-          }
-          const maxdnn_kstep ks = args.table.s[s];
-          const uint32_t fb = full_bar + 8u * stage;
-          mbar_arrive_expect_tx(fb, tx_bytes);
-          tma_load_4d(base + a_off + (uint32_t)stage * g.a_stage_bytes, &map_filt, fb, o0, ks.kw0,
-                      ks.kh, ks.c0);
-          uint32_t dst = base + b_off + (uint32_t)stage * g.b_stage_bytes;
-          int w = w0 + ks.kw0;
-          for (int t = 0; t < g.b_boxes; ++t) {
-            tma_load_4d(dst, &map_in, fb, n0, w, h0 + ks.kh, ks.c0);
-            dst += g.b_slot_bytes;
-            w += w_step;
-          }
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
-        }
+  if constexpr (!INLINE) {
+    if (warp == kFfmaConsumerWarps) {
+      // ---------------------------------------------------- producer warp
+      if (lane == 0) {
+        prefetch_tensormap(&map_filt);
+        prefetch_tensormap(&map_in);
+        FfmaProducer p;
+        p.init(g, Mt);
+        bool ok = true;
+        while (ok && p.has_work(g))
+          ok = p.template issue<true>(args, &map_filt, &map_in, base + a_off, base + b_off, full_bar,
+                                      empty_bar, Mt);
+        if (!ok) p.drain(g, full_bar);
       }
-      if (!ok) {
-        // Leaving early: let every copy already issued land before the CTA's
-        // shared memory is released.
-        for (int s = 0; s < stages; ++s) {
-          const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-          mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
-        }
-      }
+      return;
     }
-    return;
   }
 
   // -------------------------------------------------------------- consumers
+  FfmaProducer prod;          // used by warp 0 only, and only when INLINE
+  bool prod_ok = true;
+  prod.init(g, Mt);
+  if constexpr (INLINE) {
+    if (warp == 0) {
+      if (lane == 0) {
+        prefetch_tensormap(&map_filt);
+        prefetch_tensormap(&map_in);
+        for (int s = 0; s + 2 < stages && prod_ok && prod.has_work(g); ++s)
+          prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off, base + b_off,
+                                               full_bar, empty_bar, Mt);
+      }
+      __syncwarp();
+    }
+  }
+
   const int wo = warp >> 1, wn = warp & 1;
   const int to = wo * 4 + (lane >> 3);   // 0..15 along the filter axis
   const int tn = wn * 8 + (lane & 7);    // 0..15 along the column axis
   const int a_elem = (MR % 4 == 0) ? 4 * to : 2 * to;
 
-  // This thread's two groups of four columns -> (pixel, image) and smem offset.
+  // This thread's groups of four columns -> (pixel, image) and smem offset.
   const int used_cols = g.tile_px * g.tile_n;
-  int col_px[2], col_n[2];
-  uint32_t b_elem[2];
+  int col_px[NH], col_n[NH];
+  uint32_t b_elem[NH];
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
+  for (int h = 0; h < NH; ++h) {
     const int col = 4 * tn + 64 * h;
     const bool live = col < used_cols;
     col_px[h] = live ? col / g.tile_n : -1;
@@ -187,61 +252,79 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     else
       b_elem[h] = live ? (uint32_t)(col_px[h] * (g.b_slot_bytes >> 2) + col_n[h]) : 0u;
   }
-  const int b_pitch = FIXED ? kTileCols : g.tile_n;   // floats between patch rows
+  const int b_pitch = FIXED ? Nt : g.tile_n;   // floats between patch rows
 
   int stage = 0;
   uint32_t phase = 0;
   bool ok = true;
 
-  for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
-    float2 P[MR / 2][4], Q[MR / 2][4];
+  for (int tile = g.tile_begin + blockIdx.x; tile < g.tile_end && ok; tile += gridDim.x) {
+    float2 P[MR / 2][NR / 2], Q[MR / 2][NR / 2];
 #pragma unroll
     for (int i = 0; i < MR / 2; ++i)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < NR / 2; ++j) {
         P[i][j] = make_float2(0.f, 0.f);
         Q[i][j] = make_float2(0.f, 0.f);
       }
 
-    Frag<MR> f0, f1;
+    Frag<MR, NR> f0, f1;
     ok = mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull);
     if (!ok) break;
-    const float* a_ptr =
-        reinterpret_cast<const float*>(base_ptr + a_off + (size_t)stage * g.a_stage_bytes) + a_elem;
-    const float* bs_ptr =
-        reinterpret_cast<const float*>(base_ptr + b_off + (size_t)stage * g.b_stage_bytes);
-    const float* b0_ptr = bs_ptr + b_elem[0];
-    const float* b1_ptr = bs_ptr + b_elem[1];
-    load_frag<MR>(f0, MAXDNN_ROW_PTRS(0));
+    const float* a_ptr;
+    const float* b_ptr[NH];
+    auto point_at_stage = [&](int st) {
+      a_ptr = reinterpret_cast<const float*>(base_ptr + a_off + (size_t)st * g.a_stage_bytes) + a_elem;
+      const float* bs = reinterpret_cast<const float*>(base_ptr + b_off + (size_t)st * g.b_stage_bytes);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) b_ptr[h] = bs + b_elem[h];
+    };
+    point_at_stage(stage);
+    load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(0));
 
     for (int s = 0; s < n_ksteps; ++s) {
+      if constexpr (INLINE) {
+        // Refill the slot this CTA finished two steps ago (every warp has released it
+        // by now, so the wait does not hold warp 0 back) with the K step that is
+        // (stages - 2) ahead of the one being consumed.
+        if (warp == 0) {
+          if (lane == 0 && prod_ok && prod.has_work(g))
+            prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off,
+                                                 base + b_off, full_bar, empty_bar, Mt);
+          __syncwarp();
+        }
+      }
       // f0 holds row 0 of this stage.  Four rows per iteration while the row
       // after the block is still inside the stage.
       int r = 0;
 #pragma unroll 1
       for (; r + 4 < rows; r += 4) {
-        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
-        fma_block<MR>(f0, P, Q);
-        load_frag<MR>(f0, MAXDNN_ROW_PTRS(2));
-        fma_block<MR>(f1, P, Q);
-        load_frag<MR>(f1, MAXDNN_ROW_PTRS(3));
-        fma_block<MR>(f0, P, Q);
-        load_frag<MR>(f0, MAXDNN_ROW_PTRS(4));
-        fma_block<MR>(f1, P, Q);
-        a_ptr += 4 * Mt; b0_ptr += 4 * b_pitch; b1_ptr += 4 * b_pitch;
+        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        fma_block<MR, NR>(f0, P, Q);
+        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(2));
+        fma_block<MR, NR>(f1, P, Q);
+        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(3));
+        fma_block<MR, NR>(f0, P, Q);
+        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(4));
+        fma_block<MR, NR>(f1, P, Q);
+        a_ptr += 4 * Mt;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) b_ptr[h] += 4 * b_pitch;
       }
 #pragma unroll 1
       for (; rows - r > 2; r += 2) {   // 3 or 4 rows left: two of them here
-        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
-        fma_block<MR>(f0, P, Q);
-        load_frag<MR>(f0, MAXDNN_ROW_PTRS(2));
-        fma_block<MR>(f1, P, Q);
-        a_ptr += 2 * Mt; b0_ptr += 2 * b_pitch; b1_ptr += 2 * b_pitch;
+        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        fma_block<MR, NR>(f0, P, Q);
+        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(2));
+        fma_block<MR, NR>(f1, P, Q);
+        a_ptr += 2 * Mt;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) b_ptr[h] += 2 * b_pitch;
       }
       const bool two_left = (rows - r == 2);
       if (two_left) {
-        load_frag<MR>(f1, MAXDNN_ROW_PTRS(1));
-        fma_block<MR>(f0, P, Q);
+        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        fma_block<MR, NR>(f0, P, Q);
       }
       // The last row of this stage is in f1 (two_left) or f0.  Prefetch row 0 of
       // the next stage into the other buffer before computing it.
@@ -251,18 +334,14 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       if (more) {
         ok = mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull);
         if (!ok) break;
-        a_ptr = reinterpret_cast<const float*>(base_ptr + a_off + (size_t)stage * g.a_stage_bytes) +
-                a_elem;
-        bs_ptr = reinterpret_cast<const float*>(base_ptr + b_off + (size_t)stage * g.b_stage_bytes);
-        b0_ptr = bs_ptr + b_elem[0];
-        b1_ptr = bs_ptr + b_elem[1];
+        point_at_stage(stage);
       }
       if (two_left) {
-        if (more) load_frag<MR>(f0, MAXDNN_ROW_PTRS(0));
-        fma_block<MR>(f1, P, Q);
+        if (more) load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(0));
+        fma_block<MR, NR>(f1, P, Q);
       } else {
-        if (more) load_frag<MR>(f1, MAXDNN_ROW_PTRS(0));
-        fma_block<MR>(f0, P, Q);
+        if (more) load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(0));
+        fma_block<MR, NR>(f0, P, Q);
         f0 = f1;
       }
       __syncwarp();
@@ -291,7 +370,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         if (o >= g.No) continue;
         const int i2 = i >> 1, ia = i & 1;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < NH; ++h) {
           const int x = x0 + col_px[h];
           const int n = n0 + col_n[h];
           if (col_px[h] < 0 || x >= g.Wo || n >= g.Nb) continue;
@@ -308,7 +387,11 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
     }
   }
+
+  if constexpr (INLINE) {
+    if (warp == 0 && lane == 0 && !(ok && prod_ok)) prod.drain(g, full_bar);
+  }
 }
-#undef MAXDNN_ROW_PTRS
+#undef MAXDNN_ROW
 
 }  // namespace maxdnn

@@ -90,10 +90,10 @@ int env_int(const char* name) {
   return v ? atoi(v) : 0;
 }
 
-template <int MR, bool FIXED>
+template <int MR, int NR, bool FIXED>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
-  auto kern = ffma_conv_kernel<MR, FIXED>;
+  auto kern = ffma_conv_kernel<MR, NR, FIXED>;
   if (!ds->ffma_attr[slot]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
         cudaSuccess) {
@@ -102,10 +102,30 @@ maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, cons
     }
     ds->ffma_attr[slot] = true;
   }
-  kern<<<args.g.grid, ffma_threads(MR), args.g.smem_bytes, stream>>>(mf, mi, args);
+  kern<<<args.g.grid, ffma_threads(MR, NR), args.g.smem_bytes, stream>>>(mf, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return MAXDNN_OK;
+}
+
+// Picks the kernel instance built for the plan's tile shape.
+maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                            const FfmaArgs& args, cudaStream_t stream) {
+  const ConvGeom& g = args.g;
+  const bool fx = g.fixed_pitch != 0;
+#define MAXDNN_FFMA_CASE(M, C, MR, NR, SLOT)                                             \
+  if (g.tile_m == (M) && g.tile_cols == (C))                                             \
+    return fx ? launch_ffma<MR, NR, true>(ds, (SLOT), mf, mi, args, stream)              \
+              : launch_ffma<MR, NR, false>(ds, (SLOT) + 1, mf, mi, args, stream);
+  MAXDNN_FFMA_CASE(256, 128, 16, 8, 0)
+  MAXDNN_FFMA_CASE(128, 256, 8, 16, 2)
+  MAXDNN_FFMA_CASE(96, 256, 6, 16, 4)
+  MAXDNN_FFMA_CASE(128, 128, 8, 8, 6)
+  MAXDNN_FFMA_CASE(96, 128, 6, 8, 8)
+  MAXDNN_FFMA_CASE(64, 128, 4, 8, 10)
+  MAXDNN_FFMA_CASE(32, 128, 2, 8, 12)
+#undef MAXDNN_FFMA_CASE
+  return MAXDNN_NOT_SUPPORTED;
 }
 
 maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const float* filt,
@@ -121,7 +141,8 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
-  st = plan_ffma(*desc, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), &args.g, &args.table);
+  st = plan_ffma(*desc, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
+                 &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   args.out = out;
   args.status = ds->status;
@@ -148,18 +169,7 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
-  const bool fx = g.fixed_pitch != 0;
-  switch (g.tile_m) {
-    case 128: return fx ? launch_ffma<8, true>(ds, 2, mf, mi, args, stream)
-                        : launch_ffma<8, false>(ds, 3, mf, mi, args, stream);
-    case 96: return fx ? launch_ffma<6, true>(ds, 4, mf, mi, args, stream)
-                       : launch_ffma<6, false>(ds, 5, mf, mi, args, stream);
-    case 64: return fx ? launch_ffma<4, true>(ds, 6, mf, mi, args, stream)
-                       : launch_ffma<4, false>(ds, 7, mf, mi, args, stream);
-    case 32: return fx ? launch_ffma<2, true>(ds, 8, mf, mi, args, stream)
-                       : launch_ffma<2, false>(ds, 9, mf, mi, args, stream);
-    default: return MAXDNN_NOT_SUPPORTED;
-  }
+  return dispatch_ffma(ds, mf, mi, args, stream);
 }
 
 template <bool BF16>
@@ -325,7 +335,7 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;
-  st = plan_ffma(*desc, ds->sm_count, 0, &args.g, &args.table);
+  st = plan_ffma(*desc, ds->sm_count, 0, 0, &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
   args.out = out;
@@ -357,18 +367,7 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
-  const bool fx = g.fixed_pitch != 0;
-  switch (g.tile_m) {
-    case 128: return fx ? launch_ffma<8, true>(ds, 2, mf, mi, args, stream)
-                        : launch_ffma<8, false>(ds, 3, mf, mi, args, stream);
-    case 96: return fx ? launch_ffma<6, true>(ds, 4, mf, mi, args, stream)
-                       : launch_ffma<6, false>(ds, 5, mf, mi, args, stream);
-    case 64: return fx ? launch_ffma<4, true>(ds, 6, mf, mi, args, stream)
-                       : launch_ffma<4, false>(ds, 7, mf, mi, args, stream);
-    case 32: return fx ? launch_ffma<2, true>(ds, 8, mf, mi, args, stream)
-                       : launch_ffma<2, false>(ds, 9, mf, mi, args, stream);
-    default: return MAXDNN_NOT_SUPPORTED;
-  }
+  return dispatch_ffma(ds, mf, mi, args, stream);
 }
 
 }  // namespace
@@ -432,7 +431,7 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   static thread_local KStepTable t;
   switch (kind) {
     case MAXDNN_KERNEL_FP32:
-      st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), &g, &t);
+      st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
       break;
     case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;
     case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;

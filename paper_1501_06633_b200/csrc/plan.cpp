@@ -30,16 +30,14 @@ static maxdnn_status common_limits(const maxdnn_conv_desc& d, int elem_bytes) {
   return MAXDNN_OK;
 }
 
-// Relative cost per multiply-accumulate of a filter tile of height m (smaller
-// register blocks spend a larger share of issue slots on operand loads).
-static double tile_m_cost(int m) {
-  switch (m) {
-    case 128: return 1.00;
-    case 96: return 1.03;
-    case 64: return 1.10;
-    default: return 1.35;
-  }
-}
+// Tile shapes the fp32 kernel is built for, with the relative cost per
+// multiply-accumulate measured for each (smaller register blocks spend a larger
+// share of issue slots on operand loads).
+struct FfmaShape { int m, cols; double cost; };
+static const FfmaShape kFfmaShapes[] = {
+    {128, 256, 0.97}, {256, 128, 0.99}, {128, 128, 1.00}, {96, 128, 1.10},
+    {96, 256, 1.12},  {64, 128, 1.18},  {32, 128, 1.50},
+};
 
 static void build_table(const maxdnn_conv_desc& d, int kc, int kwc, KStepTable* t, int* n) {
   int k = 0;
@@ -56,8 +54,24 @@ static void build_table(const maxdnn_conv_desc& d, int kc, int kwc, KStepTable* 
   *n = k;
 }
 
-maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, ConvGeom* g,
-                        KStepTable* t) {
+// Columns of a tile: tile_px adjacent output pixels x tile_n images <= cols.
+static double pick_columns(const maxdnn_conv_desc& d, int Wo, int cols, int* nn_out, int* T_out) {
+  int best_nn = 4, best_T = 1;
+  double best_eff = -1.0;
+  for (int nn = (d.Nb < cols ? d.Nb : cols); nn >= 4; nn -= 4) {
+    int T = cols / nn;
+    if (T > Wo) T = Wo;
+    const double eff =
+        ((double)d.Nb * Wo) / ((double)ceil_div(d.Nb, nn) * ceil_div(Wo, T) * (double)cols);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best_nn = nn; best_T = T; }
+  }
+  *nn_out = best_nn;
+  *T_out = best_T;
+  return best_eff;
+}
+
+maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, int force_cols,
+                        ConvGeom* g, KStepTable* t) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -69,48 +83,46 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
   g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
 
-  // Columns of a tile: tile_px adjacent output pixels x tile_n images <= 128.
-  int best_nn = 4, best_T = 1;
-  double best_eff = -1.0;
-  for (int nn = (d.Nb < kTileCols ? d.Nb : kTileCols); nn >= 4; nn -= 4) {
-    int T = kTileCols / nn;
-    if (T > Wo) T = Wo;
-    const double eff = ((double)d.Nb * Wo) /
-                       ((double)ceil_div(d.Nb, nn) * ceil_div(Wo, T) * (double)kTileCols);
-    if (eff > best_eff + 1e-9) { best_eff = eff; best_nn = nn; best_T = T; }
+  // Tile shape: fewest SM-time units over whole waves of persistent CTAs.
+  double best_t = 1e300;
+  int best_m = 0, best_cols = 0, best_nn = 0, best_T = 0;
+  for (const FfmaShape& sh : kFfmaShapes) {
+    if (force_tile_m > 0 && sh.m != force_tile_m) continue;
+    if (force_cols > 0 && sh.cols != force_cols) continue;
+    if (force_tile_m <= 0 && sh.m > align_up(d.No, 32) && sh.m != 32) continue;
+    int nn, T;
+    pick_columns(d, Wo, sh.cols, &nn, &T);
+    if (force_cols <= 0 && sh.cols > 128 && nn * T <= 128) continue;   // would not fill it
+    const int64_t tiles = (int64_t)ceil_div(d.No, sh.m) * ceil_div(Wo, T) * Ho * ceil_div(d.Nb, nn);
+    const int64_t waves = (tiles + sm_count - 1) / sm_count;
+    const double tm = (double)waves * sh.m * sh.cols * sh.cost;
+    if (tm < best_t - 1e-9) { best_t = tm; best_m = sh.m; best_cols = sh.cols; best_nn = nn; best_T = T; }
   }
+  if (best_m == 0) return MAXDNN_NOT_SUPPORTED;
+  g->tile_m = best_m;
+  g->tile_cols = best_cols;
   g->tile_n = best_nn;
   g->tile_px = best_T;
   g->n_chunks = ceil_div(d.Nb, best_nn);
   g->x_runs = ceil_div(Wo, best_T);
-
-  // Filter-tile height: fewest SM-time units over whole waves of persistent CTAs.
-  const int cand[4] = {128, 96, 64, 32};
-  int best_m = 32;
-  double best_t = 1e300;
-  for (int i = 0; i < 4; ++i) {
-    const int m = cand[i];
-    if (force_tile_m > 0 && m != force_tile_m) continue;
-    if (m > align_up(d.No, 32) && m != 32) continue;
-    const int64_t tiles = (int64_t)ceil_div(d.No, m) * g->x_runs * Ho * g->n_chunks;
-    const int64_t waves = (tiles + sm_count - 1) / sm_count;
-    const double tm = (double)waves * m * tile_m_cost(m);
-    if (tm < best_t - 1e-9) { best_t = tm; best_m = m; }
-  }
-  g->tile_m = best_m;
   g->o_blocks = ceil_div(d.No, best_m);
   const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
   if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_tiles = (int32_t)tiles;
+  g->tile_begin = 0;
+  g->tile_end = g->n_tiles;
 
   // K step: kc channels of one filter tap, or (few channels) kc channels of a
   // whole filter row of Sk taps.
   int kc, kwc;
+  // Tiles whose first consumer warp issues the copies keep one ring slot as slack.
+  const bool inline_producer = (best_m / 16) * (best_cols / 16) >= 96;
   if (d.Nc >= 8) {
     kwc = 1;
-    kc = 32;
+    const int kc_max = 32;
+    kc = kc_max;
     int best_pad = 1 << 30;
-    for (int c = 32; c >= 8; c -= 4) {
+    for (int c = kc_max; c >= 8; c -= 4) {
       const int padded = ceil_div(d.Nc, c) * c;
       if (padded < best_pad) { best_pad = padded; kc = c; }
     }
@@ -131,14 +143,14 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
 
   g->a_box_bytes = g->rows * g->tile_m * 4;
   g->a_stage_bytes = g->a_box_bytes;
-  // One box per stage whenever the 128 columns are one contiguous run of the map
+  // One box per stage whenever the tile's columns are one contiguous run of the map
   // (one pixel, or adjacent pixels of a stride-1 layer); else one box per pixel.
-  g->fixed_pitch = (g->tile_px * g->tile_n == kTileCols &&
+  g->fixed_pitch = (g->tile_px * g->tile_n == g->tile_cols &&
                     (g->tile_px == 1 || (d.stride == 1 && kwc == 1))) ? 1 : 0;
   if (g->fixed_pitch) {
     g->b_boxes = 1;
     g->b_box_w = g->tile_px > 1 ? g->tile_px : kwc;
-    g->b_box_bytes = g->rows * kTileCols * 4;
+    g->b_box_bytes = g->rows * g->tile_cols * 4;
     g->b_slot_bytes = g->b_box_bytes;
     g->b_stage_bytes = g->b_box_bytes;
   } else {
@@ -152,9 +164,9 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   const int budget = 200 * 1024;
   int stages = budget / stage;
   if (stages > 8) stages = 8;
-  if (stages < 2) return MAXDNN_NOT_SUPPORTED;
+  if (stages < (inline_producer ? 3 : 2)) return MAXDNN_NOT_SUPPORTED;
   g->stages = stages;
-  g->smem_bytes = stages * stage + 1024;   // + barriers, + slack for 1024-byte alignment
+  g->smem_bytes = stages * stage + 1024;   // + barriers, + slack for alignment
   g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
   return MAXDNN_OK;
 }
@@ -195,6 +207,9 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
   if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_tiles = (int32_t)tiles;
+  g->tile_begin = 0;
+  g->tile_end = g->n_tiles;
+  g->tile_cols = max_cols;
 
   // K step: kc channels of one filter tap; kc a multiple of the MMA's K
   // (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).

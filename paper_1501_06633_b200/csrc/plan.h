@@ -10,7 +10,6 @@
 namespace maxdnn {
 
 constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel parameters
-constexpr int kTileCols = 128;     // GEMM-block columns (pixels x images) of the FFMA kernel
 
 // What a kernel needs to know about the problem and its tiling.  Passed by
 // value in kernel parameter space together with the K-step table.
@@ -27,6 +26,8 @@ struct ConvGeom {
   int32_t stages;
   int32_t o_blocks, n_chunks, x_runs;
   int32_t n_tiles;
+  int32_t tile_begin, tile_end;   // tiles this launch walks: [tile_begin, tile_end)
+  int32_t tile_cols;       // columns of a tile the kernel is built for (128 or 256)
   int32_t a_stage_bytes;   // filter box bytes per stage
   int32_t a_box_bytes;
   int32_t fixed_pitch;     // 1: one patch box per stage, rows 128 floats apart
@@ -48,9 +49,9 @@ inline int align_up(int a, int b) { return ceil_div(a, b) * b; }
 
 maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo);
 
-// FFMA kernel plan.  force_tile_m > 0 pins the filter-tile height (ablations).
-maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, ConvGeom* g,
-                        KStepTable* t);
+// FFMA kernel plan.  force_tile_m / force_cols > 0 pin the tile shape (ablations).
+maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, int force_cols,
+                        ConvGeom* g, KStepTable* t);
 
 // Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
 maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,

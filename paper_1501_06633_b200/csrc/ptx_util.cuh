@@ -85,17 +85,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return mbar_wait_slow(bar, parity, status, code);
 }
 
-// Producer-side wait: sleeps between polls so that a warp waiting for a ring
-// slot does not take issue slots from the arithmetic warps of its scheduler.
+#ifndef MAXDNN_PRODUCER_SLEEP_NS
+#define MAXDNN_PRODUCER_SLEEP_NS 250
+#endif
+
+// Producer-side wait: sleeps between polls, so that a warp waiting for a ring slot
+// does not take issue slots from the arithmetic warps of its scheduler.  Same 2 s
+// budget as mbar_wait.
+__device__ __noinline__ bool mbar_wait_sleep_slow(uint32_t bar, uint32_t parity, uint32_t* status,
+                                                  uint32_t code) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+#if MAXDNN_PRODUCER_SLEEP_NS > 0
+      __nanosleep(MAXDNN_PRODUCER_SLEEP_NS);
+#endif
+      if (mbar_try_wait(bar, parity)) return true;
+    }
+    if (globaltimer_ns() - t0 > kWaitBudgetNs) break;
+    if (status && *reinterpret_cast<volatile uint32_t*>(status) != 0) break;
+  }
+  if (status) atomicCAS(status, 0u, code);
+  return false;
+}
+
 __device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, uint32_t* status,
                                                   uint32_t code) {
   if (mbar_try_wait(bar, parity)) return true;
-#pragma unroll 1
-  for (int i = 0; i < 64; ++i) {
-    __nanosleep(200);
-    if (mbar_try_wait(bar, parity)) return true;
-  }
-  return mbar_wait_slow(bar, parity, status, code);
+  return mbar_wait_sleep_slow(bar, parity, status, code);
 }
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {

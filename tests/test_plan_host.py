@@ -88,7 +88,7 @@ def emulate_fp32_plan(w, inp, filt, sm_count=148):
     n_chunks = -(-w.Nb // Nn)
     x_runs = -(-Wo // T)
     assert info.n_tiles == o_blocks * n_chunks * x_runs * Ho
-    assert T * Nn <= 128 and Nn % 4 == 0 and Mt in (32, 64, 96, 128)
+    assert T * Nn <= 256 and Nn % 4 == 0 and Mt in (32, 64, 96, 128, 256)
     assert info.grid == min(info.n_tiles, sm_count)
     # every (c, kh, kw) is covered by exactly one table entry
     seen = np.zeros((w.Nc, w.Sk, w.Sk), dtype=np.int32)
