@@ -27,6 +27,11 @@ __host__ __device__ constexpr int ffma_threads(int mr, int nr) {
   return (kFfmaConsumerWarps + (ffma_inline_producer(mr, nr) ? 0 : 1)) * 32;
 }
 
+// Multiply-add order per register-block shape (see fma_block), from timings on B200.
+__host__ __device__ constexpr int ffma_order(int mr, int nr) {
+  return (mr == 16 && nr == 8) ? 0 : (mr == 6 && nr == 8) ? 2 : 1;
+}
+
 struct FfmaArgs {
   ConvGeom g;
   float* out;
@@ -80,12 +85,23 @@ __device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR 
   }
 #pragma unroll
   for (int j = 0; j < NR / 2; ++j) bs[j] = make_float2(bn[j].y, bn[j].x);
+  // The order of the multiply-adds decides how often consecutive instructions share an
+  // operand register (and how they collide in the register banks); measured per block
+  // shape, 3-6 % apart.  All orders walk the column pairs in the outer loop.
+  constexpr int kOrder = ffma_order(MR, NR);
 #pragma unroll
-  for (int i = 0; i < MR / 2; ++i) {
+  for (int j = 0; j < NR / 2; ++j) {
 #pragma unroll
-    for (int j = 0; j < NR / 2; ++j) {
-      P[i][j] = __ffma2_rn(f.a[i], bn[j], P[i][j]);
-      Q[i][j] = __ffma2_rn(f.a[i], bs[j], Q[i][j]);
+    for (int ii = 0; ii < MR / 2; ++ii) {
+      // kOrder 0: filter pairs ascending; 1, 2: serpentine (back down on odd columns)
+      const int i = (kOrder != 0 && (j & 1)) ? (MR / 2 - 1 - ii) : ii;
+      if (kOrder == 2 && (j & 1)) {   // 2: swapped-pair product first on the way back
+        Q[i][j] = __ffma2_rn(f.a[i], bs[j], Q[i][j]);
+        P[i][j] = __ffma2_rn(f.a[i], bn[j], P[i][j]);
+      } else {
+        P[i][j] = __ffma2_rn(f.a[i], bn[j], P[i][j]);
+        Q[i][j] = __ffma2_rn(f.a[i], bs[j], Q[i][j]);
+      }
     }
   }
 }
