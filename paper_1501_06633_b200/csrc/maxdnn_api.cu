@@ -214,7 +214,12 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   args.atom = atom;
   args.umma_k = 32u / (uint32_t)elem_bytes;
   args.is_bf16 = bf16 ? 1u : 0u;
-  args.lbo_bytes = (uint32_t)g.kc * 128u;     // next group of 32 / 64 filters or images
+  // Staged layouts: filters [group of 32/64][kw][channel][128 B], patches
+  // [pixel][image group][channel][128 B].
+  args.lbo_a_bytes = (uint32_t)(g.kwc * g.kc) * 128u;
+  args.lbo_b_bytes = (uint32_t)g.kc * 128u;
+  args.tap_a_bytes = (uint32_t)g.kc * 128u;
+  args.tap_b_bytes = (uint32_t)(g.tile_n / (int)atom) * (uint32_t)g.kc * 128u;
   // next group of channel rows: 8 rows for the 16-byte-chunk swizzle, 4 rows for the
   // 32-byte-chunk swizzle of 4-byte operands
   args.sbo_bytes = bf16 ? 1024u : 512u;
@@ -238,7 +243,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
     const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Nc, (uint64_t)g.Sk, (uint64_t)g.Sk};
     const uint64_t str[3] = {(uint64_t)g.Sk * g.Sk * g.No * eb, (uint64_t)g.No * eb,
                              (uint64_t)g.Sk * g.No * eb};
-    const uint32_t box[4] = {atom, (uint32_t)g.kc, 1u, 1u};
+    const uint32_t box[4] = {atom, (uint32_t)g.kc, (uint32_t)g.kwc, 1u};
     st = encode_map(&mf, dt, 4, filt, dims, str, box, op_swz);
     if (st != MAXDNN_OK) return st;
   }

@@ -1,6 +1,7 @@
 #include "plan.h"
 
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 namespace maxdnn {
@@ -188,7 +189,8 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
 
   // Columns of a tile: tile_px adjacent pixels x tile_n images <= 256 (the MMA's N).
-  const int max_cols = 256;
+  int max_cols = 256;
+  if (const char* e = getenv("MAXDNN_UMMA_COLS")) { const int v = atoi(e); if (v >= 32 && v <= 256 && v % 32 == 0) max_cols = v; }
   int best_nn = atom, best_T = 1;
   double best_eff = -1.0;
   for (int nn = (d.Nb < max_cols ? d.Nb : max_cols) / atom * atom; nn >= atom; nn -= atom) {
@@ -211,10 +213,27 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   g->tile_end = g->n_tiles;
   g->tile_cols = max_cols;
 
-  // K step: kc channels of one filter tap; kc a multiple of the MMA's K
-  // (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
+  // K step.  Stride-1 layers with a small filter stage, per filter row, ONE strip of
+  // tile_px + Sk - 1 pixels that serves all Sk filter columns (each column's window
+  // is the strip shifted by one pixel), which cuts the patch traffic from L2 by up
+  // to Sk x; otherwise one step = kc channels of one tap.  kc is a multiple of the
+  // MMA's K (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
   const int umma_k = 32 / elem_bytes;
-  const int kc_max = 128 / elem_bytes;        // 32 (tf32) / 64 (bf16): 16 KB of filters per stage
+  const int cols = g->tile_px * g->tile_n;
+  int kwc = (d.stride == 1 && d.Sk > 1 && d.Sk <= 5 && force_kc >= 0) ? d.Sk : 1;
+  const int stage_budget = 48 * 1024;
+  auto stage_bytes = [&](int c) {
+    return (kwc * 128 + (kwc > 1 ? (g->tile_px + kwc - 1) * g->tile_n : cols)) * c * elem_bytes;
+  };
+  int kc_max = 128 / elem_bytes;              // 32 (tf32) / 64 (bf16) channels at most
+  while (kc_max > umma_k && stage_bytes(kc_max) > stage_budget) kc_max -= umma_k;
+  if (kwc > 1 && kc_max < 2 * umma_k) {
+    // The strip would leave room for one MMA per tap and stage only: the shorter
+    // K steps cost more than the saved traffic (measured on the 128-image layers).
+    kwc = 1;
+    kc_max = 128 / elem_bytes;
+    while (kc_max > umma_k && stage_bytes(kc_max) > stage_budget) kc_max -= umma_k;
+  }
   int kc = kc_max, best_pad = 1 << 30;
   for (int c = kc_max; c >= umma_k; c -= umma_k) {
     const int padded = ceil_div(d.Nc, c) * c;
@@ -222,24 +241,30 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   }
   if (force_kc > 0 && force_kc % umma_k == 0 && force_kc <= 256) kc = force_kc;
   int n = 0;
-  build_table(d, kc, 1, t, &n);
+  build_table(d, kc, kwc, t, &n);
   if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
-  g->kc = kc; g->kwc = 1; g->rows = kc; g->n_ksteps = n;
+  g->kc = kc; g->kwc = kwc; g->rows = kc * kwc; g->n_ksteps = n;
 
-  const int cols = g->tile_px * g->tile_n;
-  g->a_box_bytes = atom * kc * elem_bytes;              // one group of filters: kc rows x 128 B
-  g->a_stage_bytes = 128 * kc * elem_bytes;
-  if (g->tile_px == 1 || d.stride == 1) {
+  g->a_box_bytes = atom * kc * kwc * elem_bytes;        // one group of filters: kwc x kc rows x 128 B
+  g->a_stage_bytes = 128 * kc * kwc * elem_bytes;
+  const int strip = g->tile_px + kwc - 1;
+  if (kwc > 1) {
+    g->b_boxes = 1;
+    g->b_box_w = strip;
+    g->b_box_bytes = strip * g->tile_n * kc * elem_bytes;
+    g->b_stage_bytes = g->b_box_bytes;
+  } else if (g->tile_px == 1 || d.stride == 1) {
     g->b_boxes = 1;
     g->b_box_w = g->tile_px;
     g->b_box_bytes = cols * kc * elem_bytes;
+    g->b_stage_bytes = g->b_box_bytes;
   } else {
     g->b_boxes = g->tile_px;
     g->b_box_w = 1;
     g->b_box_bytes = g->tile_n * kc * elem_bytes;
+    g->b_stage_bytes = cols * kc * elem_bytes;
   }
   g->b_slot_bytes = g->b_box_bytes;
-  g->b_stage_bytes = cols * kc * elem_bytes;
   const int stage = g->a_stage_bytes + g->b_stage_bytes;
   const int fixed = 8 * 4096 + 1024 + 512;    // epilogue staging, alignment slack, barriers
   int stages = (227 * 1024 - fixed) / stage;

@@ -30,9 +30,12 @@ struct UmmaArgs {
   uint32_t idesc;       // instruction descriptor (formats, majors, M, N)
   uint32_t umma_k;      // channels per MMA (8 tf32, 16 bf16)
   uint32_t atom;        // elements per 128-byte row (32 fp32, 64 bf16)
-  uint32_t lbo_bytes;   // distance between 128-byte-wide column groups
-  uint32_t sbo_bytes;   // distance between 8-row groups along K
-  uint32_t kstep_bytes; // start-address step between consecutive MMAs of a stage
+  uint32_t lbo_a_bytes; // distance between groups of 32 / 64 filters in a staged filter tile
+  uint32_t lbo_b_bytes; // distance between groups of 32 / 64 columns in a staged patch tile
+  uint32_t sbo_bytes;   // distance between groups of channel rows along K
+  uint32_t kstep_bytes; // start-address step between consecutive MMAs over the channels of a tap
+  uint32_t tap_a_bytes; // filter tile: start-address step from one filter column (kw) to the next
+  uint32_t tap_b_bytes; // patch strip: start-address step of one pixel (the next kw's window)
   uint32_t is_bf16;
   uint32_t* status;
   KStepTable table;
@@ -182,10 +185,13 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       prefetch_tensormap(&map_in);
       const uint32_t tx_bytes = (uint32_t)(g.a_stage_bytes + g.b_boxes * g.b_box_bytes);
       const int m_atoms = kUmmaM / (int)args.atom;
-      const uint32_t a_atom_bytes = (uint32_t)g.kc * 128u;
+      const uint32_t a_atom_bytes = args.lbo_a_bytes;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+#ifdef MAXDNN_PROBE_MMA_ONLY
+      ok = false;   // no copies at all
+#endif
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
         int r = tile;
         const int ob = r % g.o_blocks; r /= g.o_blocks;
@@ -220,20 +226,27 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
+#ifndef MAXDNN_PROBE_MMA_ONLY
       if (!ok) {
         for (int s = 0; s < stages; ++s) {
           const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
           mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
         }
       }
+#endif
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loops (so that addresses and descriptors are computed
+    // in warp-uniform control flow); one elected lane issues each MMA and commit.
+    {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
+      // Descriptor halves that never change: offsets, version, swizzle mode.
+      const uint64_t desc_hi_a = make_smem_desc(0, args.lbo_a_bytes, args.sbo_bytes, BF16 ? 2u : 1u);
+      const uint64_t desc_hi_b = make_smem_desc(0, args.lbo_b_bytes, args.sbo_bytes, BF16 ? 2u : 1u);
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x, ++it) {
         const int acc = it & 1;
         const uint32_t acc_par = ((uint32_t)(it >> 1) & 1u) ^ 1u;
@@ -243,31 +256,39 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
+        uint32_t accumulate = 0;
         for (int s = 0; s < n_ksteps; ++s) {
+#ifndef MAXDNN_PROBE_MMA_ONLY
           if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
             ok = false;
             break;
           }
+#endif
           tcgen05_fence_after();
           const uint32_t a_addr = base + a_off + (uint32_t)stage * g.a_stage_bytes;
           const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
-          for (int j = 0; j < mma_per_step; ++j) {
-            const uint64_t adesc =
-                make_smem_desc(a_addr + (uint32_t)j * args.kstep_bytes, args.lbo_bytes, args.sbo_bytes,
-                               BF16 ? 2u : 1u);
-            const uint64_t bdesc =
-                make_smem_desc(b_addr + (uint32_t)j * args.kstep_bytes, args.lbo_bytes, args.sbo_bytes,
-                               BF16 ? 2u : 1u);
-            tcgen05_mma<BF16>(d_tmem, adesc, bdesc, args.idesc, (s | j) != 0 ? 1u : 0u);
+          // One staged strip of tile_px + kwc - 1 pixels serves all kwc filter columns
+          // of this filter row: the window of column kw starts kw pixels into the strip.
+          for (int kw = 0; kw < g.kwc; ++kw) {
+            uint64_t adesc = desc_hi_a | (uint64_t)(((a_addr + (uint32_t)kw * args.tap_a_bytes) & 0x3FFFFu) >> 4);
+            uint64_t bdesc = desc_hi_b | (uint64_t)(((b_addr + (uint32_t)kw * args.tap_b_bytes) & 0x3FFFFu) >> 4);
+            const uint64_t kstep = (uint64_t)(args.kstep_bytes >> 4);
+#pragma unroll 4
+            for (int j = 0; j < mma_per_step; ++j) {
+              if (elect_one()) tcgen05_mma<BF16>(d_tmem, adesc, bdesc, args.idesc, accumulate);
+              accumulate = 1;
+              adesc += kstep;   // next channels: the start address moves, nothing carries out
+              bdesc += kstep;
+            }
           }
-          tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
+          if (elect_one()) tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when done
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tcgen05_commit(accf_bar + 8u * acc);        // accumulator complete
+        if (elect_one()) tcgen05_commit(accf_bar + 8u * acc);        // accumulator complete
       }
       // Exit path: every MMA issued so far has finished before TMEM is released.
-      tcgen05_commit(done_bar);
+      if (elect_one()) tcgen05_commit(done_bar);
       mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
     }
   } else {
@@ -297,7 +318,11 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       tcgen05_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kAccCols;
+#ifdef MAXDNN_PROBE_NO_EPILOGUE
+      for (int col = n_cols; col < n_cols; col += 32) {
+#else
       for (int col = 0; col < n_cols; col += 32) {
+#endif
         const int p = col / g.tile_n;
         const int n = n0 + (col - p * g.tile_n);
         const int x = x0 + p;
@@ -321,10 +346,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         }
         fence_proxy_async_smem();
         __syncwarp();
+#ifndef MAXDNN_PROBE_NO_STORE
         if (lane == 0) {
           tma_store_4d(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0);
           bulk_commit();
         }
+#endif
         buf ^= 1;
       }
       // all TMEM reads of this accumulator are complete: hand it back
