@@ -19,7 +19,7 @@
 
 namespace maxdnn {
 
-constexpr int kUmmaThreads = 192;
+constexpr int kUmmaThreads = 224;   // producers: warps 0 and 6; MMA: warp 1; epilogue: warps 2-5
 constexpr int kUmmaM = 128;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
@@ -152,7 +152,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 1);
+      mbar_init(full_bar + 8u * s, 2);   // one arrival per producer warp
       mbar_init(empty_bar + 8u * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -178,12 +178,22 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int mma_per_step = g.kc / (int)args.umma_k;
   const int n_cols = g.tile_px * g.tile_n;   // MMA N
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    if (lane == 0) {
-      prefetch_tensormap(&map_filt);
-      prefetch_tensormap(&map_in);
-      const uint32_t tx_bytes = (uint32_t)(g.a_stage_bytes + g.b_boxes * g.b_box_bytes);
+  if (warp == 0 || warp == 6) {
+    // ----------------------------------------------------------- producers
+    // Warp 0 copies the patch boxes, warp 6 the filter boxes: issuing a bulk tensor
+    // copy costs the issuing warp a few hundred cycles, and a K step is short.
+    const bool patch_role = (warp == 0);
+    // The whole warp walks the loops, so coordinates and addresses are computed in
+    // warp-uniform control flow; one elected lane arms the barrier and issues the
+    // copies.  A K step lasts a few hundred nanoseconds, so this loop is short and
+    // does not sleep while it waits for a ring slot.
+    {
+      if (lane == 0) {
+        prefetch_tensormap(&map_filt);
+        prefetch_tensormap(&map_in);
+      }
+      const uint32_t tx_bytes =
+          patch_role ? (uint32_t)(g.b_boxes * g.b_box_bytes) : (uint32_t)g.a_stage_bytes;
       const int m_atoms = kUmmaM / (int)args.atom;
       const uint32_t a_atom_bytes = args.lbo_a_bytes;
       int stage = 0;
@@ -202,27 +212,36 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int na0 = (nch * g.tile_n) / (int)args.atom;
         const int h0 = y * g.stride - g.pad;
         const int w0 = xr * g.tile_px * g.stride - g.pad;
+        maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
-          if (!mbar_wait_backoff(empty_bar + 8u * stage, phase ^ 1u, args.status,
-                                 kDevTimeoutEmpty)) {
+          const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
+          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
             ok = false;
             break;
           }
-          const maxdnn_kstep ks = args.table.s[s];
           const uint32_t fb = full_bar + 8u * stage;
-          mbar_arrive_expect_tx(fb, tx_bytes);
-          uint32_t dst = base + a_off + (uint32_t)stage * g.a_stage_bytes;
-          for (int m = 0; m < m_atoms; ++m) {
-            tma_load_4d(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh);
-            dst += a_atom_bytes;
+          const uint32_t a_dst = base + a_off + (uint32_t)stage * g.a_stage_bytes;
+          const uint32_t b_dst = base + b_off + (uint32_t)stage * g.b_stage_bytes;
+          if (elect_one()) {
+            mbar_arrive_expect_tx(fb, tx_bytes);
+            if (patch_role) {
+              uint32_t dst = b_dst;
+              int w = w0 + ks.kw0;
+              for (int t = 0; t < g.b_boxes; ++t) {
+                tma_load_5d(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh);
+                dst += g.b_slot_bytes;
+                w += g.stride;
+              }
+            } else {
+              uint32_t dst = a_dst;
+              for (int m = 0; m < m_atoms; ++m) {
+                tma_load_4d(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh);
+                dst += a_atom_bytes;
+              }
+            }
           }
-          dst = base + b_off + (uint32_t)stage * g.b_stage_bytes;
-          int w = w0 + ks.kw0;
-          for (int t = 0; t < g.b_boxes; ++t) {
-            tma_load_5d(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh);
-            dst += g.b_slot_bytes;
-            w += g.stride;
-          }
+          __syncwarp();
+          ks = ks_next;
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -269,19 +288,35 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
           // One staged strip of tile_px + kwc - 1 pixels serves all kwc filter columns
           // of this filter row: the window of column kw starts kw pixels into the strip.
-          for (int kw = 0; kw < g.kwc; ++kw) {
-            uint64_t adesc = desc_hi_a | (uint64_t)(((a_addr + (uint32_t)kw * args.tap_a_bytes) & 0x3FFFFu) >> 4);
-            uint64_t bdesc = desc_hi_b | (uint64_t)(((b_addr + (uint32_t)kw * args.tap_b_bytes) & 0x3FFFFu) >> 4);
-            const uint64_t kstep = (uint64_t)(args.kstep_bytes >> 4);
+          const uint64_t a_base_desc = desc_hi_a | (uint64_t)((a_addr & 0x3FFFFu) >> 4);
+          const uint64_t b_base_desc = desc_hi_b | (uint64_t)((b_addr & 0x3FFFFu) >> 4);
+          const uint64_t kstep = (uint64_t)(args.kstep_bytes >> 4);
+          const uint64_t tap_a = (uint64_t)(args.tap_a_bytes >> 4);
+          const uint64_t tap_b = (uint64_t)(args.tap_b_bytes >> 4);
+          if (elect_one()) {
+            // start addresses only move inside the 14-bit address field: plain adds
+            uint32_t acc_flag = accumulate;
+            for (int kw = 0; kw < g.kwc; ++kw) {
+              uint64_t adesc = a_base_desc + (uint64_t)kw * tap_a;
+              uint64_t bdesc = b_base_desc + (uint64_t)kw * tap_b;
 #pragma unroll 4
-            for (int j = 0; j < mma_per_step; ++j) {
-              if (elect_one()) tcgen05_mma<BF16>(d_tmem, adesc, bdesc, args.idesc, accumulate);
-              accumulate = 1;
-              adesc += kstep;   // next channels: the start address moves, nothing carries out
-              bdesc += kstep;
+              for (int j = 0; j < mma_per_step; ++j) {
+#ifndef MAXDNN_PROBE_LOAD_ONLY
+                tcgen05_mma<BF16>(d_tmem, adesc, bdesc, args.idesc, acc_flag);
+#endif
+                acc_flag = 1;
+                adesc += kstep;
+                bdesc += kstep;
+              }
             }
+#ifdef MAXDNN_PROBE_LOAD_ONLY
+            mbar_arrive(empty_bar + 8u * stage);
+#else
+            tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
+#endif
           }
-          if (elect_one()) tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when done
+          accumulate = 1;
+          __syncwarp();
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
