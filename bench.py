@@ -32,8 +32,16 @@ UNIT = "TFLOP/s"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
                   "sm_max_mhz": 1965.0}
-# dram bytes per launch from the committed ncu summaries under profiles/ (None = not captured)
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the committed ncu summaries
+# under profiles/ (None = not captured).  Writes still sitting in L2 when the kernel ends
+# are not in these figures, which is why they are below the algorithmic bytes.
+NCU_TRAFFIC_BYTES = {
+    ("first11x11s4", "fp32"): int((79.32 + 94.30) * 1e6),
+    ("mid5x5", "fp32"): int((38.50 + 38.82) * 1e6),
+    ("large3x3", "fp32"): int((104.3 + 151.1) * 1e6),
+    ("large3x3", "bf16"): int((52.03 + 147.0) * 1e6),
+    ("large3x3", "tf32"): int((104.4 + 153.7) * 1e6),
+}
 
 
 def parse_args():
