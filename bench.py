@@ -50,7 +50,7 @@ def parse_args():
     p.add_argument("--steps", type=int, default=300)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER)
+    p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER + wl.TABLE1_ORDER)
     p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16"])
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -112,7 +112,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    w = wl.WORKLOADS[args.workload]
+    w = wl.ALL[args.workload]
     inp, filt = wl.make_inputs(w)
     Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
     Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
@@ -254,7 +254,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     peaks, peaks_kind = load_peaks()
-    w = wl.WORKLOADS[args.workload]
+    w = wl.ALL[args.workload]
     kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}[args.kernel]
     d = mx.ConvDesc.make(*w.dims)
     nbytes, Ho, Wo = workload_bytes(w, args.kernel)

@@ -64,6 +64,29 @@ WORKLOADS = {
 ORDER = ["tiny3x3", "first11x11s4", "mid5x5", "wide3x3", "large3x3"]
 
 
+def _table1(name, k, Wi, Nc, No, Sk, stride, pad):
+    return Workload(name, 128, Wi, Wi, Nc, No, Sk, stride, pad, 1.0, ("uniform", 0.0, 1.0),
+                    ("normal", 0.0, 0.01), BASE_SEED + 100 + 10 * k)
+
+
+# The ten layer shapes of the paper's Table 1 (minibatch 128; padding chosen so that the
+# printed output size results).  Shapes only: values follow the same synthetic recipe.
+TABLE1 = {w.name: w for w in [
+    _table1("alexnet_conv1", 0, 224, 3, 64, 11, 4, 2),      # 224x224x3  -> 55x55x64
+    _table1("alexnet_conv2", 1, 27, 64, 192, 5, 1, 2),      # 27x27x64   -> 27x27x192
+    _table1("alexnet_conv3", 2, 13, 192, 384, 3, 1, 1),     # 13x13x192  -> 13x13x384
+    _table1("alexnet_conv4", 3, 13, 384, 256, 3, 1, 1),     # 13x13x384  -> 13x13x256
+    _table1("alexnet_conv5", 4, 13, 256, 256, 3, 1, 1),     # 13x13x256  -> 13x13x256
+    _table1("overfeat_L1", 5, 231, 3, 96, 11, 4, 0),        # 231x231x3  -> 56x56x96
+    _table1("overfeat_L2", 6, 24, 96, 256, 5, 1, 0),        # 24x24x96   -> 20x20x256
+    _table1("overfeat_L3", 7, 12, 256, 512, 3, 1, 1),       # 12x12x256  -> 12x12x512
+    _table1("overfeat_L4", 8, 12, 512, 1024, 3, 1, 1),      # 12x12x512  -> 12x12x1024
+    _table1("overfeat_L5", 9, 12, 1024, 1024, 3, 1, 1),     # 12x12x1024 -> 12x12x1024
+]}
+TABLE1_ORDER = list(TABLE1)
+ALL = dict(WORKLOADS, **TABLE1)
+
+
 def _draw(rng: np.random.Generator, dist, shape) -> np.ndarray:
     kind, a, b = dist
     if kind == "uniform":

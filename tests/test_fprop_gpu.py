@@ -192,3 +192,25 @@ def test_error_codes_on_device():
                                ctypes.c_void_p(f.data_ptr()), ctypes.c_void_p(o.data_ptr()), None)
     assert st == mx.INVALID_VALUE
     torch.cuda.synchronize()
+
+
+# Table 1's ten layer shapes (minibatch 128), reduced in map size / channel count so the
+# oracle finishes in seconds but with the paper's filter sizes, strides, paddings and
+# filter counts.
+TABLE1_REDUCED = {
+    "alexnet_conv1": dict(Wi=51, Hi=43),
+    "alexnet_conv2": dict(Wi=11, Hi=9),
+    "alexnet_conv3": dict(Wi=6, Hi=5, Nc=96),
+    "alexnet_conv4": dict(Wi=6, Hi=5, Nc=96),
+    "alexnet_conv5": dict(Wi=6, Hi=5, Nc=128),
+    "overfeat_L1": dict(Wi=47, Hi=51),
+    "overfeat_L2": dict(Wi=10, Hi=9),
+    "overfeat_L3": dict(Wi=6, Hi=5, Nc=64),
+    "overfeat_L4": dict(Wi=5, Hi=4, Nc=64, No=1024),
+    "overfeat_L5": dict(Wi=4, Hi=4, Nc=72, No=1024),
+}
+
+
+@pytest.mark.parametrize("name", wl.TABLE1_ORDER)
+def test_table1_layer_shapes_fp32(name):
+    check_fp32(wl.TABLE1[name].scaled(**TABLE1_REDUCED[name]))

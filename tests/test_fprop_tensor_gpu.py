@@ -154,3 +154,21 @@ def test_unsupported_shapes_launch_nothing():
         o = torch.zeros(mx.conv_out_elems(d), device="cuda")
         assert mx.fprop_status(d, x, f, o, kind) == mx.NOT_SUPPORTED
     assert mx.launch_count() == before
+
+
+TABLE1_REDUCED = {
+    "alexnet_conv1": dict(Wi=51, Hi=43),
+    "alexnet_conv2": dict(Wi=11, Hi=9),
+    "alexnet_conv3": dict(Wi=6, Hi=5, Nc=96),
+    "alexnet_conv5": dict(Wi=6, Hi=5, Nc=128),
+    "overfeat_L1": dict(Wi=47, Hi=51),
+    "overfeat_L2": dict(Wi=10, Hi=9),
+    "overfeat_L4": dict(Wi=5, Hi=4, Nc=64, No=1024),
+}
+
+
+@pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+@pytest.mark.parametrize("name", list(TABLE1_REDUCED))
+def test_table1_layer_shapes(kernel, name):
+    """Table 1's layer shapes (reduced maps / channels) through the tensor-core path."""
+    check(kernel, wl.TABLE1[name].scaled(**TABLE1_REDUCED[name]))

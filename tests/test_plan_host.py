@@ -152,3 +152,19 @@ def test_benchmark_plans_fit_the_device():
     # the 96-filter first layer gets a 96-high tile (no padded filter rows), the
     # 13x13 layer a tile height that fills whole waves
     assert mx.conv_plan_query(mx.ConvDesc.make(*wl.WORKLOADS["first11x11s4"].dims))[0].tile_m == 96
+
+
+def test_table1_shapes_give_the_printed_output_sizes_and_have_plans():
+    """Table 1 prints input size, kernel and output size per layer; the workload list
+    must reproduce the output sizes, and every kernel kind must have a plan for them."""
+    printed = {"alexnet_conv1": (55, 64), "alexnet_conv2": (27, 192), "alexnet_conv3": (13, 384),
+               "alexnet_conv4": (13, 256), "alexnet_conv5": (13, 256), "overfeat_L1": (56, 96),
+               "overfeat_L2": (20, 256), "overfeat_L3": (12, 512), "overfeat_L4": (12, 1024),
+               "overfeat_L5": (12, 1024)}
+    for name, (size, filters) in printed.items():
+        w = wl.TABLE1[name]
+        d = mx.ConvDesc.make(*w.dims)
+        assert mx.conv_out_dims(d) == (size, size) and w.No == filters and w.Nb == 128
+        for kind in (mx.KERNEL_FP32, mx.KERNEL_TF32, mx.KERNEL_BF16):
+            info, steps = mx.conv_plan_query(d, kind, 148)
+            assert info.n_tiles > 0 and info.smem_bytes <= 227 * 1024 and len(steps) == info.n_ksteps
