@@ -283,7 +283,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
             break;
           }
 #endif
+#ifndef MAXDNN_PROBE_NO_STEP_FENCE
           tcgen05_fence_after();
+#endif
           const uint32_t a_addr = base + a_off + (uint32_t)stage * g.a_stage_bytes;
           const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
           // One staged strip of tile_px + kwc - 1 pixels serves all kwc filter columns
@@ -311,7 +313,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
             }
 #ifdef MAXDNN_PROBE_LOAD_ONLY
             mbar_arrive(empty_bar + 8u * stage);
-#else
+#elif !defined(MAXDNN_PROBE_NO_STEP_COMMIT)
             tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
 #endif
           }
