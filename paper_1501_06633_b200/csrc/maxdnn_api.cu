@@ -1,6 +1,7 @@
 // C ABI of the library (see include/maxdnn.h): descriptor checks, per-device
 // state, tensor-copy descriptor encoding and kernel launches.
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -9,6 +10,7 @@
 #include "ffma_conv.cuh"
 #include "plan.h"
 #include "umma_conv.cuh"
+#include "umma_pair_conv.cuh"
 
 namespace maxdnn {
 namespace {
@@ -21,7 +23,7 @@ struct DeviceState {
   int sm_count = 0;
   uint32_t* status = nullptr;   // one word of device memory
   bool ffma_attr[16] = {};
-  bool umma_attr[2] = {false, false};
+  bool umma_attr[4] = {false, false, false, false};
 };
 
 std::mutex g_mu;
@@ -173,6 +175,39 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
 }
 
 template <bool BF16>
+maxdnn_status launch_umma_pair(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                               const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
+  auto kern = umma_pair_conv_kernel<BF16>;
+  const int slot = BF16 ? 3 : 2;
+  if (!ds->umma_attr[slot]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->umma_attr[slot] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
+  cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, mf, mi, mo, args) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
+template <bool BF16>
 maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
                           const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
   auto kern = umma_conv_kernel<BF16>;
@@ -204,7 +239,8 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local UmmaArgs args;
-  st = plan_umma(*desc, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"), &args.g, &args.table);
+  st = plan_umma(*desc, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
+                 env_int("MAXDNN_UMMA_PAIR"), &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   const ConvGeom& g = args.g;
   const uint64_t eb = (uint64_t)elem_bytes;
@@ -229,7 +265,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   args.idesc = (1u << 4)                      // fp32 accumulator
                | (fmt << 7) | (fmt << 10)     // A and B formats
                | (1u << 15) | (1u << 16)      // both operands contiguous along M / N, not K
-               | ((n_cols >> 3) << 17) | ((uint32_t)(kUmmaM >> 4) << 24);
+               | ((n_cols >> 3) << 17) | ((uint32_t)(g.tile_m >> 4) << 24);
   const CUtensorMapDataType dt =
       bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
 
@@ -269,6 +305,9 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
                     CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
   }
+  if (g.pair)
+    return bf16 ? launch_umma_pair<true>(ds, mf, mi, mo, args, stream)
+                : launch_umma_pair<false>(ds, mf, mi, mo, args, stream);
   return bf16 ? launch_umma<true>(ds, mf, mi, mo, args, stream)
               : launch_umma<false>(ds, mf, mi, mo, args, stream);
 }
@@ -438,8 +477,8 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
     case MAXDNN_KERNEL_FP32:
       st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
       break;
-    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;
-    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, env_int("MAXDNN_UMMA_KC"), &g, &t); break;
+    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
+    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
     default: return MAXDNN_INVALID_VALUE;
   }
   if (st != MAXDNN_OK) return st;
@@ -511,6 +550,7 @@ maxdnn_status maxdnn_last_device_status(void* cuda_stream) {
     return MAXDNN_CUDA_ERROR;
   }
   if (word != 0) {
+    if (getenv("MAXDNN_DEBUG_STATUS")) fprintf(stderr, "maxdnn: device status word 0x%x\n", word);
     cudaMemset(ds->status, 0, 4);
     return MAXDNN_DEVICE_TIMEOUT;
   }

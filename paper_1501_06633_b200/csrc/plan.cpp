@@ -173,7 +173,7 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
 }
 
 maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
-                        ConvGeom* g, KStepTable* t) {
+                        int force_pair, ConvGeom* g, KStepTable* t) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -204,8 +204,17 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   g->tile_px = best_T;
   g->n_chunks = ceil_div(d.Nb, best_nn);
   g->x_runs = ceil_div(Wo, best_T);
-  g->tile_m = 128;
-  g->o_blocks = ceil_div(d.No, 128);
+  // Two-SM tiles (256 filters per pair of CTAs, each staging half of the pixels) when
+  // the filters fill them and the pixels split evenly.
+  // (Measured slower than one-SM tiles on every layer tried — the cross-CTA barrier
+  // round trips lengthen the per-step chain that already limits the kernel — so the
+  // two-SM path is built and tested but only taken on request.)
+  const bool pair = force_pair > 0;
+  if (pair && (g->tile_px < 2 || g->tile_px % 2 != 0 || sm_count < 2)) return MAXDNN_NOT_SUPPORTED;
+  g->pair = pair ? 1 : 0;
+  g->tile_m = pair ? 256 : 128;
+  g->o_blocks = ceil_div(d.No, g->tile_m);
+  const int px_cta = pair ? g->tile_px / 2 : g->tile_px;   // pixels whose patches one CTA stages
   const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
   if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_tiles = (int32_t)tiles;
@@ -219,25 +228,36 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   // to Sk x; otherwise one step = kc channels of one tap.  kc is a multiple of the
   // MMA's K (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
   const int umma_k = 32 / elem_bytes;
-  const int cols = g->tile_px * g->tile_n;
+  const int cols = px_cta * g->tile_n;                    // patch columns one CTA stages
   int kwc = (d.stride == 1 && d.Sk > 1 && d.Sk <= 5 && force_kc >= 0) ? d.Sk : 1;
-  const int stage_budget = 48 * 1024;
+  // A K step costs the issuing warps a fixed few hundred cycles, so a step should carry
+  // many MMAs.  With the strip, a stage of up to 96 KB (two stages) pays off when it holds
+  // at least 9 (bf16) / 12 (tf32) MMAs (measured on the 3x3 / 5x5 layers); otherwise one
+  // tap per step and 48 KB stages (four or more stages).
+  int stage_budget = kwc > 1 ? 96 * 1024 : 48 * 1024;
+  if (const char* e = getenv("MAXDNN_UMMA_STAGE_KB")) { const int v = atoi(e); if (v >= 16 && v <= 96) stage_budget = v * 1024; }
   auto stage_bytes = [&](int c) {
-    return (kwc * 128 + (kwc > 1 ? (g->tile_px + kwc - 1) * g->tile_n : cols)) * c * elem_bytes;
+    return (kwc * 128 + (kwc > 1 ? (px_cta + kwc - 1) * g->tile_n : cols)) * c * elem_bytes;
   };
-  int kc_max = 128 / elem_bytes;              // 32 (tf32) / 64 (bf16) channels at most
-  while (kc_max > umma_k && stage_bytes(kc_max) > stage_budget) kc_max -= umma_k;
-  if (kwc > 1 && kc_max < 2 * umma_k) {
-    // The strip would leave room for one MMA per tap and stage only: the shorter
-    // K steps cost more than the saved traffic (measured on the 128-image layers).
-    kwc = 1;
-    kc_max = 128 / elem_bytes;
+  // channels per step: at most 128 bytes' worth (32 tf32 / 64 bf16), within the stage
+  // budget, with the least zero padding of the channel count
+  auto pick_kc = [&]() {
+    int kc_max = 128 / elem_bytes;
     while (kc_max > umma_k && stage_bytes(kc_max) > stage_budget) kc_max -= umma_k;
-  }
-  int kc = kc_max, best_pad = 1 << 30;
-  for (int c = kc_max; c >= umma_k; c -= umma_k) {
-    const int padded = ceil_div(d.Nc, c) * c;
-    if (padded < best_pad) { best_pad = padded; kc = c; }
+    int best = kc_max, best_pad = 1 << 30;
+    for (int c = kc_max; c >= umma_k; c -= umma_k) {
+      const int padded = ceil_div(d.Nc, c) * c;
+      if (padded < best_pad) { best_pad = padded; best = c; }
+    }
+    return best;
+  };
+  int kc = pick_kc();
+  const int min_mmas = elem_bytes == 2 ? 9 : 12;
+  if (kwc > 1 && (kwc * (kc / umma_k) < min_mmas || stage_bytes(kc) > stage_budget) &&
+      !getenv("MAXDNN_UMMA_STAGE_KB")) {
+    kwc = 1;
+    stage_budget = 48 * 1024;
+    kc = pick_kc();
   }
   if (force_kc > 0 && force_kc % umma_k == 0 && force_kc <= 256) kc = force_kc;
   int n = 0;
@@ -247,19 +267,19 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
 
   g->a_box_bytes = atom * kc * kwc * elem_bytes;        // one group of filters: kwc x kc rows x 128 B
   g->a_stage_bytes = 128 * kc * kwc * elem_bytes;
-  const int strip = g->tile_px + kwc - 1;
+  const int strip = px_cta + kwc - 1;
   if (kwc > 1) {
     g->b_boxes = 1;
     g->b_box_w = strip;
     g->b_box_bytes = strip * g->tile_n * kc * elem_bytes;
     g->b_stage_bytes = g->b_box_bytes;
-  } else if (g->tile_px == 1 || d.stride == 1) {
+  } else if (px_cta == 1 || d.stride == 1) {
     g->b_boxes = 1;
-    g->b_box_w = g->tile_px;
+    g->b_box_w = px_cta;
     g->b_box_bytes = cols * kc * elem_bytes;
     g->b_stage_bytes = g->b_box_bytes;
   } else {
-    g->b_boxes = g->tile_px;
+    g->b_boxes = px_cta;
     g->b_box_w = 1;
     g->b_box_bytes = g->tile_n * kc * elem_bytes;
     g->b_stage_bytes = cols * kc * elem_bytes;
@@ -272,7 +292,12 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   if (stages < 2) return MAXDNN_NOT_SUPPORTED;
   g->stages = stages;
   g->smem_bytes = stages * stage + fixed;
-  g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  if (pair) {
+    const int pairs = sm_count / 2;
+    g->grid = 2 * (g->n_tiles < pairs ? g->n_tiles : pairs);
+  } else {
+    g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  }
   return MAXDNN_OK;
 }
 

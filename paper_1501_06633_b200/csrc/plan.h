@@ -28,6 +28,7 @@ struct ConvGeom {
   int32_t n_tiles;
   int32_t tile_begin, tile_end;   // tiles this launch walks: [tile_begin, tile_end)
   int32_t tile_cols;       // columns of a tile the kernel is built for (128 or 256)
+  int32_t pair;            // tensor-core kernel: 1 = tiles of 256 filters on a pair of CTAs
   int32_t a_stage_bytes;   // filter box bytes per stage
   int32_t a_box_bytes;
   int32_t fixed_pitch;     // 1: one patch box per stage, rows 128 floats apart
@@ -54,7 +55,8 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
                         ConvGeom* g, KStepTable* t);
 
 // Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
+// force_pair: 0 = choose, 1 = two-SM tiles (256 filters per CTA pair), -1 = one-SM tiles.
 maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
-                        ConvGeom* g, KStepTable* t);
+                        int force_pair, ConvGeom* g, KStepTable* t);
 
 }  // namespace maxdnn

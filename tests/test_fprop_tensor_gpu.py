@@ -172,3 +172,24 @@ TABLE1_REDUCED = {
 def test_table1_layer_shapes(kernel, name):
     """Table 1's layer shapes (reduced maps / channels) through the tensor-core path."""
     check(kernel, wl.TABLE1[name].scaled(**TABLE1_REDUCED[name]))
+
+
+@pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+@pytest.mark.parametrize("shape", [
+    (64, 14, 9, 128, 256, 3, 1, 1, 1.0),      # strip reuse, two tiles of 256 filters
+    (128, 9, 7, 96, 256, 5, 1, 2, 1.0),       # one pixel per CTA of the pair
+    (64, 13, 5, 72, 512, 3, 1, 1, 0.5),       # ragged pixel tail, channel tail
+    (128, 23, 19, 16, 256, 11, 4, 0, 1.0),    # stride 4: one box per pixel
+    (64, 12, 6, 24, 160, 3, 1, 1, 1.0),       # 160 filters: second CTA of the pair mostly idle
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_two_sm_tiles(kernel, shape, monkeypatch):
+    """The two-SM variant (256 filters per CTA pair, cta_group::2 MMAs), taken only on
+    request, against the oracle."""
+    monkeypatch.setenv("MAXDNN_UMMA_PAIR", "1")
+    Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha = shape
+    w = wl.Workload("pair", Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), 4321 + No)
+    d = mx.ConvDesc.make(*w.dims)
+    info, _ = mx.conv_plan_query(d, KIND[kernel], 148)
+    assert info.tile_m == 256 and info.grid % 2 == 0
+    check(kernel, w)
