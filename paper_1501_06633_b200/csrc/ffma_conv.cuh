@@ -36,6 +36,10 @@ struct FfmaArgs {
   ConvGeom g;
   float* out;
   uint32_t* status;
+  // Test hook for the bounded waits: if non-zero, CTA 0's producer arms the barrier of
+  // its drop_step-th K step but never issues the patch copy, so the consumers' wait
+  // runs out and the kernel reports kDevTimeoutFull instead of hanging.
+  uint32_t drop_step;
   KStepTable table;
 };
 
@@ -110,6 +114,7 @@ __device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR 
 struct FfmaProducer {
   int tile, step, stage;
   uint32_t phase;
+  uint32_t issued;
   int o0, n0, h0, w0;
 
   __device__ __forceinline__ void set_tile(const ConvGeom& g, int mt) {
@@ -126,7 +131,7 @@ struct FfmaProducer {
 
   __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
     tile = g.tile_begin + blockIdx.x;
-    step = 0; stage = 0; phase = 0;
+    step = 0; stage = 0; phase = 0; issued = 0;
     o0 = n0 = h0 = w0 = 0;
     if (tile < g.tile_end) set_tile(g, mt);
   }
@@ -149,7 +154,8 @@ struct FfmaProducer {
     tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, o0, ks.kw0, ks.kh, ks.c0);
     uint32_t dst = b_base + (uint32_t)stage * g.b_stage_bytes;
     int w = w0 + ks.kw0;
-    for (int t = 0; t < g.b_boxes; ++t) {
+    const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
+    for (int t = 0; t < g.b_boxes && !drop; ++t) {
       tma_load_4d(dst, map_in, fb, n0, w, h0 + ks.kh, ks.c0);
       dst += g.b_slot_bytes;
       w += g.stride;

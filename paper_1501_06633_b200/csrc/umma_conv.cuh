@@ -37,6 +37,7 @@ struct UmmaArgs {
   uint32_t tap_a_bytes; // filter tile: start-address step from one filter column (kw) to the next
   uint32_t tap_b_bytes; // patch strip: start-address step of one pixel (the next kw's window)
   uint32_t is_bf16;
+  uint32_t drop_step;   // test hook: CTA 0 skips the patch copy of this K step (0 = never)
   uint32_t* status;
   KStepTable table;
 };
@@ -198,10 +199,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const uint32_t a_atom_bytes = args.lbo_a_bytes;
       int stage = 0;
       uint32_t phase = 0;
+      uint32_t issued = 0;
       bool ok = true;
-#ifdef MAXDNN_PROBE_MMA_ONLY
-      ok = false;   // no copies at all
-#endif
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
         int r = tile;
         const int ob = r % g.o_blocks; r /= g.o_blocks;
@@ -227,7 +226,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
             if (patch_role) {
               uint32_t dst = b_dst;
               int w = w0 + ks.kw0;
-              for (int t = 0; t < g.b_boxes; ++t) {
+              const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
+              for (int t = 0; t < g.b_boxes && !drop; ++t) {
                 tma_load_5d(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh);
                 dst += g.b_slot_bytes;
                 w += g.stride;
@@ -245,14 +245,12 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
-#ifndef MAXDNN_PROBE_MMA_ONLY
       if (!ok) {
         for (int s = 0; s < stages; ++s) {
           const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
           mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
         }
       }
-#endif
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
@@ -277,15 +275,11 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
         uint32_t accumulate = 0;
         for (int s = 0; s < n_ksteps; ++s) {
-#ifndef MAXDNN_PROBE_MMA_ONLY
           if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
             ok = false;
             break;
           }
-#endif
-#ifndef MAXDNN_PROBE_NO_STEP_FENCE
           tcgen05_fence_after();
-#endif
           const uint32_t a_addr = base + a_off + (uint32_t)stage * g.a_stage_bytes;
           const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
           // One staged strip of tile_px + kwc - 1 pixels serves all kwc filter columns
@@ -303,19 +297,13 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
               uint64_t bdesc = b_base_desc + (uint64_t)kw * tap_b;
 #pragma unroll 4
               for (int j = 0; j < mma_per_step; ++j) {
-#ifndef MAXDNN_PROBE_LOAD_ONLY
                 tcgen05_mma<BF16>(d_tmem, adesc, bdesc, args.idesc, acc_flag);
-#endif
                 acc_flag = 1;
                 adesc += kstep;
                 bdesc += kstep;
               }
             }
-#ifdef MAXDNN_PROBE_LOAD_ONLY
-            mbar_arrive(empty_bar + 8u * stage);
-#elif !defined(MAXDNN_PROBE_NO_STEP_COMMIT)
             tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
-#endif
           }
           accumulate = 1;
           __syncwarp();
@@ -355,11 +343,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       tcgen05_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kAccCols;
-#ifdef MAXDNN_PROBE_NO_EPILOGUE
-      for (int col = n_cols; col < n_cols; col += 32) {
-#else
       for (int col = 0; col < n_cols; col += 32) {
-#endif
         const int p = col / g.tile_n;
         const int n = n0 + (col - p * g.tile_n);
         const int x = x0 + p;
@@ -383,12 +367,10 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         }
         fence_proxy_async_smem();
         __syncwarp();
-#ifndef MAXDNN_PROBE_NO_STORE
         if (lane == 0) {
           tma_store_4d(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0);
           bulk_commit();
         }
-#endif
         buf ^= 1;
       }
       // all TMEM reads of this accumulator are complete: hand it back

@@ -1,0 +1,45 @@
+"""Failure detection without a GPU fault: every wait inside the kernels has a time
+limit; a test hook makes one copy never arrive, the waiting warps give up after their
+limit, the kernel ends normally, the status word says so, and the context stays usable."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1501_06633_b200 as mx
+from paper_1501_06633_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _tensors(w, kernel):
+    inp, filt = wl.make_inputs(w)
+    if kernel == "bf16":
+        to_dev = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+        ref_in, ref_f = wl.from_bf16_bits(wl.to_bf16_bits(inp)), wl.from_bf16_bits(wl.to_bf16_bits(filt))
+    else:
+        to_dev = lambda a: torch.from_numpy(a).cuda()
+        ref_in, ref_f = inp, filt
+    return to_dev(inp), to_dev(filt), ref_in, ref_f
+
+
+@pytest.mark.parametrize("kernel,kind", [("fp32", mx.KERNEL_FP32), ("bf16", mx.KERNEL_BF16)])
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind, monkeypatch):
+    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
+    d = mx.ConvDesc.make(*w.dims)
+    d_in, d_f, ref_in, ref_f = _tensors(w, kernel)
+    out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    assert mx.last_device_status() == mx.OK
+
+    monkeypatch.setenv("MAXDNN_TEST_DROP_COPY", "3")     # CTA 0 never copies its 3rd patch box
+    assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # the launch itself succeeds
+    assert mx.last_device_status() == mx.DEVICE_TIMEOUT               # ...the kernel gave up waiting
+    assert mx.last_device_status() == mx.OK                           # reading clears the word
+
+    monkeypatch.delenv("MAXDNN_TEST_DROP_COPY")
+    assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # same context, next call
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_fprop(ref_in, ref_f, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = out.cpu().numpy().reshape(ref.shape)
+    err = float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref)))
+    assert err <= 1e-5
