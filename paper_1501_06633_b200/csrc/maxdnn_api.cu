@@ -257,7 +257,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   args.lbo_a_bytes = (uint32_t)(g.kwc * g.kc) * 128u;
   args.lbo_b_bytes = (uint32_t)g.kc * 128u;
   args.tap_a_bytes = (uint32_t)g.kc * 128u;
-  args.tap_b_bytes = (uint32_t)(g.tile_n / (int)atom) * (uint32_t)g.kc * 128u;
+  args.tap_b_bytes = (uint32_t)(g.cta_n / (int)atom) * (uint32_t)g.kc * 128u;
   // next group of channel rows: 8 rows for the 16-byte-chunk swizzle, 4 rows for the
   // 32-byte-chunk swizzle of 4-byte operands
   args.sbo_bytes = bf16 ? 1024u : 512u;
@@ -292,7 +292,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
                               (uint64_t)g.Hi};
     const uint64_t str[4] = {(uint64_t)g.Hi * g.Wi * g.Nb * eb, 128u, (uint64_t)g.Nb * eb,
                              (uint64_t)g.Wi * g.Nb * eb};
-    const uint32_t box[5] = {atom, (uint32_t)g.kc, (uint32_t)g.tile_n / atom, (uint32_t)g.b_box_w,
+    const uint32_t box[5] = {atom, (uint32_t)g.kc, (uint32_t)g.cta_n / atom, (uint32_t)g.b_box_w,
                              1u};
     st = encode_map(&mi, dt, 5, in, dims, str, box, op_swz);
     if (st != MAXDNN_OK) return st;

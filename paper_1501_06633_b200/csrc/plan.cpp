@@ -172,8 +172,8 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   return MAXDNN_OK;
 }
 
-maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
-                        int force_pair, ConvGeom* g, KStepTable* t) {
+static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
+                                  int force_kc, bool pair, ConvGeom* g, KStepTable* t) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -204,17 +204,29 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   g->tile_px = best_T;
   g->n_chunks = ceil_div(d.Nb, best_nn);
   g->x_runs = ceil_div(Wo, best_T);
-  // Two-SM tiles (256 filters per pair of CTAs, each staging half of the pixels) when
-  // the filters fill them and the pixels split evenly.
-  // (Measured slower than one-SM tiles on every layer tried — the cross-CTA barrier
-  // round trips lengthen the per-step chain that already limits the kernel — so the
-  // two-SM path is built and tested but only taken on request.)
-  const bool pair = force_pair > 0;
-  if (pair && (g->tile_px < 2 || g->tile_px % 2 != 0 || sm_count < 2)) return MAXDNN_NOT_SUPPORTED;
+  // Two-SM tiles: 256 filters per pair of CTAs.  Each CTA stages its 128 filters and
+  // HALF of the tile's patch columns, which cuts the bytes staged per SM and per FLOP -
+  // the shared-memory fill rate is what bounds the one-SM kernel.  The columns are
+  // split by image when the tile holds at least two 128-byte groups of images (the
+  // strip of a split image range is shorter than two strips of split pixels), else by
+  // pixel.
   g->pair = pair ? 1 : 0;
   g->tile_m = pair ? 256 : 128;
   g->o_blocks = ceil_div(d.No, g->tile_m);
-  const int px_cta = pair ? g->tile_px / 2 : g->tile_px;   // pixels whose patches one CTA stages
+  g->cta_px = g->tile_px;
+  g->cta_n = g->tile_n;
+  if (pair) {
+    if (sm_count < 2) return MAXDNN_NOT_SUPPORTED;
+    if (g->tile_n % (2 * atom) == 0) {
+      g->split_n = 1;
+      g->cta_n = g->tile_n / 2;
+    } else if (g->tile_px % 2 == 0) {
+      g->cta_px = g->tile_px / 2;
+    } else {
+      return MAXDNN_NOT_SUPPORTED;
+    }
+  }
+  const int px_cta = g->cta_px;
   const int64_t tiles = (int64_t)g->o_blocks * g->x_runs * Ho * g->n_chunks;
   if (tiles > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_tiles = (int32_t)tiles;
@@ -228,7 +240,7 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   // to Sk x; otherwise one step = kc channels of one tap.  kc is a multiple of the
   // MMA's K (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
   const int umma_k = 32 / elem_bytes;
-  const int cols = px_cta * g->tile_n;                    // patch columns one CTA stages
+  const int cols = px_cta * g->cta_n;                     // patch columns one CTA stages
   int kwc = (d.stride == 1 && d.Sk > 1 && d.Sk <= 5 && force_kc >= 0) ? d.Sk : 1;
   // A K step costs the issuing warps a fixed few hundred cycles, so a step should carry
   // many MMAs.  With the strip, a stage of up to 96 KB (two stages) pays off when it holds
@@ -237,7 +249,7 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   int stage_budget = kwc > 1 ? 96 * 1024 : 48 * 1024;
   if (const char* e = getenv("MAXDNN_UMMA_STAGE_KB")) { const int v = atoi(e); if (v >= 16 && v <= 96) stage_budget = v * 1024; }
   auto stage_bytes = [&](int c) {
-    return (kwc * 128 + (kwc > 1 ? (px_cta + kwc - 1) * g->tile_n : cols)) * c * elem_bytes;
+    return (kwc * 128 + (kwc > 1 ? (px_cta + kwc - 1) * g->cta_n : cols)) * c * elem_bytes;
   };
   // channels per step: at most 128 bytes' worth (32 tf32 / 64 bf16), within the stage
   // budget, with the least zero padding of the channel count
@@ -271,7 +283,7 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   if (kwc > 1) {
     g->b_boxes = 1;
     g->b_box_w = strip;
-    g->b_box_bytes = strip * g->tile_n * kc * elem_bytes;
+    g->b_box_bytes = strip * g->cta_n * kc * elem_bytes;
     g->b_stage_bytes = g->b_box_bytes;
   } else if (px_cta == 1 || d.stride == 1) {
     g->b_boxes = 1;
@@ -281,7 +293,7 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   } else {
     g->b_boxes = px_cta;
     g->b_box_w = 1;
-    g->b_box_bytes = g->tile_n * kc * elem_bytes;
+    g->b_box_bytes = g->cta_n * kc * elem_bytes;
     g->b_stage_bytes = cols * kc * elem_bytes;
   }
   g->b_slot_bytes = g->b_box_bytes;
@@ -297,6 +309,28 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
     g->grid = 2 * (g->n_tiles < pairs ? g->n_tiles : pairs);
   } else {
     g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  }
+  return MAXDNN_OK;
+}
+
+maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
+                        int force_pair, ConvGeom* g, KStepTable* t) {
+  if (force_pair != 0) return plan_umma_as(d, elem_bytes, sm_count, force_kc, force_pair > 0, g, t);
+  const maxdnn_status st = plan_umma_as(d, elem_bytes, sm_count, force_kc, false, g, t);
+  if (st != MAXDNN_OK) return st;
+  // Two-SM tiles when they pay: a pair's tile (twice the work of a one-SM tile on twice
+  // the SMs) takes about 0.9 of the one-SM tile's time where the steps are long enough
+  // (at least four MMAs each), so compare the waves of tiles each plan needs.
+  static thread_local ConvGeom g2;
+  static thread_local KStepTable t2;
+  if (plan_umma_as(d, elem_bytes, sm_count, force_kc, true, &g2, &t2) != MAXDNN_OK) return st;
+  const int mmas_per_step = g2.kwc * (g2.kc / (32 / elem_bytes));
+  const double one = (double)ceil_div(g->n_tiles, sm_count);
+  const double two = 0.9 * (double)ceil_div(g2.n_tiles, sm_count / 2);
+  const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);   // in every tile
+  if (mmas_per_step >= 4 && peer_has_filters && two < one) {
+    *g = g2;
+    *t = t2;
   }
   return MAXDNN_OK;
 }

@@ -29,6 +29,8 @@ struct ConvGeom {
   int32_t tile_begin, tile_end;   // tiles this launch walks: [tile_begin, tile_end)
   int32_t tile_cols;       // columns of a tile the kernel is built for (128 or 256)
   int32_t pair;            // tensor-core kernel: 1 = tiles of 256 filters on a pair of CTAs
+  int32_t split_n;         // pair: 1 = the CTAs split the tile's images, 0 = its pixels
+  int32_t cta_px, cta_n;   // pixels x images whose patches ONE CTA stages (= tile_px, tile_n if not pair)
   int32_t a_stage_bytes;   // filter box bytes per stage
   int32_t a_box_bytes;
   int32_t fixed_pitch;     // 1: one patch box per stage, rows 128 floats apart

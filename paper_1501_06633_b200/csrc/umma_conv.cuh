@@ -113,6 +113,43 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, uint32_t src,
       "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
+// L2 eviction policies for bulk copies.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_store_4d_hint(const CUtensorMap* m, uint32_t src, int c0, int c1,
+                                                  int c2, int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group.L2::cache_hint "
+      "[%0, {%2, %3, %4, %5}], [%1], %6;" ::"l"(reinterpret_cast<uint64_t>(m)),
+      "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* m, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap* m, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3, int c4,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4),
+      "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void bulk_commit() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
@@ -197,6 +234,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           patch_role ? (uint32_t)(g.b_boxes * g.b_box_bytes) : (uint32_t)g.a_stage_bytes;
       const int m_atoms = kUmmaM / (int)args.atom;
       const uint32_t a_atom_bytes = args.lbo_a_bytes;
+      const uint64_t pol_last = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase = 0;
       uint32_t issued = 0;
@@ -228,14 +266,14 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
               int w = w0 + ks.kw0;
               const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
               for (int t = 0; t < g.b_boxes && !drop; ++t) {
-                tma_load_5d(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh);
+                tma_load_5d_hint(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
                 w += g.stride;
               }
             } else {
               uint32_t dst = a_dst;
               for (int m = 0; m < m_atoms; ++m) {
-                tma_load_4d(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh);
+                tma_load_4d_hint(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh, pol_last);
                 dst += a_atom_bytes;
               }
             }
@@ -323,6 +361,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     const uint32_t stg0 = base + st_off + (uint32_t)(2 * ew) * kStageTileBytes;
     uint8_t* stg0_ptr = base_ptr + st_off + (size_t)(2 * ew) * kStageTileBytes;
     const float alpha = g.alpha;
+    const uint64_t pol_first = l2_policy_evict_first();
     bool ok = true;
     int it = 0;
     int buf = 0;
@@ -368,7 +407,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_4d(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0);
+          tma_store_4d_hint(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0, pol_first);
           bulk_commit();
         }
         buf ^= 1;

@@ -2,16 +2,19 @@
 //
 // A cluster of two CTAs (one SM each) works on one tile of 256 filters x
 // (tile_px pixels x tile_n images) <= 256 columns.  CTA r of the pair stages filters
-// [128 r, 128 r + 128) of the tile and HALF of the patch columns (pixels
-// [r tile_px / 2, (r + 1) tile_px / 2)); the leader CTA (rank 0) issues one MMA of
-// M = 256 for both, which reads each half of the patch operand from the shared memory
-// of the CTA that holds it.  Per SM and per FLOP this halves the patch bytes staged and
-// the number of MMA instructions and K steps — the fixed per-step cost is what limits
-// the one-SM kernel.  Each CTA keeps its 128 filter rows of the accumulators in its own
+// [128 r, 128 r + 128) of the tile and HALF of the patch columns (half of the tile's
+// images when it holds two 128-byte groups of them, else half of its pixels); the
+// leader CTA (rank 0) issues one MMA of M = 256 for both, which reads each half of the
+// patch operand from the shared memory of the CTA that holds it.  Per SM and per FLOP
+// this halves the patch bytes staged and read by the MMAs, and the number of MMA
+// instructions and K steps — the shared-memory fill rate (about 64 bytes per clock and
+// SM) is what bounds the one-SM kernel.  Each CTA keeps its 128 filter rows of the accumulators in its own
 // TMEM and runs its own epilogue.
 //
 // Synchronisation across the pair uses mbarriers only: both CTAs' copies complete on the
-// LEADER's "full" barrier (no multicast copy is used anywhere); the leader's commits
+// LEADER's "full" barrier (no multicast copy is used anywhere), on which only the
+// leader's producers arrive, expecting the bytes of both CTAs — an arrival on the peer's
+// barrier per step costs about a microsecond and serialises the ring; the leader's commits
 // arrive on the "empty" / "accumulator complete" barriers of both CTAs; the epilogue
 // warps of both CTAs arrive on the leader's "accumulator drained" barrier.  Every wait
 // has the same iteration limit and status word as in the one-SM kernel.
@@ -65,19 +68,21 @@ __device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar, uint16_t mask 
 // Tiled bulk tensor loads whose completion barrier may live in the peer CTA of the pair
 // (the destination is always this CTA's shared memory; nothing is multicast).
 __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar,
-                                                 int c0, int c1, int c2, int c3) {
+                                                 int c0, int c1, int c2, int c3, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      ".L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar,
-                                                 int c0, int c1, int c2, int c3, int c4) {
+                                                 int c0, int c1, int c2, int c3, int c4,
+                                                 uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      ".L2::cache_hint [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4),
+      "l"(policy)
       : "memory");
 }
 
@@ -134,7 +139,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 4);   // two producer warps in each of the two CTAs
+      mbar_init(full_bar + 8u * s, 2);   // the leader's two producer warps (they expect both CTAs' bytes)
       mbar_init(empty_bar + 8u * s, 1);  // the leader's commit
     }
     for (int a = 0; a < 2; ++a) {
@@ -162,7 +167,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int n_ksteps = g.n_ksteps;
   const int mma_per_step = g.kc / (int)args.umma_k;
   const int n_cols = g.tile_px * g.tile_n;   // MMA N (both halves)
-  const int half_px = g.tile_px >> 1;        // pixels whose patches this CTA stages
+  const int half_cols = n_cols >> 1;         // columns whose patches each CTA stages
   const uint32_t leader_full = map_to_cta(full_bar, 0);
   const uint32_t leader_acce = map_to_cta(acce_bar, 0);
 
@@ -174,12 +179,18 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         prefetch_tensormap(&map_filt);
         prefetch_tensormap(&map_in);
       }
+      // Only the leader arrives on its "full" barrier, expecting the bytes of BOTH CTAs'
+      // copies of its kind; the peer's copies merely complete on that barrier.  A copy of
+      // the peer that lands before the leader's arrival leaves the byte count negative
+      // for a moment, which a phase tolerates: it cannot end before the arrival.
       const uint32_t tx_bytes =
-          patch_role ? (uint32_t)(g.b_boxes * g.b_box_bytes) : (uint32_t)g.a_stage_bytes;
+          2u * (patch_role ? (uint32_t)(g.b_boxes * g.b_box_bytes) : (uint32_t)g.a_stage_bytes);
       const int m_atoms = kUmmaM / (int)args.atom;
       const uint32_t a_atom_bytes = args.lbo_a_bytes;
+      const uint64_t pol_last = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase = 0;
+      uint32_t issued = 0;
       bool ok = true;
       for (int tile = pair; tile < g.n_tiles && ok; tile += n_pairs) {
         int r = tile;
@@ -188,9 +199,10 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int xr = r % g.x_runs;
         const int y = r / g.x_runs;
         const int o0 = ob * 2 * kUmmaM + (int)rank * kUmmaM;          // this CTA's 128 filters
-        const int na0 = (nch * g.tile_n) / (int)args.atom;
+        // this CTA's half of the tile's columns: half of the images or half of the pixels
+        const int na0 = (nch * g.tile_n + (g.split_n ? (int)rank * g.cta_n : 0)) / (int)args.atom;
         const int h0 = y * g.stride - g.pad;
-        const int w0 = (xr * g.tile_px + (int)rank * half_px) * g.stride - g.pad;   // its pixels
+        const int w0 = (xr * g.tile_px + (g.split_n ? 0 : (int)rank * g.cta_px)) * g.stride - g.pad;
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
@@ -202,19 +214,21 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           const uint32_t a_dst = base + a_off + (uint32_t)stage * g.a_stage_bytes;
           const uint32_t b_dst = base + b_off + (uint32_t)stage * g.b_stage_bytes;
           if (elect_one()) {
-            mbar_arrive_expect_tx_cluster(fb, tx_bytes);
+            if (rank == 0) mbar_arrive_expect_tx(full_bar + 8u * stage, tx_bytes);
             if (patch_role) {
               uint32_t dst = b_dst;
               int w = w0 + ks.kw0;
-              for (int t = 0; t < g.b_boxes; ++t) {
-                tma_load_5d_pair(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh);
+              const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
+              for (int t = 0; t < g.b_boxes && !drop; ++t) {
+                tma_load_5d_pair(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
                 w += g.stride;
               }
             } else {
               uint32_t dst = a_dst;
               for (int m = 0; m < m_atoms; ++m) {
-                tma_load_4d_pair(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh);
+                tma_load_4d_pair(dst, &map_filt, fb, o0 + m * (int)args.atom, ks.c0, ks.kw0, ks.kh,
+                                 pol_last);
                 dst += a_atom_bytes;
               }
             }
@@ -296,6 +310,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     const uint32_t stg0 = base + st_off + (uint32_t)(2 * ew) * kStageTileBytes;
     uint8_t* stg0_ptr = base_ptr + st_off + (size_t)(2 * ew) * kStageTileBytes;
     const float alpha = g.alpha;
+    const uint64_t pol_first = l2_policy_evict_first();
     bool ok = true;
     int it = 0;
     int buf = 0;
@@ -317,9 +332,12 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       tcgen05_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kAccCols;
       for (int col = 0; col < n_cols; col += 32) {
-        const int p = col / g.tile_n;
-        const int n = n0 + (col - p * g.tile_n);
-        const int x = x0 + p;
+        // columns [0, half) were staged by the leader, [half, 2 half) by its peer
+        const int hr = col >= half_cols ? 1 : 0;
+        const int cl = col - hr * half_cols;
+        const int pl = cl / g.cta_n;
+        const int n = n0 + (g.split_n ? hr * g.cta_n : 0) + (cl - pl * g.cta_n);
+        const int x = x0 + (g.split_n ? 0 : hr * g.cta_px) + pl;
         const bool live = (x < g.Wo) && (n < g.Nb) && (o0 < g.No);   // warp-uniform
         if (!live) continue;
         uint32_t v[32];
@@ -340,7 +358,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_4d(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0);
+          tma_store_4d_hint(&map_out, stg0 + (uint32_t)buf * kStageTileBytes, n, x, y, o0, pol_first);
           bulk_commit();
         }
         buf ^= 1;

@@ -23,10 +23,14 @@ def _tensors(w, kernel):
     return to_dev(inp), to_dev(filt), ref_in, ref_f
 
 
-@pytest.mark.parametrize("kernel,kind", [("fp32", mx.KERNEL_FP32), ("bf16", mx.KERNEL_BF16)])
-def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind, monkeypatch):
-    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
+@pytest.mark.parametrize("kernel,kind,No", [("fp32", mx.KERNEL_FP32, 128), ("bf16", mx.KERNEL_BF16, 128),
+                                            ("bf16", mx.KERNEL_BF16, 256)],
+                         ids=["fp32", "bf16-one-sm", "bf16-two-sm"])
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind, No, monkeypatch):
+    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=No)
     d = mx.ConvDesc.make(*w.dims)
+    if kernel != "fp32":
+        assert mx.conv_plan_query(d, kind, 148)[0].tile_m == (256 if No == 256 else 128)
     d_in, d_f, ref_in, ref_f = _tensors(w, kernel)
     out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
     assert mx.last_device_status() == mx.OK
