@@ -39,8 +39,9 @@ NCU_TRAFFIC_BYTES = {
     ("first11x11s4", "fp32"): int((79.32 + 94.30) * 1e6),
     ("mid5x5", "fp32"): int((38.50 + 38.82) * 1e6),
     ("large3x3", "fp32"): int((104.3 + 151.1) * 1e6),
-    ("large3x3", "bf16"): int((52.03 + 147.0) * 1e6),
-    ("large3x3", "tf32"): int((104.4 + 153.7) * 1e6),
+    ("large3x3", "bf16"): int((52.02 + 145.9) * 1e6),
+    ("large3x3", "tf32"): int((104.1 + 149.0) * 1e6),
+    ("mid5x5", "bf16"): int((19.17 + 37.48) * 1e6),
 }
 
 
