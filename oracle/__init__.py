@@ -1,12 +1,15 @@
-"""CPU oracle for FPROP direct convolution — TEST INFRASTRUCTURE ONLY.
+"""CPU oracle for the direct convolution (FPROP and its two adjoints) — TEST INFRASTRUCTURE ONLY.
 
 A plain fp64-accumulating restatement of the paper's definition (Section 2) in
-C (``conv_oracle.c``), loaded through ctypes.  Only the tests, the smoke check
+C (``conv_oracle.c``) and of its gradients with respect to maps and filters
+(``conv_bprop_oracle.c``), loaded through ctypes.  Only the tests, the smoke check
 and the benchmark's CPU-baseline / reference legs may import this package; the
 product path never does, and this package imports nothing from the product.
 
 Pinned by ``tests/test_oracle_pins.py`` (hand-worked examples, brute-force
-loops, an im2col formulation, library convolution, closed forms, invariants).
+loops, an im2col formulation, library convolution, closed forms, invariants)
+and ``tests/test_oracle_bprop_pins.py`` (adjoint identities against the pinned
+FPROP, finite differences, brute-force loops, library autograd, closed forms).
 """
 from __future__ import annotations
 
@@ -19,6 +22,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "conv_oracle.c")
+_SRCS = [_SRC, os.path.join(_HERE, "conv_bprop_oracle.c")]
 _LIB = os.path.join(_HERE, "liboracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -35,12 +39,13 @@ class ConvDesc(ctypes.Structure):
 
 
 def build(force: bool = False) -> str:
-    """Compile ``conv_oracle.c`` into ``liboracle.so`` beside it (gcc, OpenMP)."""
+    """Compile the oracle's C files into ``liboracle.so`` beside them (gcc, OpenMP)."""
     with _lock:
-        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        stale = (not os.path.exists(_LIB)) or any(os.path.getmtime(_LIB) < os.path.getmtime(p)
+                                                  for p in _SRCS)
         if force or stale:
             tmp = _LIB + ".tmp.%d" % os.getpid()
-            cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC]
+            cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp] + _SRCS
             subprocess.run(cmd, check=True)
             os.replace(tmp, _LIB)
     return _LIB
@@ -67,6 +72,16 @@ def _load():
                                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                 ctypes.c_int32, P(ctypes.c_double)]
         lib.oracle_num_threads.restype = ctypes.c_int
+        for name in ("oracle_conv_bprop_data", "oracle_conv_bprop_filter"):
+            fn = getattr(lib, name)
+            fn.restype = ctypes.c_int
+            fn.argtypes = [P(ConvDesc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                           ctypes.c_int32]
+        for name in ("oracle_conv_bprop_data_point", "oracle_conv_bprop_filter_point"):
+            fn = getattr(lib, name)
+            fn.restype = ctypes.c_double
+            fn.argtypes = [P(ConvDesc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                           ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, P(ctypes.c_double)]
         _lib = lib
     return _lib
 
@@ -131,6 +146,74 @@ def conv_fprop_point(inp, filt, o, y, x, n, *, stride=1, pad=0, alpha=1.0):
     a = ctypes.c_double()
     v = _load().oracle_conv_fprop_point(ctypes.byref(d), inp.ctypes.data, filt.ctypes.data,
                                         int(o), int(y), int(x), int(n), ctypes.byref(a))
+    return float(v), float(a.value)
+
+
+def conv_bprop_data(dout, filt, in_hw, *, stride=1, pad=0, alpha=1.0, nthreads=0):
+    """din[Nc,Hi,Wi,Nb] from dout[No,Ho,Wo,Nb] and filt[Nc,Sk,Sk,No]; ``in_hw`` = (Hi, Wi).
+
+    The adjoint of FPROP with respect to the maps, alpha included.
+    """
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    filt = np.ascontiguousarray(filt, dtype=np.float32)
+    No, Ho, Wo, Nb = dout.shape
+    Nc, Sk, Sk2, No2 = filt.shape
+    Hi, Wi = in_hw
+    if No2 != No or Sk2 != Sk or out_dims(Nb, Wi, Hi, Nc, No, Sk, stride, pad) != (Ho, Wo):
+        raise ValueError("dout / filter bank / map size do not belong to one convolution")
+    d = _desc(Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha)
+    din = np.zeros((Nc, Hi, Wi, Nb), dtype=np.float32)
+    rc = _load().oracle_conv_bprop_data(ctypes.byref(d), dout.ctypes.data, filt.ctypes.data,
+                                        din.ctypes.data, int(nthreads))
+    if rc:
+        raise RuntimeError("oracle_conv_bprop_data failed (%d)" % rc)
+    return din
+
+
+def conv_bprop_data_point(dout, filt, in_hw, c, h, w, n, *, stride=1, pad=0, alpha=1.0):
+    """(value, abs_sum) of one element of din in fp64."""
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    filt = np.ascontiguousarray(filt, dtype=np.float32)
+    No, Ho, Wo, Nb = dout.shape
+    Nc, Sk, _, _ = filt.shape
+    d = _desc(Nb, in_hw[1], in_hw[0], Nc, No, Sk, stride, pad, alpha)
+    a = ctypes.c_double()
+    v = _load().oracle_conv_bprop_data_point(ctypes.byref(d), dout.ctypes.data, filt.ctypes.data,
+                                             int(c), int(h), int(w), int(n), ctypes.byref(a))
+    return float(v), float(a.value)
+
+
+def conv_bprop_filter(inp, dout, Sk, *, stride=1, pad=0, alpha=1.0, nthreads=0):
+    """dfilt[Nc,Sk,Sk,No] from in[Nc,Hi,Wi,Nb] and dout[No,Ho,Wo,Nb].
+
+    The adjoint of FPROP with respect to the filters, alpha included.
+    """
+    inp = np.ascontiguousarray(inp, dtype=np.float32)
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    Nc, Hi, Wi, Nb = inp.shape
+    No, Ho, Wo, Nb2 = dout.shape
+    if Nb2 != Nb or out_dims(Nb, Wi, Hi, Nc, No, Sk, stride, pad) != (Ho, Wo):
+        raise ValueError("maps / dout do not belong to one convolution")
+    d = _desc(Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha)
+    dfilt = np.zeros((Nc, Sk, Sk, No), dtype=np.float32)
+    rc = _load().oracle_conv_bprop_filter(ctypes.byref(d), inp.ctypes.data, dout.ctypes.data,
+                                          dfilt.ctypes.data, int(nthreads))
+    if rc:
+        raise RuntimeError("oracle_conv_bprop_filter failed (%d)" % rc)
+    return dfilt
+
+
+def conv_bprop_filter_point(inp, dout, Sk, c, kh, kw, o, *, stride=1, pad=0, alpha=1.0):
+    """(value, abs_sum) of one element of dfilt in fp64."""
+    inp = np.ascontiguousarray(inp, dtype=np.float32)
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    Nc, Hi, Wi, Nb = inp.shape
+    No = dout.shape[0]
+    d = _desc(Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha)
+    a = ctypes.c_double()
+    v = _load().oracle_conv_bprop_filter_point(ctypes.byref(d), inp.ctypes.data,
+                                               dout.ctypes.data, int(c), int(kh), int(kw),
+                                               int(o), ctypes.byref(a))
     return float(v), float(a.value)
 
 
