@@ -198,6 +198,47 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
 maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const float* in,
                                         const float* filt, float* out, void* cuda_stream);
 
+/*
+ * Backward propagation.  The paper builds FPROP only and names BPROP (Abstract,
+ * Section 6) as the operation its techniques should carry over to, without
+ * defining it; these entry points compute the two exact adjoints of the
+ * operation above, alpha included, with dout laid out like out, din like in and
+ * dfilt like filt:
+ *
+ *   din  [c,h,w,n]   = alpha * sum over (o,y,x,kh,kw) with y*stride-pad+kh = h and
+ *                      x*stride-pad+kw = w of filt[c,kh,kw,o] * dout[o,y,x,n]
+ *   dfilt[c,kh,kw,o] = alpha * sum_{y,x,n} in0[c, y*stride-pad+kh, x*stride-pad+kw, n]
+ *                                          * dout[o,y,x,n]
+ *
+ * Both need caller-owned device scratch (`workspace`, 16-byte aligned, at
+ * least the size the matching *_workspace call reports; may be NULL when that
+ * size is 0); the library allocates nothing.  Results are overwritten in full.
+ *
+ * maxdnn_conv_bprop_data: the gradient with respect to the maps as an FPROP of
+ * dout with the filter bank transposed (channels <-> filters) and flipped in
+ * both axes (written into the workspace by a small kernel on the same stream)
+ * and padding Sk-1-pad, on the kernel `kind` names (fp32; tf32; bf16: dout and
+ * filt are bfloat16, din fp32).  NOT_SUPPORTED: stride != 1, pad > Sk-1, or
+ * what the matching fprop entry point refuses for the transposed problem
+ * (its filter count is Nc).
+ *
+ * maxdnn_conv_bprop_filter: the gradient with respect to the filters in exact
+ * fp32, as the GEMM dfilt[k][o] = sum_r patch[k][r] * dout[o][r] with the
+ * reduction r over output pixels and images, split over CTAs whose partial
+ * sums (in the workspace) are added in a fixed order, so the result does not
+ * depend on scheduling.  NOT_SUPPORTED: Nb or No not a multiple of 4, Sk
+ * larger than the map, the limits of maxdnn_conv_fprop.
+ */
+maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
+                                               maxdnn_kernel_kind kind, size_t* bytes);
+maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     const void* dout, const void* filt, float* din,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
+maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, const float* in,
+                                       const float* dout, float* dfilt, void* workspace,
+                                       size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reads and clears the current device's
  * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside a
  * kernel ran out; its output is not valid) or MAXDNN_CUDA_ERROR. */

@@ -17,6 +17,8 @@ __all__ = [
     "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
     "last_device_status",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
+    "conv_bprop_data_workspace", "conv_bprop_data", "bprop_data_status",
+    "conv_bprop_filter_workspace", "conv_bprop_filter", "bprop_filter_status",
 ]
 
 OK, INVALID_VALUE, NOT_SUPPORTED, CUDA_ERROR, DEVICE_TIMEOUT = 0, 1, 2, 3, 4
@@ -27,7 +29,8 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv_filt_elems", "maxdnn_conv_out_elems", "maxdnn_conv_plan_query",
     "maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16",
     "maxdnn_conv_fprop_host", "maxdnn_conv_fprop_noalloc", "maxdnn_last_device_status",
-    "maxdnn_launch_count",
+    "maxdnn_launch_count", "maxdnn_conv_bprop_data_workspace", "maxdnn_conv_bprop_data",
+    "maxdnn_conv_bprop_filter_workspace", "maxdnn_conv_bprop_filter",
 ]
 
 
@@ -99,6 +102,15 @@ def load_library():
         getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_host.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.maxdnn_conv_bprop_data_workspace.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_data_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
+    lib.maxdnn_conv_bprop_data.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_data.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp,
+                                           ctypes.c_size_t, vp]
+    lib.maxdnn_conv_bprop_filter_workspace.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_filter_workspace.argtypes = [P(ConvDesc), P(ctypes.c_size_t)]
+    lib.maxdnn_conv_bprop_filter.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_filter.argtypes = [P(ConvDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.maxdnn_last_device_status.restype = ctypes.c_int
     lib.maxdnn_last_device_status.argtypes = [vp]
     lib.maxdnn_launch_count.restype = ctypes.c_uint64
@@ -226,6 +238,72 @@ def conv_fprop_host(desc: ConvDesc, kind: int, h_in, h_filt, h_out, d_in, d_filt
         ctypes.byref(desc), int(kind), ctypes.c_void_p(h_in.data_ptr()),
         ctypes.c_void_p(h_filt.data_ptr()), ctypes.c_void_p(h_out.data_ptr()), pin, pf, po,
         _stream_ptr(stream)), "maxdnn_conv_fprop_host")
+
+
+def _workspace_ptr(workspace, need):
+    import torch
+    if workspace is None:
+        if need:
+            raise ValueError("this call needs %d bytes of device workspace" % need)
+        return ctypes.c_void_p(0), 0
+    if not (isinstance(workspace, torch.Tensor) and workspace.is_cuda and workspace.is_contiguous()):
+        raise TypeError("workspace must be a contiguous CUDA tensor")
+    return ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def conv_bprop_data_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:
+    """Bytes of device scratch maxdnn_conv_bprop_data needs (the transformed filter bank)."""
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv_bprop_data_workspace(ctypes.byref(desc), int(kind),
+                                                               ctypes.byref(n))),
+           "maxdnn_conv_bprop_data_workspace")
+    return int(n.value)
+
+
+def bprop_data_status(desc: ConvDesc, dout, filt, din, workspace, kind: int = KERNEL_FP32,
+                      stream=None) -> int:
+    """Enqueue maxdnn_conv_bprop_data on torch tensors; returns the raw status code."""
+    lib = load_library()
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pg = _dev_ptr(dout, in_types, conv_out_elems(desc), "dout")
+    pf = _dev_ptr(filt, in_types, conv_filt_elems(desc), "filt")
+    pd = _dev_ptr(din, ("float32",), conv_in_elems(desc), "din")
+    pw, nbytes = _workspace_ptr(workspace, 1)
+    return int(lib.maxdnn_conv_bprop_data(ctypes.byref(desc), int(kind), pg, pf, pd, pw, nbytes,
+                                          _stream_ptr(stream)))
+
+
+def conv_bprop_data(desc: ConvDesc, dout, filt, din, workspace, kind: int = KERNEL_FP32,
+                    stream=None) -> None:
+    """maxdnn_conv_bprop_data: gradient with respect to the maps (asynchronous)."""
+    _check(bprop_data_status(desc, dout, filt, din, workspace, kind, stream),
+           "maxdnn_conv_bprop_data")
+
+
+def conv_bprop_filter_workspace(desc: ConvDesc) -> int:
+    """Bytes of device scratch maxdnn_conv_bprop_filter needs (partial sums; may be 0)."""
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv_bprop_filter_workspace(ctypes.byref(desc),
+                                                                 ctypes.byref(n))),
+           "maxdnn_conv_bprop_filter_workspace")
+    return int(n.value)
+
+
+def bprop_filter_status(desc: ConvDesc, inp, dout, dfilt, workspace, stream=None) -> int:
+    """Enqueue maxdnn_conv_bprop_filter on torch tensors; returns the raw status code."""
+    lib = load_library()
+    pi = _dev_ptr(inp, ("float32",), conv_in_elems(desc), "in")
+    pg = _dev_ptr(dout, ("float32",), conv_out_elems(desc), "dout")
+    pd = _dev_ptr(dfilt, ("float32",), conv_filt_elems(desc), "dfilt")
+    pw, nbytes = _workspace_ptr(workspace, 0)
+    return int(lib.maxdnn_conv_bprop_filter(ctypes.byref(desc), pi, pg, pd, pw, nbytes,
+                                            _stream_ptr(stream)))
+
+
+def conv_bprop_filter(desc: ConvDesc, inp, dout, dfilt, workspace, stream=None) -> None:
+    """maxdnn_conv_bprop_filter: gradient with respect to the filters, exact fp32."""
+    _check(bprop_filter_status(desc, inp, dout, dfilt, workspace, stream),
+           "maxdnn_conv_bprop_filter")
 
 
 def last_device_status(stream=None) -> int:

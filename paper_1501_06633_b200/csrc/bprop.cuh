@@ -1,0 +1,269 @@
+// Backward-propagation kernels (the adjoints of the operation of Section 2; the paper
+// names BPROP in its Abstract and Section 6 as where its techniques should carry over).
+//
+//  - flip_transpose_kernel: filt[c][kh][kw][o] -> ft[o][Sk-1-kh][Sk-1-kw][c], the filter
+//    bank with which the gradient with respect to the maps is an FPROP of the output
+//    gradient (stride 1).
+//  - wgrad_kernel: gradient with respect to the filters in exact fp32.  The same
+//    technique as the forward kernel — bulk tensor copies into a ring of shared-memory
+//    stages, a register-blocked multiply-accumulate inner loop of packed FFMA2 — with
+//    the reduction running over output pixels and images:
+//        dfilt[k][o] = alpha * sum_r patch[k][r] * dout[o][r],  r = (y, x, n).
+//    Both operands arrive with r contiguous (32 images = one 128-byte row per gradient
+//    row / filter), so a thread reads 16 bytes = 4 values of r from each of its 8 + 8
+//    rows and the two halves of a packed multiply-add accumulate even and odd r, added
+//    at the end.
+//  - wgrad_reduce_kernel: adds the partial sums of the reduction splits in a fixed order.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "plan.h"
+#include "ptx_util.cuh"
+
+namespace maxdnn {
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int Sk, int No) {
+  __shared__ T tile[32][33];
+  const int taps = Sk * Sk;
+  const int tap = blockIdx.z;              // kh * Sk + kw
+  const int tap_t = taps - 1 - tap;        // (Sk-1-kh) * Sk + (Sk-1-kw)
+  const int o0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int c = c0 + i, o = o0 + threadIdx.x;
+    if (c < Nc && o < No) tile[i][threadIdx.x] = filt[((size_t)c * taps + tap) * No + o];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int o = o0 + i, c = c0 + threadIdx.x;
+    if (c < Nc && o < No) ft[((size_t)o * taps + tap_t) * Nc + c] = tile[threadIdx.x][i];
+  }
+}
+
+constexpr int kWgThreads = 256;               // 8 warps: 16 x 16 threads, 8 x 8 results each
+constexpr uint32_t kWgOperandBytes = 128 * 128;   // 128 rows x 32 floats
+
+struct WgradArgs {
+  WgradGeom g;
+  float* dfilt;        // result when g.splits == 1
+  float* partial;      // [splits][Nc Sk^2][No] otherwise
+  uint32_t* status;
+};
+
+// Which (tile, split, reduction step) comes next; the copy-issuing lane and the
+// arithmetic warps walk the same sequence.
+struct WgradCursor {
+  int item;            // index over (tile, split); >= n_items: done
+  int r, r_end;        // reduction steps of this item: [r, r_end)
+  int y, x, nc;        // r = (y * Wo + x) * n_chunks + nc
+  int ob, cb, khb, split;
+
+  __device__ __forceinline__ void start(const WgradGeom& g, int it) {
+    item = it;
+    if (it >= g.n_items) return;
+    int t = it;
+    split = t % g.splits; t /= g.splits;
+    ob = t % g.o_blocks; t /= g.o_blocks;
+    cb = t % g.c_blocks;
+    khb = t / g.c_blocks;
+    r = split * g.steps_per_split;
+    r_end = r + g.steps_per_split < g.r_steps ? r + g.steps_per_split : g.r_steps;
+    nc = r % g.n_chunks;
+    const int px = r / g.n_chunks;
+    x = px % g.Wo;
+    y = px / g.Wo;
+  }
+  __device__ __forceinline__ bool done(const WgradGeom& g) const { return item >= g.n_items; }
+  // Next reduction step; moves to this CTA's next item when the current one is exhausted.
+  __device__ __forceinline__ void advance(const WgradGeom& g) {
+    if (++r < r_end) {
+      if (++nc == g.n_chunks) {
+        nc = 0;
+        if (++x == g.Wo) { x = 0; ++y; }
+      }
+    } else {
+      start(g, item + (int)gridDim.x);
+    }
+  }
+};
+
+__global__ void __launch_bounds__(kWgThreads, 1)
+wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant__ CUtensorMap map_in,
+             const __grid_constant__ WgradArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  const WgradGeom& g = args.g;
+  // Stage s: [filters' output gradient: 128 rows x 128 B][patch rows: 128 x 128 B], both
+  // written by the copy engine with the 128-byte swizzle (16-byte chunk index XOR row
+  // index mod 8), which needs 1024-byte aligned buffers.
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const int stages = g.stages;
+  const uint32_t stage_bytes = 2u * kWgOperandBytes;
+  const uint32_t full_bar = base + (uint32_t)stages * stage_bytes;
+  const uint32_t empty_bar = full_bar + 8u * stages;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full_bar + 8u * s, 1);
+      mbar_init(empty_bar + 8u * s, kWgThreads / 32);
+    }
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  // ------------------------------------------------ copy issue (warp 0, lane 0)
+  WgradCursor pc;
+  int p_stage = 0;
+  uint32_t p_phase = 0;
+  bool p_ok = true;
+  const uint32_t tx_bytes = (uint32_t)(g.box_o + g.rows) * 128u;
+  auto produce = [&]() {
+    if (!p_ok || pc.done(g)) return;
+    if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+      p_ok = false;
+      return;
+    }
+    const uint32_t fb = full_bar + 8u * p_stage;
+    const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
+    mbar_arrive_expect_tx(fb, tx_bytes);
+    tma_load_4d(dst, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
+    tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride - g.pad,
+                pc.y * g.stride - g.pad + pc.khb * g.bh, pc.cb * g.bc);
+    if (++p_stage == stages) { p_stage = 0; p_phase ^= 1u; }
+    pc.advance(g);
+  };
+  const bool issuer = (warp == 0 && lane == 0);
+  if (issuer) {
+    prefetch_tensormap(&map_dout);
+    prefetch_tensormap(&map_in);
+    pc.start(g, blockIdx.x);
+    for (int s = 0; s + 2 < stages; ++s) produce();
+  }
+  __syncwarp();
+
+  // ------------------------------------------------ arithmetic (all 8 warps)
+  const int wo = warp >> 1, wn = warp & 1;
+  const int to = wo * 4 + (lane >> 3);    // filters 8 to .. 8 to + 7 of the tile
+  const int tk = wn * 8 + (lane & 7);     // gradient rows tk + 16 i, i = 0..7
+  const uint32_t t7 = (uint32_t)tk & 7u;
+  // A thread walks the eight 16-byte chunks of its patch rows in PHYSICAL order p; the
+  // chunk's logical position is p ^ t7 (rows tk + 16 i all have row mod 8 = t7).  The
+  // matching chunk of filter row 8 to + j sits at physical (p ^ t7) ^ j.
+  uint32_t g_off[8];
+#pragma unroll
+  for (int m = 0; m < 8; ++m) g_off[m] = (uint32_t)to * 1024u + (((uint32_t)m ^ t7) << 4);
+  const uint32_t p_off = kWgOperandBytes + (uint32_t)tk * 128u;
+
+  WgradCursor cc;
+  cc.start(g, blockIdx.x);
+  int stage = 0;
+  uint32_t phase = 0;
+  bool ok = true;
+
+  while (ok && !cc.done(g)) {
+    float2 acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = make_float2(0.f, 0.f);
+    const int item = cc.item;
+    const int ob = cc.ob, cb = cc.cb, khb = cc.khb, split = cc.split;
+    const int n_steps = cc.r_end - cc.r;
+
+    for (int s = 0; s < n_steps; ++s) {
+      if (issuer) produce();
+      __syncwarp();
+      if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+        ok = false;
+        break;
+      }
+      const uint8_t* sg = base_ptr + (size_t)stage * stage_bytes;
+      const uint8_t* sp = sg + p_off;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        float4 G[8], P[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          G[j] = *reinterpret_cast<const float4*>(sg + g_off[p ^ j] + j * 128);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          P[i] = *reinterpret_cast<const float4*>(sp + i * 2048 + p * 16);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+          for (int ii = 0; ii < 8; ++ii) {
+            const int i = (j & 1) ? 7 - ii : ii;
+            acc[i][j] = __ffma2_rn(make_float2(P[i].x, P[i].y), make_float2(G[j].x, G[j].y), acc[i][j]);
+            acc[i][j] = __ffma2_rn(make_float2(P[i].z, P[i].w), make_float2(G[j].z, G[j].w), acc[i][j]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar + 8u * stage);
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+    }
+    if (!ok) break;
+    // move the cursor past this item
+    cc.start(g, item + (int)gridDim.x);
+
+    // ---------------------------------------------- store this item's 128 x 128 block
+    const bool direct = (g.splits == 1);
+    const size_t K = (size_t)g.Nc * g.Sk * g.Sk;
+    float* dst_base = direct ? args.dfilt : args.partial + (size_t)split * K * g.No;
+    const float scale = direct ? g.alpha : 1.0f;
+    const int o = ob * 128 + to * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = tk + 16 * i;                  // (c_l * bh + h_l) * bw + w_l
+      if (row >= g.rows) continue;
+      const int w_l = row % g.bw;
+      const int t = row / g.bw;
+      const int h_l = t % g.bh;
+      const int c = cb * g.bc + t / g.bh;
+      const int kh = khb * g.bh + h_l;
+      if (c >= g.Nc || kh >= g.Sk) continue;
+      float* dst = dst_base + (((size_t)c * g.Sk + kh) * g.Sk + w_l) * g.No + o;
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = (acc[i][j].x + acc[i][j].y) * scale;
+      if (o + 8 <= g.No) {
+        *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (o + j < g.No) dst[j] = v[j];
+      }
+    }
+  }
+
+  // Exit path of the issuing lane after a wait ran out: let copies in flight land.
+  if (issuer && (!ok || !p_ok)) {
+    for (int s = 0; s < stages; ++s) {
+      const uint32_t par = (s < p_stage) ? p_phase : (p_phase ^ 1u);
+      mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
+    }
+  }
+}
+
+// dfilt[i] = alpha * (partial[0][i] + partial[1][i] + ... ), four elements per thread.
+__global__ void __launch_bounds__(256)
+wgrad_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dfilt, size_t n4,
+                    int splits, float alpha) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4* p = reinterpret_cast<const float4*>(partial);
+  float4 s = p[i];
+  for (int k = 1; k < splits; ++k) {
+    const float4 v = p[(size_t)k * n4 + i];
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  reinterpret_cast<float4*>(dfilt)[i] = make_float4(s.x * alpha, s.y * alpha, s.z * alpha, s.w * alpha);
+}
+
+}  // namespace maxdnn

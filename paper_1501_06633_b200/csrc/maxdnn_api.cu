@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "../../include/maxdnn.h"
+#include "bprop.cuh"
 #include "ffma_conv.cuh"
 #include "plan.h"
 #include "umma_conv.cuh"
@@ -24,6 +25,7 @@ struct DeviceState {
   uint32_t* status = nullptr;   // one word of device memory
   bool ffma_attr[16] = {};
   bool umma_attr[4] = {false, false, false, false};
+  bool wgrad_attr = false;
 };
 
 std::mutex g_mu;
@@ -315,6 +317,122 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
 }
 
 // ---------------------------------------------------------------------------
+// Backward propagation.
+// ---------------------------------------------------------------------------
+bool kind_ok(maxdnn_kernel_kind k) {
+  return k == MAXDNN_KERNEL_FP32 || k == MAXDNN_KERNEL_TF32 || k == MAXDNN_KERNEL_BF16;
+}
+
+// Checks that the forward kernel of `kind` takes the transposed problem.
+maxdnn_status dgrad_plan_check(const maxdnn_conv_desc& fd, maxdnn_kernel_kind kind, int sm_count) {
+  static thread_local ConvGeom g;
+  static thread_local KStepTable t;
+  if (kind == MAXDNN_KERNEL_FP32)
+    return plan_ffma(fd, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
+  return plan_umma(fd, kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
+                   env_int("MAXDNN_UMMA_PAIR"), &g, &t);
+}
+
+maxdnn_status bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* dout,
+                         const void* filt, float* din, void* ws, size_t ws_bytes,
+                         cudaStream_t stream) {
+  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  maxdnn_conv_desc fd;
+  maxdnn_status st = plan_dgrad(*desc, &fd);
+  if (st != MAXDNN_OK) return st;
+  if (!dout || !filt || !din || !ws) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(dout) || !aligned16(filt) || !aligned16(din) || !aligned16(ws))
+    return MAXDNN_INVALID_VALUE;
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  const size_t need = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * eb;
+  if (ws_bytes < need) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  st = dgrad_plan_check(fd, kind, ds->sm_count);
+  if (st != MAXDNN_OK) return st;
+  const dim3 grid((unsigned)ceil_div(desc->No, 32), (unsigned)ceil_div(desc->Nc, 32),
+                  (unsigned)(desc->Sk * desc->Sk));
+  const dim3 block(32, 8);
+  if (eb == 2)
+    flip_transpose_kernel<uint16_t><<<grid, block, 0, stream>>>(
+        static_cast<const uint16_t*>(filt), static_cast<uint16_t*>(ws), desc->Nc, desc->Sk, desc->No);
+  else
+    flip_transpose_kernel<float><<<grid, block, 0, stream>>>(
+        static_cast<const float*>(filt), static_cast<float*>(ws), desc->Nc, desc->Sk, desc->No);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (kind == MAXDNN_KERNEL_FP32)
+    return fprop_fp32(&fd, static_cast<const float*>(dout), static_cast<const float*>(ws), din, stream);
+  return fprop_umma(&fd, (int)eb, dout, ws, din, stream);
+}
+
+maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, const float* in, const float* dout,
+                           float* dfilt, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  if (!in || !dout || !dfilt) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(dout) || !aligned16(dfilt) || !aligned16(ws))
+    return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  static thread_local WgradArgs args;
+  st = plan_wgrad(*desc, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &args.g);
+  if (st != MAXDNN_OK) return st;
+  const WgradGeom& g = args.g;
+  const size_t kno = (size_t)g.Nc * g.Sk * g.Sk * g.No;
+  const size_t need = g.splits > 1 ? (size_t)g.splits * kno * 4 : 0;
+  if (need > 0 && (!ws || ws_bytes < need)) return MAXDNN_INVALID_VALUE;
+  args.dfilt = dfilt;
+  args.partial = static_cast<float*>(ws);
+  args.status = ds->status;
+  CUtensorMap mg, mi;
+  {
+    // output gradient as (n, x, y, o): one box = 32 images of one pixel x the tile's filters
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
+                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
+    const uint32_t box[4] = {32u, 1u, 1u, (uint32_t)g.box_o};
+    st = encode_map(&mg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, dout, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    // maps as (n, w, h, c): one box = 32 images of a bh x bw window of pixels x bc channels
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
+                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
+    st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != MAXDNN_OK) return st;
+  }
+  if (!ds->wgrad_attr) {
+    if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->wgrad_attr = true;
+  }
+  wgrad_kernel<<<g.grid, kWgThreads, g.smem_bytes, stream>>>(mg, mi, args);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g.splits > 1) {
+    const size_t n4 = kno / 4;
+    wgrad_reduce_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, stream>>>(
+        static_cast<const float*>(ws), dfilt, n4, g.splits, g.alpha);
+    if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  }
+  return MAXDNN_OK;
+}
+
+// ---------------------------------------------------------------------------
 // Allocation-free fp32 entry point.  The status block its kernel reports into
 // lives in this file-scope device array instead of cudaMalloc'd memory.  Every
 // device that loads the library carries these 256 bytes until the process ends.
@@ -538,6 +656,46 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
     return MAXDNN_CUDA_ERROR;
   }
   return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
+                                               maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!desc || !bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  maxdnn_conv_desc fd;
+  const maxdnn_status st = plan_dgrad(*desc, &fd);
+  if (st != MAXDNN_OK) return st;
+  *bytes = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                     const void* dout, const void* filt, float* din,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return bprop_data(desc, kind, dout, filt, din, workspace, workspace_bytes,
+                    static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
+  if (!desc || !bytes) return MAXDNN_INVALID_VALUE;
+  int sm_count = env_int("MAXDNN_SM_COUNT");   // planning without a device (tests)
+  if (sm_count <= 0) {
+    DeviceState* ds = nullptr;
+    const maxdnn_status st = device_state(&ds);
+    if (st != MAXDNN_OK) return st;
+    sm_count = ds->sm_count;
+  }
+  WgradGeom g;
+  const maxdnn_status st = plan_wgrad(*desc, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
+  if (st != MAXDNN_OK) return st;
+  *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Sk * g.Sk * g.No * 4 : 0;
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, const float* in,
+                                       const float* dout, float* dfilt, void* workspace,
+                                       size_t workspace_bytes, void* cuda_stream) {
+  return bprop_filter(desc, in, dout, dfilt, workspace, workspace_bytes,
+                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_last_device_status(void* cuda_stream) {

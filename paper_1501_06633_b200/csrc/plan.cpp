@@ -335,4 +335,70 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
   return MAXDNN_OK;
 }
 
+maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* f) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  if (!f) return MAXDNN_INVALID_VALUE;
+  if (d.stride != 1 || d.pad > d.Sk - 1) return MAXDNN_NOT_SUPPORTED;
+  f->Nb = d.Nb; f->Wi = Wo; f->Hi = Ho; f->Nc = d.No; f->No = d.Nc; f->Sk = d.Sk;
+  f->stride = 1; f->pad = d.Sk - 1 - d.pad; f->alpha = d.alpha;
+  return MAXDNN_OK;
+}
+
+maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int sm_count, int force_splits, WgradGeom* g) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  st = common_limits(d, 4);
+  if (st != MAXDNN_OK) return st;
+  if (!g || sm_count <= 0) return MAXDNN_INVALID_VALUE;
+  if (d.Nb % 4 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule
+  if (d.Sk > d.Wi || d.Sk > d.Hi) return MAXDNN_NOT_SUPPORTED;       // a copy box must fit the map
+  memset(g, 0, sizeof(*g));
+  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
+  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+  g->bw = d.Sk;
+  g->bh = d.Sk < 128 / g->bw ? d.Sk : 128 / g->bw;
+  if (g->bh < 1) return MAXDNN_NOT_SUPPORTED;
+  g->bc = 128 / (g->bw * g->bh);
+  if (g->bc > d.Nc) g->bc = d.Nc;
+  g->rows = g->bc * g->bh * g->bw;
+  g->box_o = d.No < 128 ? d.No : 128;
+  g->c_blocks = ceil_div(d.Nc, g->bc);
+  g->kh_blocks = ceil_div(d.Sk, g->bh);
+  g->o_blocks = ceil_div(d.No, 128);
+  g->n_chunks = ceil_div(d.Nb, 32);
+  const int64_t r_steps = (int64_t)Ho * Wo * g->n_chunks;
+  const int64_t tiles = (int64_t)g->c_blocks * g->kh_blocks * g->o_blocks;
+  if (r_steps > 0x3fffffff || tiles > 0x3fffffff) return MAXDNN_NOT_SUPPORTED;
+  g->r_steps = (int32_t)r_steps;
+  // Split the reduction so that the items fill whole waves of persistent CTAs (about
+  // four waves when the tiles alone are fewer), each split keeping at least 64 steps.
+  int splits = 1;
+  if (force_splits > 0) {
+    splits = force_splits;
+  } else if (tiles < 4 * (int64_t)sm_count) {
+    const int64_t want = ceil_div(4 * sm_count, (int)tiles);
+    const int64_t most = r_steps / 64 > 0 ? r_steps / 64 : 1;
+    splits = (int)(want < most ? want : most);
+    // round the item count to whole waves where that is cheap
+    const int64_t items = tiles * splits;
+    const int64_t waves = (items + sm_count - 1) / sm_count;
+    const int64_t fit = waves * sm_count / tiles;
+    if (fit >= 1 && fit <= most) splits = (int)fit;
+  }
+  if (splits > r_steps) splits = (int)r_steps;
+  if (splits < 1) splits = 1;
+  g->steps_per_split = ceil_div(g->r_steps, splits);
+  g->splits = ceil_div(g->r_steps, g->steps_per_split);
+  const int64_t items = tiles * g->splits;
+  if (items > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
+  g->n_items = (int32_t)items;
+  g->stages = 6;
+  g->smem_bytes = g->stages * 2 * 128 * 128 + 1024 + 256;
+  g->grid = g->n_items < sm_count ? g->n_items : sm_count;
+  return MAXDNN_OK;
+}
+
 }  // namespace maxdnn

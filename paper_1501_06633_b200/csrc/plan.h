@@ -61,4 +61,39 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
 maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
                         int force_pair, ConvGeom* g, KStepTable* t);
 
+// ---------------------------------------------------------------------------
+// Backward propagation (the adjoints of the operation; the paper names BPROP in
+// its Abstract and Section 6 as the place its techniques should carry over to).
+// ---------------------------------------------------------------------------
+
+// Gradient with respect to the maps, stride 1: FPROP of the output gradient with
+// the filter bank transposed (channels <-> filters) and flipped in both axes and
+// padding Sk - 1 - pad.  Fills the descriptor of that FPROP.  NOT_SUPPORTED for
+// stride != 1 or pad > Sk - 1.
+maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* fprop_desc);
+
+// Gradient with respect to the filters: the (Nc Sk^2) x No matrix
+//   dfilt[k][o] = alpha * sum_r patch[k][r] * dout[o][r],   r = (y, x, n),
+// as a GEMM whose reduction runs over output pixels and images.  One tile = up to
+// 128 gradient rows (bc channels x bh filter rows x bw = Sk filter columns: one
+// bulk copy of a bh x bw window of input pixels) x up to 128 filters; a reduction
+// step = 32 images of one output pixel.  The reduction is split over `splits`
+// CTAs per tile whose partial sums a second kernel adds in a fixed order.
+struct WgradGeom {
+  int32_t Nb, Wi, Hi, Nc, No, Sk, stride, pad, Ho, Wo;
+  float alpha;
+  int32_t bc, bh, bw;        // channels x filter rows x filter columns per tile
+  int32_t rows;              // bc * bh * bw <= 128
+  int32_t box_o;             // filters per tile, min(128, No)
+  int32_t c_blocks, kh_blocks, o_blocks;
+  int32_t n_chunks;          // groups of 32 images
+  int32_t r_steps;           // Ho * Wo * n_chunks
+  int32_t splits, steps_per_split;
+  int32_t n_items;           // tiles x splits
+  int32_t stages, grid, smem_bytes;
+};
+
+// force_splits > 0 pins the number of reduction splits (tests, ablations).
+maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int sm_count, int force_splits, WgradGeom* g);
+
 }  // namespace maxdnn

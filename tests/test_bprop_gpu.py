@@ -1,0 +1,130 @@
+"""Parity of the backward-propagation entry points against the CPU oracle, through the
+C ABI: the gradient with respect to the maps (an FPROP of the output gradient with the
+transformed filter bank, on all three kernels) and with respect to the filters (exact
+fp32, split reduction with a fixed-order sum)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1501_06633_b200 as mx
+from paper_1501_06633_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+KIND = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}
+TOL = {"fp32": 1e-5, "tf32": 5e-3, "bf16": 2e-2}
+
+
+def make(shape, seed):
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("bprop", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), seed)
+    inp, filt = wl.make_inputs(w)
+    Ho, Wo = oracle.out_dims(*w.dims)
+    rng = np.random.default_rng(seed + 2)
+    dout = rng.uniform(-1.0, 1.0, size=(No, Ho, Wo, Nb)).astype(np.float32)
+    return w, inp, filt, dout
+
+
+def rel_err(got, ref):
+    return float(np.max(np.abs(got.astype(np.float64) - ref))) / max(float(np.max(np.abs(ref))), 1e-30)
+
+
+def dev(a, kernel):
+    if kernel == "bf16":
+        return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(a).cuda()
+
+
+def rounded(a, kernel):
+    """What the kernel's operands really are: bf16 operands are the caller's rounding."""
+    return wl.from_bf16_bits(wl.to_bf16_bits(a)) if kernel == "bf16" else a
+
+
+DGRAD_SHAPES = [
+    # Nb Wi Hi Nc No Sk stride pad alpha
+    (64, 14, 9, 64, 96, 3, 1, 1, 1.0),
+    (128, 9, 7, 32, 64, 5, 1, 2, 0.5),
+    (64, 12, 10, 128, 32, 3, 1, 0, 1.0),      # no padding: din gets pad' = Sk - 1
+    (64, 8, 8, 64, 64, 1, 1, 0, 2.0),         # 1x1
+    (64, 10, 6, 96, 160, 4, 1, 3, 1.0),       # even filter, pad = Sk - 1
+]
+
+
+@pytest.mark.parametrize("kernel", ["fp32", "tf32", "bf16"])
+@pytest.mark.parametrize("shape", DGRAD_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_data(kernel, shape):
+    w, inp, filt, dout = make(shape, 900 + shape[5])
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_workspace(d, KIND[kernel]), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data(d, dev(dout, kernel), dev(filt, kernel), din, ws, KIND[kernel])
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_data(rounded(dout, kernel), rounded(filt, kernel), (w.Hi, w.Wi),
+                                 stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = din.cpu().numpy().reshape(ref.shape)
+    assert np.all(np.isfinite(got))
+    assert rel_err(got, ref) <= TOL[kernel]
+
+
+def test_bprop_data_refusals():
+    d = mx.ConvDesc.make(64, 16, 16, 32, 32, 3, 2, 1, 1.0)          # stride 2
+    with pytest.raises(mx.MaxdnnError) as e:
+        mx.conv_bprop_data_workspace(d)
+    assert e.value.status == mx.NOT_SUPPORTED
+    d = mx.ConvDesc.make(64, 16, 16, 32, 32, 3, 1, 1, 1.0)
+    need = mx.conv_bprop_data_workspace(d)
+    assert need == 32 * 9 * 32 * 4
+    g = torch.zeros(mx.conv_out_elems(d), device="cuda")
+    f = torch.zeros(mx.conv_filt_elems(d), device="cuda")
+    x = torch.zeros(mx.conv_in_elems(d), device="cuda")
+    small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
+    assert mx.bprop_data_status(d, g, f, x, small) == mx.INVALID_VALUE
+
+
+WGRAD_SHAPES = [
+    # Nb Wi Hi Nc No Sk stride pad alpha
+    (64, 14, 9, 20, 96, 3, 1, 1, 1.0),        # 14 channels per tile: two channel blocks
+    (128, 9, 7, 12, 64, 5, 1, 2, 0.5),        # 5 channels per tile, ragged last block
+    (32, 23, 19, 3, 96, 11, 4, 0, 1.0),       # the first-layer shape: all 121 taps x 1 channel
+    (36, 12, 10, 16, 132, 3, 2, 1, 1.0),      # images and filters not multiples of 32 / 128
+    (64, 8, 8, 160, 64, 1, 1, 0, 2.0),        # 1x1: 128 channels per tile
+    (8, 30, 30, 4, 8, 13, 1, 6, 1.0),         # 13x13 filter: 9 filter rows per tile, two row blocks
+    (64, 10, 6, 8, 256, 4, 1, 3, -1.0),       # two filter blocks
+]
+
+
+@pytest.mark.parametrize("splits", [0, 1, 3])
+@pytest.mark.parametrize("shape", WGRAD_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_filter(shape, splits, monkeypatch):
+    if splits:
+        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+    w, inp, filt, dout = make(shape, 1700 + shape[5])
+    d = mx.ConvDesc.make(*w.dims)
+    need = mx.conv_bprop_filter_workspace(d)
+    if splits == 1:
+        assert need == 0
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    dfilt = torch.full((mx.conv_filt_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_filter(d, torch.from_numpy(inp).cuda(), torch.from_numpy(dout).cuda(), dfilt, ws)
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_filter(inp, dout, w.Sk, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = dfilt.cpu().numpy().reshape(ref.shape)
+    assert np.all(np.isfinite(got))
+    assert rel_err(got, ref) <= 1e-5
+
+
+def test_bprop_filter_is_reproducible():
+    """Partial sums are added in a fixed order: two runs agree bit for bit."""
+    w, inp, filt, dout = make((64, 14, 9, 20, 96, 3, 1, 1, 1.0), 77)
+    d = mx.ConvDesc.make(*w.dims)
+    need = mx.conv_bprop_filter_workspace(d)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    a = torch.empty(mx.conv_filt_elems(d), device="cuda")
+    b = torch.empty_like(a)
+    x, g = torch.from_numpy(inp).cuda(), torch.from_numpy(dout).cuda()
+    mx.conv_bprop_filter(d, x, g, a, ws)
+    mx.conv_bprop_filter(d, x, g, b, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)

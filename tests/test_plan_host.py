@@ -168,3 +168,28 @@ def test_table1_shapes_give_the_printed_output_sizes_and_have_plans():
         for kind in (mx.KERNEL_FP32, mx.KERNEL_TF32, mx.KERNEL_BF16):
             info, steps = mx.conv_plan_query(d, kind, 148)
             assert info.n_tiles > 0 and info.smem_bytes <= 227 * 1024 and len(steps) == info.n_ksteps
+
+
+def test_bprop_workspace_sizes_and_refusals(monkeypatch):
+    """Host-side planning of the backward entry points (no device needed: the SM count
+    is given)."""
+    monkeypatch.setenv("MAXDNN_SM_COUNT", "148")
+    d = mx.ConvDesc.make(128, 27, 27, 96, 256, 5, 1, 2, 1.0)
+    assert mx.conv_bprop_data_workspace(d, mx.KERNEL_FP32) == 96 * 25 * 256 * 4
+    assert mx.conv_bprop_data_workspace(d, mx.KERNEL_BF16) == 96 * 25 * 256 * 2
+    for bad in (mx.ConvDesc.make(128, 227, 227, 3, 96, 11, 4, 0, 1.0),      # stride 4
+                mx.ConvDesc.make(64, 16, 16, 8, 8, 3, 1, 3, 1.0)):          # pad > Sk - 1
+        with pytest.raises(mx.MaxdnnError) as e:
+            mx.conv_bprop_data_workspace(bad)
+        assert e.value.status == mx.NOT_SUPPORTED
+    # filter gradient: partial sums of `splits` reduction splits, or nothing for one split
+    kno = 96 * 25 * 256 * 4
+    need = mx.conv_bprop_filter_workspace(d)
+    assert need % kno == 0 and 2 <= need // kno <= 64          # 40 tiles: the reduction is split
+    big = mx.ConvDesc.make(128, 12, 12, 1024, 1024, 3, 1, 1, 1.0)   # 592 tiles: 4 whole waves
+    assert mx.conv_bprop_filter_workspace(big) == 0
+    monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", "5")
+    assert mx.conv_bprop_filter_workspace(d) == 5 * kno
+    with pytest.raises(mx.MaxdnnError) as e:
+        mx.conv_bprop_filter_workspace(mx.ConvDesc.make(30, 16, 16, 8, 8, 3, 1, 1, 1.0))   # Nb % 4
+    assert e.value.status == mx.NOT_SUPPORTED
