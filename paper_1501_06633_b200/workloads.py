@@ -107,6 +107,15 @@ def make_inputs(w: Workload, seed_offset: int = 0):
     return maps, filt
 
 
+def make_dout(w: Workload, seed_offset: int = 0):
+    """Output gradient for the backward-propagation entry points: uniform [-1, 1) in the
+    output's storage layout [No][Ho][Wo][Nb], PCG64 from ``seed + 2``."""
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
+    rng = np.random.default_rng(w.seed + 1000 * seed_offset + 2)
+    return rng.uniform(-1.0, 1.0, size=(w.No, Ho, Wo, w.Nb)).astype(np.float32)
+
+
 def to_bf16_bits(a: np.ndarray) -> np.ndarray:
     """fp32 -> bf16 storage (uint16), round-to-nearest-even; finite inputs."""
     u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)

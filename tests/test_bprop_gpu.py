@@ -21,10 +21,7 @@ def make(shape, seed):
     w = wl.Workload("bprop", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
                     ("uniform", -1.0, 1.0), seed)
     inp, filt = wl.make_inputs(w)
-    Ho, Wo = oracle.out_dims(*w.dims)
-    rng = np.random.default_rng(seed + 2)
-    dout = rng.uniform(-1.0, 1.0, size=(No, Ho, Wo, Nb)).astype(np.float32)
-    return w, inp, filt, dout
+    return w, inp, filt, wl.make_dout(w)
 
 
 def rel_err(got, ref):
@@ -128,3 +125,55 @@ def test_bprop_filter_is_reproducible():
     mx.conv_bprop_filter(d, x, g, b, ws)
     torch.cuda.synchronize()
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["first11x11s4", "mid5x5", "wide3x3"])
+def test_full_size_sampled_bprop_filter(name):
+    """Benchmark sizes, in the launch configuration the bench times: random single
+    gradient elements against the oracle, within the a-priori bound of an fp32 sum."""
+    w = wl.WORKLOADS[name]
+    inp, _ = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+    d = mx.ConvDesc.make(*w.dims)
+    need = mx.conv_bprop_filter_workspace(d)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    dfilt = torch.full((mx.conv_filt_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_filter(d, torch.from_numpy(inp).cuda(), torch.from_numpy(dout).cuda(), dfilt, ws)
+    assert mx.last_device_status() == mx.OK
+    got = dfilt.cpu().numpy().reshape(w.Nc, w.Sk, w.Sk, w.No)
+    assert np.isfinite(got).all()
+    R = dout.shape[1] * dout.shape[2] * w.Nb
+    rng = np.random.default_rng(4)
+    for _ in range(200):
+        c, kh, kw, o = (int(rng.integers(0, s)) for s in got.shape)
+        v, a = oracle.conv_bprop_filter_point(inp, dout, w.Sk, c, kh, kw, o, stride=w.stride,
+                                              pad=w.pad, alpha=w.alpha)
+        # pairwise-ish summation order on the GPU: the plain bound R u |terms| is loose but safe
+        assert abs(float(got[c, kh, kw, o]) - v) <= 64 * np.sqrt(R) * 2.0 ** -24 * abs(w.alpha) * a + 1e-30
+
+
+@pytest.mark.parametrize("name,kernel", [("mid5x5", "fp32"), ("large3x3", "bf16"), ("wide3x3", "tf32")])
+def test_full_size_sampled_bprop_data(name, kernel):
+    w = wl.WORKLOADS[name]
+    _, filt = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_workspace(d, KIND[kernel]), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data(d, dev(dout, kernel), dev(filt, kernel), din, ws, KIND[kernel])
+    assert mx.last_device_status() == mx.OK
+    got = din.cpu().numpy().reshape(w.Nc, w.Hi, w.Wi, w.Nb)
+    assert np.isfinite(got).all()
+    rd, rf = rounded(dout, kernel), rounded(filt, kernel)
+    rng = np.random.default_rng(5)
+    pts = [tuple(int(rng.integers(0, s)) for s in got.shape) for _ in range(200)]
+    pts += [(0, 0, 0, 0), (w.Nc - 1, w.Hi - 1, w.Wi - 1, w.Nb - 1), (1, 0, w.Wi - 1, 3)]   # corners: apron
+    vals = [oracle.conv_bprop_data_point(rd, rf, (w.Hi, w.Wi), *p, stride=w.stride, pad=w.pad,
+                                         alpha=w.alpha) for p in pts]
+    scale = max(abs(v) for v, _ in vals)
+    K = w.No * w.Sk ** 2
+    for p, (v, a) in zip(pts, vals):
+        if kernel == "fp32":
+            assert abs(float(got[p]) - v) <= (K + 3) * 2.0 ** -24 * abs(w.alpha) * a + 1e-30
+        else:
+            assert abs(float(got[p]) - v) <= TOL[kernel] * scale
