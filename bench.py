@@ -53,6 +53,8 @@ def parse_args():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER + wl.TABLE1_ORDER)
     p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16"])
+    p.add_argument("--op", default="fprop", choices=["fprop", "dgrad", "wgrad"],
+                   help="fprop (the headline path) or one of its two adjoints (BPROP)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=12.0,
@@ -68,14 +70,18 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def workload_bytes(w, kernel):
-    """Algorithmic HBM bytes of one step: every map and filter element read
-    once, every output written once."""
+def workload_bytes(w, kernel, op="fprop"):
+    """Algorithmic HBM bytes of one step: every operand element read once, every
+    result element written once (results are fp32)."""
     eb = 2 if kernel == "bf16" else 4
     Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
     Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
-    return (w.Nc * w.Hi * w.Wi * w.Nb * eb + w.Nc * w.Sk * w.Sk * w.No * eb
-            + w.No * Ho * Wo * w.Nb * 4), Ho, Wo
+    maps, filt, out = w.Nc * w.Hi * w.Wi * w.Nb, w.Nc * w.Sk * w.Sk * w.No, w.No * Ho * Wo * w.Nb
+    if op == "dgrad":
+        return out * eb + filt * eb + maps * 4, Ho, Wo
+    if op == "wgrad":
+        return maps * eb + out * eb + filt * 4, Ho, Wo
+    return maps * eb + filt * eb + out * 4, Ho, Wo
 
 
 def flops(w, Ho, Wo):
@@ -106,6 +112,30 @@ def oracle_sample(w, target_seconds):
     dt = time.perf_counter() - t0
     fl = flops(w, rows, Wo) * repeats
     return fl / dt / 1e12, dt, rows, Ho, repeats, oracle.num_threads()
+
+
+def oracle_sample_bprop(w, op, target_seconds):
+    """The BPROP oracle on the first `cs` channels of the workload (a gradient with respect
+    to a subset of channels is that subset of the work), sized to about `target_seconds`."""
+    import oracle
+    inp, filt = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+
+    def run(cs):
+        t0 = time.perf_counter()
+        if op == "dgrad":
+            oracle.conv_bprop_data(dout, filt[:cs], (w.Hi, w.Wi), stride=w.stride, pad=w.pad, alpha=w.alpha)
+        else:
+            oracle.conv_bprop_filter(inp[:cs], dout, w.Sk, stride=w.stride, pad=w.pad, alpha=w.alpha)
+        return max(time.perf_counter() - t0, 1e-6)
+
+    t1 = run(1)
+    cs = int(max(1, min(w.Nc, target_seconds / t1)))
+    dt = run(cs) if cs > 1 else t1
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    Wo = (w.Wi + 2 * w.pad - w.Sk) // w.stride + 1
+    fl = flops(w, Ho, Wo) * cs / w.Nc
+    return fl / dt / 1e12, dt, cs, oracle.num_threads()
 
 
 def run_reference(args):
@@ -258,26 +288,54 @@ def run_ours(args):
     w = wl.ALL[args.workload]
     kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}[args.kernel]
     d = mx.ConvDesc.make(*w.dims)
-    nbytes, Ho, Wo = workload_bytes(w, args.kernel)
-    C = mx.conv_flops(d)
+    op = args.op
+    if op == "wgrad" and args.kernel != "fp32":
+        raise SystemExit("the filter gradient is built in fp32 only")
+    nbytes, Ho, Wo = workload_bytes(w, args.kernel, op)
+    C = mx.conv_flops(d)          # the same bilinear form: all three operations cost C
     assert C == flops(w, Ho, Wo)
 
-    # Each rank holds its own batch shard (same recipe, its own seed); FPROP needs
-    # no exchange between shards.  Buffer sets are rotated so that no step finds
-    # its inputs in L2.
+    # Each rank holds its own batch shard (same recipe, its own seed); neither FPROP nor
+    # the map gradient needs an exchange between shards (the filter gradient of a sharded
+    # batch would need a sum over ranks, which this benchmark does not time).  Buffer
+    # sets are rotated so that no step finds its operands in L2.
     inp, filt = shard_inputs(w, rank)
+    dout = wl.make_dout(w, seed_offset=rank) if op != "fprop" else None
     n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / nbytes)))
-    if args.kernel == "bf16":
-        to_dev = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+    bf16 = args.kernel == "bf16"
+    if bf16:
+        to_host = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).reshape(-1)
+        as_op = lambda t: t.view(torch.bfloat16)
     else:
-        to_dev = lambda a: torch.from_numpy(a).cuda()
-    d_filt = to_dev(filt).reshape(-1)
-    base_in = to_dev(inp).reshape(-1)
-    d_ins = [base_in] + [base_in.clone() for _ in range(n_sets - 1)]
-    d_outs = [torch.empty(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
-              for _ in range(n_sets)]
+        to_host = lambda a: torch.from_numpy(a).reshape(-1)
+        as_op = lambda t: t
+    # operands: (big streamed operand, second operand); result: fp32
+    if op == "fprop":
+        h_a, h_b, n_res = to_host(inp), to_host(filt), mx.conv_out_elems(d)
+    elif op == "dgrad":
+        h_a, h_b, n_res = to_host(dout), to_host(filt), mx.conv_in_elems(d)
+    else:
+        h_a, h_b, n_res = to_host(inp), to_host(dout), mx.conv_filt_elems(d)
+    h_a, h_b = h_a.pin_memory(), h_b.pin_memory()
+    d_as = [h_a.cuda() for _ in range(n_sets)]
+    d_bs = [h_b.cuda() for _ in range(n_sets if op == "wgrad" else 1)]
+    d_res = [torch.empty(n_res, dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+    ws = None
+    if op == "dgrad":
+        ws = torch.empty(mx.conv_bprop_data_workspace(d, kind), dtype=torch.uint8, device="cuda")
+    elif op == "wgrad":
+        ws = torch.empty(max(16, mx.conv_bprop_filter_workspace(d)), dtype=torch.uint8, device="cuda")
     fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
              mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
+
+    def step(i):
+        a, b, r = d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets]
+        if op == "fprop":
+            fprop(d, as_op(a), as_op(b), r)
+        elif op == "dgrad":
+            mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws, kind)
+        else:
+            mx.conv_bprop_filter(d, a, b, r, ws)
 
     def barrier():
         if world > 1:
@@ -285,7 +343,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     for i in range(max(3, args.warmup)):
-        fprop(d, d_ins[i % n_sets], d_filt, d_outs[i % n_sets])
+        step(i)
     barrier()
 
     sampler = ClockSampler(local_rank)
@@ -295,7 +353,7 @@ def run_ours(args):
     barrier()
     ev0.record()
     for i in range(args.steps):
-        fprop(d, d_ins[i % n_sets], d_filt, d_outs[i % n_sets])
+        step(i)
     ev1.record()
     barrier()
     clocks = sampler.stop()
@@ -304,22 +362,29 @@ def run_ours(args):
     if mx.last_device_status() != mx.OK:
         raise SystemExit("a kernel reported a timed-out wait; results are not valid")
 
-    # end to end: pinned host buffers through maxdnn_conv_fprop_host
-    h_in = torch.from_numpy(wl.to_bf16_bits(inp).view(np.int16) if args.kernel == "bf16" else inp
-                            ).reshape(-1).pin_memory()
-    h_f = torch.from_numpy(wl.to_bf16_bits(filt).view(np.int16) if args.kernel == "bf16" else filt
-                           ).reshape(-1).pin_memory()
-    h_out = torch.empty(mx.conv_out_elems(d), dtype=torch.float32).pin_memory()
-    s_in = d_ins[0].view(torch.int16) if args.kernel == "bf16" else d_ins[0]
-    s_f = d_filt.view(torch.int16) if args.kernel == "bf16" else d_filt
+    # end to end from pinned host buffers: host -> device copies of both operands, the
+    # kernel(s), device -> host copy of the result, every step.  FPROP goes through
+    # maxdnn_conv_fprop_host; the gradients through the same copies around their call.
+    h_out = torch.empty(n_res, dtype=torch.float32).pin_memory()
+    h_in, h_f = h_a, h_b
+
+    def e2e_step():
+        if op == "fprop":
+            mx.conv_fprop_host(d, kind, h_a, h_b, h_out, d_as[0], d_bs[0], d_res[0])
+        else:
+            d_as[0].copy_(h_a, non_blocking=True)
+            d_bs[0].copy_(h_b, non_blocking=True)
+            step(0)
+            h_out.copy_(d_res[0], non_blocking=True)
+
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     for _ in range(2):
-        mx.conv_fprop_host(d, kind, h_in, h_f, h_out, s_in, s_f, d_outs[0])
+        e2e_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
-        mx.conv_fprop_host(d, kind, h_in, h_f, h_out, s_in, s_f, d_outs[0])
+        e2e_step()
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
@@ -352,7 +417,7 @@ def run_ours(args):
             "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[args.kernel],
             "data": "synthetic",
             "config": {
-                "workload": w.name, "kernel": args.kernel, "Nb": w.Nb, "Wi": w.Wi, "Hi": w.Hi,
+                "workload": w.name, "op": op, "kernel": args.kernel, "Nb": w.Nb, "Wi": w.Wi, "Hi": w.Hi,
                 "Nc": w.Nc, "No": w.No, "Sk": w.Sk, "stride": w.stride, "pad": w.pad,
                 "alpha": w.alpha, "flops_per_step": C, "algorithmic_bytes_per_step": nbytes,
                 "l2": "rotating %d buffer sets (%.0f MB) > L2 (126 MB)" % (n_sets, n_sets * nbytes / 1e6),
@@ -366,7 +431,8 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "roofline": {
                 "bound": bound, "achieved": per_gpu, "peak": peak, "unit": "TFLOP/s",
-                "frac": per_gpu / peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.kernel)),
+                "frac": per_gpu / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.kernel)) if op == "fprop" else None,
                 "peak_source": peak_note,
                 "roofline_time_us": max(t_compute, t_hbm) * 1e6,
                 "frac_of_roofline_time": max(t_compute, t_hbm) / (ms_step * 1e-3),
@@ -377,7 +443,12 @@ def run_ours(args):
             # the paper's clock-independent efficiency: C / (2*128*SMs*elapsed SM cycles)
             cycles = ms_step * 1e-3 * clocks["sm_mhz"] * 1e6
             line["roofline"]["ce_at_sampled_clock"] = C / (2.0 * 128 * sm_count * cycles)
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and op != "fprop":
+            tf, secs, cs, threads = oracle_sample_bprop(w, op, args.cpu_seconds)
+            line["cpu_baseline"] = {
+                "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
+                "sample": "%s of %s restricted to %d of %d channels, %.1f s" % (op, w.name, cs, w.Nc, secs)}
+        elif world == 1 and not args.no_cpu_baseline:
             tf, secs, rows, Ho_, reps, threads = oracle_sample(w, args.cpu_seconds)
             line["cpu_baseline"] = {
                 "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
