@@ -247,7 +247,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   if (issuer && (!ok || !p_ok)) {
     for (int s = 0; s < stages; ++s) {
       const uint32_t par = (s < p_stage) ? p_phase : (p_phase ^ 1u);
-      mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
+      mbar_wait_grace(full_bar + 8u * s, par);
     }
   }
 }

@@ -36,10 +36,10 @@ struct FfmaArgs {
   ConvGeom g;
   float* out;
   uint32_t* status;
-  // Test hook for the bounded waits: if non-zero, CTA 0's producer arms the barrier of
-  // its drop_step-th K step but never issues the patch copy, so the consumers' wait
+  // Test hook for the bounded waits: if non-zero, CTA 0 initialises its "full" barriers
+  // to expect one arrival more than they will ever get, so the consumers' first wait
   // runs out and the kernel reports kDevTimeoutFull instead of hanging.
-  uint32_t drop_step;
+  uint32_t test_missing_arrival;
   KStepTable table;
 };
 
@@ -114,7 +114,6 @@ __device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR 
 struct FfmaProducer {
   int tile, step, stage;
   uint32_t phase;
-  uint32_t issued;
   int o0, n0, h0, w0;
 
   __device__ __forceinline__ void set_tile(const ConvGeom& g, int mt) {
@@ -131,7 +130,7 @@ struct FfmaProducer {
 
   __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
     tile = g.tile_begin + blockIdx.x;
-    step = 0; stage = 0; phase = 0; issued = 0;
+    step = 0; stage = 0; phase = 0;
     o0 = n0 = h0 = w0 = 0;
     if (tile < g.tile_end) set_tile(g, mt);
   }
@@ -154,8 +153,7 @@ struct FfmaProducer {
     tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, o0, ks.kw0, ks.kh, ks.c0);
     uint32_t dst = b_base + (uint32_t)stage * g.b_stage_bytes;
     int w = w0 + ks.kw0;
-    const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
-    for (int t = 0; t < g.b_boxes && !drop; ++t) {
+    for (int t = 0; t < g.b_boxes; ++t) {
       tma_load_4d(dst, map_in, fb, n0, w, h0 + ks.kh, ks.c0);
       dst += g.b_slot_bytes;
       w += g.stride;
@@ -174,7 +172,7 @@ struct FfmaProducer {
   __device__ __forceinline__ void drain(const ConvGeom& g, uint32_t full_bar) {
     for (int s = 0; s < g.stages; ++s) {
       const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-      mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
+      mbar_wait_grace(full_bar + 8u * s, par);
     }
   }
 };
@@ -207,8 +205,9 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    const uint32_t extra = (args.test_missing_arrival != 0 && blockIdx.x == 0) ? 1u : 0u;
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 1);
+      mbar_init(full_bar + 8u * s, 1 + extra);
       mbar_init(empty_bar + 8u * s, kFfmaConsumerWarps);
     }
     fence_mbar_init();

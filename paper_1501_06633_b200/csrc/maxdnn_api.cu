@@ -150,7 +150,7 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   if (st != MAXDNN_OK) return st;
   args.out = out;
   args.status = ds->status;
-  args.drop_step = (uint32_t)env_int("MAXDNN_TEST_DROP_COPY");   // test hook, see FfmaArgs
+  args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see FfmaArgs
   const ConvGeom& g = args.g;
 
   CUtensorMap mf, mi;
@@ -253,7 +253,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   args.atom = atom;
   args.umma_k = 32u / (uint32_t)elem_bytes;
   args.is_bf16 = bf16 ? 1u : 0u;
-  args.drop_step = (uint32_t)env_int("MAXDNN_TEST_DROP_COPY");   // test hook, see UmmaArgs
+  args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see UmmaArgs
   // Staged layouts: filters [group of 32/64][kw][channel][128 B], patches
   // [pixel][image group][channel][128 B].
   args.lbo_a_bytes = (uint32_t)(g.kwc * g.kc) * 128u;
@@ -504,7 +504,7 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
   args.out = out;
   args.status = ds->status;
-  args.drop_step = 0;
+  args.test_missing_arrival = 0;
   const ConvGeom& g = args.g;
 
   CUtensorMap mf, mi;

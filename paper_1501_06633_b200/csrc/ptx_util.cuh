@@ -85,6 +85,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
   return mbar_wait_slow(bar, parity, status, code);
 }
 
+// Exit-path wait after another wait ran out: copies already issued land within
+// microseconds; give their barrier one millisecond, then move on without a code.
+__device__ __noinline__ void mbar_wait_grace(uint32_t bar, uint32_t parity) {
+  const uint64_t t0 = globaltimer_ns();
+  while (!mbar_try_wait(bar, parity))
+    if (globaltimer_ns() - t0 > 1000000ull) break;
+}
+
 #ifndef MAXDNN_PRODUCER_SLEEP_NS
 #define MAXDNN_PRODUCER_SLEEP_NS 250
 #endif

@@ -37,7 +37,7 @@ struct UmmaArgs {
   uint32_t tap_a_bytes; // filter tile: start-address step from one filter column (kw) to the next
   uint32_t tap_b_bytes; // patch strip: start-address step of one pixel (the next kw's window)
   uint32_t is_bf16;
-  uint32_t drop_step;   // test hook: CTA 0 skips the patch copy of this K step (0 = never)
+  uint32_t test_missing_arrival;   // test hook: CTA 0's full barriers expect an arrival that never comes
   uint32_t* status;
   KStepTable table;
 };
@@ -189,8 +189,9 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    const uint32_t extra = (args.test_missing_arrival != 0 && blockIdx.x == 0) ? 1u : 0u;   // test hook
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 2);   // one arrival per producer warp
+      mbar_init(full_bar + 8u * s, 2 + extra);   // one arrival per producer warp
       mbar_init(empty_bar + 8u * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -237,7 +238,6 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const uint64_t pol_last = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase = 0;
-      uint32_t issued = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
         int r = tile;
@@ -264,8 +264,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
             if (patch_role) {
               uint32_t dst = b_dst;
               int w = w0 + ks.kw0;
-              const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
-              for (int t = 0; t < g.b_boxes && !drop; ++t) {
+              for (int t = 0; t < g.b_boxes; ++t) {
                 tma_load_5d_hint(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
                 w += g.stride;
@@ -286,7 +285,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       if (!ok) {
         for (int s = 0; s < stages; ++s) {
           const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-          mbar_wait(full_bar + 8u * s, par, nullptr, kDevTimeoutDrain);
+          mbar_wait_grace(full_bar + 8u * s, par);
         }
       }
     }

@@ -138,8 +138,9 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
+    const uint32_t extra = (args.test_missing_arrival != 0 && blockIdx.x == 0) ? 1u : 0u;   // test hook
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 2);   // the leader's two producer warps (they expect both CTAs' bytes)
+      mbar_init(full_bar + 8u * s, 2 + extra);   // the leader's two producer warps (they expect both CTAs' bytes)
       mbar_init(empty_bar + 8u * s, 1);  // the leader's commit
     }
     for (int a = 0; a < 2; ++a) {
@@ -190,7 +191,6 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const uint64_t pol_last = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase = 0;
-      uint32_t issued = 0;
       bool ok = true;
       for (int tile = pair; tile < g.n_tiles && ok; tile += n_pairs) {
         int r = tile;
@@ -218,8 +218,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
             if (patch_role) {
               uint32_t dst = b_dst;
               int w = w0 + ks.kw0;
-              const bool drop = args.drop_step != 0 && blockIdx.x == 0 && ++issued == args.drop_step;
-              for (int t = 0; t < g.b_boxes && !drop; ++t) {
+              for (int t = 0; t < g.b_boxes; ++t) {
                 tma_load_5d_pair(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
                 w += g.stride;

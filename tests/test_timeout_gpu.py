@@ -1,5 +1,6 @@
 """Failure detection without a GPU fault: every wait inside the kernels has a time
-limit; a test hook makes one copy never arrive, the waiting warps give up after their
+limit; a test hook makes one CTA's barriers expect an arrival that never comes, the waiting
+warps give up after their
 limit, the kernel ends normally, the status word says so, and the context stays usable."""
 import numpy as np
 import pytest
@@ -35,12 +36,12 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind,
     out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
     assert mx.last_device_status() == mx.OK
 
-    monkeypatch.setenv("MAXDNN_TEST_DROP_COPY", "3")     # CTA 0 never copies its 3rd patch box
+    monkeypatch.setenv("MAXDNN_TEST_MISSING_ARRIVAL", "1")     # CTA 0 waits for an arrival that never comes
     assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # the launch itself succeeds
     assert mx.last_device_status() == mx.DEVICE_TIMEOUT               # ...the kernel gave up waiting
     assert mx.last_device_status() == mx.OK                           # reading clears the word
 
-    monkeypatch.delenv("MAXDNN_TEST_DROP_COPY")
+    monkeypatch.delenv("MAXDNN_TEST_MISSING_ARRIVAL")
     assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # same context, next call
     assert mx.last_device_status() == mx.OK
     ref = oracle.conv_fprop(ref_in, ref_f, stride=w.stride, pad=w.pad, alpha=w.alpha)
