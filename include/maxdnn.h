@@ -200,7 +200,7 @@ maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const floa
 
 /*
  * Backward propagation.  The paper builds FPROP only and names BPROP (Abstract,
- * Section 6) as the operation its techniques should carry over to, without
+ * Section 3.5 "Conclusion") as the operation its techniques should carry over to, without
  * defining it; these entry points compute the two exact adjoints of the
  * operation above, alpha included, with dout laid out like out, din like in and
  * dfilt like filt:

@@ -4,7 +4,7 @@
  * TEST INFRASTRUCTURE ONLY.  Shares no code with the CUDA path; nothing in the
  * product may call it.
  *
- * The paper builds FPROP only and states (Abstract, Section 6) that the same
+ * The paper builds FPROP only and states (Abstract, Section 3.5 "Conclusion") that the same
  * techniques should carry over to BPROP without defining it.  BPROP is taken
  * here as what the word means for Section 2's operation
  *

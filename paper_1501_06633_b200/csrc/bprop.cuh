@@ -1,5 +1,5 @@
 // Backward-propagation kernels (the adjoints of the operation of Section 2; the paper
-// names BPROP in its Abstract and Section 6 as where its techniques should carry over).
+// names BPROP in its Abstract and Section 3.5 ("Conclusion") as where its techniques should carry over).
 //
 //  - flip_transpose_kernel: filt[c][kh][kw][o] -> ft[o][Sk-1-kh][Sk-1-kw][c], the filter
 //    bank with which the gradient with respect to the maps is an FPROP of the output

@@ -63,7 +63,7 @@ maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
 
 // ---------------------------------------------------------------------------
 // Backward propagation (the adjoints of the operation; the paper names BPROP in
-// its Abstract and Section 6 as the place its techniques should carry over to).
+// its Abstract and Section 3.5 ("Conclusion") as the place its techniques should carry over to).
 // ---------------------------------------------------------------------------
 
 // Gradient with respect to the maps, stride 1: FPROP of the output gradient with
