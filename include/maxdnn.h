@@ -199,6 +199,25 @@ maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const floa
                                         const float* filt, float* out, void* cuda_stream);
 
 /*
+ * FPROP for shapes the entry points above refuse because of the 16-byte row rule
+ * (Nb or No not a multiple of 4 for fp32; of 32 / 64 and 32 for tf32 / bf16): the
+ * maps and filters are copied into zero-padded staging tensors in the caller's
+ * workspace (Nb, No rounded up), the matching kernel runs on the padded problem,
+ * and the result is copied back without the padding.  Same arguments and result
+ * as the matching entry point; `workspace` as for the backward entry points
+ * below (size from maxdnn_conv_fprop_ragged_workspace; 0 when the shape needs no
+ * padding, in which case the kernel runs directly on the caller's tensors).
+ * The paper has no counterpart (Section 3.3 only notes that its kernel wants
+ * multiples of 64 filters and 8 images for efficiency).
+ */
+maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,
+                                                 maxdnn_kernel_kind kind, size_t* bytes);
+maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                       const void* in, const void* filt, float* out,
+                                       void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream);
+
+/*
  * Backward propagation.  The paper builds FPROP only and names BPROP (Abstract,
  * Section 3.5 "Conclusion") as the operation its techniques should carry over to, without
  * defining it; these entry points compute the two exact adjoints of the

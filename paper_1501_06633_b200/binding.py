@@ -17,6 +17,7 @@ __all__ = [
     "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
     "last_device_status",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
+    "conv_fprop_ragged_workspace", "conv_fprop_ragged", "fprop_ragged_status",
     "conv_bprop_data_workspace", "conv_bprop_data", "bprop_data_status",
     "conv_bprop_filter_workspace", "conv_bprop_filter", "bprop_filter_status",
 ]
@@ -31,6 +32,7 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv_fprop_host", "maxdnn_conv_fprop_noalloc", "maxdnn_last_device_status",
     "maxdnn_launch_count", "maxdnn_conv_bprop_data_workspace", "maxdnn_conv_bprop_data",
     "maxdnn_conv_bprop_filter_workspace", "maxdnn_conv_bprop_filter",
+    "maxdnn_conv_fprop_ragged_workspace", "maxdnn_conv_fprop_ragged",
 ]
 
 
@@ -102,6 +104,11 @@ def load_library():
         getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_host.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.maxdnn_conv_fprop_ragged_workspace.restype = ctypes.c_int
+    lib.maxdnn_conv_fprop_ragged_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
+    lib.maxdnn_conv_fprop_ragged.restype = ctypes.c_int
+    lib.maxdnn_conv_fprop_ragged.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp,
+                                             ctypes.c_size_t, vp]
     lib.maxdnn_conv_bprop_data_workspace.restype = ctypes.c_int
     lib.maxdnn_conv_bprop_data_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
     lib.maxdnn_conv_bprop_data.restype = ctypes.c_int
@@ -249,6 +256,35 @@ def _workspace_ptr(workspace, need):
     if not (isinstance(workspace, torch.Tensor) and workspace.is_cuda and workspace.is_contiguous()):
         raise TypeError("workspace must be a contiguous CUDA tensor")
     return ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def conv_fprop_ragged_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:
+    """Bytes of device scratch maxdnn_conv_fprop_ragged needs (0: the shape needs no padding)."""
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv_fprop_ragged_workspace(ctypes.byref(desc), int(kind),
+                                                                 ctypes.byref(n))),
+           "maxdnn_conv_fprop_ragged_workspace")
+    return int(n.value)
+
+
+def fprop_ragged_status(desc: ConvDesc, inp, filt, out, workspace, kind: int = KERNEL_FP32,
+                        stream=None) -> int:
+    """Enqueue maxdnn_conv_fprop_ragged on torch tensors; returns the raw status code."""
+    lib = load_library()
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pin = _dev_ptr(inp, in_types, conv_in_elems(desc), "in")
+    pf = _dev_ptr(filt, in_types, conv_filt_elems(desc), "filt")
+    po = _dev_ptr(out, ("float32",), conv_out_elems(desc), "out")
+    pw, nbytes = _workspace_ptr(workspace, 0)
+    return int(lib.maxdnn_conv_fprop_ragged(ctypes.byref(desc), int(kind), pin, pf, po, pw, nbytes,
+                                            _stream_ptr(stream)))
+
+
+def conv_fprop_ragged(desc: ConvDesc, inp, filt, out, workspace, kind: int = KERNEL_FP32,
+                      stream=None) -> None:
+    """maxdnn_conv_fprop_ragged: FPROP for any Nb / No, through zero-padded staging tensors."""
+    _check(fprop_ragged_status(desc, inp, filt, out, workspace, kind, stream),
+           "maxdnn_conv_fprop_ragged")
 
 
 def conv_bprop_data_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:

@@ -42,6 +42,29 @@ flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, in
   }
 }
 
+// Staging copies for shapes the bulk tensor copies cannot address (row pitches that are
+// not multiples of 16 bytes): dst[row][j] = src[row][j] for j < n, 0 for n <= j < n_pad
+// (pad_inner), and the reverse for results (unpad_inner drops the padding columns).
+template <typename T>
+__global__ void __launch_bounds__(256)
+pad_inner_kernel(const T* __restrict__ src, T* __restrict__ dst, size_t rows, int n, int n_pad) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * (size_t)n_pad) return;
+  const size_t row = i / (size_t)n_pad;
+  const int j = (int)(i - row * (size_t)n_pad);
+  dst[i] = j < n ? src[row * (size_t)n + j] : T(0);
+}
+
+__global__ void __launch_bounds__(256)
+unpad_inner_kernel(const float* __restrict__ src, float* __restrict__ dst, size_t rows, int n,
+                   int n_pad) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * (size_t)n) return;
+  const size_t row = i / (size_t)n;
+  const int j = (int)(i - row * (size_t)n);
+  dst[i] = src[row * (size_t)n_pad + j];
+}
+
 constexpr int kWgThreads = 256;               // 8 warps: 16 x 16 threads, 8 x 8 results each (stride 16)
 constexpr uint32_t kWgOperandBytes = 128 * 128;   // 128 rows x 32 floats
 

@@ -433,6 +433,97 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, const float* in, const 
 }
 
 // ---------------------------------------------------------------------------
+// FPROP through zero-padded staging tensors (shapes outside the 16-byte row rule).
+// ---------------------------------------------------------------------------
+struct RaggedPlan {
+  maxdnn_conv_desc padded;
+  bool direct;                        // the shape needs no padding
+  size_t in_bytes, filt_bytes, out_bytes;   // staging tensors, each rounded up to 256 bytes
+};
+
+size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+maxdnn_status plan_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, RaggedPlan* p) {
+  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  int32_t Ho, Wo;
+  const maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  const int nb_mult = kind == MAXDNN_KERNEL_FP32 ? 4 : (kind == MAXDNN_KERNEL_TF32 ? 32 : 64);
+  const int no_mult = kind == MAXDNN_KERNEL_FP32 ? 4 : 32;
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  p->padded = *desc;
+  p->padded.Nb = align_up(desc->Nb, nb_mult);
+  p->padded.No = align_up(desc->No, no_mult);
+  p->direct = p->padded.Nb == desc->Nb && p->padded.No == desc->No;
+  p->in_bytes = round256((size_t)desc->Nc * desc->Hi * desc->Wi * p->padded.Nb * eb);
+  p->filt_bytes = round256((size_t)desc->Nc * desc->Sk * desc->Sk * p->padded.No * eb);
+  p->out_bytes = round256((size_t)p->padded.No * Ho * Wo * p->padded.Nb * 4);
+  return MAXDNN_OK;
+}
+
+template <typename T>
+maxdnn_status launch_pad(const void* src, void* dst, size_t rows, int n, int n_pad,
+                         cudaStream_t stream) {
+  const size_t total = rows * (size_t)n_pad;
+  pad_inner_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+      static_cast<const T*>(src), static_cast<T*>(dst), rows, n, n_pad);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
+maxdnn_status fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* in,
+                           const void* filt, float* out, void* ws, size_t ws_bytes,
+                           cudaStream_t stream) {
+  RaggedPlan p;
+  maxdnn_status st = plan_ragged(desc, kind, &p);
+  if (st != MAXDNN_OK) return st;
+  const int eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  if (p.direct) {
+    if (kind == MAXDNN_KERNEL_FP32)
+      return fprop_fp32(desc, static_cast<const float*>(in), static_cast<const float*>(filt), out, stream);
+    return fprop_umma(desc, eb, in, filt, out, stream);
+  }
+  if (!in || !filt || !out || !ws) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(ws) || ws_bytes < p.in_bytes + p.filt_bytes + p.out_bytes) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  st = dgrad_plan_check(p.padded, kind, ds->sm_count);   // the padded problem must have a plan
+  if (st != MAXDNN_OK) return st;
+  int32_t Ho, Wo;
+  check_desc(desc, &Ho, &Wo);
+  uint8_t* w_in = static_cast<uint8_t*>(ws);
+  uint8_t* w_filt = w_in + p.in_bytes;
+  float* w_out = reinterpret_cast<float*>(w_filt + p.filt_bytes);
+  const size_t in_rows = (size_t)desc->Nc * desc->Hi * desc->Wi;
+  const size_t f_rows = (size_t)desc->Nc * desc->Sk * desc->Sk;
+  if (eb == 2) {
+    st = launch_pad<uint16_t>(in, w_in, in_rows, desc->Nb, p.padded.Nb, stream);
+    if (st == MAXDNN_OK) st = launch_pad<uint16_t>(filt, w_filt, f_rows, desc->No, p.padded.No, stream);
+  } else {
+    st = launch_pad<float>(in, w_in, in_rows, desc->Nb, p.padded.Nb, stream);
+    if (st == MAXDNN_OK) st = launch_pad<float>(filt, w_filt, f_rows, desc->No, p.padded.No, stream);
+  }
+  if (st != MAXDNN_OK) return st;
+  if (kind == MAXDNN_KERNEL_FP32)
+    st = fprop_fp32(&p.padded, reinterpret_cast<const float*>(w_in),
+                    reinterpret_cast<const float*>(w_filt), w_out, stream);
+  else
+    st = fprop_umma(&p.padded, eb, w_in, w_filt, w_out, stream);
+  if (st != MAXDNN_OK) return st;
+  // out[o][y][x][n] for o < No, n < Nb: the first No filter slabs, padding images dropped
+  const size_t out_rows = (size_t)desc->No * Ho * Wo;
+  const size_t total = out_rows * (size_t)desc->Nb;
+  unpad_inner_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(w_out, out, out_rows,
+                                                                         desc->Nb, p.padded.Nb);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
+// ---------------------------------------------------------------------------
 // Allocation-free fp32 entry point.  The status block its kernel reports into
 // lives in this file-scope device array instead of cudaMalloc'd memory.  Every
 // device that loads the library carries these 256 bytes until the process ends.
@@ -656,6 +747,24 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
     return MAXDNN_CUDA_ERROR;
   }
   return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,
+                                                 maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!bytes) return MAXDNN_INVALID_VALUE;
+  RaggedPlan p;
+  const maxdnn_status st = plan_ragged(desc, kind, &p);
+  if (st != MAXDNN_OK) return st;
+  *bytes = p.direct ? 0 : p.in_bytes + p.filt_bytes + p.out_bytes;
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                       const void* in, const void* filt, float* out,
+                                       void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream) {
+  return fprop_ragged(desc, kind, in, filt, out, workspace, workspace_bytes,
+                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,

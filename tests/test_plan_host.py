@@ -193,3 +193,18 @@ def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     with pytest.raises(mx.MaxdnnError) as e:
         mx.conv_bprop_filter_workspace(mx.ConvDesc.make(30, 16, 16, 8, 8, 3, 1, 1, 1.0))   # Nb % 4
     assert e.value.status == mx.NOT_SUPPORTED
+
+
+def test_ragged_workspace_sizes():
+    """Staging tensors of the relaxed-boundary entry point: Nb and No rounded up to what the
+    kernel of each kind needs, each tensor rounded to 256 bytes; nothing for aligned shapes."""
+    r256 = lambda b: (b + 255) // 256 * 256
+    d = mx.ConvDesc.make(30, 14, 9, 16, 50, 3, 1, 1, 1.0)
+    Ho, Wo = 9, 14
+    assert mx.conv_fprop_ragged_workspace(d, mx.KERNEL_FP32) == \
+        r256(16 * 9 * 14 * 32 * 4) + r256(16 * 9 * 52 * 4) + r256(52 * Ho * Wo * 32 * 4)
+    assert mx.conv_fprop_ragged_workspace(d, mx.KERNEL_BF16) == \
+        r256(16 * 9 * 14 * 64 * 2) + r256(16 * 9 * 64 * 2) + r256(64 * Ho * Wo * 64 * 4)
+    assert mx.conv_fprop_ragged_workspace(mx.ConvDesc.make(32, 14, 9, 16, 64, 3, 1, 1, 1.0)) == 0
+    assert mx.conv_fprop_ragged_workspace(mx.ConvDesc.make(32, 14, 9, 16, 64, 3, 1, 1, 1.0),
+                                          mx.KERNEL_BF16) > 0          # bf16 wants 64 images
