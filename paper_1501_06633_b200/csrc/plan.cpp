@@ -173,7 +173,8 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
 }
 
 static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
-                                  int force_kc, bool pair, ConvGeom* g, KStepTable* t) {
+                                  int force_kc, bool pair, int max_cols, ConvGeom* g,
+                                  KStepTable* t) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -189,8 +190,6 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
 
   // Columns of a tile: tile_px adjacent pixels x tile_n images <= 256 (the MMA's N).
-  int max_cols = 256;
-  if (const char* e = getenv("MAXDNN_UMMA_COLS")) { const int v = atoi(e); if (v >= 32 && v <= 256 && v % 32 == 0) max_cols = v; }
   int best_nn = atom, best_T = 1;
   double best_eff = -1.0;
   for (int nn = (d.Nb < max_cols ? d.Nb : max_cols) / atom * atom; nn >= atom; nn -= atom) {
@@ -315,24 +314,50 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
 
 maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
                         int force_pair, ConvGeom* g, KStepTable* t) {
-  if (force_pair != 0) return plan_umma_as(d, elem_bytes, sm_count, force_kc, force_pair > 0, g, t);
-  const maxdnn_status st = plan_umma_as(d, elem_bytes, sm_count, force_kc, false, g, t);
-  if (st != MAXDNN_OK) return st;
-  // Two-SM tiles when they pay: a pair's tile (twice the work of a one-SM tile on twice
-  // the SMs) takes about 0.9 of the one-SM tile's time where the steps are long enough
-  // (at least four MMAs each), so compare the waves of tiles each plan needs.
-  static thread_local ConvGeom g2;
-  static thread_local KStepTable t2;
-  if (plan_umma_as(d, elem_bytes, sm_count, force_kc, true, &g2, &t2) != MAXDNN_OK) return st;
-  const int mmas_per_step = g2.kwc * (g2.kc / (32 / elem_bytes));
-  const double one = (double)ceil_div(g->n_tiles, sm_count);
-  const double two = 0.9 * (double)ceil_div(g2.n_tiles, sm_count / 2);
-  const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);   // in every tile
-  if (mmas_per_step >= 4 && peer_has_filters && two < one) {
-    *g = g2;
-    *t = t2;
+  // Candidates: tiles of at most 256 / 192 / 128 columns, on one SM or on a pair.  A
+  // tile's time goes with (columns + 128) — the 128 filter rows are staged whatever the
+  // columns — and a pair's tile (twice the work on twice the SMs) takes about 0.9 of
+  // that where its steps are long enough (at least four MMAs each); the plan that
+  // needs the least (waves of tiles) x (tile time) wins; a narrower tile has to win by 5 %.
+  // (Measured: the 13 x 13 Alexnet layers gain 14-24 % from 192-column tiles, the 5 x 5
+  // and long-K 3 x 3 layers 5-20 % from pairs.)  MAXDNN_UMMA_COLS / the pair argument
+  // pin a choice.
+  int cols_list[3] = {256, 192, 128};
+  int n_cols = 3;
+  if (const char* e = getenv("MAXDNN_UMMA_COLS")) {
+    const int v = atoi(e);
+    if (v >= 32 && v <= 256 && v % 32 == 0) { cols_list[0] = v; n_cols = 1; }
   }
-  return MAXDNN_OK;
+  static thread_local ConvGeom gc;
+  static thread_local KStepTable tc;
+  maxdnn_status first = MAXDNN_NOT_SUPPORTED;
+  double best = 1e300;
+  bool have = false;
+  const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);   // in every tile
+  for (int ci = 0; ci < n_cols; ++ci) {
+    for (int pair = 0; pair < 2; ++pair) {
+      if ((force_pair > 0 && !pair) || (force_pair < 0 && pair)) continue;
+      const maxdnn_status st = plan_umma_as(d, elem_bytes, sm_count, force_kc, pair != 0,
+                                            cols_list[ci], &gc, &tc);
+      if (ci == 0 && pair == (force_pair > 0 ? 1 : 0)) first = st;
+      if (st != MAXDNN_OK) continue;
+      if (pair && force_pair == 0) {
+        const int mmas_per_step = gc.kwc * (gc.kc / (32 / elem_bytes));
+        if (mmas_per_step < 4 || !peer_has_filters) continue;
+      }
+      const int units = pair ? sm_count / 2 : sm_count;
+      const double cost = (double)ceil_div(gc.n_tiles, units) * (gc.tile_px * gc.tile_n + 128) *
+                          (pair ? 0.9 : 1.0);
+      // a narrower tile must promise at least 5 % (its steps carry fewer MMAs)
+      if (!have || cost < (ci == 0 ? best - 1e-9 : 0.95 * best)) {
+        best = cost;
+        have = true;
+        *g = gc;
+        *t = tc;
+      }
+    }
+  }
+  return have ? MAXDNN_OK : first;
 }
 
 maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* f) {
