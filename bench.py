@@ -289,8 +289,6 @@ def run_ours(args):
     kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}[args.kernel]
     d = mx.ConvDesc.make(*w.dims)
     op = args.op
-    if op == "wgrad" and args.kernel != "fp32":
-        raise SystemExit("the filter gradient is built in fp32 only")
     nbytes, Ho, Wo = workload_bytes(w, args.kernel, op)
     C = mx.conv_flops(d)          # the same bilinear form: all three operations cost C
     assert C == flops(w, Ho, Wo)
@@ -324,7 +322,8 @@ def run_ours(args):
     if op == "dgrad":
         ws = torch.empty(mx.conv_bprop_data_workspace(d, kind), dtype=torch.uint8, device="cuda")
     elif op == "wgrad":
-        ws = torch.empty(max(16, mx.conv_bprop_filter_workspace(d)), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(max(16, mx.conv_bprop_filter_workspace(d, kind)), dtype=torch.uint8,
+                         device="cuda")
     fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
              mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
 
@@ -335,7 +334,7 @@ def run_ours(args):
         elif op == "dgrad":
             mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws, kind)
         else:
-            mx.conv_bprop_filter(d, a, b, r, ws)
+            mx.conv_bprop_filter(d, as_op(a), as_op(b), r, ws, kind)
 
     def barrier():
         if world > 1:
@@ -384,7 +383,7 @@ def run_ours(args):
                 if op == "dgrad":
                     mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws_e2e[k], kind, stream=stream)
                 else:
-                    mx.conv_bprop_filter(d, a, b, r, ws_e2e[k], stream=stream)
+                    mx.conv_bprop_filter(d, as_op(a), as_op(b), r, ws_e2e[k], kind, stream=stream)
                 h_outs[k].copy_(r, non_blocking=True)
 
     ws_e2e = [ws, None if ws is None else torch.empty_like(ws)]

@@ -241,22 +241,27 @@ maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kern
  * what the matching fprop entry point refuses for the transposed problem
  * (its filter count is Nc).
  *
- * maxdnn_conv_bprop_filter: the gradient with respect to the filters in exact
- * fp32, as the GEMM dfilt[k][o] = sum_r patch[k][r] * dout[o][r] with the
- * reduction r over output pixels and images, split over CTAs whose partial
- * sums (in the workspace) are added in a fixed order, so the result does not
- * depend on scheduling.  NOT_SUPPORTED: Nb or No not a multiple of 4, Sk
- * larger than the map, the limits of maxdnn_conv_fprop.
+ * maxdnn_conv_bprop_filter: the gradient with respect to the filters as the GEMM
+ * dfilt[k][o] = sum_r patch[k][r] * dout[o][r] with the reduction r over output
+ * pixels and images, split over CTAs whose partial sums (in the workspace) are
+ * added in a fixed order, so the result does not depend on scheduling.  `kind`
+ * fp32: exact fp32 on the CUDA cores; tf32: the same fp32 buffers on the tensor
+ * cores; bf16: `in` and `dout` are bfloat16.  dfilt is fp32 for every kind.
+ * NOT_SUPPORTED: a row of images not a multiple of 16 bytes (Nb % 4 for fp32 /
+ * tf32, % 8 for bf16), No not a multiple of 4, Sk larger than the map, the
+ * limits of maxdnn_conv_fprop.
  */
 maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
                                                maxdnn_kernel_kind kind, size_t* bytes);
 maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
                                      const void* dout, const void* filt, float* din,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
-maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
-maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, const float* in,
-                                       const float* dout, float* dfilt, void* workspace,
-                                       size_t workspace_bytes, void* cuda_stream);
+maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
+                                                 maxdnn_kernel_kind kind, size_t* bytes);
+maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                       const void* in, const void* dout, float* dfilt,
+                                       void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream);
 
 /* Synchronises `cuda_stream`, then reads and clears the current device's
  * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside a

@@ -115,9 +115,10 @@ def load_library():
     lib.maxdnn_conv_bprop_data.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp,
                                            ctypes.c_size_t, vp]
     lib.maxdnn_conv_bprop_filter_workspace.restype = ctypes.c_int
-    lib.maxdnn_conv_bprop_filter_workspace.argtypes = [P(ConvDesc), P(ctypes.c_size_t)]
+    lib.maxdnn_conv_bprop_filter_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
     lib.maxdnn_conv_bprop_filter.restype = ctypes.c_int
-    lib.maxdnn_conv_bprop_filter.argtypes = [P(ConvDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.maxdnn_conv_bprop_filter.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp,
+                                             ctypes.c_size_t, vp]
     lib.maxdnn_last_device_status.restype = ctypes.c_int
     lib.maxdnn_last_device_status.argtypes = [vp]
     lib.maxdnn_launch_count.restype = ctypes.c_uint64
@@ -316,29 +317,32 @@ def conv_bprop_data(desc: ConvDesc, dout, filt, din, workspace, kind: int = KERN
            "maxdnn_conv_bprop_data")
 
 
-def conv_bprop_filter_workspace(desc: ConvDesc) -> int:
+def conv_bprop_filter_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:
     """Bytes of device scratch maxdnn_conv_bprop_filter needs (partial sums; may be 0)."""
     n = ctypes.c_size_t()
-    _check(int(load_library().maxdnn_conv_bprop_filter_workspace(ctypes.byref(desc),
+    _check(int(load_library().maxdnn_conv_bprop_filter_workspace(ctypes.byref(desc), int(kind),
                                                                  ctypes.byref(n))),
            "maxdnn_conv_bprop_filter_workspace")
     return int(n.value)
 
 
-def bprop_filter_status(desc: ConvDesc, inp, dout, dfilt, workspace, stream=None) -> int:
+def bprop_filter_status(desc: ConvDesc, inp, dout, dfilt, workspace, kind: int = KERNEL_FP32,
+                        stream=None) -> int:
     """Enqueue maxdnn_conv_bprop_filter on torch tensors; returns the raw status code."""
     lib = load_library()
-    pi = _dev_ptr(inp, ("float32",), conv_in_elems(desc), "in")
-    pg = _dev_ptr(dout, ("float32",), conv_out_elems(desc), "dout")
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pi = _dev_ptr(inp, in_types, conv_in_elems(desc), "in")
+    pg = _dev_ptr(dout, in_types, conv_out_elems(desc), "dout")
     pd = _dev_ptr(dfilt, ("float32",), conv_filt_elems(desc), "dfilt")
     pw, nbytes = _workspace_ptr(workspace, 0)
-    return int(lib.maxdnn_conv_bprop_filter(ctypes.byref(desc), pi, pg, pd, pw, nbytes,
+    return int(lib.maxdnn_conv_bprop_filter(ctypes.byref(desc), int(kind), pi, pg, pd, pw, nbytes,
                                             _stream_ptr(stream)))
 
 
-def conv_bprop_filter(desc: ConvDesc, inp, dout, dfilt, workspace, stream=None) -> None:
-    """maxdnn_conv_bprop_filter: gradient with respect to the filters, exact fp32."""
-    _check(bprop_filter_status(desc, inp, dout, dfilt, workspace, stream),
+def conv_bprop_filter(desc: ConvDesc, inp, dout, dfilt, workspace, kind: int = KERNEL_FP32,
+                      stream=None) -> None:
+    """maxdnn_conv_bprop_filter: gradient with respect to the filters (fp32 / tf32 / bf16)."""
+    _check(bprop_filter_status(desc, inp, dout, dfilt, workspace, kind, stream),
            "maxdnn_conv_bprop_filter")
 
 

@@ -86,8 +86,12 @@ struct WgradCursor {
   __device__ __forceinline__ void start(const WgradGeom& g, int it) {
     item = it;
     if (it >= g.n_items) return;
-    int t = it;
-    split = t % g.splits; t /= g.splits;
+    // Items are ordered split-major: the CTAs that run at the same time work on the same
+    // range of output pixels for different tiles, so each slice of the two operands is
+    // fetched from HBM once and served to the other tiles' CTAs by L2.
+    const int tiles = g.n_items / g.splits;
+    split = it / tiles;
+    int t = it - split * tiles;
     ob = t % g.o_blocks; t /= g.o_blocks;
     cb = t % g.c_blocks;
     khb = t / g.c_blocks;

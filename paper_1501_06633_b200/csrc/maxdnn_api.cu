@@ -12,6 +12,7 @@
 #include "plan.h"
 #include "umma_conv.cuh"
 #include "umma_pair_conv.cuh"
+#include "wgrad_umma.cuh"
 
 namespace maxdnn {
 namespace {
@@ -26,6 +27,7 @@ struct DeviceState {
   bool ffma_attr[16] = {};
   bool umma_attr[4] = {false, false, false, false};
   bool wgrad_attr = false;
+  bool wgrad_umma_attr[2] = {false, false};
 };
 
 std::mutex g_mu;
@@ -368,9 +370,10 @@ maxdnn_status bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, 
   return fprop_umma(&fd, (int)eb, dout, ws, din, stream);
 }
 
-maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, const float* in, const float* dout,
-                           float* dfilt, void* ws, size_t ws_bytes, cudaStream_t stream) {
-  if (!desc) return MAXDNN_INVALID_VALUE;
+maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* in,
+                           const void* dout, float* dfilt, void* ws, size_t ws_bytes,
+                           cudaStream_t stream) {
+  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
   maxdnn_status st = check_desc(desc, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
   if (!in || !dout || !dfilt) return MAXDNN_INVALID_VALUE;
@@ -380,46 +383,72 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, const float* in, const 
   st = device_state(&ds);
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
-  static thread_local WgradArgs args;
-  st = plan_wgrad(*desc, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &args.g);
+  const bool tensor = kind != MAXDNN_KERNEL_FP32;
+  const bool bf16 = kind == MAXDNN_KERNEL_BF16;
+  const int eb = bf16 ? 2 : 4;
+  static thread_local WgradArgs fargs;
+  static thread_local WgradUmmaArgs uargs;
+  WgradGeom& g = tensor ? uargs.g : fargs.g;
+  st = plan_wgrad(*desc, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
   if (st != MAXDNN_OK) return st;
-  const WgradGeom& g = args.g;
   const size_t kno = (size_t)g.Nc * g.Sk * g.Sk * g.No;
   const size_t need = g.splits > 1 ? (size_t)g.splits * kno * 4 : 0;
   if (need > 0 && (!ws || ws_bytes < need)) return MAXDNN_INVALID_VALUE;
-  args.dfilt = dfilt;
-  args.partial = static_cast<float*>(ws);
-  args.status = ds->status;
+  const CUtensorMapDataType dt =
+      bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  const uint32_t chunk = 128u / (uint32_t)eb;     // images per reduction step = one 128-byte row
   CUtensorMap mg, mi;
   {
-    // output gradient as (n, x, y, o): one box = 32 images of one pixel x the tile's filters
+    // output gradient as (n, x, y, o): one box = 128 bytes of images of one pixel x the tile's filters
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
-                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
-    const uint32_t box[4] = {32u, 1u, 1u, (uint32_t)g.box_o};
-    st = encode_map(&mg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, dout, dims, str, box,
-                    CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint64_t str[3] = {(uint64_t)g.Nb * eb, (uint64_t)g.Wo * g.Nb * eb,
+                             (uint64_t)g.Ho * g.Wo * g.Nb * eb};
+    const uint32_t box[4] = {chunk, 1u, 1u, (uint32_t)g.box_o};
+    st = encode_map(&mg, dt, 4, dout, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
   }
   {
-    // maps as (n, w, h, c): one box = 32 images of a bh x bw window of pixels x bc channels
+    // maps as (n, w, h, c): one box = 128 bytes of images of a bh x bw window of pixels x bc channels
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
-                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
-    const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
-    st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
-                    CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint64_t str[3] = {(uint64_t)g.Nb * eb, (uint64_t)g.Wi * g.Nb * eb,
+                             (uint64_t)g.Hi * g.Wi * g.Nb * eb};
+    const uint32_t box[4] = {chunk, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
+    st = encode_map(&mi, dt, 4, in, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
   }
-  if (!ds->wgrad_attr) {
-    if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024) != cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
+  if (!tensor) {
+    fargs.dfilt = dfilt;
+    fargs.partial = static_cast<float*>(ws);
+    fargs.status = ds->status;
+    if (!ds->wgrad_attr) {
+      if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               227 * 1024) != cudaSuccess) {
+        cudaGetLastError();
+        return MAXDNN_CUDA_ERROR;
+      }
+      ds->wgrad_attr = true;
     }
-    ds->wgrad_attr = true;
+    wgrad_kernel<<<g.grid, kWgThreads, g.smem_bytes, stream>>>(mg, mi, fargs);
+  } else {
+    uargs.dfilt = dfilt;
+    uargs.partial = static_cast<float*>(ws);
+    uargs.status = ds->status;
+    uargs.atom = chunk;
+    const uint32_t fmt = bf16 ? 1u : 2u;
+    const uint32_t n_mma = (uint32_t)align_up(g.rows, 16);
+    uargs.idesc = (1u << 4) | (fmt << 7) | (fmt << 10)      // fp32 accumulate, operand formats;
+                  | ((n_mma >> 3) << 17) | ((128u >> 4) << 24);   // both operands K-major; N, M
+    auto kern = bf16 ? wgrad_umma_kernel<true> : wgrad_umma_kernel<false>;
+    if (!ds->wgrad_umma_attr[bf16 ? 1 : 0]) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+          cudaSuccess) {
+        cudaGetLastError();
+        return MAXDNN_CUDA_ERROR;
+      }
+      ds->wgrad_umma_attr[bf16 ? 1 : 0] = true;
+    }
+    kern<<<g.grid, kWgUmmaThreads, g.smem_bytes, stream>>>(mg, mi, uargs);
   }
-  wgrad_kernel<<<g.grid, kWgThreads, g.smem_bytes, stream>>>(mg, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (g.splits > 1) {
@@ -784,8 +813,9 @@ maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel
                     static_cast<cudaStream_t>(cuda_stream));
 }
 
-maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
-  if (!desc || !bytes) return MAXDNN_INVALID_VALUE;
+maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
+                                                 maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!desc || !bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
   int sm_count = env_int("MAXDNN_SM_COUNT");   // planning without a device (tests)
   if (sm_count <= 0) {
     DeviceState* ds = nullptr;
@@ -794,16 +824,18 @@ maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc, s
     sm_count = ds->sm_count;
   }
   WgradGeom g;
-  const maxdnn_status st = plan_wgrad(*desc, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
+  const int eb = kind == MAXDNN_KERNEL_FP32 ? 0 : (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
+  const maxdnn_status st = plan_wgrad(*desc, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
   if (st != MAXDNN_OK) return st;
   *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Sk * g.Sk * g.No * 4 : 0;
   return MAXDNN_OK;
 }
 
-maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, const float* in,
-                                       const float* dout, float* dfilt, void* workspace,
-                                       size_t workspace_bytes, void* cuda_stream) {
-  return bprop_filter(desc, in, dout, dfilt, workspace, workspace_bytes,
+maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                       const void* in, const void* dout, float* dfilt,
+                                       void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream) {
+  return bprop_filter(desc, kind, in, dout, dfilt, workspace, workspace_bytes,
                       static_cast<cudaStream_t>(cuda_stream));
 }
 

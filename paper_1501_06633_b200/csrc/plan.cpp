@@ -371,29 +371,36 @@ maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* f) {
   return MAXDNN_OK;
 }
 
-maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int sm_count, int force_splits, WgradGeom* g) {
+maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
+                         WgradGeom* g) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
-  st = common_limits(d, 4);
+  if (elem_bytes != 0 && elem_bytes != 4 && elem_bytes != 2) return MAXDNN_INVALID_VALUE;
+  const bool tensor = elem_bytes != 0;
+  const int eb = tensor ? elem_bytes : 4;
+  const int max_rows = tensor ? 256 : 128;
+  const int chunk = 128 / eb;                                         // images per reduction step
+  st = common_limits(d, eb);
   if (st != MAXDNN_OK) return st;
   if (!g || sm_count <= 0) return MAXDNN_INVALID_VALUE;
-  if (d.Nb % 4 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule
+  if ((d.Nb * eb) % 16 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule
   if (d.Sk > d.Wi || d.Sk > d.Hi) return MAXDNN_NOT_SUPPORTED;       // a copy box must fit the map
   memset(g, 0, sizeof(*g));
   g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
   g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
   g->bw = d.Sk;
-  g->bh = d.Sk < 128 / g->bw ? d.Sk : 128 / g->bw;
+  g->bh = d.Sk < max_rows / g->bw ? d.Sk : max_rows / g->bw;
   if (g->bh < 1) return MAXDNN_NOT_SUPPORTED;
-  g->bc = 128 / (g->bw * g->bh);
+  g->bc = max_rows / (g->bw * g->bh);
+  if (g->bc > 256) g->bc = 256;                                       // a copy box has at most 256 per axis
   if (g->bc > d.Nc) g->bc = d.Nc;
   g->rows = g->bc * g->bh * g->bw;
   g->box_o = d.No < 128 ? d.No : 128;
   g->c_blocks = ceil_div(d.Nc, g->bc);
   g->kh_blocks = ceil_div(d.Sk, g->bh);
   g->o_blocks = ceil_div(d.No, 128);
-  g->n_chunks = ceil_div(d.Nb, 32);
+  g->n_chunks = ceil_div(d.Nb, chunk);
   const int64_t r_steps = (int64_t)Ho * Wo * g->n_chunks;
   const int64_t tiles = (int64_t)g->c_blocks * g->kh_blocks * g->o_blocks;
   if (r_steps > 0x3fffffff || tiles > 0x3fffffff) return MAXDNN_NOT_SUPPORTED;
@@ -420,8 +427,8 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int sm_count, int force_spli
   const int64_t items = tiles * g->splits;
   if (items > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_items = (int32_t)items;
-  g->stages = 6;
-  g->smem_bytes = g->stages * 2 * 128 * 128 + 1024 + 256;
+  g->stages = tensor ? 4 : 6;
+  g->smem_bytes = g->stages * (128 + max_rows) * 128 + 1024 + 1024 + (tensor ? 2048 : 0);   // ring, alignment slack, barriers, row table
   g->grid = g->n_items < sm_count ? g->n_items : sm_count;
   return MAXDNN_OK;
 }

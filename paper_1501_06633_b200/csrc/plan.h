@@ -94,6 +94,9 @@ struct WgradGeom {
 };
 
 // force_splits > 0 pins the number of reduction splits (tests, ablations).
-maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int sm_count, int force_splits, WgradGeom* g);
+// elem_bytes 0: the fp32 FFMA2 kernel (128 gradient rows per tile, 32 images per step);
+// 4 / 2: the tensor-core kernel with TF32 / BF16 operands (256 rows; 32 / 64 images).
+maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
+                         WgradGeom* g);
 
 }  // namespace maxdnn

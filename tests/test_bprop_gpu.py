@@ -112,6 +112,35 @@ def test_bprop_filter(shape, splits, monkeypatch):
     assert rel_err(got, ref) <= 1e-5
 
 
+WGRAD_TC_SHAPES = WGRAD_SHAPES + [
+    (64, 14, 9, 40, 96, 3, 1, 1, 1.0),        # 28 channels x 9 taps = 252 rows per tile, two blocks
+    (128, 9, 7, 24, 64, 5, 1, 2, 0.5),        # 10 channels x 25 taps
+    (64, 8, 8, 300, 64, 1, 1, 0, 2.0),        # 1x1: 256 channels per tile, ragged second block
+]
+
+
+@pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+@pytest.mark.parametrize("splits", [0, 2])
+@pytest.mark.parametrize("shape", WGRAD_TC_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_filter_tensor_cores(shape, splits, kernel, monkeypatch):
+    if kernel == "bf16" and shape[0] % 8:
+        pytest.skip("a row of bf16 images must be a multiple of 16 bytes")
+    if splits:
+        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+    w, inp, filt, dout = make(shape, 2600 + shape[5])
+    d = mx.ConvDesc.make(*w.dims)
+    need = mx.conv_bprop_filter_workspace(d, KIND[kernel])
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    dfilt = torch.full((mx.conv_filt_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_filter(d, dev(inp, kernel), dev(dout, kernel), dfilt, ws, KIND[kernel])
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_filter(rounded(inp, kernel), rounded(dout, kernel), w.Sk,
+                                   stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = dfilt.cpu().numpy().reshape(ref.shape)
+    assert np.all(np.isfinite(got))
+    assert rel_err(got, ref) <= TOL[kernel]
+
+
 def test_bprop_filter_is_reproducible():
     """Partial sums are added in a fixed order: two runs agree bit for bit."""
     w, inp, filt, dout = make((64, 14, 9, 20, 96, 3, 1, 1, 1.0), 77)

@@ -188,6 +188,7 @@ def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     assert need % kno == 0 and 2 <= need // kno <= 64          # 40 tiles: the reduction is split
     big = mx.ConvDesc.make(128, 12, 12, 1024, 1024, 3, 1, 1, 1.0)   # 592 tiles: 4 whole waves
     assert mx.conv_bprop_filter_workspace(big) == 0
+    assert mx.conv_bprop_filter_workspace(d, mx.KERNEL_BF16) % kno == 0     # 10 channels x 25 taps per tile
     monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", "5")
     assert mx.conv_bprop_filter_workspace(d) == 5 * kno
     with pytest.raises(mx.MaxdnnError) as e:
