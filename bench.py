@@ -264,6 +264,15 @@ def shard_inputs(w, rank):
     return wl.make_inputs(w, seed_offset=rank)
 
 
+def sum_gradient_over_ranks(t, world):
+    """The one data-path collective of the sharded job: the filter gradient of a minibatch
+    split over ranks is the sum of the ranks' filter gradients (in place, all ranks)."""
+    import torch.distributed as dist
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t
+
+
 def whole_job_tflops(flops_per_rank, world, ms_step):
     return world * flops_per_rank / (ms_step * 1e-3) / 1e12
 
@@ -294,8 +303,8 @@ def run_ours(args):
     assert C == flops(w, Ho, Wo)
 
     # Each rank holds its own batch shard (same recipe, its own seed); neither FPROP nor
-    # the map gradient needs an exchange between shards (the filter gradient of a sharded
-    # batch would need a sum over ranks, which this benchmark does not time).  Buffer
+    # the map gradient needs an exchange between shards; the filter gradient of a sharded
+    # batch is summed over ranks (all-reduce, inside the timed step).  Buffer
     # sets are rotated so that no step finds its operands in L2.
     inp, filt = shard_inputs(w, rank)
     dout = wl.make_dout(w, seed_offset=rank) if op != "fprop" else None
@@ -335,6 +344,7 @@ def run_ours(args):
             mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws, kind)
         else:
             mx.conv_bprop_filter(d, as_op(a), as_op(b), r, ws, kind)
+            sum_gradient_over_ranks(r, world)      # NCCL all-reduce over the batch shards
 
     def barrier():
         if world > 1:
@@ -441,7 +451,9 @@ def run_ours(args):
                 "Nc": w.Nc, "No": w.No, "Sk": w.Sk, "stride": w.stride, "pad": w.pad,
                 "alpha": w.alpha, "flops_per_step": C, "algorithmic_bytes_per_step": nbytes,
                 "l2": "rotating %d buffer sets (%.0f MB) > L2 (126 MB)" % (n_sets, n_sets * nbytes / 1e6),
-                "parallelism": "batch shards, no collective" if world > 1 else "single GPU",
+                "parallelism": ("single GPU" if world == 1 else
+                                "batch shards, filter gradient all-reduced" if op == "wgrad" else
+                                "batch shards, no collective"),
             },
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps, "streams": 2,

@@ -1,6 +1,6 @@
 """The N > 1 path of bench.py on CPU: two gloo ranks exercise the launcher
 environment parsing, the per-rank batch shards (no data-path collective: FPROP
-has no exchange step), the max-over-ranks timing reduction and the whole-job
+has no exchange step; the filter gradient's sum over ranks is the one exception), the max-over-ranks timing reduction and the whole-job
 throughput; and the reference arm under a 2-rank launcher prints exactly one line."""
 import json
 import os
@@ -26,6 +26,9 @@ def _worker(rank, world, port, q):
     inp, filt = bench.shard_inputs(w, rank)
     # each rank "measures" a different time; everyone must end up with the slowest
     ms_total, e2e_ms = bench.max_over_ranks([10.0 + rank, 100.0 - rank], "cpu", world)
+    import torch
+    grad = bench.sum_gradient_over_ranks(torch.full((5,), float(rank + 1)), world)
+    assert bool((grad == 3.0).all())               # 1 + 2: every rank holds the summed gradient
     dist.barrier()
     q.put((rank, float(inp.sum()), float(filt.sum()), ms_total, e2e_ms))
     dist.destroy_process_group()
