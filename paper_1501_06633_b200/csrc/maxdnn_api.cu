@@ -285,7 +285,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
     const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Nc, (uint64_t)g.Sk, (uint64_t)g.Sk};
     const uint64_t str[3] = {(uint64_t)g.Sk * g.Sk * g.No * eb, (uint64_t)g.No * eb,
                              (uint64_t)g.Sk * g.No * eb};
-    const uint32_t box[4] = {atom, (uint32_t)g.kc, (uint32_t)g.kwc, 1u};
+    const uint32_t box[4] = {atom, (uint32_t)g.box_c, (uint32_t)g.box_kw, (uint32_t)g.box_kh};
     st = encode_map(&mf, dt, 4, filt, dims, str, box, op_swz);
     if (st != MAXDNN_OK) return st;
   }
@@ -296,8 +296,8 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
                               (uint64_t)g.Hi};
     const uint64_t str[4] = {(uint64_t)g.Hi * g.Wi * g.Nb * eb, 128u, (uint64_t)g.Nb * eb,
                              (uint64_t)g.Wi * g.Nb * eb};
-    const uint32_t box[5] = {atom, (uint32_t)g.kc, (uint32_t)g.cta_n / atom, (uint32_t)g.b_box_w,
-                             1u};
+    const uint32_t box[5] = {atom, (uint32_t)g.box_c, (uint32_t)g.cta_n / atom, (uint32_t)g.b_box_w,
+                             (uint32_t)g.box_kh};
     st = encode_map(&mi, dt, 5, in, dims, str, box, op_swz);
     if (st != MAXDNN_OK) return st;
   }

@@ -199,6 +199,22 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
                        ((double)ceil_div(d.Nb, nn) * ceil_div(Wo, T) * (double)max_cols);
     if (eff > best_eff + 1e-9) { best_eff = eff; best_nn = nn; best_T = T; }
   }
+  // Few-channel layers (Nc below the MMA's K: the 3-channel first layers): a K step per
+  // tap would be mostly zero padding (3 of 16 rows), so the filter COLUMNS are merged
+  // into the K dimension.  One box of box_kw pixels x box_c channels per output pixel and
+  // filter row lands as box_kw * box_c consecutive K rows, the filter box in the same
+  // (kw, c) order; box_c >= Nc and box_kw >= Sk are rounded up so that the row count is
+  // a multiple of the MMA's K, the surplus rows being out-of-bounds zeros in the filter
+  // operand (c >= Nc in both, kw >= Sk in the filter box).  11 x 11 x 3: 33 of 48 rows
+  // carry data instead of 3 of 16.  Needs one 128-byte group of images per tile column
+  // group, so the tile is 256 / atom pixels x atom images.
+  const int umma_k0 = 32 / elem_bytes;
+  const bool merged = d.Nc < umma_k0 && d.Sk > 1 && !pair && force_kc == 0 &&
+                      !(getenv("MAXDNN_UMMA_MERGE") && atoi(getenv("MAXDNN_UMMA_MERGE")) < 0);
+  if (merged) {
+    best_nn = atom;
+    best_T = max_cols / atom < Wo ? max_cols / atom : Wo;
+  }
   g->tile_n = best_nn;
   g->tile_px = best_T;
   g->n_chunks = ceil_div(d.Nb, best_nn);
@@ -272,14 +288,39 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   }
   if (force_kc > 0 && force_kc % umma_k == 0 && force_kc <= 256) kc = force_kc;
   int n = 0;
-  build_table(d, kc, kwc, t, &n);
+  if (merged) {
+    const int box_c = align_up(d.Nc, 4);
+    int box_kw = d.Sk;
+    while ((box_kw * box_c) % umma_k != 0) ++box_kw;
+    const int rows1 = box_kw * box_c;                     // K rows of one filter row
+    int khc = 1;   // filter rows per step: stages of at most 40 KB (a deep ring beat longer steps)
+    while (khc < d.Sk && (128 + cols) * rows1 * (khc + 1) * elem_bytes <= 40 * 1024) ++khc;
+    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Sk) khc = v; }
+    if (box_kw > 256 || rows1 * khc > 1024) return MAXDNN_NOT_SUPPORTED;
+    kc = rows1 * khc;
+    kwc = 1;
+    for (int kh = 0; kh < d.Sk; kh += khc) {
+      if (n >= kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
+      t->s[n].c0 = 0; t->s[n].kh = (int8_t)kh; t->s[n].kw0 = 0;
+      ++n;
+    }
+    g->box_c = box_c; g->box_kw = box_kw; g->box_kh = khc;
+  } else {
+    build_table(d, kc, kwc, t, &n);
+    g->box_c = kc; g->box_kw = kwc; g->box_kh = 1;
+  }
   if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
   g->kc = kc; g->kwc = kwc; g->rows = kc * kwc; g->n_ksteps = n;
 
   g->a_box_bytes = atom * kc * kwc * elem_bytes;        // one group of filters: kwc x kc rows x 128 B
   g->a_stage_bytes = 128 * kc * kwc * elem_bytes;
   const int strip = px_cta + kwc - 1;
-  if (kwc > 1) {
+  if (merged) {
+    g->b_boxes = px_cta;                                // one window per output pixel
+    g->b_box_w = g->box_kw;
+    g->b_box_bytes = g->cta_n * kc * elem_bytes;
+    g->b_stage_bytes = px_cta * g->b_box_bytes;
+  } else if (kwc > 1) {
     g->b_boxes = 1;
     g->b_box_w = strip;
     g->b_box_bytes = strip * g->cta_n * kc * elem_bytes;

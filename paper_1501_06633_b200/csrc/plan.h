@@ -21,6 +21,7 @@ struct ConvGeom {
   int32_t tile_px;    // adjacent output pixels (x) per tile
   int32_t tile_n;     // images per tile
   int32_t kc, kwc;    // channels / filter columns per K step
+  int32_t box_c, box_kw, box_kh;   // tensor kernels: extents of the copy boxes along c, kw (w), kh (h)
   int32_t rows;       // patch rows per K step = kc * kwc
   int32_t n_ksteps;
   int32_t stages;

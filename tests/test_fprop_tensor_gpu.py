@@ -175,6 +175,34 @@ def test_table1_layer_shapes(kernel, name):
 
 
 @pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+@pytest.mark.parametrize("khc", [0, 2])
+@pytest.mark.parametrize("shape", [
+    (128, 47, 39, 3, 96, 11, 4, 0, 1.0),      # the first-layer shape: 12 columns x 4 channels = 48 K rows
+    (64, 23, 19, 3, 64, 11, 4, 2, 0.5),       # with padding: windows reach into the apron
+    (64, 14, 11, 1, 32, 3, 1, 1, 1.0),        # one channel, stride 1: overlapping windows per pixel
+    (64, 12, 9, 5, 160, 5, 2, 2, 1.0),        # 5 channels -> boxes of 8, stride 2
+    (128, 9, 9, 7, 32, 7, 1, 3, 1.0),         # 7 x 7 x 7
+    (64, 10, 8, 2, 32, 2, 1, 0, 1.0),         # 2 x 2 filter, 2 channels
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_few_channel_layers_merge_filter_columns_into_k(kernel, shape, khc, monkeypatch):
+    """Layers with fewer channels than the MMA's K take K steps that span all filter columns
+    (and khc filter rows) of a few channels; surplus K rows are out-of-bounds zeros."""
+    if khc:
+        monkeypatch.setenv("MAXDNN_UMMA_MERGE", str(khc))
+    Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha = shape
+    w = wl.Workload("merged", Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), 8800 + Sk)
+    d = mx.ConvDesc.make(*w.dims)
+    try:
+        info, _ = mx.conv_plan_query(d, KIND[kernel], 148)
+    except mx.MaxdnnError:
+        assert khc                       # only a forced step size may not fit shared memory
+        pytest.skip("two filter rows per step do not fit two stages for this shape")
+    assert info.kwc == 1 and info.kc >= Nc * Sk and info.n_ksteps <= Sk   # merged plan taken
+    check(kernel, w)
+
+
+@pytest.mark.parametrize("kernel", ["tf32", "bf16"])
 @pytest.mark.parametrize("shape", [
     (64, 14, 9, 128, 256, 3, 1, 1, 1.0),      # strip reuse, two tiles of 256 filters
     (128, 9, 7, 96, 256, 5, 1, 2, 1.0),       # the CTAs of the pair split the images
