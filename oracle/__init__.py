@@ -72,6 +72,11 @@ def _load():
                                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                 ctypes.c_int32, P(ctypes.c_double)]
         lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_conv2_out_dims.restype = ctypes.c_int
+        lib.oracle_conv2_out_dims.argtypes = [P(ConvDesc2), P(ctypes.c_int32), P(ctypes.c_int32)]
+        lib.oracle_conv2_fprop.restype = ctypes.c_int
+        lib.oracle_conv2_fprop.argtypes = [P(ConvDesc2), ctypes.c_void_p, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_int32]
         for name in ("oracle_conv_bprop_data", "oracle_conv_bprop_filter"):
             fn = getattr(lib, name)
             fn.restype = ctypes.c_int
@@ -84,6 +89,14 @@ def _load():
                            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, P(ctypes.c_double)]
         _lib = lib
     return _lib
+
+
+class ConvDesc2(ctypes.Structure):
+    """Per-axis filter size, stride and padding (w before h, as in the C struct)."""
+
+    _fields_ = [(n, ctypes.c_int32) for n in ("Nb", "Wi", "Hi", "Nc", "No", "Skw", "Skh",
+                                              "stride_w", "stride_h", "pad_w", "pad_h")] + \
+               [("alpha", ctypes.c_float)]
 
 
 def _desc(Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha) -> ConvDesc:
@@ -147,6 +160,28 @@ def conv_fprop_point(inp, filt, o, y, x, n, *, stride=1, pad=0, alpha=1.0):
     v = _load().oracle_conv_fprop_point(ctypes.byref(d), inp.ctypes.data, filt.ctypes.data,
                                         int(o), int(y), int(x), int(n), ctypes.byref(a))
     return float(v), float(a.value)
+
+
+def conv2_fprop(inp, filt, *, stride=(1, 1), pad=(0, 0), alpha=1.0, nthreads=0):
+    """out[No,Ho,Wo,Nb] from in[Nc,Hi,Wi,Nb] and filt[Nc,Skh,Skw,No] with per-axis
+    ``stride=(stride_h, stride_w)`` and ``pad=(pad_h, pad_w)``."""
+    inp = np.ascontiguousarray(inp, dtype=np.float32)
+    filt = np.ascontiguousarray(filt, dtype=np.float32)
+    Nc, Hi, Wi, Nb = inp.shape
+    Nc2, Skh, Skw, No = filt.shape
+    if Nc2 != Nc:
+        raise ValueError("filter bank does not match the maps")
+    d = ConvDesc2(Nb, Wi, Hi, Nc, No, Skw, Skh, int(stride[1]), int(stride[0]), int(pad[1]),
+                  int(pad[0]), float(alpha))
+    ho, wo = ctypes.c_int32(), ctypes.c_int32()
+    if _load().oracle_conv2_out_dims(ctypes.byref(d), ctypes.byref(ho), ctypes.byref(wo)):
+        raise ValueError("invalid convolution descriptor")
+    out = np.zeros((No, ho.value, wo.value, Nb), dtype=np.float32)
+    rc = _load().oracle_conv2_fprop(ctypes.byref(d), inp.ctypes.data, filt.ctypes.data,
+                                    out.ctypes.data, int(nthreads))
+    if rc:
+        raise RuntimeError("oracle_conv2_fprop failed (%d)" % rc)
+    return out
 
 
 def conv_bprop_data(dout, filt, in_hw, *, stride=1, pad=0, alpha=1.0, nthreads=0):

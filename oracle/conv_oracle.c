@@ -169,3 +169,81 @@ int oracle_num_threads(void) {
   return 1;
 #endif
 }
+
+/*
+ * The same operation with per-axis filter size, stride and padding (Section 2 states one
+ * square size, one stride and one padding; this is the plain generalisation of its sum,
+ * used to check the library's relaxed-boundary entry point):
+ *
+ *   out[o,y,x,n] = alpha * sum_{c,kh,kw} filt[c,kh,kw,o]
+ *                    * in0[c, y*stride_h - pad_h + kh, x*stride_w - pad_w + kw, n]
+ *
+ * kh < Skh, kw < Skw; filt is [Nc][Skh][Skw][No]; Ho = floor((Hi + 2 pad_h - Skh)/stride_h) + 1,
+ * Wo likewise with the w quantities.  Same arithmetic as above.
+ */
+typedef struct oracle_conv_desc2 {
+  int32_t Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w, stride_h, pad_w, pad_h;
+  float alpha;
+} oracle_conv_desc2;
+
+int oracle_conv2_out_dims(const oracle_conv_desc2* d, int32_t* Ho, int32_t* Wo) {
+  if (!d || d->Nb <= 0 || d->Wi <= 0 || d->Hi <= 0 || d->Nc <= 0 || d->No <= 0 || d->Skw <= 0 ||
+      d->Skh <= 0 || d->stride_w <= 0 || d->stride_h <= 0 || d->pad_w < 0 || d->pad_h < 0)
+    return 1;
+  int ho = out_dim(d->Hi, d->pad_h, d->Skh, d->stride_h);
+  int wo = out_dim(d->Wi, d->pad_w, d->Skw, d->stride_w);
+  if (ho <= 0 || wo <= 0) return 1;
+  if (Ho) *Ho = ho;
+  if (Wo) *Wo = wo;
+  return 0;
+}
+
+int oracle_conv2_fprop(const oracle_conv_desc2* d, const float* in, const float* filt, float* out,
+                       int32_t nthreads) {
+  int32_t Ho, Wo;
+  if (!in || !filt || !out || oracle_conv2_out_dims(d, &Ho, &Wo)) return 1;
+  const int Nb = d->Nb, Wi = d->Wi, Hi = d->Hi, Nc = d->Nc, No = d->No;
+  const int Skw = d->Skw, Skh = d->Skh;
+  const double alpha = (double)d->alpha;
+  int bad_alloc = 0;
+#ifdef _OPENMP
+  if (nthreads > 0) omp_set_num_threads(nthreads);
+#else
+  (void)nthreads;
+#endif
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)Nb);
+    if (!s) {
+#pragma omp atomic write
+      bad_alloc = 1;
+    }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+    for (int o = 0; o < No; ++o) {
+      for (int y = 0; y < Ho; ++y) {
+        if (!s) continue;
+        for (int x = 0; x < Wo; ++x) {
+          for (int n = 0; n < Nb; ++n) s[n] = 0.0;
+          for (int c = 0; c < Nc; ++c) {
+            for (int kh = 0; kh < Skh; ++kh) {
+              const int h = y * d->stride_h - d->pad_h + kh;
+              if (h < 0 || h >= Hi) continue;
+              for (int kw = 0; kw < Skw; ++kw) {
+                const int w = x * d->stride_w - d->pad_w + kw;
+                if (w < 0 || w >= Wi) continue;
+                const double f =
+                    (double)filt[(((size_t)c * Skh + kh) * Skw + kw) * (size_t)No + o];
+                const float* px = in + (((size_t)c * Hi + h) * Wi + w) * (size_t)Nb;
+                for (int n = 0; n < Nb; ++n) s[n] += f * (double)px[n];
+              }
+            }
+          }
+          float* dst = out + (((size_t)o * Ho + y) * Wo + x) * (size_t)Nb;
+          for (int n = 0; n < Nb; ++n) dst[n] = (float)(alpha * s[n]);
+        }
+      }
+    }
+    free(s);
+  }
+  return bad_alloc;
+}

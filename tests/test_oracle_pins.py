@@ -306,3 +306,58 @@ def test_bf16_and_tf32_helpers():
     np.testing.assert_array_equal(b, ref)
     t = wl.truncate_to_tf32(a)
     assert np.all(np.abs(t) <= np.abs(a)) and np.all(np.abs(t - a) <= np.abs(a) * 2.0 ** -10)
+
+
+# ----------------------------------------------------------------------------
+# per-axis filter size / stride / padding (the relaxed-boundary generalisation)
+# ----------------------------------------------------------------------------
+def brute_force2(inp, filt, stride, pad, alpha):
+    """The sum with separate h / w quantities, index maps by hand, python floats."""
+    Nc, Hi, Wi, Nb = inp.shape
+    _, Skh, Skw, No = filt.shape
+    (sh, sw), (ph, pw) = stride, pad
+    Ho = (Hi + 2 * ph - Skh) // sh + 1
+    Wo = (Wi + 2 * pw - Skw) // sw + 1
+    fin = [float(v) for v in inp.reshape(-1)]
+    ff = [float(v) for v in filt.reshape(-1)]
+    out = np.zeros(No * Ho * Wo * Nb, dtype=np.float64)
+    for o in range(No):
+        for y in range(Ho):
+            for x in range(Wo):
+                for n in range(Nb):
+                    s = 0.0
+                    for c in range(Nc):
+                        for kh in range(Skh):
+                            for kw in range(Skw):
+                                h = y * sh - ph + kh
+                                w = x * sw - pw + kw
+                                if 0 <= h < Hi and 0 <= w < Wi:
+                                    s += (ff[((c * Skh + kh) * Skw + kw) * No + o]
+                                          * fin[((c * Hi + h) * Wi + w) * Nb + n])
+                    out[((o * Ho + y) * Wo + x) * Nb + n] = alpha * s
+    return out.reshape(No, Ho, Wo, Nb)
+
+
+RECT_SHAPES = [
+    # Nb Wi Hi Nc No Skw Skh (sh, sw) (ph, pw) alpha
+    (2, 7, 5, 2, 3, 3, 1, (1, 1), (0, 1), 1.0),        # 1 x 3 row filter
+    (2, 6, 8, 1, 2, 2, 5, (2, 1), (2, 0), 0.5),        # 5 x 2, stride 2 down only
+    (1, 9, 7, 2, 2, 4, 3, (1, 3), (1, 2), -1.5),
+    (3, 5, 5, 2, 2, 3, 3, (2, 2), (1, 1), 1.0),        # square: must equal the square oracle
+]
+
+
+@pytest.mark.parametrize("shape", RECT_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_per_axis_oracle_matches_brute_force_and_library(shape):
+    Nb, Wi, Hi, Nc, No, Skw, Skh, stride, pad, alpha = shape
+    rng = np.random.default_rng(31 + Skw * 7 + Skh)
+    inp = rng.uniform(-1, 1, size=(Nc, Hi, Wi, Nb)).astype(np.float32)
+    filt = rng.uniform(-1, 1, size=(Nc, Skh, Skw, No)).astype(np.float32)
+    got = oracle.conv2_fprop(inp, filt, stride=stride, pad=pad, alpha=alpha)
+    assert close(got, brute_force2(inp, filt, stride, pad, alpha), 2 * F32_ROUND)
+    x = torch.from_numpy(inp).double().permute(3, 0, 1, 2)
+    w = torch.from_numpy(filt).double().permute(3, 0, 1, 2)
+    lib = (alpha * torch.nn.functional.conv2d(x, w, stride=stride, padding=pad)).permute(1, 2, 3, 0).numpy()
+    assert close(got, lib, 2 * F32_ROUND)
+    if Skw == Skh and stride[0] == stride[1] and pad[0] == pad[1]:
+        np.testing.assert_array_equal(got, oracle.conv_fprop(inp, filt, stride=stride[0], pad=pad[0], alpha=alpha))
