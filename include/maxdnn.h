@@ -218,6 +218,27 @@ maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kern
                                        void* cuda_stream);
 
 /*
+ * FPROP with per-axis filter size, stride and padding (Section 2 states one square filter
+ * size, one stride and one padding; this lifts that restriction for the same kernels):
+ *
+ *   out[o,y,x,n] = alpha * sum_{c,kh,kw} filt[c,kh,kw,o]
+ *                    * in0[c, y*stride_h - pad_h + kh, x*stride_w - pad_w + kw, n]
+ *
+ * with kh < Skh, kw < Skw, filt laid out [Nc][Skh][Skw][No], Ho = floor((Hi + 2 pad_h -
+ * Skh)/stride_h) + 1 and Wo likewise with the w quantities.  `kind` selects the kernel as
+ * in the entry points above (bf16: in and filt are bfloat16); same conventions, limits and
+ * NOT_SUPPORTED cases, with Sk read as max(Skw, Skh).
+ */
+typedef struct maxdnn_conv_desc2 {
+  int32_t Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w, stride_h, pad_w, pad_h;
+  float alpha;
+} maxdnn_conv_desc2;
+
+maxdnn_status maxdnn_conv2_out_dims(const maxdnn_conv_desc2* desc, int32_t* Ho, int32_t* Wo);
+maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                 const void* in, const void* filt, float* out, void* cuda_stream);
+
+/*
  * Backward propagation.  The paper builds FPROP only and names BPROP (Abstract,
  * Section 3.5 "Conclusion") as the operation its techniques should carry over to, without
  * defining it; these entry points compute the two exact adjoints of the

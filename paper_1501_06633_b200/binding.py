@@ -17,6 +17,7 @@ __all__ = [
     "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
     "last_device_status",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
+    "ConvDesc2", "conv2_out_dims", "conv2_fprop", "conv2_fprop_status",
     "conv_fprop_ragged_workspace", "conv_fprop_ragged", "fprop_ragged_status",
     "conv_bprop_data_workspace", "conv_bprop_data", "bprop_data_status",
     "conv_bprop_filter_workspace", "conv_bprop_filter", "bprop_filter_status",
@@ -33,6 +34,7 @@ EXPORTED_SYMBOLS = [
     "maxdnn_launch_count", "maxdnn_conv_bprop_data_workspace", "maxdnn_conv_bprop_data",
     "maxdnn_conv_bprop_filter_workspace", "maxdnn_conv_bprop_filter",
     "maxdnn_conv_fprop_ragged_workspace", "maxdnn_conv_fprop_ragged",
+    "maxdnn_conv2_out_dims", "maxdnn_conv2_fprop",
 ]
 
 
@@ -55,6 +57,20 @@ class ConvDesc(ctypes.Structure):
     def make(cls, Nb, Wi, Hi, Nc, No, Sk, stride=1, pad=0, alpha=1.0) -> "ConvDesc":
         return cls(int(Nb), int(Wi), int(Hi), int(Nc), int(No), int(Sk), int(stride), int(pad),
                    float(alpha))
+
+
+class ConvDesc2(ctypes.Structure):
+    """maxdnn_conv_desc2: per-axis filter size, stride and padding (w before h)."""
+
+    _fields_ = [(n, ctypes.c_int32) for n in ("Nb", "Wi", "Hi", "Nc", "No", "Skw", "Skh",
+                                              "stride_w", "stride_h", "pad_w", "pad_h")] + \
+               [("alpha", ctypes.c_float)]
+
+    @classmethod
+    def make(cls, Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w=1, stride_h=1, pad_w=0, pad_h=0,
+             alpha=1.0) -> "ConvDesc2":
+        return cls(int(Nb), int(Wi), int(Hi), int(Nc), int(No), int(Skw), int(Skh), int(stride_w),
+                   int(stride_h), int(pad_w), int(pad_h), float(alpha))
 
 
 class KStep(ctypes.Structure):
@@ -104,6 +120,10 @@ def load_library():
         getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_host.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.maxdnn_conv2_out_dims.restype = ctypes.c_int
+    lib.maxdnn_conv2_out_dims.argtypes = [P(ConvDesc2), P(ctypes.c_int32), P(ctypes.c_int32)]
+    lib.maxdnn_conv2_fprop.restype = ctypes.c_int
+    lib.maxdnn_conv2_fprop.argtypes = [P(ConvDesc2), ctypes.c_int, vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_ragged_workspace.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_ragged_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
     lib.maxdnn_conv_fprop_ragged.restype = ctypes.c_int
@@ -257,6 +277,30 @@ def _workspace_ptr(workspace, need):
     if not (isinstance(workspace, torch.Tensor) and workspace.is_cuda and workspace.is_contiguous()):
         raise TypeError("workspace must be a contiguous CUDA tensor")
     return ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def conv2_out_dims(desc: ConvDesc2):
+    ho, wo = ctypes.c_int32(), ctypes.c_int32()
+    _check(int(load_library().maxdnn_conv2_out_dims(ctypes.byref(desc), ctypes.byref(ho),
+                                                     ctypes.byref(wo))), "maxdnn_conv2_out_dims")
+    return ho.value, wo.value
+
+
+def conv2_fprop_status(desc: ConvDesc2, inp, filt, out, kind: int = KERNEL_FP32, stream=None) -> int:
+    """Enqueue maxdnn_conv2_fprop on torch tensors; returns the raw status code."""
+    lib = load_library()
+    Ho, Wo = conv2_out_dims(desc)
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pin = _dev_ptr(inp, in_types, desc.Nc * desc.Hi * desc.Wi * desc.Nb, "in")
+    pf = _dev_ptr(filt, in_types, desc.Nc * desc.Skh * desc.Skw * desc.No, "filt")
+    po = _dev_ptr(out, ("float32",), desc.No * Ho * Wo * desc.Nb, "out")
+    return int(lib.maxdnn_conv2_fprop(ctypes.byref(desc), int(kind), pin, pf, po,
+                                      _stream_ptr(stream)))
+
+
+def conv2_fprop(desc: ConvDesc2, inp, filt, out, kind: int = KERNEL_FP32, stream=None) -> None:
+    """maxdnn_conv2_fprop: FPROP with per-axis filter size, stride and padding."""
+    _check(conv2_fprop_status(desc, inp, filt, out, kind, stream), "maxdnn_conv2_fprop")
 
 
 def conv_fprop_ragged_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:

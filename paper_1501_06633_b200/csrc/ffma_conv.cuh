@@ -124,8 +124,8 @@ struct FfmaProducer {
     const int y = r / g.x_runs;
     o0 = ob * mt;
     n0 = nch * g.tile_n;
-    h0 = y * g.stride - g.pad;
-    w0 = xr * g.tile_px * g.stride - g.pad;
+    h0 = y * g.stride_h - g.pad_h;
+    w0 = xr * g.tile_px * g.stride_w - g.pad_w;
   }
 
   __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
@@ -156,7 +156,7 @@ struct FfmaProducer {
     for (int t = 0; t < g.b_boxes; ++t) {
       tma_load_4d(dst, map_in, fb, n0, w, h0 + ks.kh, ks.c0);
       dst += g.b_slot_bytes;
-      w += g.stride;
+      w += g.stride_w;
     }
     if (++stage == g.stages) { stage = 0; phase ^= 1u; }
     if (++step == g.n_ksteps) {

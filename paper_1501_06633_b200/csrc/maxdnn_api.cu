@@ -134,10 +134,10 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   return MAXDNN_NOT_SUPPORTED;
 }
 
-maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const float* filt,
-                         float* out, cudaStream_t stream) {
+maxdnn_status fprop_fp32(const ConvDims& dims, const float* in, const float* filt, float* out,
+                         cudaStream_t stream) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  maxdnn_status st = check_dims(dims, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
@@ -147,7 +147,7 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
-  st = plan_ffma(*desc, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
+  st = plan_ffma(dims, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
                  &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   args.out = out;
@@ -158,9 +158,9 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   CUtensorMap mf, mi;
   {
     // filter bank as (o, kw, kh, c)
-    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Sk, (uint64_t)g.Sk, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Sk * g.No * 4,
-                             (uint64_t)g.Sk * g.Sk * g.No * 4};
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Skh, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skw * g.No * 4,
+                             (uint64_t)g.Skh * g.Skw * g.No * 4};
     const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
     st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -177,6 +177,12 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
     if (st != MAXDNN_OK) return st;
   }
   return dispatch_ffma(ds, mf, mi, args, stream);
+}
+
+maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                         float* out, cudaStream_t stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return fprop_fp32(dims_from(*desc), in, filt, out, stream);
 }
 
 template <bool BF16>
@@ -231,10 +237,10 @@ maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensor
   return MAXDNN_OK;
 }
 
-maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const void* in,
-                         const void* filt, float* out, cudaStream_t stream) {
+maxdnn_status fprop_umma(const ConvDims& dims, int elem_bytes, const void* in, const void* filt,
+                         float* out, cudaStream_t stream) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  maxdnn_status st = check_dims(dims, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
@@ -244,7 +250,7 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local UmmaArgs args;
-  st = plan_umma(*desc, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
+  st = plan_umma(dims, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
                  env_int("MAXDNN_UMMA_PAIR"), &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   const ConvGeom& g = args.g;
@@ -282,9 +288,9 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
   CUtensorMap mf, mi, mo;
   {
     // filter bank as (o, c, kw, kh); one box = 128 bytes of filters x kc channels of a tap
-    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Nc, (uint64_t)g.Sk, (uint64_t)g.Sk};
-    const uint64_t str[3] = {(uint64_t)g.Sk * g.Sk * g.No * eb, (uint64_t)g.No * eb,
-                             (uint64_t)g.Sk * g.No * eb};
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Nc, (uint64_t)g.Skw, (uint64_t)g.Skh};
+    const uint64_t str[3] = {(uint64_t)g.Skh * g.Skw * g.No * eb, (uint64_t)g.No * eb,
+                             (uint64_t)g.Skw * g.No * eb};
     const uint32_t box[4] = {atom, (uint32_t)g.box_c, (uint32_t)g.box_kw, (uint32_t)g.box_kh};
     st = encode_map(&mf, dt, 4, filt, dims, str, box, op_swz);
     if (st != MAXDNN_OK) return st;
@@ -318,6 +324,12 @@ maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const voi
               : launch_umma<false>(ds, mf, mi, mo, args, stream);
 }
 
+maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const void* in,
+                         const void* filt, float* out, cudaStream_t stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return fprop_umma(dims_from(*desc), elem_bytes, in, filt, out, stream);
+}
+
 // ---------------------------------------------------------------------------
 // Backward propagation.
 // ---------------------------------------------------------------------------
@@ -330,8 +342,8 @@ maxdnn_status dgrad_plan_check(const maxdnn_conv_desc& fd, maxdnn_kernel_kind ki
   static thread_local ConvGeom g;
   static thread_local KStepTable t;
   if (kind == MAXDNN_KERNEL_FP32)
-    return plan_ffma(fd, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
-  return plan_umma(fd, kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
+    return plan_ffma(dims_from(fd), sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
+  return plan_umma(dims_from(fd), kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
                    env_int("MAXDNN_UMMA_PAIR"), &g, &t);
 }
 
@@ -619,7 +631,7 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;
-  st = plan_ffma(*desc, ds->sm_count, 0, 0, &args.g, &args.table);
+  st = plan_ffma(dims_from(*desc), ds->sm_count, 0, 0, &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
   args.out = out;
@@ -629,9 +641,9 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
 
   CUtensorMap mf, mi;
   {
-    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Sk, (uint64_t)g.Sk, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Sk * g.No * 4,
-                             (uint64_t)g.Sk * g.Sk * g.No * 4};
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Skh, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skw * g.No * 4,
+                             (uint64_t)g.Skh * g.Skw * g.No * 4};
     const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
     st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -716,10 +728,10 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   static thread_local KStepTable t;
   switch (kind) {
     case MAXDNN_KERNEL_FP32:
-      st = plan_ffma(*desc, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
+      st = plan_ffma(dims_from(*desc), sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
       break;
-    case MAXDNN_KERNEL_TF32: st = plan_umma(*desc, 4, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
-    case MAXDNN_KERNEL_BF16: st = plan_umma(*desc, 2, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
+    case MAXDNN_KERNEL_TF32: st = plan_umma(dims_from(*desc), 4, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
+    case MAXDNN_KERNEL_BF16: st = plan_umma(dims_from(*desc), 2, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
     default: return MAXDNN_INVALID_VALUE;
   }
   if (st != MAXDNN_OK) return st;
@@ -776,6 +788,29 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
     return MAXDNN_CUDA_ERROR;
   }
   return MAXDNN_OK;
+}
+
+static maxdnn::ConvDims dims_from2(const maxdnn_conv_desc2& d) {
+  maxdnn::ConvDims c;
+  c.Nb = d.Nb; c.Wi = d.Wi; c.Hi = d.Hi; c.Nc = d.Nc; c.No = d.No;
+  c.Skw = d.Skw; c.Skh = d.Skh; c.stride_w = d.stride_w; c.stride_h = d.stride_h;
+  c.pad_w = d.pad_w; c.pad_h = d.pad_h; c.alpha = d.alpha;
+  return c;
+}
+
+maxdnn_status maxdnn_conv2_out_dims(const maxdnn_conv_desc2* desc, int32_t* Ho, int32_t* Wo) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return check_dims(dims_from2(*desc), Ho, Wo);
+}
+
+maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                 const void* in, const void* filt, float* out, void* cuda_stream) {
+  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (kind == MAXDNN_KERNEL_FP32)
+    return fprop_fp32(dims_from2(*desc), static_cast<const float*>(in),
+                      static_cast<const float*>(filt), out, stream);
+  return fprop_umma(dims_from2(*desc), kind == MAXDNN_KERNEL_BF16 ? 2 : 4, in, filt, out, stream);
 }
 
 maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,

@@ -20,15 +20,44 @@ maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo) {
   return MAXDNN_OK;
 }
 
-static maxdnn_status common_limits(const maxdnn_conv_desc& d, int elem_bytes) {
-  if (d.Sk > 127 || d.Nc > 32767) return MAXDNN_NOT_SUPPORTED;
+ConvDims dims_from(const maxdnn_conv_desc& d) {
+  ConvDims c;
+  c.Nb = d.Nb; c.Wi = d.Wi; c.Hi = d.Hi; c.Nc = d.Nc; c.No = d.No;
+  c.Skw = c.Skh = d.Sk; c.stride_w = c.stride_h = d.stride; c.pad_w = c.pad_h = d.pad;
+  c.alpha = d.alpha;
+  return c;
+}
+
+maxdnn_status check_dims(const ConvDims& d, int32_t* Ho, int32_t* Wo) {
+  if (d.Nb <= 0 || d.Wi <= 0 || d.Hi <= 0 || d.Nc <= 0 || d.No <= 0 || d.Skw <= 0 || d.Skh <= 0 ||
+      d.stride_w <= 0 || d.stride_h <= 0 || d.pad_w < 0 || d.pad_h < 0)
+    return MAXDNN_INVALID_VALUE;
+  if (!isfinite(d.alpha)) return MAXDNN_INVALID_VALUE;
+  const int64_t span_h = (int64_t)d.Hi + 2 * (int64_t)d.pad_h - d.Skh;
+  const int64_t span_w = (int64_t)d.Wi + 2 * (int64_t)d.pad_w - d.Skw;
+  if (span_h < 0 || span_w < 0) return MAXDNN_INVALID_VALUE;
+  if (Ho) *Ho = (int32_t)(span_h / d.stride_h + 1);
+  if (Wo) *Wo = (int32_t)(span_w / d.stride_w + 1);
+  return MAXDNN_OK;
+}
+
+static maxdnn_status common_limits(const ConvDims& d, int elem_bytes) {
+  if (d.Skw > 127 || d.Skh > 127 || d.Nc > 32767) return MAXDNN_NOT_SUPPORTED;
   // Row pitches of the tensor-copy descriptors are 32-bit-safe byte counts here.
   const int64_t plane = (int64_t)d.Hi * d.Wi * d.Nb * elem_bytes;
-  const int64_t frow = (int64_t)d.Sk * d.Sk * d.No * elem_bytes;
+  const int64_t frow = (int64_t)d.Skh * d.Skw * d.No * elem_bytes;
   if (plane >= ((int64_t)1 << 40) || frow >= ((int64_t)1 << 40)) return MAXDNN_NOT_SUPPORTED;
   const int64_t out_elems = (int64_t)d.No * d.Nb;
   if (out_elems <= 0) return MAXDNN_INVALID_VALUE;
   return MAXDNN_OK;
+}
+
+// Copies the problem into the geometry the kernels read.
+static void fill_geom(const ConvDims& d, int32_t Ho, int32_t Wo, ConvGeom* g) {
+  memset(g, 0, sizeof(*g));
+  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No;
+  g->Skw = d.Skw; g->Skh = d.Skh; g->stride_w = d.stride_w; g->stride_h = d.stride_h;
+  g->pad_w = d.pad_w; g->pad_h = d.pad_h; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
 }
 
 // Tile shapes the fp32 kernel is built for, with the relative cost per
@@ -40,10 +69,10 @@ static const FfmaShape kFfmaShapes[] = {
     {96, 256, 1.12},  {64, 128, 1.18},  {32, 128, 1.50},
 };
 
-static void build_table(const maxdnn_conv_desc& d, int kc, int kwc, KStepTable* t, int* n) {
+static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* n) {
   int k = 0;
-  for (int kh = 0; kh < d.Sk; ++kh)
-    for (int kw0 = 0; kw0 < d.Sk; kw0 += kwc)
+  for (int kh = 0; kh < d.Skh; ++kh)
+    for (int kw0 = 0; kw0 < d.Skw; kw0 += kwc)
       for (int c0 = 0; c0 < d.Nc; c0 += kc) {
         if (k < kMaxKSteps) {
           t->s[k].c0 = (int16_t)c0;
@@ -56,7 +85,7 @@ static void build_table(const maxdnn_conv_desc& d, int kc, int kwc, KStepTable* 
 }
 
 // Columns of a tile: tile_px adjacent output pixels x tile_n images <= cols.
-static double pick_columns(const maxdnn_conv_desc& d, int Wo, int cols, int* nn_out, int* T_out) {
+static double pick_columns(const ConvDims& d, int Wo, int cols, int* nn_out, int* T_out) {
   int best_nn = 4, best_T = 1;
   double best_eff = -1.0;
   for (int nn = (d.Nb < cols ? d.Nb : cols); nn >= 4; nn -= 4) {
@@ -71,18 +100,16 @@ static double pick_columns(const maxdnn_conv_desc& d, int Wo, int cols, int* nn_
   return best_eff;
 }
 
-maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, int force_cols,
+maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
                         ConvGeom* g, KStepTable* t) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   st = common_limits(d, 4);
   if (st != MAXDNN_OK) return st;
   if (d.Nb % 4 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;
   if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
-  memset(g, 0, sizeof(*g));
-  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
-  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+  fill_geom(d, Ho, Wo, g);
 
   // Tile shape: fewest SM-time units over whole waves of persistent CTAs.
   double best_t = 1e300;
@@ -128,8 +155,8 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
       if (padded < best_pad) { best_pad = padded; kc = c; }
     }
   } else {
-    kwc = d.Sk;
-    kc = 40 / d.Sk;
+    kwc = d.Skw;
+    kc = 40 / d.Skw;
     if (kc < 1) kc = 1;
     if (kc > d.Nc) kc = d.Nc;
   }
@@ -147,7 +174,7 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   // One box per stage whenever the tile's columns are one contiguous run of the map
   // (one pixel, or adjacent pixels of a stride-1 layer); else one box per pixel.
   g->fixed_pitch = (g->tile_px * g->tile_n == g->tile_cols &&
-                    (g->tile_px == 1 || (d.stride == 1 && kwc == 1))) ? 1 : 0;
+                    (g->tile_px == 1 || (d.stride_w == 1 && kwc == 1))) ? 1 : 0;
   if (g->fixed_pitch) {
     g->b_boxes = 1;
     g->b_box_w = g->tile_px > 1 ? g->tile_px : kwc;
@@ -172,11 +199,11 @@ maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_
   return MAXDNN_OK;
 }
 
-static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int sm_count,
+static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_count,
                                   int force_kc, bool pair, int max_cols, ConvGeom* g,
                                   KStepTable* t) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   st = common_limits(d, elem_bytes);
   if (st != MAXDNN_OK) return st;
@@ -185,9 +212,7 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   if (d.Nb % atom != 0) return MAXDNN_NOT_SUPPORTED;
   if (d.No % 32 != 0) return MAXDNN_NOT_SUPPORTED;
   if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
-  memset(g, 0, sizeof(*g));
-  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
-  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+  fill_geom(d, Ho, Wo, g);
 
   // Columns of a tile: tile_px adjacent pixels x tile_n images <= 256 (the MMA's N).
   int best_nn = atom, best_T = 1;
@@ -209,7 +234,7 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   // carry data instead of 3 of 16.  Needs one 128-byte group of images per tile column
   // group, so the tile is 256 / atom pixels x atom images.
   const int umma_k0 = 32 / elem_bytes;
-  const bool merged = d.Nc < umma_k0 && d.Sk > 1 && !pair && force_kc == 0 &&
+  const bool merged = d.Nc < umma_k0 && d.Skw > 1 && !pair && force_kc == 0 &&
                       !(getenv("MAXDNN_UMMA_MERGE") && atoi(getenv("MAXDNN_UMMA_MERGE")) < 0);
   if (merged) {
     best_nn = atom;
@@ -256,7 +281,7 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   // MMA's K (32 bytes of channel index: 8 for 4-byte, 16 for 2-byte elements).
   const int umma_k = 32 / elem_bytes;
   const int cols = px_cta * g->cta_n;                     // patch columns one CTA stages
-  int kwc = (d.stride == 1 && d.Sk > 1 && d.Sk <= 5 && force_kc >= 0) ? d.Sk : 1;
+  int kwc = (d.stride_w == 1 && d.Skw > 1 && d.Skw <= 5 && force_kc >= 0) ? d.Skw : 1;
   // A K step costs the issuing warps a fixed few hundred cycles, so a step should carry
   // many MMAs.  With the strip, a stage of up to 96 KB (two stages) pays off when it holds
   // at least 9 (bf16) / 12 (tf32) MMAs (measured on the 3x3 / 5x5 layers); otherwise one
@@ -290,16 +315,16 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   int n = 0;
   if (merged) {
     const int box_c = align_up(d.Nc, 4);
-    int box_kw = d.Sk;
+    int box_kw = d.Skw;
     while ((box_kw * box_c) % umma_k != 0) ++box_kw;
     const int rows1 = box_kw * box_c;                     // K rows of one filter row
     int khc = 1;   // filter rows per step: stages of at most 40 KB (a deep ring beat longer steps)
-    while (khc < d.Sk && (128 + cols) * rows1 * (khc + 1) * elem_bytes <= 40 * 1024) ++khc;
-    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Sk) khc = v; }
+    while (khc < d.Skh && (128 + cols) * rows1 * (khc + 1) * elem_bytes <= 40 * 1024) ++khc;
+    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Skh) khc = v; }
     if (box_kw > 256 || rows1 * khc > 1024) return MAXDNN_NOT_SUPPORTED;
     kc = rows1 * khc;
     kwc = 1;
-    for (int kh = 0; kh < d.Sk; kh += khc) {
+    for (int kh = 0; kh < d.Skh; kh += khc) {
       if (n >= kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
       t->s[n].c0 = 0; t->s[n].kh = (int8_t)kh; t->s[n].kw0 = 0;
       ++n;
@@ -325,7 +350,7 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
     g->b_box_w = strip;
     g->b_box_bytes = strip * g->cta_n * kc * elem_bytes;
     g->b_stage_bytes = g->b_box_bytes;
-  } else if (px_cta == 1 || d.stride == 1) {
+  } else if (px_cta == 1 || d.stride_w == 1) {
     g->b_boxes = 1;
     g->b_box_w = px_cta;
     g->b_box_bytes = cols * kc * elem_bytes;
@@ -353,7 +378,7 @@ static maxdnn_status plan_umma_as(const maxdnn_conv_desc& d, int elem_bytes, int
   return MAXDNN_OK;
 }
 
-maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
+maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int force_kc,
                         int force_pair, ConvGeom* g, KStepTable* t) {
   // Candidates: tiles of at most 256 / 192 / 128 columns, on one SM or on a pair.  A
   // tile's time goes with (columns + 128) — the 128 filter rows are staged whatever the
@@ -422,7 +447,7 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   const int eb = tensor ? elem_bytes : 4;
   const int max_rows = tensor ? 256 : 128;
   const int chunk = 128 / eb;                                         // images per reduction step
-  st = common_limits(d, eb);
+  st = common_limits(dims_from(d), eb);
   if (st != MAXDNN_OK) return st;
   if (!g || sm_count <= 0) return MAXDNN_INVALID_VALUE;
   if ((d.Nb * eb) % 16 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule

@@ -11,10 +11,20 @@ namespace maxdnn {
 
 constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel parameters
 
+// The operation with per-axis filter size, stride and padding (Section 2 has one of each:
+// the public square descriptor maps to Skw = Skh = Sk and so on).
+struct ConvDims {
+  int32_t Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w, stride_h, pad_w, pad_h;
+  float alpha;
+};
+
+ConvDims dims_from(const maxdnn_conv_desc& d);
+maxdnn_status check_dims(const ConvDims& d, int32_t* Ho, int32_t* Wo);
+
 // What a kernel needs to know about the problem and its tiling.  Passed by
 // value in kernel parameter space together with the K-step table.
 struct ConvGeom {
-  int32_t Nb, Wi, Hi, Nc, No, Sk, stride, pad;
+  int32_t Nb, Wi, Hi, Nc, No, Skw, stride_w, pad_w;   // the w-axis filter size, stride, padding
   int32_t Ho, Wo;
   float alpha;
   int32_t tile_m;     // filters per tile
@@ -42,6 +52,7 @@ struct ConvGeom {
   int32_t b_stage_bytes;   // patch bytes per stage
   int32_t grid;
   int32_t smem_bytes;
+  int32_t Skh, stride_h, pad_h;                       // the h-axis filter size, stride, padding
 };
 
 struct KStepTable {
@@ -54,12 +65,12 @@ inline int align_up(int a, int b) { return ceil_div(a, b) * b; }
 maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo);
 
 // FFMA kernel plan.  force_tile_m / force_cols > 0 pin the tile shape (ablations).
-maxdnn_status plan_ffma(const maxdnn_conv_desc& d, int sm_count, int force_tile_m, int force_cols,
+maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
                         ConvGeom* g, KStepTable* t);
 
 // Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
 // force_pair: 0 = choose, 1 = two-SM tiles (256 filters per CTA pair), -1 = one-SM tiles.
-maxdnn_status plan_umma(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_kc,
+maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int force_kc,
                         int force_pair, ConvGeom* g, KStepTable* t);
 
 // ---------------------------------------------------------------------------

@@ -247,8 +247,8 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int y = r / g.x_runs;
         const int o0 = ob * kUmmaM;
         const int na0 = (nch * g.tile_n) / (int)args.atom;
-        const int h0 = y * g.stride - g.pad;
-        const int w0 = xr * g.tile_px * g.stride - g.pad;
+        const int h0 = y * g.stride_h - g.pad_h;
+        const int w0 = xr * g.tile_px * g.stride_w - g.pad_w;
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
@@ -267,7 +267,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
               for (int t = 0; t < g.b_boxes; ++t) {
                 tma_load_5d_hint(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
-                w += g.stride;
+                w += g.stride_w;
               }
             } else {
               uint32_t dst = a_dst;

@@ -201,8 +201,8 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int o0 = ob * 2 * kUmmaM + (int)rank * kUmmaM;          // this CTA's 128 filters
         // this CTA's half of the tile's columns: half of the images or half of the pixels
         const int na0 = (nch * g.tile_n + (g.split_n ? (int)rank * g.cta_n : 0)) / (int)args.atom;
-        const int h0 = y * g.stride - g.pad;
-        const int w0 = (xr * g.tile_px + (g.split_n ? 0 : (int)rank * g.cta_px)) * g.stride - g.pad;
+        const int h0 = y * g.stride_h - g.pad_h;
+        const int w0 = (xr * g.tile_px + (g.split_n ? 0 : (int)rank * g.cta_px)) * g.stride_w - g.pad_w;
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
@@ -221,7 +221,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
               for (int t = 0; t < g.b_boxes; ++t) {
                 tma_load_5d_pair(dst, &map_in, fb, 0, ks.c0, na0, w, h0 + ks.kh, pol_last);
                 dst += g.b_slot_bytes;
-                w += g.stride;
+                w += g.stride_w;
               }
             } else {
               uint32_t dst = a_dst;
