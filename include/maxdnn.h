@@ -254,13 +254,17 @@ maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_ki
  * least the size the matching *_workspace call reports; may be NULL when that
  * size is 0); the library allocates nothing.  Results are overwritten in full.
  *
- * maxdnn_conv_bprop_data: the gradient with respect to the maps as an FPROP of
- * dout with the filter bank transposed (channels <-> filters) and flipped in
- * both axes (written into the workspace by a small kernel on the same stream)
- * and padding Sk-1-pad, on the kernel `kind` names (fp32; tf32; bf16: dout and
- * filt are bfloat16, din fp32).  NOT_SUPPORTED: stride != 1, pad > Sk-1, or
- * what the matching fprop entry point refuses for the transposed problem
- * (its filter count is Nc).
+ * maxdnn_conv_bprop_data: the gradient with respect to the maps on the kernel `kind`
+ * names (fp32; tf32; bf16: dout and filt are bfloat16, din fp32).  Stride 1: an FPROP
+ * of dout with the filter bank transposed (channels <-> filters) and flipped in both
+ * axes (written into the workspace by a small kernel on the same stream) and padding
+ * Sk-1-pad.  Stride s > 1: the map positions split into s x s classes by
+ * (h+pad) mod s, (w+pad) mod s; each class meets only the taps kh = rho_h + s j,
+ * kw = rho_w + s i and is, on its own grid, a stride-1 FPROP of dout with that
+ * sub-filter (flipped, transposed), whose dense result a copy kernel scatters onto
+ * the grid; positions no tap reaches are zero.  NOT_SUPPORTED: stride 1 with
+ * pad > Sk-1, Nb not a multiple of 4 (stride > 1), or what the matching fprop
+ * entry point refuses for the transposed problem (its filter count is Nc).
  *
  * maxdnn_conv_bprop_filter: the gradient with respect to the filters as the GEMM
  * dfilt[k][o] = sum_r patch[k][r] * dout[o][r] with the reduction r over output

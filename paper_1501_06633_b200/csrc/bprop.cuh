@@ -42,6 +42,42 @@ flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, in
   }
 }
 
+// Strided map gradient: the sub-filter of one class, flipped and transposed:
+//   ft[o][j'][i'][c] = filt[c][rho_h + s (Jh-1-j')][rho_w + s (Jw-1-i')][o]
+template <typename T>
+__global__ void __launch_bounds__(256)
+subfilter_flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int Sk,
+                                int No, int s, int rho_h, int rho_w, int Jh, int Jw) {
+  __shared__ T tile[32][33];
+  const int jp = blockIdx.z / Jw, ip = blockIdx.z % Jw;     // position in the transformed bank
+  const int kh = rho_h + s * (Jh - 1 - jp), kw = rho_w + s * (Jw - 1 - ip);
+  const int o0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int c = c0 + i, o = o0 + threadIdx.x;
+    if (c < Nc && o < No) tile[i][threadIdx.x] = filt[(((size_t)c * Sk + kh) * Sk + kw) * No + o];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int o = o0 + i, c = c0 + threadIdx.x;
+    if (c < Nc && o < No) ft[(((size_t)o * Jh + jp) * Jw + ip) * Nc + c] = tile[threadIdx.x][i];
+  }
+}
+
+// din[c][h_first + s a][w_first + s b][n] = sub[c][a][b][n]: the class's gradient onto its grid.
+__global__ void __launch_bounds__(256)
+dgrad_scatter_kernel(const float4* __restrict__ sub, float4* __restrict__ din, int Nc, int n_h,
+                     int n_w, int nb4, int Hi, int Wi, int s, int h_first, int w_first) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t total = (size_t)Nc * n_h * n_w * nb4;
+  if (i >= total) return;
+  size_t r = i;
+  const int n = (int)(r % nb4); r /= nb4;
+  const int b = (int)(r % n_w); r /= n_w;
+  const int a = (int)(r % n_h);
+  const int c = (int)(r / n_h);
+  din[(((size_t)c * Hi + h_first + s * a) * Wi + w_first + s * b) * nb4 + n] = sub[i];
+}
+
 // Staging copies for shapes the bulk tensor copies cannot address (row pitches that are
 // not multiples of 16 bytes): dst[row][j] = src[row][j] for j < n, 0 for n <= j < n_pad
 // (pad_inner), and the reverse for results (unpad_inner drops the padding columns).

@@ -89,6 +89,16 @@ maxdnn_status encode_map(CUtensorMap* m, CUtensorMapDataType dt, int rank, const
   return r == CUDA_SUCCESS ? MAXDNN_OK : MAXDNN_CUDA_ERROR;
 }
 
+// Element pitch of the rows / channels of the maps: the caller's, or dense.
+uint64_t dims_in_h(const ConvGeom& g, int64_t given) {
+  return given > 0 ? (uint64_t)given : (uint64_t)g.Wi * g.Nb;
+}
+uint64_t dims_in_c(const ConvGeom& g, int64_t given) {
+  return given > 0 ? (uint64_t)given : (uint64_t)g.Hi * g.Wi * g.Nb;
+}
+
+size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int env_int(const char* name) {
@@ -134,10 +144,10 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   return MAXDNN_NOT_SUPPORTED;
 }
 
-maxdnn_status fprop_fp32(const ConvDims& dims, const float* in, const float* filt, float* out,
+maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt, float* out,
                          cudaStream_t stream) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_dims(dims, &Ho, &Wo);
+  maxdnn_status st = check_dims(cd, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
@@ -147,7 +157,7 @@ maxdnn_status fprop_fp32(const ConvDims& dims, const float* in, const float* fil
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
-  st = plan_ffma(dims, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
+  st = plan_ffma(cd, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
                  &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   args.out = out;
@@ -169,8 +179,8 @@ maxdnn_status fprop_fp32(const ConvDims& dims, const float* in, const float* fil
   {
     // maps as (n, w, h, c)
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
-                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint64_t hs = dims_in_h(g, cd.in_h_stride), cs = dims_in_c(g, cd.in_c_stride);
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, hs * 4, cs * 4};
     const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -237,10 +247,10 @@ maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensor
   return MAXDNN_OK;
 }
 
-maxdnn_status fprop_umma(const ConvDims& dims, int elem_bytes, const void* in, const void* filt,
+maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, const void* filt,
                          float* out, cudaStream_t stream) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_dims(dims, &Ho, &Wo);
+  maxdnn_status st = check_dims(cd, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
@@ -250,7 +260,7 @@ maxdnn_status fprop_umma(const ConvDims& dims, int elem_bytes, const void* in, c
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local UmmaArgs args;
-  st = plan_umma(dims, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
+  st = plan_umma(cd, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
                  env_int("MAXDNN_UMMA_PAIR"), &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   const ConvGeom& g = args.g;
@@ -300,8 +310,8 @@ maxdnn_status fprop_umma(const ConvDims& dims, int elem_bytes, const void* in, c
     // [pixel][image group][channel][128 bytes of images]
     const uint64_t dims[5] = {atom, (uint64_t)g.Nc, (uint64_t)g.Nb / atom, (uint64_t)g.Wi,
                               (uint64_t)g.Hi};
-    const uint64_t str[4] = {(uint64_t)g.Hi * g.Wi * g.Nb * eb, 128u, (uint64_t)g.Nb * eb,
-                             (uint64_t)g.Wi * g.Nb * eb};
+    const uint64_t str[4] = {dims_in_c(g, cd.in_c_stride) * eb, 128u, (uint64_t)g.Nb * eb,
+                             dims_in_h(g, cd.in_h_stride) * eb};
     const uint32_t box[5] = {atom, (uint32_t)g.box_c, (uint32_t)g.cta_n / atom, (uint32_t)g.b_box_w,
                              (uint32_t)g.box_kh};
     st = encode_map(&mi, dt, 5, in, dims, str, box, op_swz);
@@ -347,16 +357,115 @@ maxdnn_status dgrad_plan_check(const maxdnn_conv_desc& fd, maxdnn_kernel_kind ki
                    env_int("MAXDNN_UMMA_PAIR"), &g, &t);
 }
 
+// Workspace of the strided map gradient: the largest transformed sub-filter bank and the
+// largest class's dense result, each rounded up to 256 bytes.
+struct DgradStridedPlan {
+  size_t ft_bytes, sub_bytes;
+};
+
+maxdnn_status plan_dgrad_strided(const maxdnn_conv_desc& d, size_t eb, DgradStridedPlan* p) {
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  const int s = d.stride;
+  size_t jmax = 0, nmax = 0;
+  for (int rh = 0; rh < s; ++rh)
+    for (int rw = 0; rw < s; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, d.Sk, s, d.pad, d.Hi), aw = dgrad_axis(rw, d.Sk, s, d.pad, d.Wi);
+      const size_t j = (size_t)ah.J * aw.J, n = (size_t)ah.n * aw.n;
+      if (j > jmax) jmax = j;
+      if (n > nmax) nmax = n;
+    }
+  p->ft_bytes = round256((size_t)d.No * jmax * d.Nc * eb);
+  p->sub_bytes = round256((size_t)d.Nc * nmax * d.Nb * 4);
+  return MAXDNN_OK;
+}
+
+maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
+                                 const void* dout, const void* filt, float* din, void* ws,
+                                 size_t ws_bytes, cudaStream_t stream) {
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  DgradStridedPlan p;
+  maxdnn_status st = plan_dgrad_strided(*desc, eb, &p);
+  if (st != MAXDNN_OK) return st;
+  if (ws_bytes < p.ft_bytes + p.sub_bytes) return MAXDNN_INVALID_VALUE;
+  if (desc->Nb % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  int32_t Ho, Wo;
+  check_desc(desc, &Ho, &Wo);
+  const int s = desc->stride;
+  uint8_t* w_ft = static_cast<uint8_t*>(ws);
+  float* w_sub = reinterpret_cast<float*>(w_ft + p.ft_bytes);
+  // Positions that no tap reaches (a class without taps, or whose window lies outside
+  // dout) keep the zeros written here.
+  if (cudaMemsetAsync(din, 0, (size_t)desc->Nc * desc->Hi * desc->Wi * desc->Nb * 4, stream) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  for (int rh = 0; rh < s; ++rh) {
+    for (int rw = 0; rw < s; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, desc->Sk, s, desc->pad, desc->Hi);
+      const DgradAxis aw = dgrad_axis(rw, desc->Sk, s, desc->pad, desc->Wi);
+      if (ah.J == 0 || aw.J == 0 || ah.n == 0 || aw.n == 0) continue;
+      if (ah.crop >= Ho || aw.crop >= Wo) continue;            // its windows miss dout entirely
+      ConvDims fd;
+      fd.Nb = desc->Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = desc->No;
+      fd.No = desc->Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
+      fd.pad_w = aw.pad; fd.pad_h = ah.pad; fd.alpha = desc->alpha;
+      fd.in_h_stride = (int64_t)Wo * desc->Nb;
+      fd.in_c_stride = (int64_t)Ho * Wo * desc->Nb;
+      fd.Ho_given = ah.n; fd.Wo_given = aw.n;
+      const dim3 grid((unsigned)ceil_div(desc->No, 32), (unsigned)ceil_div(desc->Nc, 32),
+                      (unsigned)(ah.J * aw.J));
+      const dim3 block(32, 8);
+      if (eb == 2)
+        subfilter_flip_transpose_kernel<uint16_t><<<grid, block, 0, stream>>>(
+            static_cast<const uint16_t*>(filt), reinterpret_cast<uint16_t*>(w_ft), desc->Nc,
+            desc->Sk, desc->No, s, ah.rho, aw.rho, ah.J, aw.J);
+      else
+        subfilter_flip_transpose_kernel<float><<<grid, block, 0, stream>>>(
+            static_cast<const float*>(filt), reinterpret_cast<float*>(w_ft), desc->Nc, desc->Sk,
+            desc->No, s, ah.rho, aw.rho, ah.J, aw.J);
+      if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      const uint8_t* src = static_cast<const uint8_t*>(dout) +
+                           ((size_t)ah.crop * Wo + aw.crop) * desc->Nb * eb;
+      if (kind == MAXDNN_KERNEL_FP32)
+        st = fprop_fp32(fd, reinterpret_cast<const float*>(src),
+                        reinterpret_cast<const float*>(w_ft), w_sub, stream);
+      else
+        st = fprop_umma(fd, (int)eb, src, w_ft, w_sub, stream);
+      if (st != MAXDNN_OK) return st;
+      const int nb4 = desc->Nb / 4;
+      const size_t total = (size_t)desc->Nc * ah.n * aw.n * nb4;
+      dgrad_scatter_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+          reinterpret_cast<const float4*>(w_sub), reinterpret_cast<float4*>(din), desc->Nc, ah.n,
+          aw.n, nb4, desc->Hi, desc->Wi, s, ah.first, aw.first);
+      if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+  }
+  return MAXDNN_OK;
+}
+
 maxdnn_status bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* dout,
                          const void* filt, float* din, void* ws, size_t ws_bytes,
                          cudaStream_t stream) {
   if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  maxdnn_conv_desc fd;
-  maxdnn_status st = plan_dgrad(*desc, &fd);
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
   if (!dout || !filt || !din || !ws) return MAXDNN_INVALID_VALUE;
   if (!aligned16(dout) || !aligned16(filt) || !aligned16(din) || !aligned16(ws))
     return MAXDNN_INVALID_VALUE;
+  if (desc->stride != 1)
+    return bprop_data_strided(desc, kind, dout, filt, din, ws, ws_bytes, stream);
+  maxdnn_conv_desc fd;
+  st = plan_dgrad(*desc, &fd);
+  if (st != MAXDNN_OK) return st;
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   const size_t need = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * eb;
   if (ws_bytes < need) return MAXDNN_INVALID_VALUE;
@@ -482,7 +591,6 @@ struct RaggedPlan {
   size_t in_bytes, filt_bytes, out_bytes;   // staging tensors, each rounded up to 256 bytes
 };
 
-size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 maxdnn_status plan_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, RaggedPlan* p) {
   if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
@@ -651,8 +759,8 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   }
   {
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
-                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint64_t hs = dims_in_h(g, 0), cs = dims_in_c(g, 0);
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, hs * 4, cs * 4};
     const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -795,6 +903,8 @@ static maxdnn::ConvDims dims_from2(const maxdnn_conv_desc2& d) {
   c.Nb = d.Nb; c.Wi = d.Wi; c.Hi = d.Hi; c.Nc = d.Nc; c.No = d.No;
   c.Skw = d.Skw; c.Skh = d.Skh; c.stride_w = d.stride_w; c.stride_h = d.stride_h;
   c.pad_w = d.pad_w; c.pad_h = d.pad_h; c.alpha = d.alpha;
+  c.in_h_stride = c.in_c_stride = 0;
+  c.Ho_given = c.Wo_given = 0;
   return c;
 }
 
@@ -834,10 +944,20 @@ maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kern
 maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
                                                maxdnn_kernel_kind kind, size_t* bytes) {
   if (!desc || !bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  maxdnn_conv_desc fd;
-  const maxdnn_status st = plan_dgrad(*desc, &fd);
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
-  *bytes = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  if (desc->stride != 1) {
+    DgradStridedPlan p;
+    st = plan_dgrad_strided(*desc, eb, &p);
+    if (st != MAXDNN_OK) return st;
+    *bytes = p.ft_bytes + p.sub_bytes;
+    return MAXDNN_OK;
+  }
+  maxdnn_conv_desc fd;
+  st = plan_dgrad(*desc, &fd);
+  if (st != MAXDNN_OK) return st;
+  *bytes = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * eb;
   return MAXDNN_OK;
 }
 

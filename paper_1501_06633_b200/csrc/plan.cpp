@@ -25,6 +25,8 @@ ConvDims dims_from(const maxdnn_conv_desc& d) {
   c.Nb = d.Nb; c.Wi = d.Wi; c.Hi = d.Hi; c.Nc = d.Nc; c.No = d.No;
   c.Skw = c.Skh = d.Sk; c.stride_w = c.stride_h = d.stride; c.pad_w = c.pad_h = d.pad;
   c.alpha = d.alpha;
+  c.in_h_stride = c.in_c_stride = 0;
+  c.Ho_given = c.Wo_given = 0;
   return c;
 }
 
@@ -33,12 +35,35 @@ maxdnn_status check_dims(const ConvDims& d, int32_t* Ho, int32_t* Wo) {
       d.stride_w <= 0 || d.stride_h <= 0 || d.pad_w < 0 || d.pad_h < 0)
     return MAXDNN_INVALID_VALUE;
   if (!isfinite(d.alpha)) return MAXDNN_INVALID_VALUE;
+  if (d.Ho_given > 0 && d.Wo_given > 0) {      // output size stated by the caller
+    if (Ho) *Ho = d.Ho_given;
+    if (Wo) *Wo = d.Wo_given;
+    return MAXDNN_OK;
+  }
   const int64_t span_h = (int64_t)d.Hi + 2 * (int64_t)d.pad_h - d.Skh;
   const int64_t span_w = (int64_t)d.Wi + 2 * (int64_t)d.pad_w - d.Skw;
   if (span_h < 0 || span_w < 0) return MAXDNN_INVALID_VALUE;
   if (Ho) *Ho = (int32_t)(span_h / d.stride_h + 1);
   if (Wo) *Wo = (int32_t)(span_w / d.stride_w + 1);
   return MAXDNN_OK;
+}
+
+DgradAxis dgrad_axis(int rho, int Sk, int s, int pad, int size_in) {
+  DgradAxis c;
+  c.rho = rho;
+  c.J = rho < Sk ? (Sk - rho + s - 1) / s : 0;
+  // positions s a + rho - pad in [0, size_in):  a >= (pad - rho) / s  (pad - rho > -s)
+  c.a_min = pad > rho ? (pad - rho + s - 1) / s : 0;
+  const int top = size_in - 1 + pad - rho;                 // s a <= top
+  const int a_max = top >= 0 ? top / s : -1;
+  c.n = a_max >= c.a_min ? a_max - c.a_min + 1 : 0;
+  c.first = s * c.a_min + rho - pad;
+  // grid index a reads dout rows a - J + 1 .. a: FPROP's window of output a - a_min starts at
+  // (a - a_min) - pad, so pad = J - 1 - a_min; a negative value skips rows instead
+  const int p = c.J - 1 - c.a_min;
+  c.pad = p > 0 ? p : 0;
+  c.crop = p < 0 ? -p : 0;
+  return c;
 }
 
 static maxdnn_status common_limits(const ConvDims& d, int elem_bytes) {

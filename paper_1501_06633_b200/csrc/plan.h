@@ -16,6 +16,12 @@ constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel pa
 struct ConvDims {
   int32_t Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w, stride_h, pad_w, pad_h;
   float alpha;
+  // Host-side extras (0 = not used), for the sub-convolutions of the strided map gradient:
+  // the maps are a window of a larger tensor (element pitches of its rows and channels),
+  // and the number of output rows / columns is given instead of derived (the window may
+  // end before or after the last full filter position; what it lacks reads as zeros).
+  int64_t in_h_stride, in_c_stride;
+  int32_t Ho_given, Wo_given;
 };
 
 ConvDims dims_from(const maxdnn_conv_desc& d);
@@ -83,6 +89,22 @@ maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int for
 // padding Sk - 1 - pad.  Fills the descriptor of that FPROP.  NOT_SUPPORTED for
 // stride != 1 or pad > Sk - 1.
 maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* fprop_desc);
+
+// Gradient with respect to the maps, stride s > 1: the map positions split into s x s
+// classes by (h + pad) mod s, (w + pad) mod s; a class only meets the filter taps
+// kh = rho_h + s j, kw = rho_w + s i, and on its own grid (h = s a + rho_h - pad) the
+// gradient is a stride-1 convolution of dout with that sub-filter: an FPROP with the
+// sub-filter flipped and transposed.  One axis of one class:
+struct DgradAxis {
+  int32_t rho;      // residue of (position + pad) mod s
+  int32_t J;        // taps of the class along this axis (0: none, the gradient is zero)
+  int32_t a_min;    // first grid index whose position s a + rho - pad is inside the map
+  int32_t n;        // number of grid positions inside the map
+  int32_t first;    // position of grid index a_min
+  int32_t pad;      // padding of the equivalent FPROP (>= 0)
+  int32_t crop;     // leading rows / columns of dout that FPROP's input window skips
+};
+DgradAxis dgrad_axis(int rho, int Sk, int s, int pad, int size_in);
 
 // Gradient with respect to the filters: the (Nc Sk^2) x No matrix
 //   dfilt[k][o] = alpha * sum_r patch[k][r] * dout[o][r],   r = (y, x, n),

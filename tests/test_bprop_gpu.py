@@ -65,8 +65,40 @@ def test_bprop_data(kernel, shape):
     assert rel_err(got, ref) <= TOL[kernel]
 
 
+DGRAD_STRIDED_SHAPES = [
+    # Nb Wi Hi Nc No Sk stride pad alpha
+    (64, 15, 11, 32, 64, 3, 2, 1, 1.0),       # classes with 2x2, 2x1, 1x2, 1x1 taps
+    (64, 16, 12, 32, 32, 2, 2, 0, 0.5),       # filter = stride: one tap per class
+    (64, 35, 27, 8, 32, 11, 4, 0, 1.0),       # the first-layer geometry: 16 classes, 3x3 / 3x2 / 2x2 taps
+    (64, 23, 19, 4, 32, 11, 4, 2, 1.0),       # with padding: classes start at different rows
+    (64, 23, 19, 32, 64, 7, 4, 3, 1.0),       # the same with 32 channels (tensor kernels too)
+    (64, 14, 14, 32, 32, 2, 3, 0, 1.0),       # stride > filter: a class without taps stays zero
+    (64, 13, 10, 32, 32, 3, 2, 2, 1.0),       # pad = Sk - 1: a class whose window skips a row of dout
+    (64, 9, 9, 32, 32, 5, 3, 1, -1.0),
+]
+
+
+@pytest.mark.parametrize("kernel", ["fp32", "tf32", "bf16"])
+@pytest.mark.parametrize("shape", DGRAD_STRIDED_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_data_strided(kernel, shape):
+    """Stride > 1: one FPROP per residue class of the map positions, scattered onto its grid."""
+    if kernel != "fp32" and shape[3] % 32:
+        pytest.skip("the tensor-core kernels want a multiple of 32 'filters' (here: channels)")
+    w, inp, filt, dout = make(shape, 1300 + shape[5])
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_workspace(d, KIND[kernel]), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data(d, dev(dout, kernel), dev(filt, kernel), din, ws, KIND[kernel])
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_data(rounded(dout, kernel), rounded(filt, kernel), (w.Hi, w.Wi),
+                                 stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = din.cpu().numpy().reshape(ref.shape)
+    assert np.all(np.isfinite(got))
+    assert rel_err(got, ref) <= TOL[kernel]
+
+
 def test_bprop_data_refusals():
-    d = mx.ConvDesc.make(64, 16, 16, 32, 32, 3, 2, 1, 1.0)          # stride 2
+    d = mx.ConvDesc.make(64, 16, 16, 32, 32, 3, 1, 3, 1.0)          # pad > Sk - 1, stride 1
     with pytest.raises(mx.MaxdnnError) as e:
         mx.conv_bprop_data_workspace(d)
     assert e.value.status == mx.NOT_SUPPORTED

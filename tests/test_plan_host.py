@@ -177,8 +177,11 @@ def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     d = mx.ConvDesc.make(128, 27, 27, 96, 256, 5, 1, 2, 1.0)
     assert mx.conv_bprop_data_workspace(d, mx.KERNEL_FP32) == 96 * 25 * 256 * 4
     assert mx.conv_bprop_data_workspace(d, mx.KERNEL_BF16) == 96 * 25 * 256 * 2
-    for bad in (mx.ConvDesc.make(128, 227, 227, 3, 96, 11, 4, 0, 1.0),      # stride 4
-                mx.ConvDesc.make(64, 16, 16, 8, 8, 3, 1, 3, 1.0)):          # pad > Sk - 1
+    strided = mx.ConvDesc.make(128, 227, 227, 3, 96, 11, 4, 0, 1.0)        # stride 4: 16 classes
+    r256 = lambda b: (b + 255) // 256 * 256
+    assert mx.conv_bprop_data_workspace(strided) == \
+        r256(96 * 9 * 3 * 4) + r256(3 * 57 * 57 * 128 * 4)     # 3 x 3 taps at most; 57 x 57 positions
+    for bad in (mx.ConvDesc.make(64, 16, 16, 8, 8, 3, 1, 3, 1.0),):         # pad > Sk - 1
         with pytest.raises(mx.MaxdnnError) as e:
             mx.conv_bprop_data_workspace(bad)
         assert e.value.status == mx.NOT_SUPPORTED
