@@ -261,8 +261,8 @@ maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_ki
  * Sk-1-pad.  Stride s > 1: the map positions split into s x s classes by
  * (h+pad) mod s, (w+pad) mod s; each class meets only the taps kh = rho_h + s j,
  * kw = rho_w + s i and is, on its own grid, a stride-1 FPROP of dout with that
- * sub-filter (flipped, transposed), whose dense result a copy kernel scatters onto
- * the grid; positions no tap reaches are zero.  NOT_SUPPORTED: stride 1 with
+ * sub-filter (flipped, transposed), written onto the class's grid inside din;
+ * positions no tap reaches are zero.  NOT_SUPPORTED: stride 1 with
  * pad > Sk-1, Nb not a multiple of 4 (stride > 1), or what the matching fprop
  * entry point refuses for the transposed problem (its filter count is Nc).
  *

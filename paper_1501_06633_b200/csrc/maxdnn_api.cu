@@ -149,6 +149,7 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(cd, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
+  if (cd.out_x_stride != 0) return MAXDNN_INVALID_VALUE;   // this kernel writes dense results only
   if (!in || !filt || !out) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(filt) || !aligned16(out)) return MAXDNN_INVALID_VALUE;
   DeviceState* ds = nullptr;
@@ -320,8 +321,10 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   {
     // output as (n, x, y, o): one store = 32 filters x 32 images
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
-                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
+    const bool sub = cd.out_x_stride > 0;     // the result is a sub-grid of a larger tensor
+    const uint64_t str[3] = {(sub ? (uint64_t)cd.out_x_stride : (uint64_t)g.Nb) * 4,
+                             (sub ? (uint64_t)cd.out_y_stride : (uint64_t)g.Wo * g.Nb) * 4,
+                             (sub ? (uint64_t)cd.out_o_stride : (uint64_t)g.Ho * g.Wo * g.Nb) * 4};
     const uint32_t box[4] = {32u, 1u, 1u, 32u};
     st = encode_map(&mo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_128B);
@@ -400,12 +403,25 @@ maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kin
   uint8_t* w_ft = static_cast<uint8_t*>(ws);
   float* w_sub = reinterpret_cast<float*>(w_ft + p.ft_bytes);
   // Positions that no tap reaches (a class without taps, or whose window lies outside
-  // dout) keep the zeros written here.
-  if (cudaMemsetAsync(din, 0, (size_t)desc->Nc * desc->Hi * desc->Wi * desc->Nb * 4, stream) !=
-      cudaSuccess) {
+  // dout) must read zero: clear din first if there is such a class.
+  bool all_covered = true;
+  for (int rh = 0; rh < s; ++rh)
+    for (int rw = 0; rw < s; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, desc->Sk, s, desc->pad, desc->Hi);
+      const DgradAxis aw = dgrad_axis(rw, desc->Sk, s, desc->pad, desc->Wi);
+      if (ah.n == 0 || aw.n == 0) continue;                     // no positions: nothing to cover
+      if (ah.J == 0 || aw.J == 0 || ah.crop >= Ho || aw.crop >= Wo) all_covered = false;
+    }
+  if (!all_covered &&
+      cudaMemsetAsync(din, 0, (size_t)desc->Nc * desc->Hi * desc->Wi * desc->Nb * 4, stream) !=
+          cudaSuccess) {
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
+  // The tensor-core kernels store through a tensor map, which can address the class's
+  // grid inside din directly; the fp32 kernel writes a dense scratch tensor that a copy
+  // kernel scatters.
+  const bool direct = kind != MAXDNN_KERNEL_FP32;
   for (int rh = 0; rh < s; ++rh) {
     for (int rw = 0; rw < s; ++rw) {
       const DgradAxis ah = dgrad_axis(rh, desc->Sk, s, desc->pad, desc->Hi);
@@ -434,11 +450,17 @@ maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kin
       g_launches.fetch_add(1, std::memory_order_relaxed);
       const uint8_t* src = static_cast<const uint8_t*>(dout) +
                            ((size_t)ah.crop * Wo + aw.crop) * desc->Nb * eb;
-      if (kind == MAXDNN_KERNEL_FP32)
-        st = fprop_fp32(fd, reinterpret_cast<const float*>(src),
-                        reinterpret_cast<const float*>(w_ft), w_sub, stream);
-      else
-        st = fprop_umma(fd, (int)eb, src, w_ft, w_sub, stream);
+      if (direct) {
+        fd.out_x_stride = (int64_t)s * desc->Nb;
+        fd.out_y_stride = (int64_t)s * desc->Wi * desc->Nb;
+        fd.out_o_stride = (int64_t)desc->Hi * desc->Wi * desc->Nb;
+        float* dst = din + ((size_t)ah.first * desc->Wi + aw.first) * desc->Nb;
+        st = fprop_umma(fd, (int)eb, src, w_ft, dst, stream);
+        if (st != MAXDNN_OK) return st;
+        continue;
+      }
+      st = fprop_fp32(fd, reinterpret_cast<const float*>(src), reinterpret_cast<const float*>(w_ft),
+                      w_sub, stream);
       if (st != MAXDNN_OK) return st;
       const int nb4 = desc->Nb / 4;
       const size_t total = (size_t)desc->Nc * ah.n * aw.n * nb4;
@@ -905,6 +927,7 @@ static maxdnn::ConvDims dims_from2(const maxdnn_conv_desc2& d) {
   c.pad_w = d.pad_w; c.pad_h = d.pad_h; c.alpha = d.alpha;
   c.in_h_stride = c.in_c_stride = 0;
   c.Ho_given = c.Wo_given = 0;
+  c.out_x_stride = c.out_y_stride = c.out_o_stride = 0;
   return c;
 }
 

@@ -27,6 +27,7 @@ ConvDims dims_from(const maxdnn_conv_desc& d) {
   c.alpha = d.alpha;
   c.in_h_stride = c.in_c_stride = 0;
   c.Ho_given = c.Wo_given = 0;
+  c.out_x_stride = c.out_y_stride = c.out_o_stride = 0;
   return c;
 }
 

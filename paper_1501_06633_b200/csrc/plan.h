@@ -22,6 +22,9 @@ struct ConvDims {
   // end before or after the last full filter position; what it lacks reads as zeros).
   int64_t in_h_stride, in_c_stride;
   int32_t Ho_given, Wo_given;
+  // element pitches of the result's pixels / rows / filters when it is a sub-grid of a larger
+  // tensor (tensor-core kernels only: their stores go through a tensor map)
+  int64_t out_x_stride, out_y_stride, out_o_stride;
 };
 
 ConvDims dims_from(const maxdnn_conv_desc& d);
