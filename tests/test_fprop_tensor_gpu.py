@@ -135,6 +135,35 @@ def test_full_size_large3x3_sampled(kernel):
     assert np.isfinite(got).all()
 
 
+@pytest.mark.parametrize("name,kernel", [
+    ("first11x11s4", "bf16"), ("first11x11s4", "tf32"),      # filter columns merged into K
+    ("mid5x5", "bf16"), ("mid5x5", "tf32"),                  # two-SM tiles, images split, 5-column strips
+    ("wide3x3", "bf16"),                                     # one-SM tiles, 384 filters
+    ("alexnet_conv4", "bf16"), ("alexnet_conv5", "tf32"),    # 192-column tiles (3 pixels x 64 images)
+    ("alexnet_conv1", "bf16"),                               # merged columns, 64 of 128 filter rows
+    ("overfeat_L2", "tf32"),
+])
+def test_full_size_sampled_in_the_benchmarked_plans(name, kernel):
+    """Every kind of plan the planner picks at full size (the launch configuration the bench
+    and the Table 1 run time): first / middle / last output row and random single outputs."""
+    w = wl.ALL[name]
+    inp, filt = wl.make_inputs(w)
+    got, r_in, r_f = run(kernel, w, inp, filt)
+    assert np.isfinite(got).all()
+    Ho = got.shape[1]
+    scale = float(np.max(np.abs(got)))
+    for y in sorted({0, Ho // 2, Ho - 1}):
+        refr = oracle.conv_fprop(r_in, r_f, stride=w.stride, pad=w.pad, alpha=w.alpha,
+                                 rows=(y, y + 1))[:, y]
+        assert float(np.max(np.abs(got[:, y].astype(np.float64) - refr))) <= TOL_ROUNDED * scale
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        o, y, x, n = (int(rng.integers(0, s)) for s in got.shape)
+        v, _ = oracle.conv_fprop_point(r_in, r_f, o, y, x, n, stride=w.stride, pad=w.pad,
+                                       alpha=w.alpha)
+        assert abs(float(got[o, y, x, n]) - v) <= TOL_ROUNDED * scale
+
+
 @pytest.mark.parametrize("kernel", ["tf32", "bf16"])
 def test_run_to_run_bitwise_identical(kernel):
     w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
