@@ -139,15 +139,16 @@ struct WgradCursor {
     y = px / g.Wo;
   }
   __device__ __forceinline__ bool done(const WgradGeom& g) const { return item >= g.n_items; }
-  // Next reduction step; moves to this CTA's next item when the current one is exhausted.
-  __device__ __forceinline__ void advance(const WgradGeom& g) {
+  // Next reduction step; moves to this CTA's (or CTA pair's) next item, `item_stride`
+  // further, when the current one is exhausted.
+  __device__ __forceinline__ void advance(const WgradGeom& g, int item_stride) {
     if (++r < r_end) {
       if (++nc == g.n_chunks) {
         nc = 0;
         if (++x == g.Wo) { x = 0; ++y; }
       }
     } else {
-      start(g, item + (int)gridDim.x);
+      start(g, item + item_stride);
     }
   }
 };
@@ -198,7 +199,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
     tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride - g.pad,
                 pc.y * g.stride - g.pad + pc.khb * g.bh, pc.cb * g.bc);
     if (++p_stage == stages) { p_stage = 0; p_phase ^= 1u; }
-    pc.advance(g);
+    pc.advance(g, (int)gridDim.x);
   };
   const bool issuer = (warp == 0 && lane == 0);
   if (issuer) {

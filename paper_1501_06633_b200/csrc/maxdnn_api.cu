@@ -13,6 +13,7 @@
 #include "umma_conv.cuh"
 #include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
+#include "wgrad_umma_pair.cuh"
 
 namespace maxdnn {
 namespace {
@@ -27,7 +28,7 @@ struct DeviceState {
   bool ffma_attr[16] = {};
   bool umma_attr[4] = {false, false, false, false};
   bool wgrad_attr = false;
-  bool wgrad_umma_attr[2] = {false, false};
+  bool wgrad_umma_attr[4] = {false, false, false, false};
 };
 
 std::mutex g_mu;
@@ -532,7 +533,8 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
   static thread_local WgradArgs fargs;
   static thread_local WgradUmmaArgs uargs;
   WgradGeom& g = tensor ? uargs.g : fargs.g;
-  st = plan_wgrad(*desc, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
+  st = plan_wgrad(*desc, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
+                  env_int("MAXDNN_WGRAD_PAIR"));
   if (st != MAXDNN_OK) return st;
   const size_t kno = (size_t)g.Nc * g.Sk * g.Sk * g.No;
   const size_t need = g.splits > 1 ? (size_t)g.splits * kno * 4 : 0;
@@ -555,7 +557,9 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
     const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
     const uint64_t str[3] = {(uint64_t)g.Nb * eb, (uint64_t)g.Wi * g.Nb * eb,
                              (uint64_t)g.Hi * g.Wi * g.Nb * eb};
-    const uint32_t box[4] = {chunk, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
+    // (a pair's CTA stages half of the tile's channels)
+    const uint32_t box[4] = {chunk, (uint32_t)g.bw, (uint32_t)g.bh,
+                             (uint32_t)(g.pair ? g.bc_h : g.bc)};
     st = encode_map(&mi, dt, 4, in, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
   }
@@ -578,19 +582,49 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
     uargs.status = ds->status;
     uargs.atom = chunk;
     const uint32_t fmt = bf16 ? 1u : 2u;
-    const uint32_t n_mma = (uint32_t)align_up(g.rows, 16);
+    const uint32_t n_mma = (uint32_t)g.n_mma;
+    const uint32_t m_mma = g.pair ? 256u : 128u;
     uargs.idesc = (1u << 4) | (fmt << 7) | (fmt << 10)      // fp32 accumulate, operand formats;
-                  | ((n_mma >> 3) << 17) | ((128u >> 4) << 24);   // both operands K-major; N, M
-    auto kern = bf16 ? wgrad_umma_kernel<true> : wgrad_umma_kernel<false>;
-    if (!ds->wgrad_umma_attr[bf16 ? 1 : 0]) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-          cudaSuccess) {
+                  | ((n_mma >> 3) << 17) | ((m_mma >> 4) << 24);   // both operands K-major; N, M
+    const int slot = (bf16 ? 1 : 0) + (g.pair ? 2 : 0);
+    if (g.pair) {
+      auto kern = bf16 ? wgrad_umma_pair_kernel<true> : wgrad_umma_pair_kernel<false>;
+      if (!ds->wgrad_umma_attr[slot]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess) {
+          cudaGetLastError();
+          return MAXDNN_CUDA_ERROR;
+        }
+        ds->wgrad_umma_attr[slot] = true;
+      }
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
+      cfg.blockDim = dim3(kWgUmmaThreads, 1, 1);
+      cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaLaunchKernelEx(&cfg, kern, mg, mi, uargs) != cudaSuccess) {
         cudaGetLastError();
         return MAXDNN_CUDA_ERROR;
       }
-      ds->wgrad_umma_attr[bf16 ? 1 : 0] = true;
+    } else {
+      auto kern = bf16 ? wgrad_umma_kernel<true> : wgrad_umma_kernel<false>;
+      if (!ds->wgrad_umma_attr[slot]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess) {
+          cudaGetLastError();
+          return MAXDNN_CUDA_ERROR;
+        }
+        ds->wgrad_umma_attr[slot] = true;
+      }
+      kern<<<g.grid, kWgUmmaThreads, g.smem_bytes, stream>>>(mg, mi, uargs);
     }
-    kern<<<g.grid, kWgUmmaThreads, g.smem_bytes, stream>>>(mg, mi, uargs);
   }
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -1003,7 +1037,8 @@ maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
   }
   WgradGeom g;
   const int eb = kind == MAXDNN_KERNEL_FP32 ? 0 : (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
-  const maxdnn_status st = plan_wgrad(*desc, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g);
+  const maxdnn_status st = plan_wgrad(*desc, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
+                                      env_int("MAXDNN_WGRAD_PAIR"));
   if (st != MAXDNN_OK) return st;
   *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Sk * g.Sk * g.No * 4 : 0;
   return MAXDNN_OK;

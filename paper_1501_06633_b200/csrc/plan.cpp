@@ -464,7 +464,7 @@ maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* f) {
 }
 
 maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
-                         WgradGeom* g) {
+                         WgradGeom* g, int force_pair) {
   int32_t Ho, Wo;
   maxdnn_status st = check_desc(&d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -487,11 +487,24 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   g->bc = max_rows / (g->bw * g->bh);
   if (g->bc > 256) g->bc = 256;                                       // a copy box has at most 256 per axis
   if (g->bc > d.Nc) g->bc = d.Nc;
+  // Two-SM tiles (tensor-core kernel): 256 filters per pair of CTAs, each CTA staging its
+  // 128 filters and half of the tile's channels — per SM and per MMA 8 KB instead of 12 KB
+  // are staged, and the kernel is bound by that fill rate.  Taken when the second CTA of
+  // every tile has filters and the channels split evenly.
+  const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);
+  g->pair = (tensor && force_pair >= 0 && (peer_has_filters || force_pair > 0) && g->bc >= 2 &&
+             sm_count >= 2) ? 1 : 0;
+  if (g->pair) {
+    g->bc &= ~1;
+    g->bc_h = g->bc / 2;
+  }
   g->rows = g->bc * g->bh * g->bw;
+  g->rows_h = g->pair ? g->rows / 2 : g->rows;
+  g->n_mma = g->pair ? 2 * align_up(g->rows_h, 8) : align_up(g->rows, 16);
   g->box_o = d.No < 128 ? d.No : 128;
   g->c_blocks = ceil_div(d.Nc, g->bc);
   g->kh_blocks = ceil_div(d.Sk, g->bh);
-  g->o_blocks = ceil_div(d.No, 128);
+  g->o_blocks = ceil_div(d.No, g->pair ? 256 : 128);
   g->n_chunks = ceil_div(d.Nb, chunk);
   const int64_t r_steps = (int64_t)Ho * Wo * g->n_chunks;
   const int64_t tiles = (int64_t)g->c_blocks * g->kh_blocks * g->o_blocks;
@@ -499,17 +512,18 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   g->r_steps = (int32_t)r_steps;
   // Split the reduction so that the items fill whole waves of persistent CTAs (about
   // four waves when the tiles alone are fewer), each split keeping at least 64 steps.
+  const int units = g->pair ? sm_count / 2 : sm_count;
   int splits = 1;
   if (force_splits > 0) {
     splits = force_splits;
-  } else if (tiles < 4 * (int64_t)sm_count) {
-    const int64_t want = ceil_div(4 * sm_count, (int)tiles);
+  } else if (tiles < 4 * (int64_t)units) {
+    const int64_t want = ceil_div(4 * units, (int)tiles);
     const int64_t most = r_steps / 64 > 0 ? r_steps / 64 : 1;
     splits = (int)(want < most ? want : most);
     // round the item count to whole waves where that is cheap
     const int64_t items = tiles * splits;
-    const int64_t waves = (items + sm_count - 1) / sm_count;
-    const int64_t fit = waves * sm_count / tiles;
+    const int64_t waves = (items + units - 1) / units;
+    const int64_t fit = waves * units / tiles;
     if (fit >= 1 && fit <= most) splits = (int)fit;
   }
   if (splits > r_steps) splits = (int)r_steps;
@@ -519,9 +533,15 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   const int64_t items = tiles * g->splits;
   if (items > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   g->n_items = (int32_t)items;
-  g->stages = tensor ? 4 : 6;
-  g->smem_bytes = g->stages * (128 + max_rows) * 128 + 1024 + 1024 + (tensor ? 2048 : 0);   // ring, alignment slack, barriers, row table
-  g->grid = g->n_items < sm_count ? g->n_items : sm_count;
+  g->stages = tensor ? (g->pair ? 6 : 4) : 6;
+  g->smem_bytes = g->stages * (128 + (g->pair ? 128 : max_rows)) * 128 + 1024 + 1024 +
+                  (tensor ? 2048 : 0);   // ring, alignment slack, barriers, row table
+  if (g->pair) {
+    const int pairs = sm_count / 2;
+    g->grid = 2 * (g->n_items < pairs ? g->n_items : pairs);
+  } else {
+    g->grid = g->n_items < sm_count ? g->n_items : sm_count;
+  }
   return MAXDNN_OK;
 }
 

@@ -128,12 +128,15 @@ struct WgradGeom {
   int32_t splits, steps_per_split;
   int32_t n_items;           // tiles x splits
   int32_t stages, grid, smem_bytes;
+  // tensor-core kernel on a pair of CTAs (256 filters per tile; each CTA stages its 128
+  // filters and half of the tile's channels): channels / gradient rows per CTA, MMA N
+  int32_t pair, bc_h, rows_h, n_mma;
 };
 
 // force_splits > 0 pins the number of reduction splits (tests, ablations).
 // elem_bytes 0: the fp32 FFMA2 kernel (128 gradient rows per tile, 32 images per step);
 // 4 / 2: the tensor-core kernel with TF32 / BF16 operands (256 rows; 32 / 64 images).
 maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
-                         WgradGeom* g);
+                         WgradGeom* g, int force_pair = 0);
 
 }  // namespace maxdnn

@@ -122,7 +122,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       }
       __syncwarp();
       if (++stage == stages) { stage = 0; phase ^= 1u; }
-      pc.advance(g);
+      pc.advance(g, (int)gridDim.x);
     }
     if (!ok) {
       for (int s = 0; s < stages; ++s) {

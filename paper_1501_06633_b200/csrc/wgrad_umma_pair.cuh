@@ -1,0 +1,234 @@
+// Two-SM variant of the tensor-core filter-gradient kernel (tcgen05 MMA with
+// cta_group::2): a cluster of two CTAs works on a tile of 256 filters x up to 256
+// gradient rows.  CTA r stages its 128 filters of the output gradient and the gradient
+// rows of HALF of the tile's channels; the leader issues MMAs of M = 256 that read each
+// half of the row operand from the CTA that holds it.  Per SM and per MMA 8 KB instead of
+// 12 KB are staged — the one-SM kernel is bound by that fill rate — and the ring holds
+// six stages of 32 KB.  Synchronisation as in the two-SM forward kernel: both CTAs'
+// copies complete on the leader's "full" barrier, on which only the leader arrives
+// (expecting both CTAs' bytes); the leader's commits reach the "empty" / "accumulator
+// complete" barriers of both CTAs; both CTAs' epilogue warps arrive on the leader's
+// "accumulator drained" barrier.  Every wait is bounded.
+#pragma once
+#include "umma_pair_conv.cuh"
+#include "wgrad_umma.cuh"
+
+namespace maxdnn {
+
+template <bool BF16>
+__global__ void __launch_bounds__(kWgUmmaThreads, 1)
+wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
+                       const __grid_constant__ CUtensorMap map_in,
+                       const __grid_constant__ WgradUmmaArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  const WgradGeom& g = args.g;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const int stages = g.stages;
+  const uint32_t half_b_bytes = 128u * 128u;                 // up to 128 gradient rows per CTA
+  const uint32_t stage_bytes = kWgUmmaABytes + half_b_bytes;
+  const uint32_t bar_off = (uint32_t)stages * stage_bytes;
+  const uint32_t full_bar = base + bar_off;                  // the leader's are used
+  const uint32_t empty_bar = full_bar + 8u * stages;
+  const uint32_t accf_bar = empty_bar + 8u * stages;         // 2
+  const uint32_t acce_bar = accf_bar + 16u;                  // 2; the leader's are used
+  const uint32_t done_bar = acce_bar + 16u;
+  const uint32_t tmem_slot = done_bar + 8u;
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(base_ptr + bar_off + 16u * stages + 40u);
+  int2* row_tab = reinterpret_cast<int2*>(base_ptr + bar_off + 1024u);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
+  const int hcols = g.n_mma >> 1;                            // accumulator columns per half
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full_bar + 8u * s, 1);     // the leader's copy warp (expects both CTAs' bytes)
+      mbar_init(empty_bar + 8u * s, 1);    // the leader's commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar + 8u * a, 1);     // the leader's commit
+      mbar_init(acce_bar + 8u * a, 8);     // four epilogue warps in each of the two CTAs
+    }
+    mbar_init(done_bar, 1);
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot),
+                 "r"(kWgUmmaTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  // accumulator column -> {dfilt row offset relative to the tile's first row; channel << 16 | filter row}
+  for (int col = threadIdx.x; col < 256; col += kWgUmmaThreads) {
+    const int half = col >= hcols ? 1 : 0;
+    const int row = col - half * hcols;
+    if (row < g.rows_h) {
+      const int w_l = row % g.bw;
+      const int t = row / g.bw;
+      const int h_l = t % g.bh;
+      const int c_l = half * g.bc_h + t / g.bh;
+      row_tab[col] = make_int2((c_l * g.Sk + h_l) * g.Sk + w_l, (c_l << 16) | h_l);
+    } else {
+      row_tab[col] = make_int2(0, 0x7fff << 16);             // no such row: never stored
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  const uint32_t leader_full = map_to_cta(full_bar, 0);
+  const uint32_t leader_acce = map_to_cta(acce_bar, 0);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- copies
+    if (lane == 0) {
+      prefetch_tensormap(&map_dout);
+      prefetch_tensormap(&map_in);
+    }
+    const uint32_t tx_bytes = 2u * (uint32_t)(g.box_o + g.rows_h) * 128u;   // both CTAs' boxes
+    const uint64_t pol_last = l2_policy_evict_last();
+    WgradCursor pc;
+    pc.start(g, pair);
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    while (ok && !pc.done(g)) {
+      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+        ok = false;
+        break;
+      }
+      const uint32_t fb = leader_full + 8u * stage;
+      const uint32_t dst = base + (uint32_t)stage * stage_bytes;
+      const int n0 = pc.nc * (int)args.atom;
+      if (elect_one()) {
+        if (rank == 0) mbar_arrive_expect_tx(full_bar + 8u * stage, tx_bytes);
+        tma_load_4d_pair(dst, &map_dout, fb, n0, pc.x, pc.y, pc.ob * 256 + (int)rank * 128, pol_last);
+        tma_load_4d_pair(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride - g.pad,
+                         pc.y * g.stride - g.pad + pc.khb * g.bh,
+                         pc.cb * g.bc + (int)rank * g.bc_h, pol_last);
+      }
+      __syncwarp();
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      pc.advance(g, n_pairs);
+    }
+    if (!ok) {
+      // Leaving early: give copies already issued time to land (their barrier lives in
+      // the leader CTA and cannot be polled from the peer).
+      const uint64_t t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) {}
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------- MMA issue (leader only)
+    if (rank == 0) {
+      WgradCursor cc;
+      cc.start(g, pair);
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t it = 0;
+      bool ok = true;
+      const uint64_t desc_hi = make_smem_desc(0, 0, 1024, 2u);
+      while (ok && !cc.done(g)) {
+        const int n_steps = cc.r_end - cc.r;
+        const uint32_t acc = it & 1u;
+        if (!mbar_wait(acce_bar + 8u * acc, ((it >> 1) & 1u) ^ 1u, args.status, kDevTimeoutAccFree)) {
+          ok = false;
+          break;
+        }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * 256u;
+        uint32_t accumulate = 0;
+        for (int s = 0; s < n_steps; ++s) {
+          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+            ok = false;
+            break;
+          }
+          tcgen05_fence_after();
+          const uint32_t a_addr = base + (uint32_t)stage * stage_bytes;
+          const uint64_t adesc0 = desc_hi | (uint64_t)((a_addr & 0x3FFFFu) >> 4);
+          const uint64_t bdesc0 = desc_hi | (uint64_t)(((a_addr + kWgUmmaABytes) & 0x3FFFFu) >> 4);
+          if (elect_one()) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              tcgen05_mma_pair<BF16>(d_tmem, adesc0 + (uint64_t)(2 * j), bdesc0 + (uint64_t)(2 * j),
+                                     args.idesc, accumulate | (uint32_t)(j > 0));
+            }
+            tcgen05_commit_pair(empty_bar + 8u * stage);       // frees the stage in both CTAs
+          }
+          accumulate = 1;
+          __syncwarp();
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (elect_one()) tcgen05_commit_pair(accf_bar + 8u * acc);
+        __syncwarp();
+        cc.start(g, cc.item + n_pairs);
+        ++it;
+      }
+      if (elect_one()) tcgen05_commit_pair(done_bar, 1);
+      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (both CTAs)
+    const int q = warp & 3;
+    WgradCursor cc;
+    cc.start(g, pair);
+    uint32_t it = 0;
+    bool ok = true;
+    const bool direct = (g.splits == 1);
+    const size_t K = (size_t)g.Nc * g.Sk * g.Sk;
+    const float scale = direct ? g.alpha : 1.0f;
+    while (ok && !cc.done(g)) {
+      const uint32_t acc = it & 1u;
+      if (!mbar_wait(accf_bar + 8u * acc, (it >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+        ok = false;
+        break;
+      }
+      tcgen05_fence_after();
+      const int o = cc.ob * 256 + (int)rank * 128 + q * 32 + lane;
+      const int c_lim = g.Nc - cc.cb * g.bc;
+      const int h_lim = g.Sk - cc.khb * g.bh;
+      float* dst = (direct ? args.dfilt : args.partial + (size_t)cc.split * K * g.No) +
+                   ((size_t)(cc.cb * g.bc) * g.Sk + (size_t)cc.khb * g.bh) * g.Sk * g.No + o;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256u;
+      for (int col = 0; col < g.n_mma; col += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32(t_row + (uint32_t)col, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int2 e = row_tab[col + j];
+          if (col + j < g.n_mma && (e.y >> 16) < c_lim && (e.y & 0xffff) < h_lim && o < g.No)
+            dst[(size_t)e.x * g.No] = __uint_as_float(v[j]) * scale;
+        }
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_acce + 8u * acc);
+      cc.start(g, cc.item + n_pairs);
+      ++it;
+    }
+  }
+
+  // Neither CTA leaves (or frees TMEM) while its peer may still arrive on its barriers,
+  // have copies in flight that report to it, or run MMAs that read its shared memory.
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 1) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(kWgUmmaTmemCols)
+                 : "memory");
+  }
+}
+
+}  // namespace maxdnn

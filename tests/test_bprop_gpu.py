@@ -152,11 +152,20 @@ WGRAD_TC_SHAPES = WGRAD_SHAPES + [
 
 
 @pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+@pytest.mark.parametrize("pair", [-1, 1])
 @pytest.mark.parametrize("splits", [0, 2])
-@pytest.mark.parametrize("shape", WGRAD_TC_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
-def test_bprop_filter_tensor_cores(shape, splits, kernel, monkeypatch):
+@pytest.mark.parametrize("shape", WGRAD_TC_SHAPES + [(64, 9, 9, 64, 512, 3, 1, 1, 1.0),
+                                                     (64, 9, 9, 33, 384, 3, 1, 1, 1.0)],
+                         ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_filter_tensor_cores(shape, splits, pair, kernel, monkeypatch):
+    """pair = -1: one-SM tiles of 128 filters; 1: two-SM tiles of 256 filters (each CTA stages
+    its 128 filters and half of the tile's channels), forced also where the planner would not
+    take them (fewer than 129 filters: the second CTA's filters are all out of range)."""
     if kernel == "bf16" and shape[0] % 8:
         pytest.skip("a row of bf16 images must be a multiple of 16 bytes")
+    if pair == 1 and shape[3] == 3 and shape[5] == 11:
+        pytest.skip("one channel per tile (121 taps): nothing to split between two CTAs")
+    monkeypatch.setenv("MAXDNN_WGRAD_PAIR", str(pair))
     if splits:
         monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
     w, inp, filt, dout = make(shape, 2600 + shape[5])
