@@ -52,7 +52,7 @@ def parse_args():
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER + wl.TABLE1_ORDER)
-    p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16"])
+    p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16", "tf32x3"])
     p.add_argument("--op", default="fprop", choices=["fprop", "dgrad", "wgrad"],
                    help="fprop (the headline path) or one of its two adjoints (BPROP)")
     p.add_argument("--e2e-steps", type=int, default=10)
@@ -295,7 +295,11 @@ def run_ours(args):
 
     peaks, peaks_kind = load_peaks()
     w = wl.ALL[args.workload]
-    kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16}[args.kernel]
+    x3 = args.kernel == "tf32x3"            # three TF32 products: fp32 buffers, FPROP only
+    if x3 and args.op != "fprop":
+        raise SystemExit("--kernel tf32x3 is an FPROP mode")
+    kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16,
+            "tf32x3": mx.KERNEL_TF32}[args.kernel]
     d = mx.ConvDesc.make(*w.dims)
     op = args.op
     nbytes, Ho, Wo = workload_bytes(w, args.kernel, op)
@@ -335,6 +339,9 @@ def run_ours(args):
                          device="cuda")
     fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
              mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
+    if x3:
+        ws = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+        fprop = lambda dd, a, b, r, stream=None: mx.conv_fprop_tf32x3(dd, a, b, r, ws, stream=stream)
 
     def step(i):
         a, b, r = d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets]
@@ -384,8 +391,14 @@ def run_ours(args):
 
     def e2e_step(k, stream):
         a, b, r = d_as[k % n_sets], d_bs[k % len(d_bs)], d_res[k % n_sets]
-        if op == "fprop":
+        if op == "fprop" and not x3:
             mx.conv_fprop_host(d, kind, h_a, h_b, h_outs[k], a, b, r, stream=stream)
+        elif op == "fprop":
+            with torch.cuda.stream(stream):
+                a.copy_(h_a, non_blocking=True)
+                b.copy_(h_b, non_blocking=True)
+                mx.conv_fprop_tf32x3(d, a, b, r, ws_e2e[k], stream=stream)
+                h_outs[k].copy_(r, non_blocking=True)
         else:
             with torch.cuda.stream(stream):
                 a.copy_(h_a, non_blocking=True)
@@ -435,16 +448,20 @@ def run_ours(args):
         else:
             bf16 = float(peaks["bf16_tflops"])
             peak = bf16 if args.kernel == "bf16" else bf16 * (1.1 / 2.25)
+            if x3:
+                peak /= 3.0          # three TF32 products per product of the paper's count
             bound = "tensor"
             peak_note = ("cuBLAS bf16 burst (%s)" % peaks_kind) if args.kernel == "bf16" else \
                 ("cuBLAS bf16 burst (%s) x nominal tf32/bf16 ratio 1.1/2.25" % peaks_kind)
+            if x3:
+                peak_note += " / 3 (three TF32 products per product counted)"
         t_compute = C / (peak * 1e12)
         t_hbm = nbytes / (float(peaks["hbm_gbs"]) * 1e9)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16"}[args.kernel],
+            "dtype": {"fp32": "f32", "tf32": "tf32", "bf16": "bf16", "tf32x3": "tf32x3"}[args.kernel],
             "data": "synthetic",
             "config": {
                 "workload": w.name, "op": op, "kernel": args.kernel, "Nb": w.Nb, "Wi": w.Wi, "Hi": w.Hi,

@@ -17,6 +17,7 @@ __all__ = [
     "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
     "last_device_status",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
+    "conv_fprop_tf32x3_workspace", "conv_fprop_tf32x3",
     "ConvDesc2", "conv2_out_dims", "conv2_fprop", "conv2_fprop_status",
     "conv_fprop_ragged_workspace", "conv_fprop_ragged", "fprop_ragged_status",
     "conv_bprop_data_workspace", "conv_bprop_data", "bprop_data_status",
@@ -35,6 +36,7 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv_bprop_filter_workspace", "maxdnn_conv_bprop_filter",
     "maxdnn_conv_fprop_ragged_workspace", "maxdnn_conv_fprop_ragged",
     "maxdnn_conv2_out_dims", "maxdnn_conv2_fprop",
+    "maxdnn_conv_fprop_tf32x3_workspace", "maxdnn_conv_fprop_tf32x3",
 ]
 
 
@@ -120,6 +122,10 @@ def load_library():
         getattr(lib, name).argtypes = [P(ConvDesc), vp, vp, vp, vp]
     lib.maxdnn_conv_fprop_host.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_host.argtypes = [P(ConvDesc), ctypes.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.maxdnn_conv_fprop_tf32x3_workspace.restype = ctypes.c_int
+    lib.maxdnn_conv_fprop_tf32x3_workspace.argtypes = [P(ConvDesc), P(ctypes.c_size_t)]
+    lib.maxdnn_conv_fprop_tf32x3.restype = ctypes.c_int
+    lib.maxdnn_conv_fprop_tf32x3.argtypes = [P(ConvDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.maxdnn_conv2_out_dims.restype = ctypes.c_int
     lib.maxdnn_conv2_out_dims.argtypes = [P(ConvDesc2), P(ctypes.c_int32), P(ctypes.c_int32)]
     lib.maxdnn_conv2_fprop.restype = ctypes.c_int
@@ -277,6 +283,26 @@ def _workspace_ptr(workspace, need):
     if not (isinstance(workspace, torch.Tensor) and workspace.is_cuda and workspace.is_contiguous()):
         raise TypeError("workspace must be a contiguous CUDA tensor")
     return ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def conv_fprop_tf32x3_workspace(desc: ConvDesc) -> int:
+    """Bytes of device scratch maxdnn_conv_fprop_tf32x3 needs (the split maps and filters)."""
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv_fprop_tf32x3_workspace(ctypes.byref(desc),
+                                                                 ctypes.byref(n))),
+           "maxdnn_conv_fprop_tf32x3_workspace")
+    return int(n.value)
+
+
+def conv_fprop_tf32x3(desc: ConvDesc, inp, filt, out, workspace, stream=None) -> None:
+    """maxdnn_conv_fprop_tf32x3: fp32-level accuracy on the tensor cores (three TF32 products)."""
+    lib = load_library()
+    pin = _dev_ptr(inp, ("float32",), conv_in_elems(desc), "in")
+    pf = _dev_ptr(filt, ("float32",), conv_filt_elems(desc), "filt")
+    po = _dev_ptr(out, ("float32",), conv_out_elems(desc), "out")
+    pw, nbytes = _workspace_ptr(workspace, 1)
+    _check(int(lib.maxdnn_conv_fprop_tf32x3(ctypes.byref(desc), pin, pf, po, pw, nbytes,
+                                            _stream_ptr(stream))), "maxdnn_conv_fprop_tf32x3")
 
 
 def conv2_out_dims(desc: ConvDesc2):

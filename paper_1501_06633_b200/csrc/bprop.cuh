@@ -78,6 +78,26 @@ dgrad_scatter_kernel(const float4* __restrict__ sub, float4* __restrict__ din, i
   din[(((size_t)c * Hi + h_first + s * a) * Wi + w_first + s * b) * nb4 + n] = sub[i];
 }
 
+// Split of fp32 values for the three-product TF32 scheme: hi = the value with its low 13
+// mantissa bits cleared (what a TF32 tensor core reads from an fp32 word), lo = value - hi
+// (exact in fp32).  dst holds three copies of the tensor back to back along its outermost
+// (channel) axis: part p is hi where bit p of `lo_mask` is clear, lo where it is set.
+__global__ void __launch_bounds__(256)
+tf32_split3_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t n4,
+                   uint32_t lo_mask) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 a = src[i];
+  float4 hi, lo;
+  hi.x = __uint_as_float(__float_as_uint(a.x) & 0xFFFFE000u);
+  hi.y = __uint_as_float(__float_as_uint(a.y) & 0xFFFFE000u);
+  hi.z = __uint_as_float(__float_as_uint(a.z) & 0xFFFFE000u);
+  hi.w = __uint_as_float(__float_as_uint(a.w) & 0xFFFFE000u);
+  lo.x = a.x - hi.x; lo.y = a.y - hi.y; lo.z = a.z - hi.z; lo.w = a.w - hi.w;
+#pragma unroll
+  for (int p = 0; p < 3; ++p) dst[(size_t)p * n4 + i] = ((lo_mask >> p) & 1u) ? lo : hi;
+}
+
 // Staging copies for shapes the bulk tensor copies cannot address (row pitches that are
 // not multiples of 16 bytes): dst[row][j] = src[row][j] for j < n, 0 for n <= j < n_pad
 // (pad_inner), and the reverse for results (unpad_inner drops the padding columns).

@@ -729,6 +729,51 @@ maxdnn_status fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
 }
 
 // ---------------------------------------------------------------------------
+// fp32-level accuracy on the tensor cores: three TF32 products as one FPROP over 3 Nc channels.
+// ---------------------------------------------------------------------------
+maxdnn_status tf32x3_sizes(const maxdnn_conv_desc* desc, size_t* in_bytes, size_t* filt_bytes) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  const maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  if (desc->Nc > 32767 / 3) return MAXDNN_NOT_SUPPORTED;
+  if (desc->Nb % 4 != 0 || desc->No % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+  *in_bytes = round256((size_t)3 * desc->Nc * desc->Hi * desc->Wi * desc->Nb * 4);
+  *filt_bytes = round256((size_t)3 * desc->Nc * desc->Sk * desc->Sk * desc->No * 4);
+  return MAXDNN_OK;
+}
+
+maxdnn_status fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in, const float* filt,
+                           float* out, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  size_t in_bytes = 0, filt_bytes = 0;
+  maxdnn_status st = tf32x3_sizes(desc, &in_bytes, &filt_bytes);
+  if (st != MAXDNN_OK) return st;
+  if (!in || !filt || !out || !ws) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(filt) || !aligned16(out) || !aligned16(ws)) return MAXDNN_INVALID_VALUE;
+  if (ws_bytes < in_bytes + filt_bytes) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  maxdnn_conv_desc d3 = *desc;
+  d3.Nc = 3 * desc->Nc;
+  st = dgrad_plan_check(d3, MAXDNN_KERNEL_TF32, ds->sm_count);   // the 3 Nc-channel problem has a plan
+  if (st != MAXDNN_OK) return st;
+  float* w_in = static_cast<float*>(ws);
+  float* w_filt = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + in_bytes);
+  const size_t n4_in = (size_t)desc->Nc * desc->Hi * desc->Wi * desc->Nb / 4;
+  const size_t n4_f = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No / 4;
+  // maps [hi; hi; lo] x filters [hi; lo; hi]  ->  hi*hi + hi*lo + lo*hi
+  tf32_split3_kernel<<<(unsigned)((n4_in + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(in), reinterpret_cast<float4*>(w_in), n4_in, 0x4u);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  tf32_split3_kernel<<<(unsigned)((n4_f + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(filt), reinterpret_cast<float4*>(w_filt), n4_f, 0x2u);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(2, std::memory_order_relaxed);
+  return fprop_umma(&d3, 4, w_in, w_filt, out, stream);
+}
+
+// ---------------------------------------------------------------------------
 // Allocation-free fp32 entry point.  The status block its kernel reports into
 // lives in this file-scope device array instead of cudaMalloc'd memory.  Every
 // device that loads the library carries these 256 bytes until the process ends.
@@ -978,6 +1023,22 @@ maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_ki
     return fprop_fp32(dims_from2(*desc), static_cast<const float*>(in),
                       static_cast<const float*>(filt), out, stream);
   return fprop_umma(dims_from2(*desc), kind == MAXDNN_KERNEL_BF16 ? 2 : 4, in, filt, out, stream);
+}
+
+maxdnn_status maxdnn_conv_fprop_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
+  if (!bytes) return MAXDNN_INVALID_VALUE;
+  size_t a = 0, b = 0;
+  const maxdnn_status st = tf32x3_sizes(desc, &a, &b);
+  if (st != MAXDNN_OK) return st;
+  *bytes = a + b;
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in,
+                                       const float* filt, float* out, void* workspace,
+                                       size_t workspace_bytes, void* cuda_stream) {
+  return fprop_tf32x3(desc, in, filt, out, workspace, workspace_bytes,
+                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,

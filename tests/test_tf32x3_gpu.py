@@ -1,0 +1,62 @@
+"""Three-product TF32 FPROP (fp32 operands split into hi + lo, one TF32 launch over 3 Nc
+channels): accuracy class between exact fp32 (<= 1e-5 required, ~1e-6 measured) and plain
+TF32 (<= 5e-3 required, ~7e-4 measured) — required here: <= 5e-5 of the largest output."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1501_06633_b200 as mx
+from paper_1501_06633_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+TOL_X3 = 5e-5
+
+
+def run(w, inp, filt):
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    out = torch.full((mx.conv_out_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_fprop_tf32x3(d, torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda(), out, ws)
+    assert mx.last_device_status() == mx.OK
+    Ho, Wo = mx.conv_out_dims(d)
+    return out.cpu().numpy().reshape(w.No, Ho, Wo, w.Nb)
+
+
+@pytest.mark.parametrize("shape", [
+    (64, 14, 9, 32, 64, 3, 1, 1, 1.0),
+    (128, 9, 7, 48, 96, 5, 1, 2, 0.5),
+    (32, 23, 19, 3, 96, 11, 4, 0, 1.0),      # 9 split channels: filter columns merged into K
+    (64, 12, 10, 100, 256, 3, 2, 1, 1.0),
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_tf32x3_small(shape):
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("x3", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), 4400 + Sk)
+    inp, filt = wl.make_inputs(w)
+    got = run(w, inp, filt)
+    ref = oracle.conv_fprop(inp, filt, stride=stride, pad=pad, alpha=alpha)
+    assert np.isfinite(got).all()
+    err = float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref)))
+    assert err <= TOL_X3
+    # and it really is better than one TF32 product: the plain TF32 kernel on the same data
+    d = mx.ConvDesc.make(*w.dims)
+    out1 = torch.empty(mx.conv_out_elems(d), device="cuda")
+    mx.conv_fprop_tf32(d, torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda(), out1)
+    err1 = float(np.max(np.abs(out1.cpu().numpy().reshape(ref.shape).astype(np.float64) - ref))) / \
+        float(np.max(np.abs(ref)))
+    assert err < err1 / 8
+
+
+@pytest.mark.parametrize("name", ["mid5x5", "large3x3", "first11x11s4"])
+def test_tf32x3_full_size_sampled(name):
+    w = wl.WORKLOADS[name]
+    inp, filt = wl.make_inputs(w)
+    got = run(w, inp, filt)
+    assert np.isfinite(got).all()
+    Ho = got.shape[1]
+    for y in sorted({0, Ho // 2, Ho - 1}):
+        ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha,
+                                rows=(y, y + 1))[:, y]
+        err = float(np.max(np.abs(got[:, y].astype(np.float64) - ref))) / float(np.max(np.abs(ref)))
+        assert err <= TOL_X3
