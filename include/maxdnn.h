@@ -293,8 +293,7 @@ maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_ki
  * fp32: exact fp32 on the CUDA cores; tf32: the same fp32 buffers on the tensor
  * cores; bf16: `in` and `dout` are bfloat16.  dfilt is fp32 for every kind.
  * NOT_SUPPORTED: a row of images not a multiple of 16 bytes (Nb % 4 for fp32 /
- * tf32, % 8 for bf16), No not a multiple of 4, Sk larger than the map, the
- * limits of maxdnn_conv_fprop.
+ * tf32, % 8 for bf16), No not a multiple of 4, the limits of maxdnn_conv_fprop.
  */
 maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
                                                maxdnn_kernel_kind kind, size_t* bytes);

@@ -477,7 +477,6 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   if (st != MAXDNN_OK) return st;
   if (!g || sm_count <= 0) return MAXDNN_INVALID_VALUE;
   if ((d.Nb * eb) % 16 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule
-  if (d.Sk > d.Wi || d.Sk > d.Hi) return MAXDNN_NOT_SUPPORTED;       // a copy box must fit the map
   memset(g, 0, sizeof(*g));
   g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
   g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
