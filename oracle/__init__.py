@@ -77,6 +77,11 @@ def _load():
         lib.oracle_conv2_fprop.restype = ctypes.c_int
         lib.oracle_conv2_fprop.argtypes = [P(ConvDesc2), ctypes.c_void_p, ctypes.c_void_p,
                                            ctypes.c_void_p, ctypes.c_int32]
+        for name in ("oracle_conv2_bprop_data", "oracle_conv2_bprop_filter"):
+            fn = getattr(lib, name)
+            fn.restype = ctypes.c_int
+            fn.argtypes = [P(ConvDesc2), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                           ctypes.c_int32]
         for name in ("oracle_conv_bprop_data", "oracle_conv_bprop_filter"):
             fn = getattr(lib, name)
             fn.restype = ctypes.c_int
@@ -182,6 +187,40 @@ def conv2_fprop(inp, filt, *, stride=(1, 1), pad=(0, 0), alpha=1.0, nthreads=0):
     if rc:
         raise RuntimeError("oracle_conv2_fprop failed (%d)" % rc)
     return out
+
+
+def conv2_bprop_data(dout, filt, in_hw, *, stride=(1, 1), pad=(0, 0), alpha=1.0, nthreads=0):
+    """din[Nc,Hi,Wi,Nb] for the per-axis operation; ``stride`` / ``pad`` are (h, w) pairs."""
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    filt = np.ascontiguousarray(filt, dtype=np.float32)
+    No, Ho, Wo, Nb = dout.shape
+    Nc, Skh, Skw, _ = filt.shape
+    Hi, Wi = in_hw
+    d = ConvDesc2(Nb, Wi, Hi, Nc, No, Skw, Skh, int(stride[1]), int(stride[0]), int(pad[1]),
+                  int(pad[0]), float(alpha))
+    din = np.zeros((Nc, Hi, Wi, Nb), dtype=np.float32)
+    rc = _load().oracle_conv2_bprop_data(ctypes.byref(d), dout.ctypes.data, filt.ctypes.data,
+                                         din.ctypes.data, int(nthreads))
+    if rc:
+        raise RuntimeError("oracle_conv2_bprop_data failed (%d)" % rc)
+    return din
+
+
+def conv2_bprop_filter(inp, dout, filt_hw, *, stride=(1, 1), pad=(0, 0), alpha=1.0, nthreads=0):
+    """dfilt[Nc,Skh,Skw,No] for the per-axis operation; ``filt_hw`` = (Skh, Skw)."""
+    inp = np.ascontiguousarray(inp, dtype=np.float32)
+    dout = np.ascontiguousarray(dout, dtype=np.float32)
+    Nc, Hi, Wi, Nb = inp.shape
+    No = dout.shape[0]
+    Skh, Skw = filt_hw
+    d = ConvDesc2(Nb, Wi, Hi, Nc, No, Skw, Skh, int(stride[1]), int(stride[0]), int(pad[1]),
+                  int(pad[0]), float(alpha))
+    dfilt = np.zeros((Nc, Skh, Skw, No), dtype=np.float32)
+    rc = _load().oracle_conv2_bprop_filter(ctypes.byref(d), inp.ctypes.data, dout.ctypes.data,
+                                           dfilt.ctypes.data, int(nthreads))
+    if rc:
+        raise RuntimeError("oracle_conv2_bprop_filter failed (%d)" % rc)
+    return dfilt
 
 
 def conv_bprop_data(dout, filt, in_hw, *, stride=1, pad=0, alpha=1.0, nthreads=0):

@@ -199,3 +199,103 @@ double oracle_conv_bprop_filter_point(const oracle_conv_desc* d, const float* in
   if (abs_sum) *abs_sum = a;
   return (double)d->alpha * s;
 }
+
+/*
+ * The same two adjoints for the operation with per-axis filter size, stride and padding
+ * (the relaxed-boundary generalisation; filt and dfilt are [Nc][Skh][Skw][No]):
+ *
+ *   din  [c,h,w,n]   = alpha * sum over (o,y,x,kh,kw) with y*stride_h-pad_h+kh = h and
+ *                      x*stride_w-pad_w+kw = w of filt[c,kh,kw,o] * dout[o,y,x,n]
+ *   dfilt[c,kh,kw,o] = alpha * sum_{y,x,n} in0[c, y*stride_h-pad_h+kh, x*stride_w-pad_w+kw, n]
+ *                                          * dout[o,y,x,n]
+ */
+typedef struct oracle_conv_desc2 {
+  int32_t Nb, Wi, Hi, Nc, No, Skw, Skh, stride_w, stride_h, pad_w, pad_h;
+  float alpha;
+} oracle_conv_desc2;
+
+int oracle_conv2_out_dims(const oracle_conv_desc2* d, int32_t* Ho, int32_t* Wo);
+
+int oracle_conv2_bprop_data(const oracle_conv_desc2* d, const float* dout, const float* filt,
+                            float* din, int32_t nthreads) {
+  int32_t Ho, Wo;
+  if (!dout || !filt || !din || oracle_conv2_out_dims(d, &Ho, &Wo)) return 1;
+  const int Nb = d->Nb, Wi = d->Wi, Hi = d->Hi, Nc = d->Nc, No = d->No;
+  const int Skw = d->Skw, Skh = d->Skh;
+  const double alpha = (double)d->alpha;
+  int bad_alloc = 0;
+  set_threads(nthreads);
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)Nb);
+    if (!s) {
+#pragma omp atomic write
+      bad_alloc = 1;
+    }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+    for (int c = 0; c < Nc; ++c) {
+      for (int h = 0; h < Hi; ++h) {
+        if (!s) continue;
+        for (int w = 0; w < Wi; ++w) {
+          for (int n = 0; n < Nb; ++n) s[n] = 0.0;
+          for (int kh = 0; kh < Skh; ++kh) {
+            const int ys = h + d->pad_h - kh; /* = y * stride_h */
+            if (ys < 0 || ys % d->stride_h != 0) continue;
+            const int y = ys / d->stride_h;
+            if (y >= Ho) continue;
+            for (int kw = 0; kw < Skw; ++kw) {
+              const int xs = w + d->pad_w - kw;
+              if (xs < 0 || xs % d->stride_w != 0) continue;
+              const int x = xs / d->stride_w;
+              if (x >= Wo) continue;
+              const float* frow = filt + (((size_t)c * Skh + kh) * Skw + kw) * (size_t)No;
+              for (int o = 0; o < No; ++o) {
+                const double f = (double)frow[o];
+                const float* g = dout + (((size_t)o * Ho + y) * Wo + x) * (size_t)Nb;
+                for (int n = 0; n < Nb; ++n) s[n] += f * (double)g[n];
+              }
+            }
+          }
+          float* dst = din + (((size_t)c * Hi + h) * Wi + w) * (size_t)Nb;
+          for (int n = 0; n < Nb; ++n) dst[n] = (float)(alpha * s[n]);
+        }
+      }
+    }
+    free(s);
+  }
+  return bad_alloc;
+}
+
+int oracle_conv2_bprop_filter(const oracle_conv_desc2* d, const float* in, const float* dout,
+                              float* dfilt, int32_t nthreads) {
+  int32_t Ho, Wo;
+  if (!in || !dout || !dfilt || oracle_conv2_out_dims(d, &Ho, &Wo)) return 1;
+  const int Nb = d->Nb, Wi = d->Wi, Hi = d->Hi, Nc = d->Nc, No = d->No;
+  const int Skw = d->Skw, Skh = d->Skh;
+  const double alpha = (double)d->alpha;
+  set_threads(nthreads);
+#pragma omp parallel for collapse(3) schedule(dynamic, 1)
+  for (int c = 0; c < Nc; ++c) {
+    for (int kh = 0; kh < Skh; ++kh) {
+      for (int kw = 0; kw < Skw; ++kw) {
+        float* dst = dfilt + (((size_t)c * Skh + kh) * Skw + kw) * (size_t)No;
+        for (int o = 0; o < No; ++o) {
+          double s = 0.0;
+          for (int y = 0; y < Ho; ++y) {
+            const int h = y * d->stride_h - d->pad_h + kh;
+            if (h < 0 || h >= Hi) continue;
+            for (int x = 0; x < Wo; ++x) {
+              const int w = x * d->stride_w - d->pad_w + kw;
+              if (w < 0 || w >= Wi) continue;
+              const float* px = in + (((size_t)c * Hi + h) * Wi + w) * (size_t)Nb;
+              const float* g = dout + (((size_t)o * Ho + y) * Wo + x) * (size_t)Nb;
+              for (int n = 0; n < Nb; ++n) s += (double)px[n] * (double)g[n];
+            }
+          }
+          dst[o] = (float)(alpha * s);
+        }
+      }
+    }
+  }
+  return 0;
+}

@@ -242,3 +242,45 @@ def test_points_agree_with_full_and_threads_do_not_matter():
         c, kh, kw, o = (int(rng.integers(0, s)) for s in dfilt.shape)
         v, a = oracle.conv_bprop_filter_point(inp, dout, Sk, c, kh, kw, o, stride=stride, pad=pad, alpha=alpha)
         assert np.float32(v) == dfilt[c, kh, kw, o] and a >= abs(v) / abs(alpha) - 1e-12
+
+
+# ----------------------------------------------------------------------------
+# per-axis filter size / stride / padding
+# ----------------------------------------------------------------------------
+RECT = [
+    # Nb Wi Hi Nc No Skw Skh (sh, sw) (ph, pw) alpha
+    (2, 7, 5, 2, 3, 3, 1, (1, 1), (0, 1), 1.0),
+    (2, 6, 8, 1, 2, 2, 5, (2, 1), (2, 0), 0.5),
+    (1, 9, 7, 2, 2, 4, 3, (1, 3), (1, 2), -1.5),
+    (3, 8, 6, 2, 2, 3, 2, (3, 2), (0, 1), 1.0),
+    (3, 5, 5, 2, 2, 3, 3, (2, 2), (1, 1), 1.0),        # square: must equal the square oracle
+]
+
+
+@pytest.mark.parametrize("shape", RECT, ids=lambda s: "x".join(str(v) for v in s))
+def test_per_axis_gradients_match_library_autograd_and_adjoint_identities(shape):
+    Nb, Wi, Hi, Nc, No, Skw, Skh, stride, pad, alpha = shape
+    rng = np.random.default_rng(71 + Skw * 5 + Skh)
+    inp = rng.uniform(-1, 1, size=(Nc, Hi, Wi, Nb)).astype(np.float32)
+    filt = rng.uniform(-1, 1, size=(Nc, Skh, Skw, No)).astype(np.float32)
+    out = oracle.conv2_fprop(inp, filt, stride=stride, pad=pad, alpha=alpha)
+    dout = rng.uniform(-1, 1, size=out.shape).astype(np.float32)
+    din = oracle.conv2_bprop_data(dout, filt, (Hi, Wi), stride=stride, pad=pad, alpha=alpha)
+    dfilt = oracle.conv2_bprop_filter(inp, dout, (Skh, Skw), stride=stride, pad=pad, alpha=alpha)
+    # library autograd, fp64
+    x = torch.from_numpy(inp).double().permute(3, 0, 1, 2).clone().requires_grad_(True)
+    w = torch.from_numpy(filt).double().permute(3, 0, 1, 2).clone().requires_grad_(True)
+    y = alpha * torch.nn.functional.conv2d(x, w, stride=stride, padding=pad)
+    y.backward(torch.from_numpy(dout).double().permute(3, 0, 1, 2))
+    assert close(din, x.grad.permute(1, 2, 3, 0).numpy(), 2 * F32_ROUND)
+    assert close(dfilt, w.grad.permute(1, 2, 3, 0).numpy(), 2 * F32_ROUND)
+    # adjoint identities against the per-axis forward oracle (pinned on its own)
+    lhs = float(np.sum(dout.astype(np.float64) * out))
+    scale = float(np.sum(np.abs(dout.astype(np.float64) * out))) + 1e-30
+    assert abs(lhs - float(np.sum(din.astype(np.float64) * inp))) <= 1e-5 * scale
+    assert abs(lhs - float(np.sum(dfilt.astype(np.float64) * filt))) <= 1e-5 * scale
+    if Skw == Skh and stride[0] == stride[1] and pad[0] == pad[1]:
+        np.testing.assert_array_equal(din, oracle.conv_bprop_data(dout, filt, (Hi, Wi), stride=stride[0],
+                                                                  pad=pad[0], alpha=alpha))
+        np.testing.assert_array_equal(dfilt, oracle.conv_bprop_filter(inp, dout, Skh, stride=stride[0],
+                                                                      pad=pad[0], alpha=alpha))
