@@ -257,6 +257,19 @@ typedef struct maxdnn_conv_desc2 {
 maxdnn_status maxdnn_conv2_out_dims(const maxdnn_conv_desc2* desc, int32_t* Ho, int32_t* Wo);
 maxdnn_status maxdnn_conv2_fprop(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
                                  const void* in, const void* filt, float* out, void* cuda_stream);
+/* The two gradients of the per-axis operation: as maxdnn_conv_bprop_data / _filter below,
+ * with every Sk, stride and pad read per axis (dfilt is [Nc][Skh][Skw][No]). */
+maxdnn_status maxdnn_conv2_bprop_data_workspace(const maxdnn_conv_desc2* desc,
+                                                maxdnn_kernel_kind kind, size_t* bytes);
+maxdnn_status maxdnn_conv2_bprop_data(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                      const void* dout, const void* filt, float* din,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+maxdnn_status maxdnn_conv2_bprop_filter_workspace(const maxdnn_conv_desc2* desc,
+                                                  maxdnn_kernel_kind kind, size_t* bytes);
+maxdnn_status maxdnn_conv2_bprop_filter(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                        const void* in, const void* dout, float* dfilt,
+                                        void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream);
 
 /*
  * Backward propagation.  The paper builds FPROP only and names BPROP (Abstract,

@@ -19,6 +19,8 @@ __all__ = [
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
     "conv_fprop_tf32x3_workspace", "conv_fprop_tf32x3",
     "ConvDesc2", "conv2_out_dims", "conv2_fprop", "conv2_fprop_status",
+    "conv2_bprop_data_workspace", "conv2_bprop_data", "conv2_bprop_filter_workspace",
+    "conv2_bprop_filter",
     "conv_fprop_ragged_workspace", "conv_fprop_ragged", "fprop_ragged_status",
     "conv_bprop_data_workspace", "conv_bprop_data", "bprop_data_status",
     "conv_bprop_filter_workspace", "conv_bprop_filter", "bprop_filter_status",
@@ -37,6 +39,8 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv_fprop_ragged_workspace", "maxdnn_conv_fprop_ragged",
     "maxdnn_conv2_out_dims", "maxdnn_conv2_fprop",
     "maxdnn_conv_fprop_tf32x3_workspace", "maxdnn_conv_fprop_tf32x3",
+    "maxdnn_conv2_bprop_data_workspace", "maxdnn_conv2_bprop_data",
+    "maxdnn_conv2_bprop_filter_workspace", "maxdnn_conv2_bprop_filter",
 ]
 
 
@@ -130,6 +134,12 @@ def load_library():
     lib.maxdnn_conv2_out_dims.argtypes = [P(ConvDesc2), P(ctypes.c_int32), P(ctypes.c_int32)]
     lib.maxdnn_conv2_fprop.restype = ctypes.c_int
     lib.maxdnn_conv2_fprop.argtypes = [P(ConvDesc2), ctypes.c_int, vp, vp, vp, vp]
+    for name in ("maxdnn_conv2_bprop_data_workspace", "maxdnn_conv2_bprop_filter_workspace"):
+        getattr(lib, name).restype = ctypes.c_int
+        getattr(lib, name).argtypes = [P(ConvDesc2), ctypes.c_int, P(ctypes.c_size_t)]
+    for name in ("maxdnn_conv2_bprop_data", "maxdnn_conv2_bprop_filter"):
+        getattr(lib, name).restype = ctypes.c_int
+        getattr(lib, name).argtypes = [P(ConvDesc2), ctypes.c_int, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.maxdnn_conv_fprop_ragged_workspace.restype = ctypes.c_int
     lib.maxdnn_conv_fprop_ragged_workspace.argtypes = [P(ConvDesc), ctypes.c_int, P(ctypes.c_size_t)]
     lib.maxdnn_conv_fprop_ragged.restype = ctypes.c_int
@@ -327,6 +337,56 @@ def conv2_fprop_status(desc: ConvDesc2, inp, filt, out, kind: int = KERNEL_FP32,
 def conv2_fprop(desc: ConvDesc2, inp, filt, out, kind: int = KERNEL_FP32, stream=None) -> None:
     """maxdnn_conv2_fprop: FPROP with per-axis filter size, stride and padding."""
     _check(conv2_fprop_status(desc, inp, filt, out, kind, stream), "maxdnn_conv2_fprop")
+
+
+def _conv2_sizes(desc: ConvDesc2):
+    Ho, Wo = conv2_out_dims(desc)
+    return (desc.Nc * desc.Hi * desc.Wi * desc.Nb, desc.Nc * desc.Skh * desc.Skw * desc.No,
+            desc.No * Ho * Wo * desc.Nb)
+
+
+def conv2_bprop_data_workspace(desc: ConvDesc2, kind: int = KERNEL_FP32) -> int:
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv2_bprop_data_workspace(ctypes.byref(desc), int(kind),
+                                                                ctypes.byref(n))),
+           "maxdnn_conv2_bprop_data_workspace")
+    return int(n.value)
+
+
+def conv2_bprop_data(desc: ConvDesc2, dout, filt, din, workspace, kind: int = KERNEL_FP32,
+                     stream=None) -> None:
+    """maxdnn_conv2_bprop_data: map gradient of the per-axis operation."""
+    n_in, n_f, n_out = _conv2_sizes(desc)
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pg = _dev_ptr(dout, in_types, n_out, "dout")
+    pf = _dev_ptr(filt, in_types, n_f, "filt")
+    pd = _dev_ptr(din, ("float32",), n_in, "din")
+    pw, nbytes = _workspace_ptr(workspace, 1)
+    _check(int(load_library().maxdnn_conv2_bprop_data(ctypes.byref(desc), int(kind), pg, pf, pd, pw,
+                                                      nbytes, _stream_ptr(stream))),
+           "maxdnn_conv2_bprop_data")
+
+
+def conv2_bprop_filter_workspace(desc: ConvDesc2, kind: int = KERNEL_FP32) -> int:
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv2_bprop_filter_workspace(ctypes.byref(desc), int(kind),
+                                                                  ctypes.byref(n))),
+           "maxdnn_conv2_bprop_filter_workspace")
+    return int(n.value)
+
+
+def conv2_bprop_filter(desc: ConvDesc2, inp, dout, dfilt, workspace, kind: int = KERNEL_FP32,
+                       stream=None) -> None:
+    """maxdnn_conv2_bprop_filter: filter gradient of the per-axis operation."""
+    n_in, n_f, n_out = _conv2_sizes(desc)
+    in_types = ("bfloat16", "uint16", "int16") if kind == KERNEL_BF16 else ("float32",)
+    pi = _dev_ptr(inp, in_types, n_in, "in")
+    pg = _dev_ptr(dout, in_types, n_out, "dout")
+    pd = _dev_ptr(dfilt, ("float32",), n_f, "dfilt")
+    pw, nbytes = _workspace_ptr(workspace, 0)
+    _check(int(load_library().maxdnn_conv2_bprop_filter(ctypes.byref(desc), int(kind), pi, pg, pd,
+                                                        pw, nbytes, _stream_ptr(stream))),
+           "maxdnn_conv2_bprop_filter")
 
 
 def conv_fprop_ragged_workspace(desc: ConvDesc, kind: int = KERNEL_FP32) -> int:

@@ -1,7 +1,7 @@
 // Backward-propagation kernels (the adjoints of the operation of Section 2; the paper
 // names BPROP in its Abstract and Section 3.5 ("Conclusion") as where its techniques should carry over).
 //
-//  - flip_transpose_kernel: filt[c][kh][kw][o] -> ft[o][Sk-1-kh][Sk-1-kw][c], the filter
+//  - flip_transpose_kernel: filt[c][kh][kw][o] -> ft[o][Skh-1-kh][Skw-1-kw][c], the filter
 //    bank with which the gradient with respect to the maps is an FPROP of the output
 //    gradient (stride 1).
 //  - wgrad_kernel: gradient with respect to the filters in exact fp32.  The same
@@ -25,9 +25,8 @@ namespace maxdnn {
 
 template <typename T>
 __global__ void __launch_bounds__(256)
-flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int Sk, int No) {
+flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int taps, int No) {
   __shared__ T tile[32][33];
-  const int taps = Sk * Sk;
   const int tap = blockIdx.z;              // kh * Sk + kw
   const int tap_t = taps - 1 - tap;        // (Sk-1-kh) * Sk + (Sk-1-kw)
   const int o0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
@@ -43,18 +42,19 @@ flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, in
 }
 
 // Strided map gradient: the sub-filter of one class, flipped and transposed:
-//   ft[o][j'][i'][c] = filt[c][rho_h + s (Jh-1-j')][rho_w + s (Jw-1-i')][o]
+//   ft[o][j'][i'][c] = filt[c][rho_h + s_h (Jh-1-j')][rho_w + s_w (Jw-1-i')][o]
 template <typename T>
 __global__ void __launch_bounds__(256)
-subfilter_flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int Sk,
-                                int No, int s, int rho_h, int rho_w, int Jh, int Jw) {
+subfilter_flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, int Nc, int Skh,
+                                int Skw, int No, int s_h, int s_w, int rho_h, int rho_w, int Jh,
+                                int Jw) {
   __shared__ T tile[32][33];
   const int jp = blockIdx.z / Jw, ip = blockIdx.z % Jw;     // position in the transformed bank
-  const int kh = rho_h + s * (Jh - 1 - jp), kw = rho_w + s * (Jw - 1 - ip);
+  const int kh = rho_h + s_h * (Jh - 1 - jp), kw = rho_w + s_w * (Jw - 1 - ip);
   const int o0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
   for (int i = threadIdx.y; i < 32; i += 8) {
     const int c = c0 + i, o = o0 + threadIdx.x;
-    if (c < Nc && o < No) tile[i][threadIdx.x] = filt[(((size_t)c * Sk + kh) * Sk + kw) * No + o];
+    if (c < Nc && o < No) tile[i][threadIdx.x] = filt[(((size_t)c * Skh + kh) * Skw + kw) * No + o];
   }
   __syncthreads();
   for (int i = threadIdx.y; i < 32; i += 8) {
@@ -63,10 +63,11 @@ subfilter_flip_transpose_kernel(const T* __restrict__ filt, T* __restrict__ ft, 
   }
 }
 
-// din[c][h_first + s a][w_first + s b][n] = sub[c][a][b][n]: the class's gradient onto its grid.
+// din[c][h_first + s_h a][w_first + s_w b][n] = sub[c][a][b][n]: the class's gradient onto its grid.
 __global__ void __launch_bounds__(256)
 dgrad_scatter_kernel(const float4* __restrict__ sub, float4* __restrict__ din, int Nc, int n_h,
-                     int n_w, int nb4, int Hi, int Wi, int s, int h_first, int w_first) {
+                     int n_w, int nb4, int Hi, int Wi, int s_h, int s_w, int h_first,
+                     int w_first) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t total = (size_t)Nc * n_h * n_w * nb4;
   if (i >= total) return;
@@ -75,7 +76,7 @@ dgrad_scatter_kernel(const float4* __restrict__ sub, float4* __restrict__ din, i
   const int b = (int)(r % n_w); r /= n_w;
   const int a = (int)(r % n_h);
   const int c = (int)(r / n_h);
-  din[(((size_t)c * Hi + h_first + s * a) * Wi + w_first + s * b) * nb4 + n] = sub[i];
+  din[(((size_t)c * Hi + h_first + s_h * a) * Wi + w_first + s_w * b) * nb4 + n] = sub[i];
 }
 
 // Split of fp32 values for the three-product TF32 scheme: hi = the value with its low 13
@@ -216,8 +217,8 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
     const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
     mbar_arrive_expect_tx(fb, tx_bytes);
     tma_load_4d(dst, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
-    tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride - g.pad,
-                pc.y * g.stride - g.pad + pc.khb * g.bh, pc.cb * g.bc);
+    tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride_w - g.pad_w,
+                pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc);
     if (++p_stage == stages) { p_stage = 0; p_phase ^= 1u; }
     pc.advance(g, (int)gridDim.x);
   };
@@ -306,7 +307,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
 
     // ---------------------------------------------- store this item's 128 x 128 block
     const bool direct = (g.splits == 1);
-    const size_t K = (size_t)g.Nc * g.Sk * g.Sk;
+    const size_t K = (size_t)g.Nc * g.Skh * g.Skw;
     float* dst_base = direct ? args.dfilt : args.partial + (size_t)split * K * g.No;
     const float scale = direct ? g.alpha : 1.0f;
     const int o = ob * 128 + to;
@@ -319,8 +320,8 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
       const int h_l = t % g.bh;
       const int c = cb * g.bc + t / g.bh;
       const int kh = khb * g.bh + h_l;
-      if (c >= g.Nc || kh >= g.Sk) continue;
-      float* dst = dst_base + (((size_t)c * g.Sk + kh) * g.Sk + w_l) * g.No + o;
+      if (c >= g.Nc || kh >= g.Skh) continue;
+      float* dst = dst_base + (((size_t)c * g.Skh + kh) * g.Skw + w_l) * g.No + o;
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         if (o + 16 * j < g.No) dst[16 * j] = (acc[i][j].x + acc[i][j].y) * scale;

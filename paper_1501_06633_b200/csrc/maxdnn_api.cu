@@ -352,12 +352,12 @@ bool kind_ok(maxdnn_kernel_kind k) {
 }
 
 // Checks that the forward kernel of `kind` takes the transposed problem.
-maxdnn_status dgrad_plan_check(const maxdnn_conv_desc& fd, maxdnn_kernel_kind kind, int sm_count) {
+maxdnn_status dgrad_plan_check(const ConvDims& fd, maxdnn_kernel_kind kind, int sm_count) {
   static thread_local ConvGeom g;
   static thread_local KStepTable t;
   if (kind == MAXDNN_KERNEL_FP32)
-    return plan_ffma(dims_from(fd), sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
-  return plan_umma(dims_from(fd), kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
+    return plan_ffma(fd, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
+  return plan_umma(fd, kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
                    env_int("MAXDNN_UMMA_PAIR"), &g, &t);
 }
 
@@ -367,15 +367,15 @@ struct DgradStridedPlan {
   size_t ft_bytes, sub_bytes;
 };
 
-maxdnn_status plan_dgrad_strided(const maxdnn_conv_desc& d, size_t eb, DgradStridedPlan* p) {
+maxdnn_status plan_dgrad_strided(const ConvDims& d, size_t eb, DgradStridedPlan* p) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
-  const int s = d.stride;
   size_t jmax = 0, nmax = 0;
-  for (int rh = 0; rh < s; ++rh)
-    for (int rw = 0; rw < s; ++rw) {
-      const DgradAxis ah = dgrad_axis(rh, d.Sk, s, d.pad, d.Hi), aw = dgrad_axis(rw, d.Sk, s, d.pad, d.Wi);
+  for (int rh = 0; rh < d.stride_h; ++rh)
+    for (int rw = 0; rw < d.stride_w; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, d.Skh, d.stride_h, d.pad_h, d.Hi);
+      const DgradAxis aw = dgrad_axis(rw, d.Skw, d.stride_w, d.pad_w, d.Wi);
       const size_t j = (size_t)ah.J * aw.J, n = (size_t)ah.n * aw.n;
       if (j > jmax) jmax = j;
       if (n > nmax) nmax = n;
@@ -385,37 +385,36 @@ maxdnn_status plan_dgrad_strided(const maxdnn_conv_desc& d, size_t eb, DgradStri
   return MAXDNN_OK;
 }
 
-maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
-                                 const void* dout, const void* filt, float* din, void* ws,
-                                 size_t ws_bytes, cudaStream_t stream) {
+maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, const void* dout,
+                                 const void* filt, float* din, void* ws, size_t ws_bytes,
+                                 cudaStream_t stream) {
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   DgradStridedPlan p;
-  maxdnn_status st = plan_dgrad_strided(*desc, eb, &p);
+  maxdnn_status st = plan_dgrad_strided(d, eb, &p);
   if (st != MAXDNN_OK) return st;
   if (ws_bytes < p.ft_bytes + p.sub_bytes) return MAXDNN_INVALID_VALUE;
-  if (desc->Nb % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+  if (d.Nb % 4 != 0) return MAXDNN_NOT_SUPPORTED;
   DeviceState* ds = nullptr;
   st = device_state(&ds);
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
   int32_t Ho, Wo;
-  check_desc(desc, &Ho, &Wo);
-  const int s = desc->stride;
+  check_dims(d, &Ho, &Wo);
+  const int sh = d.stride_h, sw = d.stride_w;
   uint8_t* w_ft = static_cast<uint8_t*>(ws);
   float* w_sub = reinterpret_cast<float*>(w_ft + p.ft_bytes);
   // Positions that no tap reaches (a class without taps, or whose window lies outside
   // dout) must read zero: clear din first if there is such a class.
   bool all_covered = true;
-  for (int rh = 0; rh < s; ++rh)
-    for (int rw = 0; rw < s; ++rw) {
-      const DgradAxis ah = dgrad_axis(rh, desc->Sk, s, desc->pad, desc->Hi);
-      const DgradAxis aw = dgrad_axis(rw, desc->Sk, s, desc->pad, desc->Wi);
+  for (int rh = 0; rh < sh; ++rh)
+    for (int rw = 0; rw < sw; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, d.Skh, sh, d.pad_h, d.Hi);
+      const DgradAxis aw = dgrad_axis(rw, d.Skw, sw, d.pad_w, d.Wi);
       if (ah.n == 0 || aw.n == 0) continue;                     // no positions: nothing to cover
       if (ah.J == 0 || aw.J == 0 || ah.crop >= Ho || aw.crop >= Wo) all_covered = false;
     }
   if (!all_covered &&
-      cudaMemsetAsync(din, 0, (size_t)desc->Nc * desc->Hi * desc->Wi * desc->Nb * 4, stream) !=
-          cudaSuccess) {
+      cudaMemsetAsync(din, 0, (size_t)d.Nc * d.Hi * d.Wi * d.Nb * 4, stream) != cudaSuccess) {
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
@@ -423,39 +422,40 @@ maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kin
   // grid inside din directly; the fp32 kernel writes a dense scratch tensor that a copy
   // kernel scatters.
   const bool direct = kind != MAXDNN_KERNEL_FP32;
-  for (int rh = 0; rh < s; ++rh) {
-    for (int rw = 0; rw < s; ++rw) {
-      const DgradAxis ah = dgrad_axis(rh, desc->Sk, s, desc->pad, desc->Hi);
-      const DgradAxis aw = dgrad_axis(rw, desc->Sk, s, desc->pad, desc->Wi);
+  for (int rh = 0; rh < sh; ++rh) {
+    for (int rw = 0; rw < sw; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, d.Skh, sh, d.pad_h, d.Hi);
+      const DgradAxis aw = dgrad_axis(rw, d.Skw, sw, d.pad_w, d.Wi);
       if (ah.J == 0 || aw.J == 0 || ah.n == 0 || aw.n == 0) continue;
       if (ah.crop >= Ho || aw.crop >= Wo) continue;            // its windows miss dout entirely
       ConvDims fd;
-      fd.Nb = desc->Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = desc->No;
-      fd.No = desc->Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
-      fd.pad_w = aw.pad; fd.pad_h = ah.pad; fd.alpha = desc->alpha;
-      fd.in_h_stride = (int64_t)Wo * desc->Nb;
-      fd.in_c_stride = (int64_t)Ho * Wo * desc->Nb;
+      fd.Nb = d.Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = d.No;
+      fd.No = d.Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
+      fd.pad_w = aw.pad; fd.pad_h = ah.pad; fd.alpha = d.alpha;
+      fd.in_h_stride = (int64_t)Wo * d.Nb;
+      fd.in_c_stride = (int64_t)Ho * Wo * d.Nb;
       fd.Ho_given = ah.n; fd.Wo_given = aw.n;
-      const dim3 grid((unsigned)ceil_div(desc->No, 32), (unsigned)ceil_div(desc->Nc, 32),
+      fd.out_x_stride = fd.out_y_stride = fd.out_o_stride = 0;
+      const dim3 grid((unsigned)ceil_div(d.No, 32), (unsigned)ceil_div(d.Nc, 32),
                       (unsigned)(ah.J * aw.J));
       const dim3 block(32, 8);
       if (eb == 2)
         subfilter_flip_transpose_kernel<uint16_t><<<grid, block, 0, stream>>>(
-            static_cast<const uint16_t*>(filt), reinterpret_cast<uint16_t*>(w_ft), desc->Nc,
-            desc->Sk, desc->No, s, ah.rho, aw.rho, ah.J, aw.J);
+            static_cast<const uint16_t*>(filt), reinterpret_cast<uint16_t*>(w_ft), d.Nc, d.Skh,
+            d.Skw, d.No, sh, sw, ah.rho, aw.rho, ah.J, aw.J);
       else
         subfilter_flip_transpose_kernel<float><<<grid, block, 0, stream>>>(
-            static_cast<const float*>(filt), reinterpret_cast<float*>(w_ft), desc->Nc, desc->Sk,
-            desc->No, s, ah.rho, aw.rho, ah.J, aw.J);
+            static_cast<const float*>(filt), reinterpret_cast<float*>(w_ft), d.Nc, d.Skh, d.Skw,
+            d.No, sh, sw, ah.rho, aw.rho, ah.J, aw.J);
       if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
       g_launches.fetch_add(1, std::memory_order_relaxed);
       const uint8_t* src = static_cast<const uint8_t*>(dout) +
-                           ((size_t)ah.crop * Wo + aw.crop) * desc->Nb * eb;
+                           ((size_t)ah.crop * Wo + aw.crop) * d.Nb * eb;
       if (direct) {
-        fd.out_x_stride = (int64_t)s * desc->Nb;
-        fd.out_y_stride = (int64_t)s * desc->Wi * desc->Nb;
-        fd.out_o_stride = (int64_t)desc->Hi * desc->Wi * desc->Nb;
-        float* dst = din + ((size_t)ah.first * desc->Wi + aw.first) * desc->Nb;
+        fd.out_x_stride = (int64_t)sw * d.Nb;
+        fd.out_y_stride = (int64_t)sh * d.Wi * d.Nb;
+        fd.out_o_stride = (int64_t)d.Hi * d.Wi * d.Nb;
+        float* dst = din + ((size_t)ah.first * d.Wi + aw.first) * d.Nb;
         st = fprop_umma(fd, (int)eb, src, w_ft, dst, stream);
         if (st != MAXDNN_OK) return st;
         continue;
@@ -463,11 +463,11 @@ maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kin
       st = fprop_fp32(fd, reinterpret_cast<const float*>(src), reinterpret_cast<const float*>(w_ft),
                       w_sub, stream);
       if (st != MAXDNN_OK) return st;
-      const int nb4 = desc->Nb / 4;
-      const size_t total = (size_t)desc->Nc * ah.n * aw.n * nb4;
+      const int nb4 = d.Nb / 4;
+      const size_t total = (size_t)d.Nc * ah.n * aw.n * nb4;
       dgrad_scatter_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
-          reinterpret_cast<const float4*>(w_sub), reinterpret_cast<float4*>(din), desc->Nc, ah.n,
-          aw.n, nb4, desc->Hi, desc->Wi, s, ah.first, aw.first);
+          reinterpret_cast<const float4*>(w_sub), reinterpret_cast<float4*>(din), d.Nc, ah.n, aw.n,
+          nb4, d.Hi, d.Wi, sh, sw, ah.first, aw.first);
       if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
       g_launches.fetch_add(1, std::memory_order_relaxed);
     }
@@ -475,22 +475,23 @@ maxdnn_status bprop_data_strided(const maxdnn_conv_desc* desc, maxdnn_kernel_kin
   return MAXDNN_OK;
 }
 
-maxdnn_status bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* dout,
+maxdnn_status bprop_data(const ConvDims& d, maxdnn_kernel_kind kind, const void* dout,
                          const void* filt, float* din, void* ws, size_t ws_bytes,
                          cudaStream_t stream) {
-  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (!kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_dims(d, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
   if (!dout || !filt || !din || !ws) return MAXDNN_INVALID_VALUE;
   if (!aligned16(dout) || !aligned16(filt) || !aligned16(din) || !aligned16(ws))
     return MAXDNN_INVALID_VALUE;
-  if (desc->stride != 1)
-    return bprop_data_strided(desc, kind, dout, filt, din, ws, ws_bytes, stream);
-  maxdnn_conv_desc fd;
-  st = plan_dgrad(*desc, &fd);
+  if (d.stride_w != 1 || d.stride_h != 1)
+    return bprop_data_strided(d, kind, dout, filt, din, ws, ws_bytes, stream);
+  ConvDims fd;
+  st = plan_dgrad(d, &fd);
   if (st != MAXDNN_OK) return st;
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
-  const size_t need = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * eb;
+  const int taps = d.Skh * d.Skw;
+  const size_t need = (size_t)d.Nc * taps * d.No * eb;
   if (ws_bytes < need) return MAXDNN_INVALID_VALUE;
   DeviceState* ds = nullptr;
   st = device_state(&ds);
@@ -498,27 +499,45 @@ maxdnn_status bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, 
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
   st = dgrad_plan_check(fd, kind, ds->sm_count);
   if (st != MAXDNN_OK) return st;
-  const dim3 grid((unsigned)ceil_div(desc->No, 32), (unsigned)ceil_div(desc->Nc, 32),
-                  (unsigned)(desc->Sk * desc->Sk));
+  const dim3 grid((unsigned)ceil_div(d.No, 32), (unsigned)ceil_div(d.Nc, 32), (unsigned)taps);
   const dim3 block(32, 8);
   if (eb == 2)
     flip_transpose_kernel<uint16_t><<<grid, block, 0, stream>>>(
-        static_cast<const uint16_t*>(filt), static_cast<uint16_t*>(ws), desc->Nc, desc->Sk, desc->No);
+        static_cast<const uint16_t*>(filt), static_cast<uint16_t*>(ws), d.Nc, taps, d.No);
   else
     flip_transpose_kernel<float><<<grid, block, 0, stream>>>(
-        static_cast<const float*>(filt), static_cast<float*>(ws), desc->Nc, desc->Sk, desc->No);
+        static_cast<const float*>(filt), static_cast<float*>(ws), d.Nc, taps, d.No);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (kind == MAXDNN_KERNEL_FP32)
-    return fprop_fp32(&fd, static_cast<const float*>(dout), static_cast<const float*>(ws), din, stream);
-  return fprop_umma(&fd, (int)eb, dout, ws, din, stream);
+    return fprop_fp32(fd, static_cast<const float*>(dout), static_cast<const float*>(ws), din, stream);
+  return fprop_umma(fd, (int)eb, dout, ws, din, stream);
 }
 
-maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind, const void* in,
+maxdnn_status bprop_data_workspace(const ConvDims& d, maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_dims(d, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  if (d.stride_w != 1 || d.stride_h != 1) {
+    DgradStridedPlan p;
+    st = plan_dgrad_strided(d, eb, &p);
+    if (st != MAXDNN_OK) return st;
+    *bytes = p.ft_bytes + p.sub_bytes;
+    return MAXDNN_OK;
+  }
+  ConvDims fd;
+  st = plan_dgrad(d, &fd);
+  if (st != MAXDNN_OK) return st;
+  *bytes = (size_t)d.Nc * d.Skh * d.Skw * d.No * eb;
+  return MAXDNN_OK;
+}
+
+maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const void* in,
                            const void* dout, float* dfilt, void* ws, size_t ws_bytes,
                            cudaStream_t stream) {
-  if (!desc || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (!kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_dims(d, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
   if (!in || !dout || !dfilt) return MAXDNN_INVALID_VALUE;
   if (!aligned16(in) || !aligned16(dout) || !aligned16(dfilt) || !aligned16(ws))
@@ -533,10 +552,10 @@ maxdnn_status bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
   static thread_local WgradArgs fargs;
   static thread_local WgradUmmaArgs uargs;
   WgradGeom& g = tensor ? uargs.g : fargs.g;
-  st = plan_wgrad(*desc, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
+  st = plan_wgrad(d, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
                   env_int("MAXDNN_WGRAD_PAIR"));
   if (st != MAXDNN_OK) return st;
-  const size_t kno = (size_t)g.Nc * g.Sk * g.Sk * g.No;
+  const size_t kno = (size_t)g.Nc * g.Skh * g.Skw * g.No;
   const size_t need = g.splits > 1 ? (size_t)g.splits * kno * 4 : 0;
   if (need > 0 && (!ws || ws_bytes < need)) return MAXDNN_INVALID_VALUE;
   const CUtensorMapDataType dt =
@@ -695,7 +714,7 @@ maxdnn_status fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind
   st = device_state(&ds);
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
-  st = dgrad_plan_check(p.padded, kind, ds->sm_count);   // the padded problem must have a plan
+  st = dgrad_plan_check(dims_from(p.padded), kind, ds->sm_count);   // the padded problem must have a plan
   if (st != MAXDNN_OK) return st;
   int32_t Ho, Wo;
   check_desc(desc, &Ho, &Wo);
@@ -756,7 +775,7 @@ maxdnn_status fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in, const 
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
   maxdnn_conv_desc d3 = *desc;
   d3.Nc = 3 * desc->Nc;
-  st = dgrad_plan_check(d3, MAXDNN_KERNEL_TF32, ds->sm_count);   // the 3 Nc-channel problem has a plan
+  st = dgrad_plan_check(dims_from(d3), MAXDNN_KERNEL_TF32, ds->sm_count);   // the 3 Nc-channel problem has a plan
   if (st != MAXDNN_OK) return st;
   float* w_in = static_cast<float*>(ws);
   float* w_filt = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + in_bytes);
@@ -1061,34 +1080,25 @@ maxdnn_status maxdnn_conv_fprop_ragged(const maxdnn_conv_desc* desc, maxdnn_kern
 
 maxdnn_status maxdnn_conv_bprop_data_workspace(const maxdnn_conv_desc* desc,
                                                maxdnn_kernel_kind kind, size_t* bytes) {
-  if (!desc || !bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  const maxdnn_status st = check_desc(desc, nullptr, nullptr);
   if (st != MAXDNN_OK) return st;
-  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
-  if (desc->stride != 1) {
-    DgradStridedPlan p;
-    st = plan_dgrad_strided(*desc, eb, &p);
-    if (st != MAXDNN_OK) return st;
-    *bytes = p.ft_bytes + p.sub_bytes;
-    return MAXDNN_OK;
-  }
-  maxdnn_conv_desc fd;
-  st = plan_dgrad(*desc, &fd);
-  if (st != MAXDNN_OK) return st;
-  *bytes = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * eb;
-  return MAXDNN_OK;
+  return bprop_data_workspace(dims_from(*desc), kind, bytes);
 }
 
 maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
                                      const void* dout, const void* filt, float* din,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  return bprop_data(desc, kind, dout, filt, din, workspace, workspace_bytes,
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  const maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  return bprop_data(dims_from(*desc), kind, dout, filt, din, workspace, workspace_bytes,
                     static_cast<cudaStream_t>(cuda_stream));
 }
 
-maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
-                                                 maxdnn_kernel_kind kind, size_t* bytes) {
-  if (!desc || !bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
+static maxdnn_status bprop_filter_workspace(const maxdnn::ConvDims& d, maxdnn_kernel_kind kind,
+                                            size_t* bytes) {
+  if (!bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
   int sm_count = env_int("MAXDNN_SM_COUNT");   // planning without a device (tests)
   if (sm_count <= 0) {
     DeviceState* ds = nullptr;
@@ -1098,18 +1108,58 @@ maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
   }
   WgradGeom g;
   const int eb = kind == MAXDNN_KERNEL_FP32 ? 0 : (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
-  const maxdnn_status st = plan_wgrad(*desc, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
+  const maxdnn_status st = plan_wgrad(d, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
                                       env_int("MAXDNN_WGRAD_PAIR"));
   if (st != MAXDNN_OK) return st;
-  *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Sk * g.Sk * g.No * 4 : 0;
+  *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Skh * g.Skw * g.No * 4 : 0;
   return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_filter_workspace(const maxdnn_conv_desc* desc,
+                                                 maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  const maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  return bprop_filter_workspace(dims_from(*desc), kind, bytes);
+}
+
+maxdnn_status maxdnn_conv2_bprop_filter_workspace(const maxdnn_conv_desc2* desc,
+                                                  maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return bprop_filter_workspace(dims_from2(*desc), kind, bytes);
+}
+
+maxdnn_status maxdnn_conv2_bprop_filter(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                        const void* in, const void* dout, float* dfilt,
+                                        void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return bprop_filter(dims_from2(*desc), kind, in, dout, dfilt, workspace, workspace_bytes,
+                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv2_bprop_data_workspace(const maxdnn_conv_desc2* desc,
+                                                maxdnn_kernel_kind kind, size_t* bytes) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return bprop_data_workspace(dims_from2(*desc), kind, bytes);
+}
+
+maxdnn_status maxdnn_conv2_bprop_data(const maxdnn_conv_desc2* desc, maxdnn_kernel_kind kind,
+                                      const void* dout, const void* filt, float* din,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  return bprop_data(dims_from2(*desc), kind, dout, filt, din, workspace, workspace_bytes,
+                    static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
                                        const void* in, const void* dout, float* dfilt,
                                        void* workspace, size_t workspace_bytes,
                                        void* cuda_stream) {
-  return bprop_filter(desc, kind, in, dout, dfilt, workspace, workspace_bytes,
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  const maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  return bprop_filter(dims_from(*desc), kind, in, dout, dfilt, workspace, workspace_bytes,
                       static_cast<cudaStream_t>(cuda_stream));
 }
 

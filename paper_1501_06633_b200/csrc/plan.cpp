@@ -452,36 +452,42 @@ maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int for
   return have ? MAXDNN_OK : first;
 }
 
-maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* f) {
+maxdnn_status plan_dgrad(const ConvDims& d, ConvDims* f) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (!f) return MAXDNN_INVALID_VALUE;
-  if (d.stride != 1 || d.pad > d.Sk - 1) return MAXDNN_NOT_SUPPORTED;
-  f->Nb = d.Nb; f->Wi = Wo; f->Hi = Ho; f->Nc = d.No; f->No = d.Nc; f->Sk = d.Sk;
-  f->stride = 1; f->pad = d.Sk - 1 - d.pad; f->alpha = d.alpha;
+  if (d.stride_w != 1 || d.stride_h != 1 || d.pad_w > d.Skw - 1 || d.pad_h > d.Skh - 1)
+    return MAXDNN_NOT_SUPPORTED;
+  *f = d;
+  f->Wi = Wo; f->Hi = Ho; f->Nc = d.No; f->No = d.Nc;
+  f->pad_w = d.Skw - 1 - d.pad_w; f->pad_h = d.Skh - 1 - d.pad_h;
+  f->in_h_stride = f->in_c_stride = 0;
+  f->Ho_given = f->Wo_given = 0;
+  f->out_x_stride = f->out_y_stride = f->out_o_stride = 0;
   return MAXDNN_OK;
 }
 
-maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
+maxdnn_status plan_wgrad(const ConvDims& d, int elem_bytes, int sm_count, int force_splits,
                          WgradGeom* g, int force_pair) {
   int32_t Ho, Wo;
-  maxdnn_status st = check_desc(&d, &Ho, &Wo);
+  maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   if (elem_bytes != 0 && elem_bytes != 4 && elem_bytes != 2) return MAXDNN_INVALID_VALUE;
   const bool tensor = elem_bytes != 0;
   const int eb = tensor ? elem_bytes : 4;
   const int max_rows = tensor ? 256 : 128;
   const int chunk = 128 / eb;                                         // images per reduction step
-  st = common_limits(dims_from(d), eb);
+  st = common_limits(d, eb);
   if (st != MAXDNN_OK) return st;
   if (!g || sm_count <= 0) return MAXDNN_INVALID_VALUE;
   if ((d.Nb * eb) % 16 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;   // 16-byte row rule
   memset(g, 0, sizeof(*g));
-  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No; g->Sk = d.Sk;
-  g->stride = d.stride; g->pad = d.pad; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
-  g->bw = d.Sk;
-  g->bh = d.Sk < max_rows / g->bw ? d.Sk : max_rows / g->bw;
+  g->Nb = d.Nb; g->Wi = d.Wi; g->Hi = d.Hi; g->Nc = d.Nc; g->No = d.No;
+  g->Skw = d.Skw; g->Skh = d.Skh; g->stride_w = d.stride_w; g->stride_h = d.stride_h;
+  g->pad_w = d.pad_w; g->pad_h = d.pad_h; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
+  g->bw = d.Skw;
+  g->bh = d.Skh < max_rows / g->bw ? d.Skh : max_rows / g->bw;
   if (g->bh < 1) return MAXDNN_NOT_SUPPORTED;
   g->bc = max_rows / (g->bw * g->bh);
   if (g->bc > 256) g->bc = 256;                                       // a copy box has at most 256 per axis
@@ -502,7 +508,7 @@ maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count
   g->n_mma = g->pair ? 2 * align_up(g->rows_h, 8) : align_up(g->rows, 16);
   g->box_o = d.No < 128 ? d.No : 128;
   g->c_blocks = ceil_div(d.Nc, g->bc);
-  g->kh_blocks = ceil_div(d.Sk, g->bh);
+  g->kh_blocks = ceil_div(d.Skh, g->bh);
   g->o_blocks = ceil_div(d.No, g->pair ? 256 : 128);
   g->n_chunks = ceil_div(d.Nb, chunk);
   const int64_t r_steps = (int64_t)Ho * Wo * g->n_chunks;

@@ -89,9 +89,9 @@ maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int for
 
 // Gradient with respect to the maps, stride 1: FPROP of the output gradient with
 // the filter bank transposed (channels <-> filters) and flipped in both axes and
-// padding Sk - 1 - pad.  Fills the descriptor of that FPROP.  NOT_SUPPORTED for
-// stride != 1 or pad > Sk - 1.
-maxdnn_status plan_dgrad(const maxdnn_conv_desc& d, maxdnn_conv_desc* fprop_desc);
+// padding Sk - 1 - pad (per axis).  Fills the dims of that FPROP.  NOT_SUPPORTED for
+// a stride != 1 or a pad > Sk - 1.
+maxdnn_status plan_dgrad(const ConvDims& d, ConvDims* fprop_dims);
 
 // Gradient with respect to the maps, stride s > 1: the map positions split into s x s
 // classes by (h + pad) mod s, (w + pad) mod s; a class only meets the filter taps
@@ -117,7 +117,7 @@ DgradAxis dgrad_axis(int rho, int Sk, int s, int pad, int size_in);
 // step = 32 images of one output pixel.  The reduction is split over `splits`
 // CTAs per tile whose partial sums a second kernel adds in a fixed order.
 struct WgradGeom {
-  int32_t Nb, Wi, Hi, Nc, No, Sk, stride, pad, Ho, Wo;
+  int32_t Nb, Wi, Hi, Nc, No, Skw, stride_w, pad_w, Ho, Wo;   // w-axis filter size, stride, padding
   float alpha;
   int32_t bc, bh, bw;        // channels x filter rows x filter columns per tile
   int32_t rows;              // bc * bh * bw <= 128
@@ -131,12 +131,13 @@ struct WgradGeom {
   // tensor-core kernel on a pair of CTAs (256 filters per tile; each CTA stages its 128
   // filters and half of the tile's channels): channels / gradient rows per CTA, MMA N
   int32_t pair, bc_h, rows_h, n_mma;
+  int32_t Skh, stride_h, pad_h;   // h-axis filter size, stride, padding
 };
 
 // force_splits > 0 pins the number of reduction splits (tests, ablations).
 // elem_bytes 0: the fp32 FFMA2 kernel (128 gradient rows per tile, 32 images per step);
 // 4 / 2: the tensor-core kernel with TF32 / BF16 operands (256 rows; 32 / 64 images).
-maxdnn_status plan_wgrad(const maxdnn_conv_desc& d, int elem_bytes, int sm_count, int force_splits,
+maxdnn_status plan_wgrad(const ConvDims& d, int elem_bytes, int sm_count, int force_splits,
                          WgradGeom* g, int force_pair = 0);
 
 }  // namespace maxdnn

@@ -86,7 +86,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
     const int t = row / g.bw;
     const int h_l = t % g.bh;
     const int c_l = t / g.bh;
-    row_tab[row] = make_int2((c_l * g.Sk + h_l) * g.Sk + w_l, (c_l << 16) | h_l);
+    row_tab[row] = make_int2((c_l * g.Skh + h_l) * g.Skw + w_l, (c_l << 16) | h_l);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -117,8 +117,8 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       if (elect_one()) {
         mbar_arrive_expect_tx(fb, tx_bytes);
         tma_load_4d_hint(dst, &map_dout, fb, n0, pc.x, pc.y, pc.ob * 128, pol_last);
-        tma_load_4d_hint(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride - g.pad,
-                         pc.y * g.stride - g.pad + pc.khb * g.bh, pc.cb * g.bc, pol_last);
+        tma_load_4d_hint(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride_w - g.pad_w,
+                         pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc, pol_last);
       }
       __syncwarp();
       if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -189,7 +189,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t it = 0;
     bool ok = true;
     const bool direct = (g.splits == 1);
-    const size_t K = (size_t)g.Nc * g.Sk * g.Sk;
+    const size_t K = (size_t)g.Nc * g.Skh * g.Skw;
     const float scale = direct ? g.alpha : 1.0f;
     while (ok && !cc.done(g)) {
       const uint32_t acc = it & 1u;
@@ -200,9 +200,9 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       tcgen05_fence_after();
       const int o = cc.ob * 128 + q * 32 + lane;
       const int c_lim = g.Nc - cc.cb * g.bc;          // channels / filter rows of this tile
-      const int h_lim = g.Sk - cc.khb * g.bh;         // that exist
+      const int h_lim = g.Skh - cc.khb * g.bh;         // that exist
       float* dst = (direct ? args.dfilt : args.partial + (size_t)cc.split * K * g.No) +
-                   ((size_t)(cc.cb * g.bc) * g.Sk + (size_t)cc.khb * g.bh) * g.Sk * g.No + o;
+                   ((size_t)(cc.cb * g.bc) * g.Skh + (size_t)cc.khb * g.bh) * g.Skw * g.No + o;
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256u;
       for (int col = 0; col < g.rows; col += 32) {
         uint32_t v[32];

@@ -73,7 +73,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
       const int t = row / g.bw;
       const int h_l = t % g.bh;
       const int c_l = half * g.bc_h + t / g.bh;
-      row_tab[col] = make_int2((c_l * g.Sk + h_l) * g.Sk + w_l, (c_l << 16) | h_l);
+      row_tab[col] = make_int2((c_l * g.Skh + h_l) * g.Skw + w_l, (c_l << 16) | h_l);
     } else {
       row_tab[col] = make_int2(0, 0x7fff << 16);             // no such row: never stored
     }
@@ -111,8 +111,8 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
       if (elect_one()) {
         if (rank == 0) mbar_arrive_expect_tx(full_bar + 8u * stage, tx_bytes);
         tma_load_4d_pair(dst, &map_dout, fb, n0, pc.x, pc.y, pc.ob * 256 + (int)rank * 128, pol_last);
-        tma_load_4d_pair(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride - g.pad,
-                         pc.y * g.stride - g.pad + pc.khb * g.bh,
+        tma_load_4d_pair(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride_w - g.pad_w,
+                         pc.y * g.stride_h - g.pad_h + pc.khb * g.bh,
                          pc.cb * g.bc + (int)rank * g.bc_h, pol_last);
       }
       __syncwarp();
@@ -183,7 +183,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t it = 0;
     bool ok = true;
     const bool direct = (g.splits == 1);
-    const size_t K = (size_t)g.Nc * g.Sk * g.Sk;
+    const size_t K = (size_t)g.Nc * g.Skh * g.Skw;
     const float scale = direct ? g.alpha : 1.0f;
     while (ok && !cc.done(g)) {
       const uint32_t acc = it & 1u;
@@ -194,9 +194,9 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
       tcgen05_fence_after();
       const int o = cc.ob * 256 + (int)rank * 128 + q * 32 + lane;
       const int c_lim = g.Nc - cc.cb * g.bc;
-      const int h_lim = g.Sk - cc.khb * g.bh;
+      const int h_lim = g.Skh - cc.khb * g.bh;
       float* dst = (direct ? args.dfilt : args.partial + (size_t)cc.split * K * g.No) +
-                   ((size_t)(cc.cb * g.bc) * g.Sk + (size_t)cc.khb * g.bh) * g.Sk * g.No + o;
+                   ((size_t)(cc.cb * g.bc) * g.Skh + (size_t)cc.khb * g.bh) * g.Skw * g.No + o;
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256u;
       for (int col = 0; col < g.n_mma; col += 32) {
         uint32_t v[32];

@@ -113,5 +113,24 @@ def test_random_per_axis_shapes(kernel):
         shape = (Nb, Wi, Hi, Nc, No, Skw, Skh, sw, sh, pw, ph)
         assert mx.conv2_fprop_status(d, x, f, out, KIND[kernel]) == mx.OK, shape
         assert rel(out.cpu().numpy().reshape(ref.shape), ref) <= TOL[kernel], shape
+        # both gradients of the per-axis operation
+        dout = rng.uniform(-1, 1, size=ref.shape).astype(np.float32)
+        (g,), (rg,) = operands(kernel, dout)
+        ws = torch.empty(max(16, mx.conv2_bprop_filter_workspace(d, KIND[kernel])), dtype=torch.uint8,
+                         device="cuda")
+        dfilt = torch.full((filt.size,), float("nan"), device="cuda")
+        mx.conv2_bprop_filter(d, x, g, dfilt, ws, KIND[kernel])
+        rdf = oracle.conv2_bprop_filter(rx, rg, (Skh, Skw), stride=(sh, sw), pad=(ph, pw), alpha=alpha)
+        assert rel(dfilt.cpu().numpy().reshape(rdf.shape), rdf) <= TOL[kernel], ("wgrad", shape)
+        try:
+            need = mx.conv2_bprop_data_workspace(d, KIND[kernel])
+            ws = torch.empty(max(16, need), dtype=torch.uint8, device="cuda")
+            din = torch.full((inp.size,), float("nan"), device="cuda")
+            mx.conv2_bprop_data(d, g, f, din, ws, KIND[kernel])
+        except mx.MaxdnnError as e:
+            assert e.status == mx.NOT_SUPPORTED, ("dgrad", shape)    # transposed problem refused
+        else:
+            rdi = oracle.conv2_bprop_data(rg, rf, (Hi, Wi), stride=(sh, sw), pad=(ph, pw), alpha=alpha)
+            assert rel(din.cpu().numpy().reshape(rdi.shape), rdi) <= TOL[kernel], ("dgrad", shape)
         done += 1
     assert mx.last_device_status() == mx.OK
