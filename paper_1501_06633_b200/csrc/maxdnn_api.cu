@@ -107,6 +107,26 @@ int env_int(const char* name) {
   return v ? atoi(v) : 0;
 }
 
+// What a forward plan depends on: the problem, the device's SM count and the tuning
+// switches read from the environment.  A call that repeats the previous call's key on the
+// same thread keeps the previous plan (planning costs 1.5-4 us, a third of the host time of
+// a call; small layers are launch-bound).
+struct PlanKey {
+  ConvDims d;
+  int32_t v[8];
+  bool valid = false;
+};
+
+int env_or(const char* name, int unset) {
+  const char* v = getenv(name);
+  return v ? atoi(v) : unset;
+}
+
+bool same_plan_key(const PlanKey& a, const PlanKey& b) {
+  return a.valid && b.valid && memcmp(&a.d, &b.d, sizeof(ConvDims)) == 0 &&
+         memcmp(a.v, b.v, sizeof(a.v)) == 0;
+}
+
 template <int MR, int NR, bool FIXED>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
@@ -159,9 +179,20 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
-  st = plan_ffma(cd, ds->sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"),
-                 &args.g, &args.table);
-  if (st != MAXDNN_OK) return st;
+  static thread_local PlanKey last;
+  PlanKey key;
+  memset(&key, 0, sizeof(key));
+  key.d = cd;
+  key.v[0] = ds->sm_count;
+  key.v[1] = env_int("MAXDNN_FFMA_TILE_M");
+  key.v[2] = env_int("MAXDNN_FFMA_COLS");
+  key.valid = true;
+  if (!same_plan_key(key, last)) {
+    last.valid = false;
+    st = plan_ffma(cd, ds->sm_count, key.v[1], key.v[2], &args.g, &args.table);
+    if (st != MAXDNN_OK) return st;
+    last = key;
+  }
   args.out = out;
   args.status = ds->status;
   args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see FfmaArgs
@@ -262,9 +293,24 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local UmmaArgs args;
-  st = plan_umma(cd, elem_bytes, ds->sm_count, env_int("MAXDNN_UMMA_KC"),
-                 env_int("MAXDNN_UMMA_PAIR"), &args.g, &args.table);
-  if (st != MAXDNN_OK) return st;
+  static thread_local PlanKey last;
+  PlanKey key;
+  memset(&key, 0, sizeof(key));
+  key.d = cd;
+  key.v[0] = ds->sm_count;
+  key.v[1] = elem_bytes;
+  key.v[2] = env_int("MAXDNN_UMMA_KC");
+  key.v[3] = env_int("MAXDNN_UMMA_PAIR");
+  key.v[4] = env_or("MAXDNN_UMMA_MERGE", -12345);
+  key.v[5] = env_or("MAXDNN_UMMA_STAGE_KB", -12345);
+  key.v[6] = env_or("MAXDNN_UMMA_COLS", -12345);
+  key.valid = true;
+  if (!same_plan_key(key, last)) {
+    last.valid = false;
+    st = plan_umma(cd, elem_bytes, ds->sm_count, key.v[2], key.v[3], &args.g, &args.table);
+    if (st != MAXDNN_OK) return st;
+    last = key;
+  }
   const ConvGeom& g = args.g;
   const uint64_t eb = (uint64_t)elem_bytes;
   const uint32_t atom = 128u / (uint32_t)elem_bytes;
