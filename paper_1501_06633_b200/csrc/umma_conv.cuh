@@ -7,9 +7,10 @@
 // swizzle, which is exactly the shared-memory layout the MMA descriptors read.
 //
 // A persistent CTA per SM walks tiles of 128 filters x (tile_px pixels x tile_n
-// images) <= 256 columns.  Warp 0: one lane walks the K-step table and issues the
-// copies (apron zero-filled by the copy engine).  Warp 1: one lane issues the MMAs
-// into one of two TMEM accumulators and commits to the ring's "empty" barriers.
+// images) <= 256 columns.  Warps 0 and 6 walk the K-step table and issue the copies of
+// the patch boxes and of the filter boxes (one elected lane each; apron zero-filled by
+// the copy engine).  Warp 1: one lane issues the MMAs into one of two TMEM
+// accumulators and commits to the ring's "empty" barriers.
 // Warps 2-5: epilogue — TMEM -> registers, alpha, swizzled staging tile in shared
 // memory, bulk tensor store of 32 filters x 32 images (full 128-byte lines), while
 // the MMA warp already fills the other accumulator.
