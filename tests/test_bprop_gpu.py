@@ -254,3 +254,29 @@ def test_full_size_sampled_bprop_data(name, kernel):
             assert abs(float(got[p]) - v) <= (K + 3) * 2.0 ** -24 * abs(w.alpha) * a + 1e-30
         else:
             assert abs(float(got[p]) - v) <= TOL[kernel] * scale
+
+
+@pytest.mark.parametrize("kernel", ["fp32", "bf16"])
+def test_full_size_sampled_strided_bprop_data(kernel):
+    """A full-size stride-2 layer (56 x 56 x 128 -> 256, 3 x 3): four classes with 2x2, 2x1, 1x2
+    and 1x1 taps; sampled elements of din, corners and both parities of h, w included."""
+    w = wl.WORKLOADS["large3x3"].scaled(stride=2)
+    _, filt = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_workspace(d, KIND[kernel]), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data(d, dev(dout, kernel), dev(filt, kernel), din, ws, KIND[kernel])
+    assert mx.last_device_status() == mx.OK
+    got = din.cpu().numpy().reshape(w.Nc, w.Hi, w.Wi, w.Nb)
+    assert np.isfinite(got).all()
+    rd, rf = rounded(dout, kernel), rounded(filt, kernel)
+    rng = np.random.default_rng(6)
+    pts = [tuple(int(rng.integers(0, s)) for s in got.shape) for _ in range(200)]
+    pts += [(0, 0, 0, 0), (0, 0, 1, 0), (0, 1, 0, 0), (0, 1, 1, 0),
+            (w.Nc - 1, w.Hi - 1, w.Wi - 1, w.Nb - 1), (5, w.Hi - 2, w.Wi - 1, 7)]
+    vals = [oracle.conv_bprop_data_point(rd, rf, (w.Hi, w.Wi), *p, stride=w.stride, pad=w.pad,
+                                         alpha=w.alpha) for p in pts]
+    scale = max(abs(v) for v, _ in vals)
+    for p, (v, a) in zip(pts, vals):
+        assert abs(float(got[p]) - v) <= 1e-5 * scale, p
