@@ -108,8 +108,8 @@ typedef struct maxdnn_plan_info {
   int32_t tile_m;      /* filters per tile (rows of the GEMM block) */
   int32_t tile_px;     /* adjacent output pixels (along x) per tile */
   int32_t tile_n;      /* images per tile */
-  int32_t kc;          /* channels per K step */
-  int32_t kwc;         /* filter columns per K step (1 or Sk) */
+  int32_t kc;          /* channels per K step (few-channel tensor plans: K rows of one filter row) */
+  int32_t kwc;         /* filter columns per K step (1 or Sk; few-channel plans with a shared strip: filter rows per step) */
   int32_t n_ksteps;    /* length of the K-step table */
   int32_t stages;      /* depth of the shared-memory ring */
   int32_t n_tiles;     /* tiles in the whole problem */

@@ -326,6 +326,14 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   args.lbo_b_bytes = (uint32_t)g.kc * 128u;
   args.tap_a_bytes = (uint32_t)g.kc * 128u;
   args.tap_b_bytes = (uint32_t)(g.cta_n / (int)atom) * (uint32_t)g.kc * 128u;
+  if (g.box_c != g.kc) {
+    // few-channel plan (filter columns merged into K): a pixel's window starts
+    // b_slot_bytes after its neighbour's (its own box, or a shift inside the one strip);
+    // with the strip the MMA warp's outer loop walks the filter rows of the step, which
+    // are one strip row (patches) / one box row (filters) apart
+    args.lbo_b_bytes = (uint32_t)g.b_slot_bytes;
+    args.tap_b_bytes = (uint32_t)(g.b_box_w * g.box_c) * 128u;
+  }
   // next group of channel rows: 8 rows for the 16-byte-chunk swizzle, 4 rows for the
   // 32-byte-chunk swizzle of 4-byte operands
   args.sbo_bytes = bf16 ? 1024u : 512u;

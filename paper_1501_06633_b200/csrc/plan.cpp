@@ -339,17 +339,30 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   }
   if (force_kc > 0 && force_kc % umma_k == 0 && force_kc <= 256) kc = force_kc;
   int n = 0;
+  bool merged_strip = false;
+  int strip_w = 0;
   if (merged) {
     const int box_c = align_up(d.Nc, 4);
     int box_kw = d.Skw;
     while ((box_kw * box_c) % umma_k != 0) ++box_kw;
     const int rows1 = box_kw * box_c;                     // K rows of one filter row
+    // The windows of adjacent output pixels overlap (stride < Sk), so ONE box of
+    // box_kw + (pixels - 1) * stride columns serves all pixels of the tile: pixel j's
+    // operand starts j * stride * box_c rows into it, which the swizzle allows when that
+    // is a whole number of 8-row groups.  11 x 11 stride 4: 24 columns instead of 4 x 12.
+    strip_w = box_kw + (px_cta - 1) * d.stride_w;
+    merged_strip = px_cta > 1 && (d.stride_w * box_c) % 8 == 0 && d.stride_w < box_kw &&
+                   strip_w <= 256;
+    const int b_rows1 = merged_strip ? strip_w * box_c * (g->cta_n / atom) : cols / atom * rows1;
     int khc = 1;   // filter rows per step: stages of at most 40 KB (a deep ring beat longer steps)
-    while (khc < d.Skh && (128 + cols) * rows1 * (khc + 1) * elem_bytes <= 40 * 1024) ++khc;
+    while (khc < d.Skh && (128 / atom * rows1 + b_rows1) * 128 * (khc + 1) <= 40 * 1024) ++khc;
     if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Skh) khc = v; }
     if (box_kw > 256 || rows1 * khc > 1024) return MAXDNN_NOT_SUPPORTED;
-    kc = rows1 * khc;
-    kwc = 1;
+    // with the strip the rows of one filter row are contiguous in both operands, the
+    // filter rows of a step are not (strip_w vs box_kw columns apart): kc counts the
+    // rows of one filter row and the MMA warp's outer loop (kwc) walks the filter rows
+    kc = merged_strip ? rows1 : rows1 * khc;
+    kwc = merged_strip ? khc : 1;
     for (int kh = 0; kh < d.Skh; kh += khc) {
       if (n >= kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
       t->s[n].c0 = 0; t->s[n].kh = (int8_t)kh; t->s[n].kw0 = 0;
@@ -366,7 +379,12 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   g->a_box_bytes = atom * kc * kwc * elem_bytes;        // one group of filters: kwc x kc rows x 128 B
   g->a_stage_bytes = 128 * kc * kwc * elem_bytes;
   const int strip = px_cta + kwc - 1;
-  if (merged) {
+  if (merged_strip) {
+    g->b_boxes = 1;
+    g->b_box_w = strip_w;
+    g->b_box_bytes = strip_w * g->box_c * g->box_kh * g->cta_n * elem_bytes;
+    g->b_stage_bytes = g->b_box_bytes;
+  } else if (merged) {
     g->b_boxes = px_cta;                                // one window per output pixel
     g->b_box_w = g->box_kw;
     g->b_box_bytes = g->cta_n * kc * elem_bytes;
@@ -388,6 +406,7 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
     g->b_stage_bytes = cols * kc * elem_bytes;
   }
   g->b_slot_bytes = g->b_box_bytes;
+  if (merged_strip) g->b_slot_bytes = d.stride_w * g->box_c * g->cta_n * elem_bytes;   // window to window
   const int stage = g->a_stage_bytes + g->b_stage_bytes;
   const int fixed = 8 * 4096 + 1024 + 512;    // epilogue staging, alignment slack, barriers
   int stages = (227 * 1024 - fixed) / stage;

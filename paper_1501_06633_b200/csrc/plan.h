@@ -57,7 +57,7 @@ struct ConvGeom {
   int32_t b_boxes;         // patch boxes per K step (1, or tile_px)
   int32_t b_box_w;         // extent of a patch box along w
   int32_t b_box_bytes;
-  int32_t b_slot_bytes;    // distance between patch boxes of one stage (128-byte multiple)
+  int32_t b_slot_bytes;    // distance between the windows of adjacent pixels in a stage (separate boxes, or inside one strip)
   int32_t b_stage_bytes;   // patch bytes per stage
   int32_t grid;
   int32_t smem_bytes;

@@ -154,6 +154,23 @@ def test_benchmark_plans_fit_the_device():
     assert mx.conv_plan_query(mx.ConvDesc.make(*wl.WORKLOADS["first11x11s4"].dims))[0].tile_m == 96
 
 
+def test_few_channel_strided_layers_stage_one_strip_per_step():
+    """3-channel 11 x 11 stride-4 layers on the tensor kernels: the windows of the tile's
+    pixels overlap, so a K step stages one strip of 12 + 4 (pixels - 1) columns instead of
+    one 12-column box per pixel, which shows as a smaller stage and a deeper ring; a
+    stride-1 few-channel layer (window shift of 4 rows, not a whole swizzle group) keeps
+    one box per pixel."""
+    d = mx.ConvDesc.make(*wl.WORKLOADS["first11x11s4"].dims)
+    bf, _ = mx.conv_plan_query(d, mx.KERNEL_BF16, 148)
+    tf, _ = mx.conv_plan_query(d, mx.KERNEL_TF32, 148)
+    assert (bf.tile_px, bf.tile_n, bf.kc, bf.n_ksteps * bf.kwc) == (4, 64, 48, 11)
+    assert (tf.tile_px, tf.tile_n, tf.kc, tf.n_ksteps * tf.kwc) == (8, 32, 48, 11)
+    # stage = 128 filters x 48 rows + strip x 4 channels x 128 B: 24 KB (bf16), 44 KB (tf32)
+    assert bf.stages == 8 and tf.stages == 4
+    s1, _ = mx.conv_plan_query(mx.ConvDesc.make(64, 14, 11, 1, 32, 3, 1, 1), mx.KERNEL_BF16, 148)
+    assert s1.kwc == 1 and s1.kc % 16 == 0
+
+
 def test_table1_shapes_give_the_printed_output_sizes_and_have_plans():
     """Table 1 prints input size, kernel and output size per layer; the workload list
     must reproduce the output sizes, and every kernel kind must have a plan for them."""
