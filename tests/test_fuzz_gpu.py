@@ -134,3 +134,39 @@ def test_random_per_axis_shapes(kernel):
             assert rel(din.cpu().numpy().reshape(rdi.shape), rdi) <= TOL[kernel], ("dgrad", shape)
         done += 1
     assert mx.last_device_status() == mx.OK
+
+
+@pytest.mark.parametrize("kernel", ["tf32", "bf16"])
+def test_random_few_channel_strided_shapes(kernel):
+    """Few channels, stride > 1, large filters: the plan that merges filter columns into K
+    and stages one patch strip per step (or one box per pixel where the window shift is not
+    a whole swizzle group), with one or several filter rows per step as the stage budget
+    decides; wide maps so that tiles hold several pixels and the last tile of a row is
+    ragged."""
+    rng = np.random.default_rng({"tf32": 44, "bf16": 55}[kernel])
+    atom = {"tf32": 32, "bf16": 64}[kernel]
+    done = 0
+    while done < 40:
+        Sk = int(rng.integers(2, 12))
+        stride = int(rng.integers(2, 5))
+        pad = int(rng.integers(0, min(Sk, 4)))
+        Wi = int(rng.integers(Sk, 64))
+        Hi = int(rng.integers(Sk, 20))
+        Nb = atom * int(rng.integers(1, 3))
+        Nc = int(rng.integers(1, 8 if kernel == "tf32" else 16))
+        No = 32 * int(rng.integers(1, 6))
+        alpha = float(rng.choice([1.0, -0.5]))
+        w = wl.Workload("fuzz_fc", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
+                        ("uniform", -1.0, 1.0), 9500 + done)
+        d = mx.ConvDesc.make(*w.dims)
+        inp, filt = wl.make_inputs(w)
+        (x, f), (rx, rf) = operands(kernel, inp, filt)
+        out = torch.full((mx.conv_out_elems(d),), float("nan"), device="cuda")
+        st = mx.fprop_status(d, x, f, out, KIND[kernel])
+        if st == mx.NOT_SUPPORTED:
+            continue                      # a step of this shape does not fit two ring stages
+        assert st == mx.OK, w.dims
+        assert mx.last_device_status() == mx.OK
+        ref = oracle.conv_fprop(rx, rf, stride=stride, pad=pad, alpha=alpha)
+        assert rel(out.cpu().numpy().reshape(ref.shape), ref) <= TOL[kernel], w.dims
+        done += 1
