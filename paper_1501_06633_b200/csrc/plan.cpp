@@ -534,21 +534,25 @@ maxdnn_status plan_wgrad(const ConvDims& d, int elem_bytes, int sm_count, int fo
   const int64_t tiles = (int64_t)g->c_blocks * g->kh_blocks * g->o_blocks;
   if (r_steps > 0x3fffffff || tiles > 0x3fffffff) return MAXDNN_NOT_SUPPORTED;
   g->r_steps = (int32_t)r_steps;
-  // Split the reduction so that the items fill whole waves of persistent CTAs (about
-  // four waves when the tiles alone are fewer), each split keeping at least 64 steps.
+  // Split the reduction over CTAs: with s splits the kernel runs ceil(tiles * s / units)
+  // waves of items, each of ceil(r_steps / s) reduction steps plus a fixed cost (filling
+  // the ring, draining the accumulator, writing the partial sums) of about a dozen steps
+  // (fitted to timings of forced split counts on the 5x5, 3x3 and 13x13 layers: the best
+  // counts are the largest that still fill a whole number of waves, and one full wave of
+  // long items beats several waves of short ones).  At least 32 steps per split.
   const int units = g->pair ? sm_count / 2 : sm_count;
   int splits = 1;
   if (force_splits > 0) {
     splits = force_splits;
-  } else if (tiles < 4 * (int64_t)units) {
-    const int64_t want = ceil_div(4 * units, (int)tiles);
-    const int64_t most = r_steps / 64 > 0 ? r_steps / 64 : 1;
-    splits = (int)(want < most ? want : most);
-    // round the item count to whole waves where that is cheap
-    const int64_t items = tiles * splits;
-    const int64_t waves = (items + units - 1) / units;
-    const int64_t fit = waves * units / tiles;
-    if (fit >= 1 && fit <= most) splits = (int)fit;
+  } else {
+    const int64_t most = r_steps / 32 > 0 ? r_steps / 32 : 1;
+    const double fixed = tensor ? 12.0 : 4.0;   // the fp32 kernel's steps are longer
+    double best = 1e300;
+    for (int64_t sp = 1; sp <= most && sp <= 4096; ++sp) {
+      const int64_t waves = (tiles * sp + units - 1) / units;
+      const double cost = (double)waves * ((double)((r_steps + sp - 1) / sp) + fixed);
+      if (cost < best * 0.995) { best = cost; splits = (int)sp; }   // more splits must pay
+    }
   }
   if (splits > r_steps) splits = (int)r_steps;
   if (splits < 1) splits = 1;
