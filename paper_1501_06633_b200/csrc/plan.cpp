@@ -518,10 +518,16 @@ maxdnn_status plan_wgrad(const ConvDims& d, int elem_bytes, int sm_count, int fo
   const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);
   g->pair = (tensor && force_pair >= 0 && (peer_has_filters || force_pair > 0) && g->bc >= 2 &&
              sm_count >= 2) ? 1 : 0;
-  if (g->pair) {
-    g->bc &= ~1;
-    g->bc_h = g->bc / 2;
+  if (g->pair) g->bc &= ~1;
+  // Same number of channel blocks, evenly filled (256 channels, 3 x 3: ten blocks of 26
+  // instead of nine of 28 and one of 4): fewer gradient rows per MMA for the same tiles.
+  {
+    const int blocks = ceil_div(d.Nc, g->bc);
+    int even = ceil_div(d.Nc, blocks);
+    if (g->pair && (even & 1)) ++even;
+    if (even < g->bc) g->bc = even;
   }
+  if (g->pair) g->bc_h = g->bc / 2;
   g->rows = g->bc * g->bh * g->bw;
   g->rows_h = g->pair ? g->rows / 2 : g->rows;
   g->n_mma = g->pair ? 2 * align_up(g->rows_h, 8) : align_up(g->rows, 16);
