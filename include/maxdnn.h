@@ -295,7 +295,12 @@ maxdnn_status maxdnn_conv2_bprop_filter(const maxdnn_conv_desc2* desc, maxdnn_ke
  * (h+pad) mod s, (w+pad) mod s; each class meets only the taps kh = rho_h + s j,
  * kw = rho_w + s i and is, on its own grid, a stride-1 FPROP of dout with that
  * sub-filter (flipped, transposed), written onto the class's grid inside din;
- * positions no tap reaches are zero.  NOT_SUPPORTED: stride 1 with
+ * positions no tap reaches are zero.  The classes are independent launches: they
+ * are queued on the given stream and on three streams the library owns, which
+ * start after the work already queued on the given stream and which the given
+ * stream waits for before the call returns to it (a fork and join by events, valid
+ * under stream capture); each class has its own part of the workspace.
+ * NOT_SUPPORTED: stride 1 with
  * pad > Sk-1, Nb not a multiple of 4 (stride > 1), or what the matching fprop
  * entry point refuses for the transposed problem (its filter count is Nc).
  *

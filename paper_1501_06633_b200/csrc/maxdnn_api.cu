@@ -29,6 +29,12 @@ struct DeviceState {
   bool umma_attr[4] = {false, false, false, false};
   bool wgrad_attr = false;
   bool wgrad_umma_attr[4] = {false, false, false, false};
+  // Side streams for the strided map gradient, whose residue classes are independent
+  // launches: run side by side, the tail wave of one class overlaps the next class.
+  cudaStream_t aux[3] = {nullptr, nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr;
+  cudaEvent_t ev_join[3] = {nullptr, nullptr, nullptr};
+  std::mutex fork_mu;   // one fork / join sequence at a time uses the events
 };
 
 std::mutex g_mu;
@@ -58,6 +64,11 @@ maxdnn_status device_state(DeviceState** out) {
     if (s.sm100) {
       if (cudaMalloc(&s.status, 256) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
       if (cudaMemset(s.status, 0, 256) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+      bool ok = cudaEventCreateWithFlags(&s.ev_fork, cudaEventDisableTiming) == cudaSuccess;
+      for (int i = 0; i < 3 && ok; ++i)
+        ok = cudaStreamCreateWithFlags(&s.aux[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&s.ev_join[i], cudaEventDisableTiming) == cudaSuccess;
+      if (!ok) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
     }
     s.ready = true;
   }
@@ -111,10 +122,10 @@ int env_int(const char* name) {
 // switches read from the environment.  A call that repeats the previous call's key on the
 // same thread keeps the previous plan (planning costs 1.5-4 us, a third of the host time of
 // a call; small layers are launch-bound).
-struct PlanKey {
+struct PlanKey {   // trivial: cleared with memset so that padding compares equal
   ConvDims d;
   int32_t v[8];
-  bool valid = false;
+  bool valid;
 };
 
 int env_or(const char* name, int unset) {
@@ -126,6 +137,29 @@ bool same_plan_key(const PlanKey& a, const PlanKey& b) {
   return a.valid && b.valid && memcmp(&a.d, &b.d, sizeof(ConvDims)) == 0 &&
          memcmp(a.v, b.v, sizeof(a.v)) == 0;
 }
+
+// The plans of the last few distinct problems of this thread (a strided map gradient
+// alternates between its classes' sub-problems; a network between its layers).
+constexpr int kPlanSlots = 8;
+template <class Args>
+struct PlanCache {
+  Args args[kPlanSlots];
+  PlanKey key[kPlanSlots];
+  int next;
+  // The slot that holds `k`'s plan, or -1.
+  int find(const PlanKey& k) const {
+    for (int i = 0; i < kPlanSlots; ++i)
+      if (same_plan_key(k, key[i])) return i;
+    return -1;
+  }
+  // The slot to plan into: the oldest one, marked invalid until the plan succeeds.
+  int take() {
+    const int i = next;
+    next = (next + 1) % kPlanSlots;
+    key[i].valid = false;
+    return i;
+  }
+};
 
 template <int MR, int NR, bool FIXED>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
@@ -178,8 +212,7 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
-  static thread_local FfmaArgs args;   // 4 KB table: keep it off the stack
-  static thread_local PlanKey last;
+  static thread_local PlanCache<FfmaArgs> cache;   // 4 KB tables: kept off the stack
   PlanKey key;
   memset(&key, 0, sizeof(key));
   key.d = cd;
@@ -187,12 +220,14 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   key.v[1] = env_int("MAXDNN_FFMA_TILE_M");
   key.v[2] = env_int("MAXDNN_FFMA_COLS");
   key.valid = true;
-  if (!same_plan_key(key, last)) {
-    last.valid = false;
-    st = plan_ffma(cd, ds->sm_count, key.v[1], key.v[2], &args.g, &args.table);
+  int slot = cache.find(key);
+  if (slot < 0) {
+    slot = cache.take();
+    st = plan_ffma(cd, ds->sm_count, key.v[1], key.v[2], &cache.args[slot].g, &cache.args[slot].table);
     if (st != MAXDNN_OK) return st;
-    last = key;
+    cache.key[slot] = key;
   }
+  FfmaArgs& args = cache.args[slot];
   args.out = out;
   args.status = ds->status;
   args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see FfmaArgs
@@ -292,8 +327,7 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
-  static thread_local UmmaArgs args;
-  static thread_local PlanKey last;
+  static thread_local PlanCache<UmmaArgs> cache;
   PlanKey key;
   memset(&key, 0, sizeof(key));
   key.d = cd;
@@ -305,12 +339,15 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   key.v[5] = env_or("MAXDNN_UMMA_STAGE_KB", -12345);
   key.v[6] = env_or("MAXDNN_UMMA_COLS", -12345);
   key.valid = true;
-  if (!same_plan_key(key, last)) {
-    last.valid = false;
-    st = plan_umma(cd, elem_bytes, ds->sm_count, key.v[2], key.v[3], &args.g, &args.table);
+  int slot = cache.find(key);
+  if (slot < 0) {
+    slot = cache.take();
+    st = plan_umma(cd, elem_bytes, ds->sm_count, key.v[2], key.v[3], &cache.args[slot].g,
+                   &cache.args[slot].table);
     if (st != MAXDNN_OK) return st;
-    last = key;
+    cache.key[slot] = key;
   }
+  UmmaArgs& args = cache.args[slot];
   const ConvGeom& g = args.g;
   const uint64_t eb = (uint64_t)elem_bytes;
   const uint32_t atom = 128u / (uint32_t)elem_bytes;
@@ -415,27 +452,40 @@ maxdnn_status dgrad_plan_check(const ConvDims& fd, maxdnn_kernel_kind kind, int 
                    env_int("MAXDNN_UMMA_PAIR"), &g, &t);
 }
 
-// Workspace of the strided map gradient: the largest transformed sub-filter bank and the
-// largest class's dense result, each rounded up to 256 bytes.
+// Workspace of the strided map gradient.  The classes run side by side, so each has its
+// own region: its transformed sub-filter bank (together the classes' banks hold every tap
+// once) and, for the fp32 kernel, its dense result (together: one din), each rounded up
+// to 256 bytes.
 struct DgradStridedPlan {
   size_t ft_bytes, sub_bytes;
 };
 
-maxdnn_status plan_dgrad_strided(const ConvDims& d, size_t eb, DgradStridedPlan* p) {
+inline size_t dgrad_class_ft_bytes(const ConvDims& d, const DgradAxis& ah, const DgradAxis& aw,
+                                   size_t eb) {
+  return round256((size_t)d.No * ah.J * aw.J * d.Nc * eb);
+}
+inline size_t dgrad_class_sub_bytes(const ConvDims& d, const DgradAxis& ah, const DgradAxis& aw) {
+  return round256((size_t)d.Nc * ah.n * aw.n * d.Nb * 4);
+}
+// A class takes part when it has positions and taps and its windows reach dout.
+inline bool dgrad_class_live(const DgradAxis& ah, const DgradAxis& aw, int Ho, int Wo) {
+  return ah.J > 0 && aw.J > 0 && ah.n > 0 && aw.n > 0 && ah.crop < Ho && aw.crop < Wo;
+}
+
+maxdnn_status plan_dgrad_strided(const ConvDims& d, maxdnn_kernel_kind kind, DgradStridedPlan* p) {
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
-  size_t jmax = 0, nmax = 0;
+  const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
+  p->ft_bytes = p->sub_bytes = 0;
   for (int rh = 0; rh < d.stride_h; ++rh)
     for (int rw = 0; rw < d.stride_w; ++rw) {
       const DgradAxis ah = dgrad_axis(rh, d.Skh, d.stride_h, d.pad_h, d.Hi);
       const DgradAxis aw = dgrad_axis(rw, d.Skw, d.stride_w, d.pad_w, d.Wi);
-      const size_t j = (size_t)ah.J * aw.J, n = (size_t)ah.n * aw.n;
-      if (j > jmax) jmax = j;
-      if (n > nmax) nmax = n;
+      if (!dgrad_class_live(ah, aw, Ho, Wo)) continue;
+      p->ft_bytes += dgrad_class_ft_bytes(d, ah, aw, eb);
+      if (kind == MAXDNN_KERNEL_FP32) p->sub_bytes += dgrad_class_sub_bytes(d, ah, aw);
     }
-  p->ft_bytes = round256((size_t)d.No * jmax * d.Nc * eb);
-  p->sub_bytes = round256((size_t)d.Nc * nmax * d.Nb * 4);
   return MAXDNN_OK;
 }
 
@@ -444,7 +494,7 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
                                  cudaStream_t stream) {
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   DgradStridedPlan p;
-  maxdnn_status st = plan_dgrad_strided(d, eb, &p);
+  maxdnn_status st = plan_dgrad_strided(d, kind, &p);
   if (st != MAXDNN_OK) return st;
   if (ws_bytes < p.ft_bytes + p.sub_bytes) return MAXDNN_INVALID_VALUE;
   if (d.Nb % 4 != 0) return MAXDNN_NOT_SUPPORTED;
@@ -455,8 +505,8 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
   int32_t Ho, Wo;
   check_dims(d, &Ho, &Wo);
   const int sh = d.stride_h, sw = d.stride_w;
-  uint8_t* w_ft = static_cast<uint8_t*>(ws);
-  float* w_sub = reinterpret_cast<float*>(w_ft + p.ft_bytes);
+  uint8_t* ft_next = static_cast<uint8_t*>(ws);
+  uint8_t* sub_next = ft_next + p.ft_bytes;
   // Positions that no tap reaches (a class without taps, or whose window lies outside
   // dout) must read zero: clear din first if there is such a class.
   bool all_covered = true;
@@ -476,12 +526,31 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
   // grid inside din directly; the fp32 kernel writes a dense scratch tensor that a copy
   // kernel scatters.
   const bool direct = kind != MAXDNN_KERNEL_FP32;
-  for (int rh = 0; rh < sh; ++rh) {
-    for (int rw = 0; rw < sw; ++rw) {
+  // Fork: class i runs on the caller's stream (i % 4 == 0) or on one of three side
+  // streams that wait for what the caller's stream has queued so far; join at the end.
+  std::lock_guard<std::mutex> fork_lock(ds->fork_mu);
+  if (cudaEventRecord(ds->ev_fork, stream) != cudaSuccess) { cudaGetLastError(); return MAXDNN_CUDA_ERROR; }
+  bool aux_used[3] = {false, false, false};
+  int class_index = 0;
+  maxdnn_status result = MAXDNN_OK;
+  for (int rh = 0; rh < sh && result == MAXDNN_OK; ++rh) {
+    for (int rw = 0; rw < sw && result == MAXDNN_OK; ++rw) {
       const DgradAxis ah = dgrad_axis(rh, d.Skh, sh, d.pad_h, d.Hi);
       const DgradAxis aw = dgrad_axis(rw, d.Skw, sw, d.pad_w, d.Wi);
-      if (ah.J == 0 || aw.J == 0 || ah.n == 0 || aw.n == 0) continue;
-      if (ah.crop >= Ho || aw.crop >= Wo) continue;            // its windows miss dout entirely
+      if (!dgrad_class_live(ah, aw, Ho, Wo)) continue;
+      uint8_t* w_ft = ft_next;
+      ft_next += dgrad_class_ft_bytes(d, ah, aw, eb);
+      float* w_sub = reinterpret_cast<float*>(sub_next);
+      if (!direct) sub_next += dgrad_class_sub_bytes(d, ah, aw);
+      const int lane = class_index++ % 4;
+      cudaStream_t cs = stream;
+      if (lane > 0) {
+        cs = ds->aux[lane - 1];
+        if (!aux_used[lane - 1]) {
+          if (cudaStreamWaitEvent(cs, ds->ev_fork, 0) != cudaSuccess) { cudaGetLastError(); result = MAXDNN_CUDA_ERROR; break; }
+          aux_used[lane - 1] = true;
+        }
+      }
       ConvDims fd;
       fd.Nb = d.Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = d.No;
       fd.No = d.Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
@@ -494,14 +563,14 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
                       (unsigned)(ah.J * aw.J));
       const dim3 block(32, 8);
       if (eb == 2)
-        subfilter_flip_transpose_kernel<uint16_t><<<grid, block, 0, stream>>>(
+        subfilter_flip_transpose_kernel<uint16_t><<<grid, block, 0, cs>>>(
             static_cast<const uint16_t*>(filt), reinterpret_cast<uint16_t*>(w_ft), d.Nc, d.Skh,
             d.Skw, d.No, sh, sw, ah.rho, aw.rho, ah.J, aw.J);
       else
-        subfilter_flip_transpose_kernel<float><<<grid, block, 0, stream>>>(
+        subfilter_flip_transpose_kernel<float><<<grid, block, 0, cs>>>(
             static_cast<const float*>(filt), reinterpret_cast<float*>(w_ft), d.Nc, d.Skh, d.Skw,
             d.No, sh, sw, ah.rho, aw.rho, ah.J, aw.J);
-      if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+      if (cudaGetLastError() != cudaSuccess) { result = MAXDNN_CUDA_ERROR; break; }
       g_launches.fetch_add(1, std::memory_order_relaxed);
       const uint8_t* src = static_cast<const uint8_t*>(dout) +
                            ((size_t)ah.crop * Wo + aw.crop) * d.Nb * eb;
@@ -510,24 +579,33 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
         fd.out_y_stride = (int64_t)sh * d.Wi * d.Nb;
         fd.out_o_stride = (int64_t)d.Hi * d.Wi * d.Nb;
         float* dst = din + ((size_t)ah.first * d.Wi + aw.first) * d.Nb;
-        st = fprop_umma(fd, (int)eb, src, w_ft, dst, stream);
-        if (st != MAXDNN_OK) return st;
+        result = fprop_umma(fd, (int)eb, src, w_ft, dst, cs);
         continue;
       }
-      st = fprop_fp32(fd, reinterpret_cast<const float*>(src), reinterpret_cast<const float*>(w_ft),
-                      w_sub, stream);
-      if (st != MAXDNN_OK) return st;
+      result = fprop_fp32(fd, reinterpret_cast<const float*>(src), reinterpret_cast<const float*>(w_ft),
+                          w_sub, cs);
+      if (result != MAXDNN_OK) break;
       const int nb4 = d.Nb / 4;
       const size_t total = (size_t)d.Nc * ah.n * aw.n * nb4;
-      dgrad_scatter_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+      dgrad_scatter_kernel<<<(unsigned)((total + 255) / 256), 256, 0, cs>>>(
           reinterpret_cast<const float4*>(w_sub), reinterpret_cast<float4*>(din), d.Nc, ah.n, aw.n,
           nb4, d.Hi, d.Wi, sh, sw, ah.first, aw.first);
-      if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+      if (cudaGetLastError() != cudaSuccess) { result = MAXDNN_CUDA_ERROR; break; }
       g_launches.fetch_add(1, std::memory_order_relaxed);
     }
   }
-  return MAXDNN_OK;
+  // Join, also after an error: the caller's stream must not run ahead of the side streams.
+  for (int i = 0; i < 3; ++i) {
+    if (!aux_used[i]) continue;
+    if (cudaEventRecord(ds->ev_join[i], ds->aux[i]) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, ds->ev_join[i], 0) != cudaSuccess) {
+      cudaGetLastError();
+      if (result == MAXDNN_OK) result = MAXDNN_CUDA_ERROR;
+    }
+  }
+  return result;
 }
+
 
 maxdnn_status bprop_data(const ConvDims& d, maxdnn_kernel_kind kind, const void* dout,
                          const void* filt, float* din, void* ws, size_t ws_bytes,
@@ -575,7 +653,7 @@ maxdnn_status bprop_data_workspace(const ConvDims& d, maxdnn_kernel_kind kind, s
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   if (d.stride_w != 1 || d.stride_h != 1) {
     DgradStridedPlan p;
-    st = plan_dgrad_strided(d, eb, &p);
+    st = plan_dgrad_strided(d, kind, &p);
     if (st != MAXDNN_OK) return st;
     *bytes = p.ft_bytes + p.sub_bytes;
     return MAXDNN_OK;

@@ -52,3 +52,60 @@ def test_forward_and_both_gradients_replay_from_a_cuda_graph():
         got = got_t.cpu().numpy().reshape(ref.shape)
         err = float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref)))
         assert err <= 1e-5
+
+
+@pytest.mark.parametrize("kernel", ["fp32", "bf16"])
+def test_strided_map_gradient_forks_and_joins(kernel):
+    """Stride 2: the four residue classes run on the caller's stream and on the library's
+    side streams.  (a) Work queued on the caller's stream before and after the call is
+    ordered with all classes: the inputs are written by a kernel just before the call and
+    the result is consumed by a kernel just after it, with no host synchronisation.  (b)
+    The same call captured into a CUDA graph (fork and join by events) replays correctly."""
+    kind = {"fp32": mx.KERNEL_FP32, "bf16": mx.KERNEL_BF16}[kernel]
+    tol = {"fp32": 1e-5, "bf16": 2e-2}[kernel]
+    w = wl.Workload("s2", 64, 20, 14, 32, 64, 3, 2, 1, 1.0, ("uniform", -1.0, 1.0),
+                    ("uniform", -1.0, 1.0), 7700)
+    d = mx.ConvDesc.make(*w.dims)
+    _, filt = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+    dt = torch.bfloat16 if kernel == "bf16" else torch.float32
+    if kernel == "bf16":
+        filt = wl.from_bf16_bits(wl.to_bf16_bits(filt))
+        dout = wl.from_bf16_bits(wl.to_bf16_bits(dout))
+    ref = oracle.conv_bprop_data(dout, filt, (w.Hi, w.Wi), stride=2, pad=1, alpha=1.0)
+    scale = float(np.max(np.abs(ref)))
+    f = torch.from_numpy(filt).cuda().to(dt)
+    g_src = torch.from_numpy(dout).cuda().to(dt)
+    g = torch.zeros_like(g_src)
+    din = torch.zeros(mx.conv_in_elems(d), device="cuda")
+    total = torch.zeros(mx.conv_in_elems(d), device="cuda")
+    ws = torch.empty(mx.conv_bprop_data_workspace(d, kind), dtype=torch.uint8, device="cuda")
+    mx.conv_bprop_data(d, g, f, din, ws, kind)          # one-time set-up outside any capture
+    torch.cuda.synchronize()
+
+    side = torch.cuda.Stream()
+
+    def run():
+        g.copy_(g_src)                                  # producer on the same stream
+        mx.conv_bprop_data(d, g, f, din, ws, kind, stream=side)
+        total.copy_(din)                                # consumer on the same stream
+
+    with torch.cuda.stream(side):
+        g.zero_(); din.fill_(float("nan")); total.zero_()
+        run()
+    side.synchronize()
+    assert mx.last_device_status() == mx.OK
+    got = total.cpu().numpy().reshape(ref.shape)
+    assert float(np.max(np.abs(got - ref))) <= tol * scale
+
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    g.zero_(); din.fill_(float("nan")); total.zero_()
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert mx.last_device_status() == mx.OK
+    got = total.cpu().numpy().reshape(ref.shape)
+    assert float(np.max(np.abs(got - ref))) <= tol * scale

@@ -196,8 +196,13 @@ def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     assert mx.conv_bprop_data_workspace(d, mx.KERNEL_BF16) == 96 * 25 * 256 * 2
     strided = mx.ConvDesc.make(128, 227, 227, 3, 96, 11, 4, 0, 1.0)        # stride 4: 16 classes
     r256 = lambda b: (b + 255) // 256 * 256
-    assert mx.conv_bprop_data_workspace(strided) == \
-        r256(96 * 9 * 3 * 4) + r256(3 * 57 * 57 * 128 * 4)     # 3 x 3 taps at most; 57 x 57 positions
+    # the 16 classes run side by side, each with its own sub-filter bank (3 or 2 taps per
+    # axis: nine classes of 3 x 3, six of 3 x 2, one of 2 x 2) and, in fp32, its own dense
+    # result (together one din)
+    banks = 9 * r256(96 * 9 * 3 * 4) + 6 * r256(96 * 6 * 3 * 4) + r256(96 * 4 * 3 * 4)
+    assert mx.conv_bprop_data_workspace(strided) == banks + 3 * 227 * 227 * 128 * 4
+    assert mx.conv_bprop_data_workspace(mx.ConvDesc.make(128, 56, 56, 64, 128, 3, 2, 1, 1.0),
+                                        mx.KERNEL_BF16) == 64 * 9 * 128 * 2   # stored in place
     for bad in (mx.ConvDesc.make(64, 16, 16, 8, 8, 3, 1, 3, 1.0),):         # pad > Sk - 1
         with pytest.raises(mx.MaxdnnError) as e:
             mx.conv_bprop_data_workspace(bad)
