@@ -506,26 +506,52 @@ maxdnn_status plan_wgrad(const ConvDims& d, int elem_bytes, int sm_count, int fo
   g->Skw = d.Skw; g->Skh = d.Skh; g->stride_w = d.stride_w; g->stride_h = d.stride_h;
   g->pad_w = d.pad_w; g->pad_h = d.pad_h; g->alpha = d.alpha; g->Ho = Ho; g->Wo = Wo;
   g->bw = d.Skw;
-  g->bh = d.Skh < max_rows / g->bw ? d.Skh : max_rows / g->bw;
-  if (g->bh < 1) return MAXDNN_NOT_SUPPORTED;
-  g->bc = max_rows / (g->bw * g->bh);
-  if (g->bc > 256) g->bc = 256;                                       // a copy box has at most 256 per axis
-  if (g->bc > d.Nc) g->bc = d.Nc;
+  if (max_rows / g->bw < 1) return MAXDNN_NOT_SUPPORTED;
   // Two-SM tiles (tensor-core kernel): 256 filters per pair of CTAs, each CTA staging its
   // 128 filters and half of the tile's channels — per SM and per MMA 8 KB instead of 12 KB
   // are staged, and the kernel is bound by that fill rate.  Taken when the second CTA of
   // every tile has filters and the channels split evenly.
   const bool peer_has_filters = (d.No % 256 == 0) || (d.No % 256 > 128);
-  g->pair = (tensor && force_pair >= 0 && (peer_has_filters || force_pair > 0) && g->bc >= 2 &&
-             sm_count >= 2) ? 1 : 0;
-  if (g->pair) g->bc &= ~1;
-  // Same number of channel blocks, evenly filled (256 channels, 3 x 3: ten blocks of 26
-  // instead of nine of 28 and one of 4): fewer gradient rows per MMA for the same tiles.
+  g->pair = (tensor && force_pair >= 0 && (peer_has_filters || force_pair > 0) && d.Nc >= 2 &&
+             max_rows / (g->bw * 1) >= 2 && sm_count >= 2) ? 1 : 0;
+  // Tile = bc channels x bh filter rows x all Skw filter columns, at most max_rows
+  // gradient rows.  Blocks of channels and of filter rows are filled evenly (256
+  // channels, 3 x 3: ten blocks of 26 channels, not nine of 28 and one of 4), and the
+  // shape that needs the fewest staged rows over all tiles wins — a tile stages its
+  // gradient rows (rounded up to the MMA's N granule) plus, on the tensor cores, 128 filter
+  // rows per step whatever its height; fewer, larger tiles win near-ties.  11 x 11 x 3:
+  // two tiles of 3 channels x 6 filter rows (198 rows) instead of 2 channels x 11 rows
+  // (242) and 1 x 11 (half empty).
   {
-    const int blocks = ceil_div(d.Nc, g->bc);
-    int even = ceil_div(d.Nc, blocks);
-    if (g->pair && (even & 1)) ++even;
-    if (even < g->bc) g->bc = even;
+    const int bh_max = d.Skh < max_rows / g->bw ? d.Skh : max_rows / g->bw;
+    double best = 1e300;
+    int best_bh = 0, best_bc = 0;
+    for (int bh = bh_max; bh >= 1; --bh) {
+      int bc = max_rows / (g->bw * bh);
+      if (bc > 256) bc = 256;                                   // a copy box has at most 256 per axis
+      if (bc > d.Nc) bc = d.Nc;
+      if (g->pair) bc &= ~1;
+      if (bc < 1) continue;
+      const int cb = ceil_div(d.Nc, bc);
+      int bce = ceil_div(d.Nc, cb);
+      if (g->pair && (bce & 1)) ++bce;
+      if (bce > bc) bce = bc;
+      const int kb = ceil_div(d.Skh, bh);
+      const int bhe = ceil_div(d.Skh, kb);
+      const int rows = bce * bhe * g->bw;
+      const int staged = !tensor ? max_rows
+                                 : 128 + (g->pair ? 2 * align_up(rows / 2, 8) : align_up(rows, 16));
+      const double cost = (double)cb * kb * staged;
+      if (cost < 0.95 * best) { best = cost; best_bh = bhe; best_bc = bce; }
+    }
+    if (best_bh == 0) {
+      if (!g->pair) return MAXDNN_NOT_SUPPORTED;
+      g->pair = 0;                                              // one channel per tile: no halves
+      best_bh = bh_max;
+      best_bc = 1;
+    }
+    g->bh = best_bh;
+    g->bc = best_bc;
   }
   if (g->pair) g->bc_h = g->bc / 2;
   g->rows = g->bc * g->bh * g->bw;
