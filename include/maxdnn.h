@@ -203,18 +203,20 @@ maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const floa
  * operand a is split into a_hi (a rounded to the nearest TF32 number, which a TF32 tensor
  * core reads unchanged) and a_lo = a - a_hi (rounded likewise), and the products
  * a_hi b_hi + a_hi b_lo + a_lo b_hi are accumulated in fp32 (the dropped a_lo b_lo term is
- * below 2^-22 of the product).
- * Because the operation sums over channels, the three products are ONE TF32 FPROP over 3 Nc
- * channels: a small kernel writes the split maps [hi; hi; lo] and filters [hi; lo; hi] into
- * the caller's workspace (size from maxdnn_conv_fprop_tf32x3_workspace) and the TF32 kernel
- * runs on them.  Same arguments, layouts and limits as maxdnn_conv_fprop_tf32 (with 3 Nc <=
- * 32767); in / filt / out are the fp32 tensors.  The paper has no counterpart (its kernel
- * is an fp32 CUDA-core kernel).  Accuracy lies between the two and depends on the length
- * K = Nc Sk^2 of the sums: the tensor core truncates its fp32 accumulator at every MMA, a
- * one-sided error that adds up linearly where the terms share a sign — measured against
- * the fp64 oracle, of the largest output: 1e-6 (K = 144), 5e-6 (363), 2e-5 (2400), 9e-5
- * (9216), about 1e-8 K (exact fp32 kernel: 5e-7 .. 4e-6; plain TF32: 7e-4) — at about
- * four times the exact kernel's speed.
+ * below 2^-22 of the product).  Because the operation sums over channels, the three
+ * products are ONE TF32 FPROP over 3 Nc channels: a small kernel writes the split maps
+ * [hi; hi; lo] and filters [hi; lo; hi] into the caller's workspace (size from
+ * maxdnn_conv_fprop_tf32x3_workspace) and a TF32 kernel runs on them.  That kernel sums K
+ * in chunks: the tensor core truncates its fp32 accumulator at every MMA, a one-sided error
+ * that over a long sum of same-signed terms reaches 1e-8 K of the result, so a fresh
+ * accumulator is started about every 768 rows of K and the finished chunks are added in
+ * registers with round-to-nearest fp32 adds.  Same arguments, layouts and limits as
+ * maxdnn_conv_fprop_tf32 (with 3 Nc <= 32767); in / filt / out are the fp32 tensors.  The
+ * paper has no counterpart (its kernel is an fp32 CUDA-core kernel).  Accuracy: the exact
+ * kernel's class — measured 1e-6 .. 3e-6 of the largest output against the fp64 oracle for
+ * K = 144 .. 9216 (exact fp32 kernel: 5e-7 .. 4e-6; plain TF32: 7e-4) — at three to four
+ * times the exact kernel's speed.  (MAXDNN_X3_CHUNK_ROWS=0 in the environment selects the
+ * one-accumulator path: 10-25 % faster, error about 1e-8 K.)
  */
 maxdnn_status maxdnn_conv_fprop_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
 maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in,

@@ -11,6 +11,7 @@
 #include "ffma_conv.cuh"
 #include "plan.h"
 #include "umma_conv.cuh"
+#include "umma_chunk_conv.cuh"
 #include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
 #include "wgrad_umma_pair.cuh"
@@ -28,6 +29,7 @@ struct DeviceState {
   bool ffma_attr[16] = {};
   bool umma_attr[4] = {false, false, false, false};
   bool wgrad_attr = false;
+  bool umma_chunk_attr = false;
   bool wgrad_umma_attr[4] = {false, false, false, false};
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
@@ -296,6 +298,23 @@ maxdnn_status launch_umma_pair(DeviceState* ds, const CUtensorMap& mf, const CUt
   return MAXDNN_OK;
 }
 
+maxdnn_status launch_umma_chunk(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                                const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
+  auto kern = umma_chunk_conv_kernel;
+  if (!ds->umma_chunk_attr) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->umma_chunk_attr = true;
+  }
+  kern<<<args.g.grid, kUmmaChunkThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
 template <bool BF16>
 maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
                           const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
@@ -315,8 +334,10 @@ maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensor
   return MAXDNN_OK;
 }
 
+// chunk_rows > 0 (TF32 only): the chunked kernel, a fresh accumulator about every
+// chunk_rows rows of K, one-SM tiles.
 maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, const void* filt,
-                         float* out, cudaStream_t stream) {
+                         float* out, cudaStream_t stream, int chunk_rows = 0) {
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(cd, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -334,7 +355,7 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   key.v[0] = ds->sm_count;
   key.v[1] = elem_bytes;
   key.v[2] = env_int("MAXDNN_UMMA_KC");
-  key.v[3] = env_int("MAXDNN_UMMA_PAIR");
+  key.v[3] = chunk_rows > 0 ? -1 : env_int("MAXDNN_UMMA_PAIR");
   key.v[4] = env_or("MAXDNN_UMMA_MERGE", -12345);
   key.v[5] = env_or("MAXDNN_UMMA_STAGE_KB", -12345);
   key.v[6] = env_or("MAXDNN_UMMA_COLS", -12345);
@@ -421,6 +442,12 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
     st = encode_map(&mo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
+  }
+  if (chunk_rows > 0) {
+    if (bf16 || g.pair) return MAXDNN_INVALID_VALUE;
+    const int steps = chunk_rows / g.rows;
+    args.chunk_steps = (uint32_t)(steps < 1 ? 1 : steps);
+    return launch_umma_chunk(ds, mf, mi, mo, args, stream);
   }
   if (g.pair)
     return bf16 ? launch_umma_pair<true>(ds, mf, mi, mo, args, stream)
@@ -921,6 +948,10 @@ maxdnn_status fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in, const 
       reinterpret_cast<const float4*>(filt), reinterpret_cast<float4*>(w_filt), n4_f, 0x2u);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(2, std::memory_order_relaxed);
+  // A fresh accumulator about every 768 rows of the split problem's K (256 of the
+  // original): the accumulator's truncation then acts on short partial sums only.
+  const int chunk_rows = env_or("MAXDNN_X3_CHUNK_ROWS", 768);
+  if (chunk_rows > 0) return fprop_umma(dims_from(d3), 4, w_in, w_filt, out, stream, chunk_rows);
   return fprop_umma(&d3, 4, w_in, w_filt, out, stream);
 }
 

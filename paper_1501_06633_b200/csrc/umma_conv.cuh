@@ -39,6 +39,7 @@ struct UmmaArgs {
   uint32_t tap_b_bytes; // patch strip: start-address step of one pixel (the next kw's window)
   uint32_t is_bf16;
   uint32_t test_missing_arrival;   // test hook: CTA 0's full barriers expect an arrival that never comes
+  uint32_t chunk_steps;            // chunked kernel only: K steps per TMEM accumulator
   uint32_t* status;
   KStepTable table;
 };

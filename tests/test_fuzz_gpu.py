@@ -170,3 +170,27 @@ def test_random_few_channel_strided_shapes(kernel):
         ref = oracle.conv_fprop(rx, rf, stride=stride, pad=pad, alpha=alpha)
         assert rel(out.cpu().numpy().reshape(ref.shape), ref) <= TOL[kernel], w.dims
         done += 1
+
+
+def test_random_shapes_three_product_tf32():
+    """maxdnn_conv_fprop_tf32x3 (chunked accumulation) on random shapes, held to the exact
+    kernel's bar: ragged tiles, dead column groups, one chunk or many, all plans."""
+    done = 0
+    for i, shape in enumerate(random_shapes("tf32", 40, 66)):
+        Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+        w = wl.Workload("fuzz_x3", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
+                        ("uniform", -1.0, 1.0), 9700 + i)
+        inp, filt = wl.make_inputs(w)
+        d = mx.ConvDesc.make(*w.dims)
+        ws = torch.empty(max(16, mx.conv_fprop_tf32x3_workspace(d)), dtype=torch.uint8, device="cuda")
+        out = torch.full((mx.conv_out_elems(d),), float("nan"), device="cuda")
+        try:
+            mx.conv_fprop_tf32x3(d, torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda(), out, ws)
+        except mx.MaxdnnError as e:
+            assert e.status == mx.NOT_SUPPORTED      # 3 Nc channels x Sk^2 taps: too many K steps
+            continue
+        assert mx.last_device_status() == mx.OK, shape
+        ref = oracle.conv_fprop(inp, filt, stride=stride, pad=pad, alpha=alpha)
+        assert rel(out.cpu().numpy().reshape(ref.shape), ref) <= 1e-5, shape
+        done += 1
+    assert done >= 30

@@ -1,9 +1,9 @@
 """Three-product TF32 FPROP (fp32 operands split into hi + lo, one TF32 launch over 3 Nc
-channels): accuracy class between exact fp32 (<= 1e-5 required, ~1e-6 measured) and plain
-TF32 (<= 5e-3 required, ~7e-4 measured).  The tensor core truncates its fp32 accumulator at
-every MMA, a one-sided error that grows linearly with the length K of the sums on same-signed
-data (measured about 1e-8 K), so the bound required here is max(5e-5, 1.2e-8 K) of the
-largest output."""
+channels, the sum over K accumulated in chunks that are added in round-to-nearest fp32):
+required here is the exact kernel's own bar, <= 1e-5 of the largest output against the fp64
+oracle, whatever the length K of the sums (measured 1e-6 .. 3e-6).  Without the chunks
+(MAXDNN_X3_CHUNK_ROWS=0) the tensor core's truncating accumulator costs about 1e-8 K on
+same-signed data; that path is kept as a switch and held to max(5e-5, 1.2e-8 K)."""
 import numpy as np
 import pytest
 import torch
@@ -13,7 +13,7 @@ import paper_1501_06633_b200 as mx
 from paper_1501_06633_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
-TOL_X3 = 5e-5
+TOL_X3 = 1e-5
 
 
 def run(w, inp, filt):
@@ -51,10 +51,17 @@ def test_tf32x3_small(shape):
     assert err < err1 / 8
 
 
-@pytest.mark.parametrize("name", ["mid5x5", "large3x3", "first11x11s4", "overfeat_L5"])
-def test_tf32x3_full_size_sampled(name):
+@pytest.mark.parametrize("chunked", [True, False])
+@pytest.mark.parametrize("name", ["mid5x5", "wide3x3", "large3x3", "first11x11s4", "alexnet_conv2",
+                                  "overfeat_L3", "overfeat_L5"])
+def test_tf32x3_full_size_sampled(name, chunked, monkeypatch):
     w = wl.ALL[name]
-    tol = max(TOL_X3, 1.2e-8 * w.Nc * w.Sk * w.Sk)        # overfeat_L5: K = 9216
+    tol = TOL_X3
+    if not chunked:
+        if name not in ("mid5x5", "overfeat_L5"):
+            pytest.skip("one-accumulator path: two layers are enough")
+        monkeypatch.setenv("MAXDNN_X3_CHUNK_ROWS", "0")
+        tol = max(5e-5, 1.2e-8 * w.Nc * w.Sk * w.Sk)      # overfeat_L5: K = 9216
     inp, filt = wl.make_inputs(w)
     got = run(w, inp, filt)
     assert np.isfinite(got).all()

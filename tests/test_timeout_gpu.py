@@ -48,3 +48,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind,
     got = out.cpu().numpy().reshape(ref.shape)
     err = float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref)))
     assert err <= 1e-5
+
+
+def test_chunked_kernel_wait_runs_out_and_the_context_survives(monkeypatch):
+    """The same for the chunked TF32 kernel behind maxdnn_conv_fprop_tf32x3 (eight epilogue
+    warps that wait for one chunk's accumulator after another)."""
+    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
+    d = mx.ConvDesc.make(*w.dims)
+    inp, filt = wl.make_inputs(w)
+    x, f = torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda()
+    ws = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    assert mx.last_device_status() == mx.OK
+    monkeypatch.setenv("MAXDNN_TEST_MISSING_ARRIVAL", "1")
+    mx.conv_fprop_tf32x3(d, x, f, out, ws)
+    assert mx.last_device_status() == mx.DEVICE_TIMEOUT
+    assert mx.last_device_status() == mx.OK
+    monkeypatch.delenv("MAXDNN_TEST_MISSING_ARRIVAL")
+    mx.conv_fprop_tf32x3(d, x, f, out, ws)
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = out.cpu().numpy().reshape(ref.shape)
+    assert float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref))) <= 1e-5
