@@ -11,14 +11,132 @@
 // Same structure as umma_conv_kernel (one SM per tile, 128 filters x <= 256 columns, two
 // accumulators in TMEM, bounded waits) with EIGHT epilogue warps: two per TMEM lane
 // quarter, each holding 128 of the tile's columns of its 32 filters in registers
-// (128 totals per thread).  Warp 0: patch copies, warp 1: MMA issue, warps 2-9: epilogue,
-// warp 10: filter copies.
+// (128 totals per thread).  Warp 0: patch copies, warp 1: MMA issue, warp 2: filter copies,
+// warps 3-10: epilogue — the three warps with short per-step loops are the oldest on their
+// schedulers, ahead of the epilogue warps that wait for a chunk.
 #pragma once
 #include "umma_conv.cuh"
 
 namespace maxdnn {
 
 constexpr int kUmmaChunkThreads = 352;
+
+// 32 lanes x 16 consecutive 32-bit columns: thread l receives row (lane base + l).
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+        "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Epilogue warps (3-10) of the chunked kernel, kept out of line: their 128 totals per
+// thread fill the register file, and inlined they made the compiler spill values that
+// the copy and MMA warps read in their short per-step loops.
+__device__ __noinline__ void chunk_epilogue_role(const CUtensorMap& map_out, const UmmaArgs& args,
+                                                 uint32_t base, uint8_t* base_ptr, uint32_t st_off,
+                                                 uint32_t accf_bar, uint32_t acce_bar,
+                                                 uint32_t tmem_base, int warp, int lane) {
+  const ConvGeom& g = args.g;
+  const int n_ksteps = g.n_ksteps;
+  const int n_cols = g.tile_px * g.tile_n;
+  {
+    // Warps 3-10.  A warp may read the TMEM lanes 32 (warp % 4) ...; the two warps of a
+    // quarter take the tile's columns 0-127 and 128-255.
+    const int q = warp & 3;
+    const int half = (warp - 3) >> 2;
+    const int ew = warp - 3;                 // 0..7: one staging tile each
+    const uint32_t stg = base + st_off + (uint32_t)ew * kStageTileBytes;
+    uint8_t* stg_ptr = base_ptr + st_off + (size_t)ew * kStageTileBytes;
+    const float alpha = g.alpha;
+    const uint64_t pol_first = l2_policy_evict_first();
+    const int chunk_steps = (int)args.chunk_steps;
+    const int chunks_per_tile = (n_ksteps + chunk_steps - 1) / chunk_steps;
+    bool ok = true;
+    uint32_t chunk = 0;
+    for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
+      int r = tile;
+      const int ob = r % g.o_blocks; r /= g.o_blocks;
+      const int nch = r % g.n_chunks; r /= g.n_chunks;
+      const int xr = r % g.x_runs;
+      const int y = r / g.x_runs;
+      const int o0 = ob * kUmmaM + q * 32;
+      const int n0 = nch * g.tile_n;
+      const int x0 = xr * g.tile_px;
+      // which of this warp's four groups of 32 columns hold results (warp-uniform bit mask)
+      uint32_t live = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int col = half * 128 + 32 * k;
+        const int p = col / g.tile_n;
+        if ((col < n_cols) && (x0 + p < g.Wo) && (n0 + (col - p * g.tile_n) < g.Nb) && (o0 < g.No))
+          live |= 1u << k;
+      }
+      float tot[128];
+      for (int c = 0; c < chunks_per_tile && ok; ++c, ++chunk) {
+        const uint32_t acc = chunk & 1u;
+        if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+          ok = false;
+          break;
+        }
+        tcgen05_fence_after();
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols +
+                               (uint32_t)(half * 128);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (!((live >> k) & 1u)) continue;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {      // 16 columns per load: the totals leave few registers
+            uint32_t v[16];
+            tmem_ld_32x16(t_row + (uint32_t)(32 * k + 16 * hh), v);
+            tmem_wait_ld();
+            if (c == 0) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) tot[32 * k + 16 * hh + j] = __uint_as_float(v[j]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) tot[32 * k + 16 * hh + j] += __uint_as_float(v[j]);   // round to nearest
+            }
+          }
+        }
+        // this accumulator may be overwritten by the chunk after next
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar + 8u * acc);
+      }
+      if (!ok) break;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (!((live >> k) & 1u)) continue;
+        // the staging tile must have been read by the previous store
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
+        uint8_t* row = stg_ptr + (size_t)lane * 128;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+          float4 o4;
+          o4.x = tot[32 * k + 4 * cc + 0] * alpha;
+          o4.y = tot[32 * k + 4 * cc + 1] * alpha;
+          o4.z = tot[32 * k + 4 * cc + 2] * alpha;
+          o4.w = tot[32 * k + 4 * cc + 3] * alpha;
+          *reinterpret_cast<float4*>(row + ((cc ^ (lane & 7)) << 4)) = o4;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int col = half * 128 + 32 * k;
+          const int p = col / g.tile_n;
+          tma_store_4d_hint(&map_out, stg, n0 + (col - p * g.tile_n), x0 + p, y, o0, pol_first);
+          bulk_commit();
+        }
+      }
+    }
+    if (lane == 0) bulk_wait_all();
+  }
+}
 
 __global__ void __launch_bounds__(kUmmaChunkThreads, 1)
 umma_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
@@ -75,9 +193,9 @@ umma_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int mma_per_step = g.kc / (int)args.umma_k;
   const int n_cols = g.tile_px * g.tile_n;   // MMA N
 
-  if (warp == 0 || warp == 10) {
+  if (warp == 0 || warp == 2) {
     // ----------------------------------------------------------- producers
-    // Warp 0 copies the patch boxes, warp 10 the filter boxes: issuing a bulk tensor
+    // Warp 0 copies the patch boxes, warp 2 the filter boxes: issuing a bulk tensor
     // copy costs the issuing warp a few hundred cycles, and a K step is short.
     const bool patch_role = (warp == 0);
     // The whole warp walks the loops, so coordinates and addresses are computed in
@@ -161,59 +279,56 @@ umma_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const uint64_t desc_hi_a = make_smem_desc(0, args.lbo_a_bytes, args.sbo_bytes, 1u);
       const uint64_t desc_hi_b = make_smem_desc(0, args.lbo_b_bytes, args.sbo_bytes, 1u);
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
-        uint32_t d_tmem = 0;
-        uint32_t accumulate = 0;
-        int left = 0;          // K steps left in the current chunk
-        for (int s = 0; s < n_ksteps; ++s) {
-          if (left == 0) {
-            // a new chunk: its accumulator must have been drained (two chunks ago)
-            const uint32_t acc = chunk & 1u;
-            if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.status,
-                           kDevTimeoutAccFree)) {
-              ok = false;
-              break;
-            }
-            tcgen05_fence_after();
-            d_tmem = tmem_base + acc * kAccCols;
-            accumulate = 0;
-            left = chunk_steps;
-          }
-          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+        // One chunk = up to chunk_steps K steps into one accumulator; the loop over its
+        // steps is the plain kernel's (nothing but the step itself inside it: a K step
+        // can be as short as four MMAs).
+        for (int s0 = 0; s0 < n_ksteps && ok; s0 += chunk_steps, ++chunk) {
+          const uint32_t acc = chunk & 1u;
+          // the accumulator must have been drained (it held the chunk before last)
+          if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.status,
+                         kDevTimeoutAccFree)) {
             ok = false;
             break;
           }
           tcgen05_fence_after();
-          const uint32_t a_addr = base + a_off + (uint32_t)stage * g.a_stage_bytes;
-          const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
-          const uint64_t a_base_desc = desc_hi_a | (uint64_t)((a_addr & 0x3FFFFu) >> 4);
-          const uint64_t b_base_desc = desc_hi_b | (uint64_t)((b_addr & 0x3FFFFu) >> 4);
-          const uint64_t kstep = (uint64_t)(args.kstep_bytes >> 4);
-          const uint64_t tap_a = (uint64_t)(args.tap_a_bytes >> 4);
-          const uint64_t tap_b = (uint64_t)(args.tap_b_bytes >> 4);
-          --left;
-          const bool chunk_ends = (left == 0) || (s + 1 == n_ksteps);
-          if (elect_one()) {
-            uint32_t acc_flag = accumulate;
-            for (int kw = 0; kw < g.kwc; ++kw) {
-              uint64_t adesc = a_base_desc + (uint64_t)kw * tap_a;
-              uint64_t bdesc = b_base_desc + (uint64_t)kw * tap_b;
-#pragma unroll 4
-              for (int j = 0; j < mma_per_step; ++j) {
-                tcgen05_mma<false>(d_tmem, adesc, bdesc, args.idesc, acc_flag);
-                acc_flag = 1;
-                adesc += kstep;
-                bdesc += kstep;
-              }
+          const uint32_t d_tmem = tmem_base + acc * kAccCols;
+          const int s1 = s0 + chunk_steps < n_ksteps ? s0 + chunk_steps : n_ksteps;
+          uint32_t accumulate = 0;
+          for (int s = s0; s < s1; ++s) {
+            if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+              ok = false;
+              break;
             }
-            tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
-            if (chunk_ends) tcgen05_commit(accf_bar + 8u * (chunk & 1u));   // chunk complete
+            tcgen05_fence_after();
+            const uint32_t a_addr = base + a_off + (uint32_t)stage * g.a_stage_bytes;
+            const uint32_t b_addr = base + b_off + (uint32_t)stage * g.b_stage_bytes;
+            const uint64_t a_base_desc = desc_hi_a | (uint64_t)((a_addr & 0x3FFFFu) >> 4);
+            const uint64_t b_base_desc = desc_hi_b | (uint64_t)((b_addr & 0x3FFFFu) >> 4);
+            const uint64_t kstep = (uint64_t)(args.kstep_bytes >> 4);
+            const uint64_t tap_a = (uint64_t)(args.tap_a_bytes >> 4);
+            const uint64_t tap_b = (uint64_t)(args.tap_b_bytes >> 4);
+            if (elect_one()) {
+              uint32_t acc_flag = accumulate;
+              for (int kw = 0; kw < g.kwc; ++kw) {
+                uint64_t adesc = a_base_desc + (uint64_t)kw * tap_a;
+                uint64_t bdesc = b_base_desc + (uint64_t)kw * tap_b;
+#pragma unroll 4
+                for (int j = 0; j < mma_per_step; ++j) {
+                  tcgen05_mma<false>(d_tmem, adesc, bdesc, args.idesc, acc_flag);
+                  acc_flag = 1;
+                  adesc += kstep;
+                  bdesc += kstep;
+                }
+              }
+              tcgen05_commit(empty_bar + 8u * stage);   // frees the stage when these MMAs finish
+            }
+            accumulate = 1;
+            __syncwarp();
+            if (++stage == stages) { stage = 0; phase ^= 1u; }
           }
-          accumulate = 1;
-          __syncwarp();
-          if (chunk_ends) { ++chunk; left = 0; }
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
+          if (!ok) break;
+          if (elect_one()) tcgen05_commit(accf_bar + 8u * acc);        // chunk complete
         }
-        if (!ok) break;
       }
       // Exit path: every MMA issued so far has finished before TMEM is released.
       if (elect_one()) tcgen05_commit(done_bar);
@@ -221,94 +336,7 @@ umma_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     }
   } else {
     // ------------------------------------------------------------ epilogue
-    // Warps 2-9.  A warp may read the TMEM lanes 32 (warp % 4) ...; the two warps of a
-    // quarter take the tile's columns 0-127 and 128-255.
-    const int q = warp & 3;
-    const int half = (warp - 2) >> 2;
-    const int ew = warp - 2;                 // 0..7: one staging tile each
-    const uint32_t stg = base + st_off + (uint32_t)ew * kStageTileBytes;
-    uint8_t* stg_ptr = base_ptr + st_off + (size_t)ew * kStageTileBytes;
-    const float alpha = g.alpha;
-    const uint64_t pol_first = l2_policy_evict_first();
-    const int chunk_steps = (int)args.chunk_steps;
-    const int chunks_per_tile = (n_ksteps + chunk_steps - 1) / chunk_steps;
-    bool ok = true;
-    uint32_t chunk = 0;
-    for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x) {
-      int r = tile;
-      const int ob = r % g.o_blocks; r /= g.o_blocks;
-      const int nch = r % g.n_chunks; r /= g.n_chunks;
-      const int xr = r % g.x_runs;
-      const int y = r / g.x_runs;
-      const int o0 = ob * kUmmaM + q * 32;
-      const int n0 = nch * g.tile_n;
-      const int x0 = xr * g.tile_px;
-      // which of this warp's four groups of 32 columns hold results (warp-uniform)
-      bool live[4];
-      int col_n[4], col_x[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int col = half * 128 + 32 * k;
-        const int p = col / g.tile_n;
-        col_n[k] = n0 + (col - p * g.tile_n);
-        col_x[k] = x0 + p;
-        live[k] = (col < n_cols) && (col_x[k] < g.Wo) && (col_n[k] < g.Nb) && (o0 < g.No);
-      }
-      float tot[128];
-      for (int c = 0; c < chunks_per_tile && ok; ++c, ++chunk) {
-        const uint32_t acc = chunk & 1u;
-        if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.status, kDevTimeoutAccum)) {
-          ok = false;
-          break;
-        }
-        tcgen05_fence_after();
-        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols +
-                               (uint32_t)(half * 128);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (!live[k]) continue;
-          uint32_t v[32];
-          tmem_ld_32x32(t_row + (uint32_t)(32 * k), v);
-          tmem_wait_ld();
-          if (c == 0) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) tot[32 * k + j] = __uint_as_float(v[j]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) tot[32 * k + j] += __uint_as_float(v[j]);   // round to nearest
-          }
-        }
-        // this accumulator may be overwritten by the chunk after next
-        tcgen05_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acce_bar + 8u * acc);
-      }
-      if (!ok) break;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (!live[k]) continue;
-        // the staging tile must have been read by the previous store
-        if (lane == 0) bulk_wait_read<0>();
-        __syncwarp();
-        uint8_t* row = stg_ptr + (size_t)lane * 128;
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
-          float4 o4;
-          o4.x = tot[32 * k + 4 * cc + 0] * alpha;
-          o4.y = tot[32 * k + 4 * cc + 1] * alpha;
-          o4.z = tot[32 * k + 4 * cc + 2] * alpha;
-          o4.w = tot[32 * k + 4 * cc + 3] * alpha;
-          *reinterpret_cast<float4*>(row + ((cc ^ (lane & 7)) << 4)) = o4;
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          tma_store_4d_hint(&map_out, stg, col_n[k], col_x[k], y, o0, pol_first);
-          bulk_commit();
-        }
-      }
-    }
-    if (lane == 0) bulk_wait_all();
+    chunk_epilogue_role(map_out, args, base, base_ptr, st_off, accf_bar, acce_bar, tmem_base, warp, lane);
   }
 
   tcgen05_fence_before();
