@@ -12,6 +12,7 @@
 #include "plan.h"
 #include "umma_conv.cuh"
 #include "umma_chunk_conv.cuh"
+#include "umma_pair_chunk_conv.cuh"
 #include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
 #include "wgrad_umma_pair.cuh"
@@ -30,6 +31,7 @@ struct DeviceState {
   bool umma_attr[4] = {false, false, false, false};
   bool wgrad_attr = false;
   bool umma_chunk_attr = false;
+  bool umma_pair_chunk_attr = false;
   bool wgrad_umma_attr[4] = {false, false, false, false};
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
@@ -315,6 +317,38 @@ maxdnn_status launch_umma_chunk(DeviceState* ds, const CUtensorMap& mf, const CU
   return MAXDNN_OK;
 }
 
+maxdnn_status launch_umma_pair_chunk(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                                     const CUtensorMap& mo, const UmmaArgs& args,
+                                     cudaStream_t stream) {
+  auto kern = umma_pair_chunk_conv_kernel;
+  if (!ds->umma_pair_chunk_attr) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->umma_pair_chunk_attr = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
+  cfg.blockDim = dim3(kUmmaChunkThreads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, mf, mi, mo, args) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
 template <bool BF16>
 maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
                           const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
@@ -334,8 +368,8 @@ maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensor
   return MAXDNN_OK;
 }
 
-// chunk_rows > 0 (TF32 only): the chunked kernel, a fresh accumulator about every
-// chunk_rows rows of K, one-SM tiles.
+// chunk_rows > 0 (TF32 only): the chunked kernels, a fresh accumulator about every
+// chunk_rows rows of K.
 maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, const void* filt,
                          float* out, cudaStream_t stream, int chunk_rows = 0) {
   int32_t Ho, Wo;
@@ -355,7 +389,7 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   key.v[0] = ds->sm_count;
   key.v[1] = elem_bytes;
   key.v[2] = env_int("MAXDNN_UMMA_KC");
-  key.v[3] = chunk_rows > 0 ? -1 : env_int("MAXDNN_UMMA_PAIR");
+  key.v[3] = env_int("MAXDNN_UMMA_PAIR");
   key.v[4] = env_or("MAXDNN_UMMA_MERGE", -12345);
   key.v[5] = env_or("MAXDNN_UMMA_STAGE_KB", -12345);
   key.v[6] = env_or("MAXDNN_UMMA_COLS", -12345);
@@ -444,10 +478,11 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
     if (st != MAXDNN_OK) return st;
   }
   if (chunk_rows > 0) {
-    if (bf16 || g.pair) return MAXDNN_INVALID_VALUE;
+    if (bf16) return MAXDNN_INVALID_VALUE;
     const int steps = chunk_rows / g.rows;
     args.chunk_steps = (uint32_t)(steps < 1 ? 1 : steps);
-    return launch_umma_chunk(ds, mf, mi, mo, args, stream);
+    return g.pair ? launch_umma_pair_chunk(ds, mf, mi, mo, args, stream)
+                  : launch_umma_chunk(ds, mf, mi, mo, args, stream);
   }
   if (g.pair)
     return bf16 ? launch_umma_pair<true>(ds, mf, mi, mo, args, stream)

@@ -191,7 +191,6 @@ umma_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   const int n_ksteps = g.n_ksteps;
   const int mma_per_step = g.kc / (int)args.umma_k;
-  const int n_cols = g.tile_px * g.tile_n;   // MMA N
 
   if (warp == 0 || warp == 2) {
     // ----------------------------------------------------------- producers

@@ -51,6 +51,31 @@ def test_tf32x3_small(shape):
     assert err < err1 / 8
 
 
+@pytest.mark.parametrize("pair", [1, -1])
+@pytest.mark.parametrize("shape", [
+    (64, 14, 9, 48, 256, 3, 1, 1, 1.0),       # strip reuse, two tiles of 256 filters
+    (128, 9, 7, 32, 256, 5, 1, 2, 1.0),       # the CTAs of a pair split the images
+    (32, 21, 5, 40, 256, 3, 1, 1, 1.0),       # 8 pixels x 32 images, split by pixel
+    (64, 13, 5, 24, 512, 3, 1, 1, 0.5),       # ragged pixel tail
+    (64, 12, 6, 24, 160, 3, 1, 1, 1.0),       # 160 filters: second CTA of the pair mostly idle
+    (64, 9, 9, 300, 256, 3, 1, 1, 1.0),       # K = 2700: several chunks per tile
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_tf32x3_both_chunked_kernels(shape, pair, monkeypatch):
+    """The chunked kernel on one-SM tiles (pair = -1) and on two-SM tiles (pair = 1, forced
+    also where the planner would not take them), against the oracle at the exact kernel's bar."""
+    monkeypatch.setenv("MAXDNN_UMMA_PAIR", str(pair))
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("x3p", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
+                    ("uniform", 0.0, 1.0), 4500 + Nc)          # same-signed terms: the hard case
+    inp, filt = wl.make_inputs(w)
+    d = mx.ConvDesc.make(Nb, Wi, Hi, 3 * Nc, No, Sk, stride, pad, alpha)
+    assert mx.conv_plan_query(d, mx.KERNEL_TF32, 148)[0].tile_m == (256 if pair == 1 else 128)
+    got = run(w, inp, filt)
+    ref = oracle.conv_fprop(inp, filt, stride=stride, pad=pad, alpha=alpha)
+    assert np.isfinite(got).all()
+    assert float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref))) <= TOL_X3
+
+
 @pytest.mark.parametrize("chunked", [True, False])
 @pytest.mark.parametrize("name", ["mid5x5", "wide3x3", "large3x3", "first11x11s4", "alexnet_conv2",
                                   "overfeat_L3", "overfeat_L5"])

@@ -50,10 +50,11 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind,
     assert err <= 1e-5
 
 
-def test_chunked_kernel_wait_runs_out_and_the_context_survives(monkeypatch):
-    """The same for the chunked TF32 kernel behind maxdnn_conv_fprop_tf32x3 (eight epilogue
-    warps that wait for one chunk's accumulator after another)."""
-    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
+@pytest.mark.parametrize("No", [128, 256], ids=["one-sm", "two-sm"])
+def test_chunked_kernel_wait_runs_out_and_the_context_survives(No, monkeypatch):
+    """The same for the chunked TF32 kernels behind maxdnn_conv_fprop_tf32x3 (eight epilogue
+    warps per CTA that wait for one chunk's accumulator after another)."""
+    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=No)
     d = mx.ConvDesc.make(*w.dims)
     inp, filt = wl.make_inputs(w)
     x, f = torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda()
