@@ -214,9 +214,9 @@ maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const floa
  * maxdnn_conv_fprop_tf32 (with 3 Nc <= 32767); in / filt / out are the fp32 tensors.  The
  * paper has no counterpart (its kernel is an fp32 CUDA-core kernel).  Accuracy: the exact
  * kernel's class — measured 1e-6 .. 3e-6 of the largest output against the fp64 oracle for
- * K = 144 .. 9216 (exact fp32 kernel: 5e-7 .. 4e-6; plain TF32: 7e-4) — at three to four
- * times the exact kernel's speed.  (MAXDNN_X3_CHUNK_ROWS=0 in the environment selects the
- * one-accumulator path: 10-25 % faster, error about 1e-8 K.)
+ * K = 144 .. 9216 (exact fp32 kernel: 5e-7 .. 4e-6; plain TF32: 7e-4) — at about four
+ * times the exact kernel's speed on 3x3 / 5x5 layers.  (MAXDNN_X3_CHUNK_ROWS=0 in the
+ * environment selects the one-accumulator path: 2-3 % faster, error about 1e-8 K.)
  */
 maxdnn_status maxdnn_conv_fprop_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
 maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in,
