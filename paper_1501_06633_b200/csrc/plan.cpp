@@ -260,7 +260,12 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   // carry data instead of 3 of 16.  Needs one 128-byte group of images per tile column
   // group, so the tile is 256 / atom pixels x atom images.
   const int umma_k0 = 32 / elem_bytes;
-  const bool merged = d.Nc < umma_k0 && d.Skw > 1 && !pair && force_kc == 0 &&
+  // Also taken just above the MMA's K where a step per tap would be less than two thirds
+  // data (9 or 10 channels in tf32 — the three-product mode of a 3-channel layer — 17 to
+  // 21 in bf16).
+  const bool few = d.Nc < umma_k0 ||
+                   (d.Nc < 2 * umma_k0 && 3 * d.Nc < 2 * align_up(d.Nc, umma_k0));
+  const bool merged = few && d.Skw > 1 && !pair && force_kc == 0 &&
                       !(getenv("MAXDNN_UMMA_MERGE") && atoi(getenv("MAXDNN_UMMA_MERGE")) < 0);
   if (merged) {
     best_nn = atom;
@@ -343,9 +348,21 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   int strip_w = 0;
   if (merged) {
     const int box_c = align_up(d.Nc, 4);
-    int box_kw = d.Skw;
-    while ((box_kw * box_c) % umma_k != 0) ++box_kw;
-    const int rows1 = box_kw * box_c;                     // K rows of one filter row
+    // A filter row whose stage would not leave two ring stages is cut into as few parts
+    // of box_kw filter columns as do (every part re-reads the strip's overlap), one K step each (the copies of a part start at its
+    // first column; columns past the filter read zeros in the filter operand).
+    int box_kw = d.Skw, kw_parts = 1;
+    for (int parts = 1; parts <= d.Skw; ++parts) {
+      int w = ceil_div(d.Skw, parts);
+      while ((w * box_c) % umma_k != 0) ++w;
+      const int sw = w + (px_cta - 1) * d.stride_w;
+      const bool strip_ok = px_cta > 1 && (d.stride_w * box_c) % 8 == 0 && d.stride_w < w && sw <= 256;
+      const int b_rows = strip_ok ? sw * box_c * (g->cta_n / atom) : cols / atom * w * box_c;
+      box_kw = w;
+      kw_parts = ceil_div(d.Skw, w);
+      if ((128 / atom * w * box_c + b_rows) * 128 <= 96 * 1024) break;   // two stages fit
+    }
+    const int rows1 = box_kw * box_c;                     // K rows of one filter row (or part of it)
     // The windows of adjacent output pixels overlap (stride < Sk), so ONE box of
     // box_kw + (pixels - 1) * stride columns serves all pixels of the tile: pixel j's
     // operand starts j * stride * box_c rows into it, which the swizzle allows when that
@@ -355,19 +372,20 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
                    strip_w <= 256;
     const int b_rows1 = merged_strip ? strip_w * box_c * (g->cta_n / atom) : cols / atom * rows1;
     int khc = 1;   // filter rows per step: stages of at most 40 KB (a deep ring beat longer steps)
-    while (khc < d.Skh && (128 / atom * rows1 + b_rows1) * 128 * (khc + 1) <= 40 * 1024) ++khc;
-    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Skh) khc = v; }
+    while (kw_parts == 1 && khc < d.Skh && (128 / atom * rows1 + b_rows1) * 128 * (khc + 1) <= 40 * 1024) ++khc;
+    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Skh && kw_parts == 1) khc = v; }
     if (box_kw > 256 || rows1 * khc > 1024) return MAXDNN_NOT_SUPPORTED;
     // with the strip the rows of one filter row are contiguous in both operands, the
     // filter rows of a step are not (strip_w vs box_kw columns apart): kc counts the
     // rows of one filter row and the MMA warp's outer loop (kwc) walks the filter rows
     kc = merged_strip ? rows1 : rows1 * khc;
     kwc = merged_strip ? khc : 1;
-    for (int kh = 0; kh < d.Skh; kh += khc) {
-      if (n >= kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
-      t->s[n].c0 = 0; t->s[n].kh = (int8_t)kh; t->s[n].kw0 = 0;
-      ++n;
-    }
+    for (int kh = 0; kh < d.Skh; kh += khc)
+      for (int part = 0; part < kw_parts; ++part) {
+        if (n >= kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
+        t->s[n].c0 = 0; t->s[n].kh = (int8_t)kh; t->s[n].kw0 = (int8_t)(part * box_kw);
+        ++n;
+      }
     g->box_c = box_c; g->box_kw = box_kw; g->box_kh = khc;
   } else {
     build_table(d, kc, kwc, t, &n);
