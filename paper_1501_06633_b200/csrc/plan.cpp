@@ -330,6 +330,8 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
     int best = kc_max, best_pad = 1 << 30;
     for (int c = kc_max; c >= umma_k; c -= umma_k) {
       const int padded = ceil_div(d.Nc, c) * c;
+      // the K-step table has room for kMaxKSteps steps (one per tap or filter row and block)
+      if ((int64_t)ceil_div(d.Nc, c) * d.Skh * (kwc > 1 ? 1 : d.Skw) > kMaxKSteps && c != kc_max) continue;
       if (padded < best_pad) { best_pad = padded; best = c; }
     }
     return best;
