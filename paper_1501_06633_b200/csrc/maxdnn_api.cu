@@ -990,6 +990,49 @@ maxdnn_status fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in, const 
   return fprop_umma(&d3, 4, w_in, w_filt, out, stream);
 }
 
+// Map gradient in the three-product TF32 mode, stride 1: the FPROP of dout with the flipped,
+// transposed filter bank (as maxdnn_conv_bprop_data), run through fprop_tf32x3.  Workspace:
+// the transformed bank (fp32, rounded up to 256 bytes), then fprop_tf32x3's own.
+maxdnn_status dgrad_tf32x3_desc(const maxdnn_conv_desc* desc, maxdnn_conv_desc* t, size_t* ft_bytes) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  if (desc->stride != 1) return MAXDNN_NOT_SUPPORTED;
+  ConvDims fd;
+  st = plan_dgrad(dims_from(*desc), &fd);
+  if (st != MAXDNN_OK) return st;
+  t->Nb = fd.Nb; t->Wi = fd.Wi; t->Hi = fd.Hi; t->Nc = fd.Nc; t->No = fd.No;
+  t->Sk = fd.Skw; t->stride = 1; t->pad = fd.pad_w; t->alpha = fd.alpha;
+  *ft_bytes = round256((size_t)desc->Nc * desc->Sk * desc->Sk * desc->No * 4);
+  return MAXDNN_OK;
+}
+
+maxdnn_status bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout, const float* filt,
+                                float* din, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  maxdnn_conv_desc t;
+  size_t ft_bytes = 0, a = 0, b = 0;
+  maxdnn_status st = dgrad_tf32x3_desc(desc, &t, &ft_bytes);
+  if (st != MAXDNN_OK) return st;
+  st = tf32x3_sizes(&t, &a, &b);
+  if (st != MAXDNN_OK) return st;
+  if (!dout || !filt || !din || !ws) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(dout) || !aligned16(filt) || !aligned16(din) || !aligned16(ws))
+    return MAXDNN_INVALID_VALUE;
+  if (ws_bytes < ft_bytes + a + b) return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  const int taps = desc->Sk * desc->Sk;
+  const dim3 grid((unsigned)ceil_div(desc->No, 32), (unsigned)ceil_div(desc->Nc, 32), (unsigned)taps);
+  flip_transpose_kernel<float><<<grid, dim3(32, 8), 0, stream>>>(filt, static_cast<float*>(ws),
+                                                               desc->Nc, taps, desc->No);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return fprop_tf32x3(&t, dout, static_cast<const float*>(ws), din,
+                      static_cast<uint8_t*>(ws) + ft_bytes, ws_bytes - ft_bytes, stream);
+}
+
 // ---------------------------------------------------------------------------
 // Allocation-free fp32 entry point.  The status block its kernel reports into
 // lives in this file-scope device array instead of cudaMalloc'd memory.  Every
@@ -1256,6 +1299,25 @@ maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float
                                        size_t workspace_bytes, void* cuda_stream) {
   return fprop_tf32x3(desc, in, filt, out, workspace, workspace_bytes,
                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_bprop_data_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
+  if (!bytes) return MAXDNN_INVALID_VALUE;
+  maxdnn_conv_desc t;
+  size_t ft_bytes = 0, a = 0, b = 0;
+  maxdnn_status st = dgrad_tf32x3_desc(desc, &t, &ft_bytes);
+  if (st != MAXDNN_OK) return st;
+  st = tf32x3_sizes(&t, &a, &b);
+  if (st != MAXDNN_OK) return st;
+  *bytes = ft_bytes + a + b;
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout,
+                                            const float* filt, float* din, void* workspace,
+                                            size_t workspace_bytes, void* cuda_stream) {
+  return bprop_data_tf32x3(desc, dout, filt, din, workspace, workspace_bytes,
+                           static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,

@@ -96,3 +96,51 @@ def test_tf32x3_full_size_sampled(name, chunked, monkeypatch):
                                 rows=(y, y + 1))[:, y]
         err = float(np.max(np.abs(got[:, y].astype(np.float64) - ref))) / float(np.max(np.abs(ref)))
         assert err <= tol
+
+
+@pytest.mark.parametrize("shape", [
+    (64, 14, 9, 64, 96, 3, 1, 1, 1.0),        # transposed problem: 96 channels -> 64 "filters"
+    (128, 9, 7, 96, 64, 5, 1, 2, 0.5),
+    (64, 12, 10, 128, 32, 3, 1, 0, 1.0),      # no padding: the gradient's FPROP pads by Sk - 1
+    (32, 16, 16, 256, 160, 3, 1, 1, -2.0),    # two-SM tiles (256 "filters"), K = 1440
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_data_tf32x3(shape):
+    """Map gradient in the three-product mode against the gradient oracle, at the exact
+    kernel's bar (same-signed operands: the case the chunked accumulation is for)."""
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("x3g", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
+                    ("uniform", 0.0, 1.0), 4600 + Nc)
+    _, filt = wl.make_inputs(w)
+    dout = np.abs(wl.make_dout(w))
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data_tf32x3(d, torch.from_numpy(dout).cuda(), torch.from_numpy(filt).cuda(), din, ws)
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_data(dout, filt, (Hi, Wi), stride=stride, pad=pad, alpha=alpha)
+    got = din.cpu().numpy().reshape(ref.shape)
+    assert np.isfinite(got).all()
+    assert float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref))) <= TOL_X3
+
+
+def test_bprop_data_tf32x3_full_size_sampled_and_refusals():
+    w = wl.WORKLOADS["large3x3"]
+    _, filt = wl.make_inputs(w)
+    dout = wl.make_dout(w)
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data_tf32x3(d, torch.from_numpy(dout).cuda(), torch.from_numpy(filt).cuda(), din, ws)
+    assert mx.last_device_status() == mx.OK
+    got = din.cpu().numpy().reshape(w.Nc, w.Hi, w.Wi, w.Nb)
+    assert np.isfinite(got).all()
+    rng = np.random.default_rng(12)
+    pts = [tuple(int(rng.integers(0, s)) for s in got.shape) for _ in range(150)]
+    pts += [(0, 0, 0, 0), (w.Nc - 1, w.Hi - 1, w.Wi - 1, w.Nb - 1)]
+    vals = [oracle.conv_bprop_data_point(dout, filt, (w.Hi, w.Wi), *p, stride=1, pad=w.pad,
+                                         alpha=w.alpha)[0] for p in pts]
+    scale = max(abs(v) for v in vals)
+    assert max(abs(float(got[p]) - v) for p, v in zip(pts, vals)) <= TOL_X3 * scale
+    with pytest.raises(mx.MaxdnnError) as e:        # stride 2: not in this mode
+        mx.conv_bprop_data_tf32x3_workspace(mx.ConvDesc.make(64, 56, 56, 128, 256, 3, 2, 1, 1.0))
+    assert e.value.status == mx.NOT_SUPPORTED
