@@ -19,6 +19,7 @@ __all__ = [
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
     "conv_fprop_tf32x3_workspace", "conv_fprop_tf32x3",
     "conv_bprop_data_tf32x3_workspace", "conv_bprop_data_tf32x3",
+    "conv_bprop_filter_tf32x3_workspace", "conv_bprop_filter_tf32x3",
     "ConvDesc2", "conv2_out_dims", "conv2_fprop", "conv2_fprop_status",
     "conv2_bprop_data_workspace", "conv2_bprop_data", "conv2_bprop_filter_workspace",
     "conv2_bprop_filter",
@@ -41,6 +42,7 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv2_out_dims", "maxdnn_conv2_fprop",
     "maxdnn_conv_fprop_tf32x3_workspace", "maxdnn_conv_fprop_tf32x3",
     "maxdnn_conv_bprop_data_tf32x3_workspace", "maxdnn_conv_bprop_data_tf32x3",
+    "maxdnn_conv_bprop_filter_tf32x3_workspace", "maxdnn_conv_bprop_filter_tf32x3",
     "maxdnn_conv2_bprop_data_workspace", "maxdnn_conv2_bprop_data",
     "maxdnn_conv2_bprop_filter_workspace", "maxdnn_conv2_bprop_filter",
 ]
@@ -136,6 +138,10 @@ def load_library():
     lib.maxdnn_conv_bprop_data_tf32x3_workspace.argtypes = [P(ConvDesc), P(ctypes.c_size_t)]
     lib.maxdnn_conv_bprop_data_tf32x3.restype = ctypes.c_int
     lib.maxdnn_conv_bprop_data_tf32x3.argtypes = [P(ConvDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.maxdnn_conv_bprop_filter_tf32x3_workspace.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_filter_tf32x3_workspace.argtypes = [P(ConvDesc), P(ctypes.c_size_t)]
+    lib.maxdnn_conv_bprop_filter_tf32x3.restype = ctypes.c_int
+    lib.maxdnn_conv_bprop_filter_tf32x3.argtypes = [P(ConvDesc), vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.maxdnn_conv2_out_dims.restype = ctypes.c_int
     lib.maxdnn_conv2_out_dims.argtypes = [P(ConvDesc2), P(ctypes.c_int32), P(ctypes.c_int32)]
     lib.maxdnn_conv2_fprop.restype = ctypes.c_int
@@ -340,6 +346,27 @@ def conv_bprop_data_tf32x3(desc: ConvDesc, dout, filt, din, workspace, stream=No
     _check(int(lib.maxdnn_conv_bprop_data_tf32x3(ctypes.byref(desc), pg, pf, px, pw, nbytes,
                                                  _stream_ptr(stream))),
            "maxdnn_conv_bprop_data_tf32x3")
+
+
+def conv_bprop_filter_tf32x3_workspace(desc: ConvDesc) -> int:
+    """Bytes of device scratch maxdnn_conv_bprop_filter_tf32x3 needs."""
+    n = ctypes.c_size_t()
+    _check(int(load_library().maxdnn_conv_bprop_filter_tf32x3_workspace(ctypes.byref(desc),
+                                                                        ctypes.byref(n))),
+           "maxdnn_conv_bprop_filter_tf32x3_workspace")
+    return int(n.value)
+
+
+def conv_bprop_filter_tf32x3(desc: ConvDesc, inp, dout, dfilt, workspace, stream=None) -> None:
+    """maxdnn_conv_bprop_filter_tf32x3: filter gradient in the three-product TF32 mode."""
+    lib = load_library()
+    px = _dev_ptr(inp, ("float32",), conv_in_elems(desc), "in")
+    pg = _dev_ptr(dout, ("float32",), conv_out_elems(desc), "dout")
+    pf = _dev_ptr(dfilt, ("float32",), conv_filt_elems(desc), "dfilt")
+    pw, nbytes = _workspace_ptr(workspace, 1)
+    _check(int(lib.maxdnn_conv_bprop_filter_tf32x3(ctypes.byref(desc), px, pg, pf, pw, nbytes,
+                                                   _stream_ptr(stream))),
+           "maxdnn_conv_bprop_filter_tf32x3")
 
 
 def conv2_out_dims(desc: ConvDesc2):

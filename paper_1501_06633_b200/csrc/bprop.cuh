@@ -109,6 +109,27 @@ tf32_split3_kernel(const float4* __restrict__ src, float4* __restrict__ dst, siz
   for (int p = 0; p < 3; ++p) dst[(size_t)p * n4 + i] = ((lo_mask >> p) & 1u) ? lo : hi;
 }
 
+// The same split with the three parts side by side along the innermost (image) axis: row r
+// of dst is [part 0 | part 1 | part 2] of row r of src, each n4 float4 long.  For the filter
+// gradient, whose reduction runs over images: maps [hi | lo | hi] x gradients [hi | hi | lo].
+__global__ void __launch_bounds__(256)
+tf32_split3_rows_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t rows,
+                        int n4, uint32_t lo_mask) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * (size_t)n4) return;
+  const size_t row = i / (size_t)n4;
+  const int j = (int)(i - row * (size_t)n4);
+  const float4 a = src[i];
+  float4 hi, lo;
+  hi.x = round_to_tf32(a.x); hi.y = round_to_tf32(a.y);
+  hi.z = round_to_tf32(a.z); hi.w = round_to_tf32(a.w);
+  lo.x = round_to_tf32(a.x - hi.x); lo.y = round_to_tf32(a.y - hi.y);
+  lo.z = round_to_tf32(a.z - hi.z); lo.w = round_to_tf32(a.w - hi.w);
+#pragma unroll
+  for (int p = 0; p < 3; ++p)
+    dst[(row * 3 + p) * (size_t)n4 + j] = ((lo_mask >> p) & 1u) ? lo : hi;
+}
+
 // Staging copies for shapes the bulk tensor copies cannot address (row pitches that are
 // not multiples of 16 bytes): dst[row][j] = src[row][j] for j < n, 0 for n <= j < n_pad
 // (pad_inner), and the reverse for results (unpad_inner drops the padding columns).

@@ -13,6 +13,7 @@
 #include "umma_conv.cuh"
 #include "umma_chunk_conv.cuh"
 #include "umma_pair_chunk_conv.cuh"
+#include "wgrad_umma_chunk.cuh"
 #include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
 #include "wgrad_umma_pair.cuh"
@@ -32,6 +33,7 @@ struct DeviceState {
   bool wgrad_attr = false;
   bool umma_chunk_attr = false;
   bool umma_pair_chunk_attr = false;
+  bool wgrad_chunk_attr = false;
   bool wgrad_umma_attr[4] = {false, false, false, false};
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
@@ -1033,6 +1035,114 @@ maxdnn_status bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout,
                       static_cast<uint8_t*>(ws) + ft_bytes, ws_bytes - ft_bytes, stream);
 }
 
+// Filter gradient in the three-product TF32 mode.  The reduction runs over pixels and
+// images, so the three products are one reduction over three times the images: maps
+// [hi | lo | hi] and gradients [hi | hi | lo] side by side along the image axis, then the
+// chunked TF32 filter-gradient kernel on the problem with 3 Nb images.  Workspace: the two
+// split tensors (each rounded up to 256 bytes), then the partial sums of the split reduction.
+struct WgradX3Plan {
+  ConvDims d3;
+  size_t in_bytes, dout_bytes, partial_bytes;
+};
+
+maxdnn_status plan_wgrad_x3(const maxdnn_conv_desc* desc, int sm_count, WgradX3Plan* p, WgradGeom* g) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  int32_t Ho, Wo;
+  maxdnn_status st = check_desc(desc, &Ho, &Wo);
+  if (st != MAXDNN_OK) return st;
+  if (desc->Nb % 32 != 0) return MAXDNN_NOT_SUPPORTED;      // whole 128-byte rows of each part
+  if ((int64_t)desc->Nb * 3 > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
+  p->d3 = dims_from(*desc);
+  p->d3.Nb = 3 * desc->Nb;
+  p->in_bytes = round256((size_t)desc->Nc * desc->Hi * desc->Wi * p->d3.Nb * 4);
+  p->dout_bytes = round256((size_t)desc->No * Ho * Wo * p->d3.Nb * 4);
+  static thread_local WgradGeom scratch;
+  WgradGeom* gg = g ? g : &scratch;
+  st = plan_wgrad(p->d3, 4, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), gg, -1);   // one-SM tiles
+  if (st != MAXDNN_OK) return st;
+  const size_t kno = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No;
+  p->partial_bytes = gg->splits > 1 ? (size_t)gg->splits * kno * 4 : 0;
+  return MAXDNN_OK;
+}
+
+maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in, const float* dout,
+                                  float* dfilt, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  if (!in || !dout || !dfilt || !ws) return MAXDNN_INVALID_VALUE;
+  if (!aligned16(in) || !aligned16(dout) || !aligned16(dfilt) || !aligned16(ws))
+    return MAXDNN_INVALID_VALUE;
+  DeviceState* ds = nullptr;
+  maxdnn_status st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
+  static thread_local WgradUmmaArgs args;
+  WgradX3Plan p;
+  st = plan_wgrad_x3(desc, ds->sm_count, &p, &args.g);
+  if (st != MAXDNN_OK) return st;
+  if (ws_bytes < p.in_bytes + p.dout_bytes + p.partial_bytes) return MAXDNN_INVALID_VALUE;
+  const WgradGeom& g = args.g;
+  float* w_in = static_cast<float*>(ws);
+  float* w_dout = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + p.in_bytes);
+  float* w_part = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + p.in_bytes + p.dout_bytes);
+  const int n4 = desc->Nb / 4;
+  const size_t rows_in = (size_t)desc->Nc * desc->Hi * desc->Wi;
+  const size_t rows_g = (size_t)desc->No * g.Ho * g.Wo;
+  // maps [hi | lo | hi] x gradients [hi | hi | lo]  ->  hi*hi + lo*hi + hi*lo
+  tf32_split3_rows_kernel<<<(unsigned)((rows_in * n4 + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(in), reinterpret_cast<float4*>(w_in), rows_in, n4, 0x2u);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  tf32_split3_rows_kernel<<<(unsigned)((rows_g * n4 + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(dout), reinterpret_cast<float4*>(w_dout), rows_g, n4, 0x4u);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(2, std::memory_order_relaxed);
+  CUtensorMap mg, mi;
+  {
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
+                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
+    const uint32_t box[4] = {32u, 1u, 1u, (uint32_t)g.box_o};
+    st = encode_map(&mg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w_dout, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != MAXDNN_OK) return st;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
+                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
+    st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w_in, dims, str, box,
+                    CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != MAXDNN_OK) return st;
+  }
+  args.dfilt = dfilt;
+  args.partial = w_part;
+  args.status = ds->status;
+  args.atom = 32u;
+  // a fresh accumulator every 24 reduction steps: 768 terms of the tripled reduction
+  const int cs = env_or("MAXDNN_X3_CHUNK_ROWS", 768) / 32;
+  args.chunk_steps = (uint32_t)(cs < 1 ? 1 : cs);
+  args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) | ((128u >> 4) << 24);
+  if (!ds->wgrad_chunk_attr) {
+    if (cudaFuncSetAttribute(wgrad_umma_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return MAXDNN_CUDA_ERROR;
+    }
+    ds->wgrad_chunk_attr = true;
+  }
+  wgrad_umma_chunk_kernel<<<g.grid, kWgChunkThreads, g.smem_bytes, stream>>>(mg, mi, args);
+  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g.splits > 1) {
+    const size_t n4f = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No / 4;
+    wgrad_reduce_kernel<<<(unsigned)((n4f + 255) / 256), 256, 0, stream>>>(w_part, dfilt, n4f,
+                                                                         g.splits, g.alpha);
+    if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  }
+  return MAXDNN_OK;
+}
+
 // ---------------------------------------------------------------------------
 // Allocation-free fp32 entry point.  The status block its kernel reports into
 // lives in this file-scope device array instead of cudaMalloc'd memory.  Every
@@ -1318,6 +1428,29 @@ maxdnn_status maxdnn_conv_bprop_data_tf32x3(const maxdnn_conv_desc* desc, const 
                                             size_t workspace_bytes, void* cuda_stream) {
   return bprop_data_tf32x3(desc, dout, filt, din, workspace, workspace_bytes,
                            static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_conv_bprop_filter_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
+  if (!bytes) return MAXDNN_INVALID_VALUE;
+  int sm = env_int("MAXDNN_SM_COUNT");
+  if (sm <= 0) {
+    DeviceState* ds = nullptr;
+    const maxdnn_status st = device_state(&ds);
+    if (st != MAXDNN_OK) return st;
+    sm = ds->sm_count;
+  }
+  WgradX3Plan p;
+  const maxdnn_status st = plan_wgrad_x3(desc, sm, &p, nullptr);
+  if (st != MAXDNN_OK) return st;
+  *bytes = p.in_bytes + p.dout_bytes + p.partial_bytes;
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
+                                              const float* dout, float* dfilt, void* workspace,
+                                              size_t workspace_bytes, void* cuda_stream) {
+  return bprop_filter_tf32x3(desc, in, dout, dfilt, workspace, workspace_bytes,
+                             static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_fprop_ragged_workspace(const maxdnn_conv_desc* desc,

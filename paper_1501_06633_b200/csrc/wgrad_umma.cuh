@@ -30,6 +30,7 @@ struct WgradUmmaArgs {
   WgradGeom g;            // rows <= 256; n_chunks counts groups of `atom` images
   uint32_t idesc;
   uint32_t atom;          // images per reduction step: 32 (tf32) or 64 (bf16)
+  uint32_t chunk_steps;   // chunked kernel only: reduction steps per TMEM accumulator
   float* dfilt;
   float* partial;
   uint32_t* status;

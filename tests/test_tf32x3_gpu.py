@@ -144,3 +144,34 @@ def test_bprop_data_tf32x3_full_size_sampled_and_refusals():
     with pytest.raises(mx.MaxdnnError) as e:        # stride 2: not in this mode
         mx.conv_bprop_data_tf32x3_workspace(mx.ConvDesc.make(64, 56, 56, 128, 256, 3, 2, 1, 1.0))
     assert e.value.status == mx.NOT_SUPPORTED
+
+
+@pytest.mark.parametrize("splits", [0, 1, 3])
+@pytest.mark.parametrize("shape", [
+    (64, 14, 9, 40, 96, 3, 1, 1, 1.0),        # 28 channels x 9 taps per tile, two channel blocks
+    (128, 9, 7, 24, 64, 5, 1, 2, 0.5),        # 10 channels x 25 taps
+    (32, 23, 19, 3, 96, 11, 4, 0, 1.0),       # the first-layer shape: two blocks of filter rows
+    (64, 8, 8, 300, 64, 1, 1, 0, 2.0),        # 1x1: 256 channels per tile, ragged second block
+    (64, 12, 10, 16, 132, 3, 2, 1, 1.0),      # filters not a multiple of 128, stride 2
+    (96, 10, 6, 8, 256, 4, 1, 3, -1.0),       # two filter blocks; 96 images = three 128-byte rows
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_filter_tf32x3(shape, splits, monkeypatch):
+    """Filter gradient in the three-product mode (the three products as one reduction over
+    three times the images, accumulated in chunks) against the gradient oracle at the exact
+    kernel's bar; same-signed operands, forced split counts."""
+    if splits:
+        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("x3w", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
+                    ("uniform", 0.0, 1.0), 4700 + Nc)
+    inp, _ = wl.make_inputs(w)
+    dout = np.abs(wl.make_dout(w))
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_filter_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    dfilt = torch.full((mx.conv_filt_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_filter_tf32x3(d, torch.from_numpy(inp).cuda(), torch.from_numpy(dout).cuda(), dfilt, ws)
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_filter(inp, dout, Sk, stride=stride, pad=pad, alpha=alpha)
+    got = dfilt.cpu().numpy().reshape(ref.shape)
+    assert np.isfinite(got).all()
+    assert float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref))) <= TOL_X3
