@@ -295,9 +295,7 @@ def run_ours(args):
 
     peaks, peaks_kind = load_peaks()
     w = wl.ALL[args.workload]
-    x3 = args.kernel == "tf32x3"            # three TF32 products: fp32 buffers, FPROP only
-    if x3 and args.op != "fprop":
-        raise SystemExit("--kernel tf32x3 is an FPROP mode")
+    x3 = args.kernel == "tf32x3"            # three TF32 products: fp32 buffers, its own entry points
     kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16,
             "tf32x3": mx.KERNEL_TF32}[args.kernel]
     d = mx.ConvDesc.make(*w.dims)
@@ -339,18 +337,27 @@ def run_ours(args):
                          device="cuda")
     fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
              mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
+    # one call of the operation: run(a, b, r, workspace, stream)
     if x3:
-        ws = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
-        fprop = lambda dd, a, b, r, stream=None: mx.conv_fprop_tf32x3(dd, a, b, r, ws, stream=stream)
+        size_fn, call_fn = {
+            "fprop": (mx.conv_fprop_tf32x3_workspace, mx.conv_fprop_tf32x3),
+            "dgrad": (mx.conv_bprop_data_tf32x3_workspace, mx.conv_bprop_data_tf32x3),
+            "wgrad": (mx.conv_bprop_filter_tf32x3_workspace, mx.conv_bprop_filter_tf32x3)}[op]
+        ws = torch.empty(max(16, size_fn(d)), dtype=torch.uint8, device="cuda")
+        run = lambda a, b, r, wsp, stream=None: call_fn(d, a, b, r, wsp, stream=stream)
+    elif op == "fprop":
+        run = lambda a, b, r, wsp, stream=None: fprop(d, as_op(a), as_op(b), r, stream=stream)
+    elif op == "dgrad":
+        run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_data(d, as_op(a), as_op(b), r, wsp, kind,
+                                                                   stream=stream)
+    else:
+        run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_filter(d, as_op(a), as_op(b), r, wsp, kind,
+                                                                     stream=stream)
 
     def step(i):
         a, b, r = d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets]
-        if op == "fprop":
-            fprop(d, as_op(a), as_op(b), r)
-        elif op == "dgrad":
-            mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws, kind)
-        else:
-            mx.conv_bprop_filter(d, as_op(a), as_op(b), r, ws, kind)
+        run(a, b, r, ws)
+        if op == "wgrad":
             sum_gradient_over_ranks(r, world)      # NCCL all-reduce over the batch shards
 
     def barrier():
@@ -393,20 +400,11 @@ def run_ours(args):
         a, b, r = d_as[k % n_sets], d_bs[k % len(d_bs)], d_res[k % n_sets]
         if op == "fprop" and not x3:
             mx.conv_fprop_host(d, kind, h_a, h_b, h_outs[k], a, b, r, stream=stream)
-        elif op == "fprop":
-            with torch.cuda.stream(stream):
-                a.copy_(h_a, non_blocking=True)
-                b.copy_(h_b, non_blocking=True)
-                mx.conv_fprop_tf32x3(d, a, b, r, ws_e2e[k], stream=stream)
-                h_outs[k].copy_(r, non_blocking=True)
         else:
             with torch.cuda.stream(stream):
                 a.copy_(h_a, non_blocking=True)
                 b.copy_(h_b, non_blocking=True)
-                if op == "dgrad":
-                    mx.conv_bprop_data(d, as_op(a), as_op(b), r, ws_e2e[k], kind, stream=stream)
-                else:
-                    mx.conv_bprop_filter(d, as_op(a), as_op(b), r, ws_e2e[k], kind, stream=stream)
+                run(a, b, r, ws_e2e[k], stream=stream)
                 h_outs[k].copy_(r, non_blocking=True)
 
     ws_e2e = [ws, None if ws is None else torch.empty_like(ws)]
