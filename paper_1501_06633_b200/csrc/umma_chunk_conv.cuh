@@ -12,8 +12,9 @@
 // accumulators in TMEM, bounded waits) with EIGHT epilogue warps: two per TMEM lane
 // quarter, each holding 128 of the tile's columns of its 32 filters in registers
 // (128 totals per thread).  Warp 0: patch copies, warp 1: MMA issue, warp 2: filter copies,
-// warps 3-10: epilogue — the three warps with short per-step loops are the oldest on their
-// schedulers, ahead of the epilogue warps that wait for a chunk.
+// warps 3-10: epilogue.  The MMA warp's loop over a chunk's K steps is exactly the plain
+// kernel's, with the chunk loop around it: a K step can be as short as four MMAs, and a
+// chunk test inside the step loop cost 17 % on such layers.
 #pragma once
 #include "umma_conv.cuh"
 
