@@ -233,10 +233,10 @@ maxdnn_status maxdnn_conv_bprop_data_tf32x3(const maxdnn_conv_desc* desc, const 
                                             size_t workspace_bytes, void* cuda_stream);
 /* The gradient with respect to the filters in the three-product mode.  Its reduction runs
  * over pixels and images, so the three products are ONE reduction over three times the
- * images: a small kernel writes maps [hi | lo | hi] and gradients [hi | hi | lo] side by side
- * along the image axis into the workspace, and a TF32 filter-gradient kernel that accumulates
- * in chunks (a fresh accumulator every 768 terms, the chunks added in round-to-nearest fp32)
- * runs on the problem with 3 Nb images; partial sums of the split reduction are added in a
+ * images: a small kernel writes both tensors as [hi | lo] side by side along the image axis
+ * into the workspace, and a TF32 filter-gradient kernel that accumulates in chunks (a fresh
+ * accumulator every 768 terms, the chunks added in round-to-nearest fp32) runs on the
+ * problem with 3 Nb images, reading for each third the parts of that product; partial sums of the split reduction are added in a
  * fixed order as in maxdnn_conv_bprop_filter.  in / dout / dfilt are the fp32 tensors.
  * NOT_SUPPORTED: Nb not a multiple of 32, No not a multiple of 4, the limits of
  * maxdnn_conv_fprop.  Accuracy: the exact kernel's class (tested to 1e-5 of the largest

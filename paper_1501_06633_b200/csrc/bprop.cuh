@@ -109,12 +109,12 @@ tf32_split3_kernel(const float4* __restrict__ src, float4* __restrict__ dst, siz
   for (int p = 0; p < 3; ++p) dst[(size_t)p * n4 + i] = ((lo_mask >> p) & 1u) ? lo : hi;
 }
 
-// The same split with the three parts side by side along the innermost (image) axis: row r
-// of dst is [part 0 | part 1 | part 2] of row r of src, each n4 float4 long.  For the filter
-// gradient, whose reduction runs over images: maps [hi | lo | hi] x gradients [hi | hi | lo].
+// The split for the filter gradient, whose reduction runs over images: row r of dst is
+// [hi | lo] of row r of src, each part n4 float4 long (the kernel reads the parts it needs
+// for each of the three products: hi x hi, lo x hi, hi x lo).
 __global__ void __launch_bounds__(256)
-tf32_split3_rows_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t rows,
-                        int n4, uint32_t lo_mask) {
+tf32_split2_rows_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t rows,
+                        int n4) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= rows * (size_t)n4) return;
   const size_t row = i / (size_t)n4;
@@ -125,9 +125,8 @@ tf32_split3_rows_kernel(const float4* __restrict__ src, float4* __restrict__ dst
   hi.z = round_to_tf32(a.z); hi.w = round_to_tf32(a.w);
   lo.x = round_to_tf32(a.x - hi.x); lo.y = round_to_tf32(a.y - hi.y);
   lo.z = round_to_tf32(a.z - hi.z); lo.w = round_to_tf32(a.w - hi.w);
-#pragma unroll
-  for (int p = 0; p < 3; ++p)
-    dst[(row * 3 + p) * (size_t)n4 + j] = ((lo_mask >> p) & 1u) ? lo : hi;
+  dst[(row * 2) * (size_t)n4 + j] = hi;
+  dst[(row * 2 + 1) * (size_t)n4 + j] = lo;
 }
 
 // Staging copies for shapes the bulk tensor copies cannot address (row pitches that are

@@ -1036,9 +1036,10 @@ maxdnn_status bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout,
 }
 
 // Filter gradient in the three-product TF32 mode.  The reduction runs over pixels and
-// images, so the three products are one reduction over three times the images: maps
-// [hi | lo | hi] and gradients [hi | hi | lo] side by side along the image axis, then the
-// chunked TF32 filter-gradient kernel on the problem with 3 Nb images.  Workspace: the two
+// images, so the three products are one reduction over three times the images: both
+// tensors are split into [hi | lo] side by side along the image axis, and the chunked TF32
+// filter-gradient kernel runs on the problem with 3 Nb images, reading for each third of
+// them the parts of that product (hi x hi, hi x lo, lo x hi).  Workspace: the two
 // split tensors (each rounded up to 256 bytes), then the partial sums of the split reduction.
 struct WgradX3Plan {
   ConvDims d3;
@@ -1054,8 +1055,8 @@ maxdnn_status plan_wgrad_x3(const maxdnn_conv_desc* desc, int sm_count, WgradX3P
   if ((int64_t)desc->Nb * 3 > 0x7fffffff) return MAXDNN_NOT_SUPPORTED;
   p->d3 = dims_from(*desc);
   p->d3.Nb = 3 * desc->Nb;
-  p->in_bytes = round256((size_t)desc->Nc * desc->Hi * desc->Wi * p->d3.Nb * 4);
-  p->dout_bytes = round256((size_t)desc->No * Ho * Wo * p->d3.Nb * 4);
+  p->in_bytes = round256((size_t)desc->Nc * desc->Hi * desc->Wi * 2 * desc->Nb * 4);     // [hi | lo]
+  p->dout_bytes = round256((size_t)desc->No * Ho * Wo * 2 * desc->Nb * 4);
   static thread_local WgradGeom scratch;
   WgradGeom* gg = g ? g : &scratch;
   st = plan_wgrad(p->d3, 4, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), gg, -1);   // one-SM tiles
@@ -1087,28 +1088,29 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
   const int n4 = desc->Nb / 4;
   const size_t rows_in = (size_t)desc->Nc * desc->Hi * desc->Wi;
   const size_t rows_g = (size_t)desc->No * g.Ho * g.Wo;
-  // maps [hi | lo | hi] x gradients [hi | hi | lo]  ->  hi*hi + lo*hi + hi*lo
-  tf32_split3_rows_kernel<<<(unsigned)((rows_in * n4 + 255) / 256), 256, 0, stream>>>(
-      reinterpret_cast<const float4*>(in), reinterpret_cast<float4*>(w_in), rows_in, n4, 0x2u);
+  // both tensors as [hi | lo] along the image axis; the kernel's three passes over the
+  // images pair them as hi*hi + hi*lo + lo*hi
+  tf32_split2_rows_kernel<<<(unsigned)((rows_in * n4 + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(in), reinterpret_cast<float4*>(w_in), rows_in, n4);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
-  tf32_split3_rows_kernel<<<(unsigned)((rows_g * n4 + 255) / 256), 256, 0, stream>>>(
-      reinterpret_cast<const float4*>(dout), reinterpret_cast<float4*>(w_dout), rows_g, n4, 0x4u);
+  tf32_split2_rows_kernel<<<(unsigned)((rows_g * n4 + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(dout), reinterpret_cast<float4*>(w_dout), rows_g, n4);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(2, std::memory_order_relaxed);
   CUtensorMap mg, mi;
   {
-    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wo * g.Nb * 4,
-                             (uint64_t)g.Ho * g.Wo * g.Nb * 4};
+    const uint64_t nb2 = 2ull * desc->Nb;      // stored images per pixel: [hi | lo]
+    const uint64_t dims[4] = {nb2, (uint64_t)g.Wo, (uint64_t)g.Ho, (uint64_t)g.No};
+    const uint64_t str[3] = {nb2 * 4, (uint64_t)g.Wo * nb2 * 4, (uint64_t)g.Ho * g.Wo * nb2 * 4};
     const uint32_t box[4] = {32u, 1u, 1u, (uint32_t)g.box_o};
     st = encode_map(&mg, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w_dout, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, (uint64_t)g.Wi * g.Nb * 4,
-                             (uint64_t)g.Hi * g.Wi * g.Nb * 4};
+    const uint64_t nb2 = 2ull * desc->Nb;
+    const uint64_t dims[4] = {nb2, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t str[3] = {nb2 * 4, (uint64_t)g.Wi * nb2 * 4, (uint64_t)g.Hi * g.Wi * nb2 * 4};
     const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w_in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_128B);
@@ -1121,6 +1123,7 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
   // a fresh accumulator every 24 reduction steps: 768 terms of the tripled reduction
   const int cs = env_or("MAXDNN_X3_CHUNK_ROWS", 768) / 32;
   args.chunk_steps = (uint32_t)(cs < 1 ? 1 : cs);
+  args.x3_per_part = (uint32_t)(desc->Nb / 32);
   args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) | ((128u >> 4) << 24);
   if (!ds->wgrad_chunk_attr) {
     if (cudaFuncSetAttribute(wgrad_umma_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -31,6 +31,7 @@ struct WgradUmmaArgs {
   uint32_t idesc;
   uint32_t atom;          // images per reduction step: 32 (tf32) or 64 (bf16)
   uint32_t chunk_steps;   // chunked kernel only: reduction steps per TMEM accumulator
+  uint32_t x3_per_part;   // chunked kernel only: reduction steps (groups of 32 images) per product part
   float* dfilt;
   float* partial;
   uint32_t* status;

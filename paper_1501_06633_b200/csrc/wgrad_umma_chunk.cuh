@@ -3,7 +3,7 @@
 // Same structure as wgrad_umma_kernel; the MMA warp starts a fresh TMEM accumulator every
 // chunk_steps reduction steps and eight epilogue warps add the chunks in registers.  Used by
 // maxdnn_conv_bprop_filter_tf32x3, whose three TF32 products are one reduction over three
-// times the images (maps [hi | lo | hi], gradients [hi | hi | lo] along the image axis).
+// times the images (three passes over tensors stored [hi | lo] along the image axis).
 // Warp 0: copies, warp 1: MMA issue and TMEM, warps 2-9: epilogue.
 #pragma once
 #include "umma_chunk_conv.cuh"
@@ -156,11 +156,18 @@ wgrad_umma_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
       }
       const uint32_t fb = full_bar + 8u * stage;
       const uint32_t dst = base + (uint32_t)stage * stage_bytes;
-      const int n0 = pc.nc * (int)args.atom;
+      // The image axis of the reduction holds the three products one after another:
+      // part 0 = gradient hi x map hi, 1 = hi x lo, 2 = lo x hi; both tensors are stored
+      // as [hi | lo] along their image axis.
+      const int per = (int)args.x3_per_part;
+      const int part = pc.nc / per;
+      const int within = pc.nc - part * per;
+      const int n_g = ((part == 2 ? per : 0) + within) * (int)args.atom;
+      const int n_x = ((part == 1 ? per : 0) + within) * (int)args.atom;
       if (elect_one()) {
         mbar_arrive_expect_tx(fb, tx_bytes);
-        tma_load_4d_hint(dst, &map_dout, fb, n0, pc.x, pc.y, pc.ob * 128, pol_last);
-        tma_load_4d_hint(dst + kWgUmmaABytes, &map_in, fb, n0, pc.x * g.stride_w - g.pad_w,
+        tma_load_4d_hint(dst, &map_dout, fb, n_g, pc.x, pc.y, pc.ob * 128, pol_last);
+        tma_load_4d_hint(dst + kWgUmmaABytes, &map_in, fb, n_x, pc.x * g.stride_w - g.pad_w,
                          pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc, pol_last);
       }
       __syncwarp();
