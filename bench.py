@@ -430,6 +430,32 @@ def run_ours(args):
     e2e_ms_single = time_e2e(1)
     e2e_ms = time_e2e(2)
 
+    # Beside the default (exact fp32) line: the same workload through the three-product TF32
+    # entry point, which holds the exact kernel's accuracy bar on the tensor cores — reported
+    # as an extra object, outside every timed region above.
+    also = None
+    if world == 1 and args.kernel == "fp32" and op == "fprop":
+        try:
+            ws3 = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+            n3 = max(1, min(args.steps, 100))
+            for i in range(3):
+                mx.conv_fprop_tf32x3(d, d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets], ws3)
+            torch.cuda.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for i in range(n3):
+                mx.conv_fprop_tf32x3(d, d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets], ws3)
+            a1.record()
+            torch.cuda.synchronize()
+            if mx.last_device_status() == mx.OK:
+                ms3 = a0.elapsed_time(a1) / n3
+                also = {"kernel": "tf32x3", "value": whole_job_tflops(C, 1, ms3), "unit": UNIT,
+                        "ms_per_step": ms3, "steps": n3,
+                        "note": "three TF32 products, K summed in chunks: tested to the exact kernel's "
+                                "bar (1e-5 of the largest output)"}
+        except mx.MaxdnnError:
+            also = None                     # a shape the tensor-core kernels do not take
+
     ms_total, e2e_ms, e2e_ms_single = max_over_ranks([ms_total, e2e_ms, e2e_ms_single], "cuda", world)
     ms_step = ms_total / args.steps
     value = whole_job_tflops(C, world, ms_step)
@@ -487,6 +513,8 @@ def run_ours(args):
                 "achieved_hbm_gbs": nbytes / (ms_step * 1e-3) / 1e9,
             },
         }
+        if also is not None:
+            line["same_accuracy_on_tensor_cores"] = also
         if clocks.get("sm_mhz"):
             # the paper's clock-independent efficiency: C / (2*128*SMs*elapsed SM cycles)
             cycles = ms_step * 1e-3 * clocks["sm_mhz"] * 1e6
