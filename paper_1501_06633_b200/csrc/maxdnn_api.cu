@@ -14,6 +14,7 @@
 #include "umma_chunk_conv.cuh"
 #include "umma_pair_chunk_conv.cuh"
 #include "wgrad_umma_chunk.cuh"
+#include "wgrad_umma_pair_chunk.cuh"
 #include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
 #include "wgrad_umma_pair.cuh"
@@ -34,6 +35,7 @@ struct DeviceState {
   bool umma_chunk_attr = false;
   bool umma_pair_chunk_attr = false;
   bool wgrad_chunk_attr = false;
+  bool wgrad_pair_chunk_attr = false;
   bool wgrad_umma_attr[4] = {false, false, false, false};
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
@@ -1059,7 +1061,7 @@ maxdnn_status plan_wgrad_x3(const maxdnn_conv_desc* desc, int sm_count, WgradX3P
   p->dout_bytes = round256((size_t)desc->No * Ho * Wo * 2 * desc->Nb * 4);
   static thread_local WgradGeom scratch;
   WgradGeom* gg = g ? g : &scratch;
-  st = plan_wgrad(p->d3, 4, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), gg, -1);   // one-SM tiles
+  st = plan_wgrad(p->d3, 4, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), gg, env_int("MAXDNN_WGRAD_PAIR"));
   if (st != MAXDNN_OK) return st;
   const size_t kno = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No;
   p->partial_bytes = gg->splits > 1 ? (size_t)gg->splits * kno * 4 : 0;
@@ -1111,7 +1113,8 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
     const uint64_t nb2 = 2ull * desc->Nb;
     const uint64_t dims[4] = {nb2, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
     const uint64_t str[3] = {nb2 * 4, (uint64_t)g.Wi * nb2 * 4, (uint64_t)g.Hi * g.Wi * nb2 * 4};
-    const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)g.bc};
+    // (a pair's CTA stages half of the tile's channels)
+    const uint32_t box[4] = {32u, (uint32_t)g.bw, (uint32_t)g.bh, (uint32_t)(g.pair ? g.bc_h : g.bc)};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w_in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_128B);
     if (st != MAXDNN_OK) return st;
@@ -1124,16 +1127,44 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
   const int cs = env_or("MAXDNN_X3_CHUNK_ROWS", 768) / 32;
   args.chunk_steps = (uint32_t)(cs < 1 ? 1 : cs);
   args.x3_per_part = (uint32_t)(desc->Nb / 32);
-  args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) | ((128u >> 4) << 24);
-  if (!ds->wgrad_chunk_attr) {
-    if (cudaFuncSetAttribute(wgrad_umma_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024) != cudaSuccess) {
+  args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) |
+               (((g.pair ? 256u : 128u) >> 4) << 24);
+  if (g.pair) {
+    if (!ds->wgrad_pair_chunk_attr) {
+      if (cudaFuncSetAttribute(wgrad_umma_pair_chunk_kernel,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+        cudaGetLastError();
+        return MAXDNN_CUDA_ERROR;
+      }
+      ds->wgrad_pair_chunk_attr = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
+    cfg.blockDim = dim3(kWgChunkThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, wgrad_umma_pair_chunk_kernel, mg, mi, args) != cudaSuccess) {
       cudaGetLastError();
       return MAXDNN_CUDA_ERROR;
     }
-    ds->wgrad_chunk_attr = true;
+  } else {
+    if (!ds->wgrad_chunk_attr) {
+      if (cudaFuncSetAttribute(wgrad_umma_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               227 * 1024) != cudaSuccess) {
+        cudaGetLastError();
+        return MAXDNN_CUDA_ERROR;
+      }
+      ds->wgrad_chunk_attr = true;
+    }
+    wgrad_umma_chunk_kernel<<<g.grid, kWgChunkThreads, g.smem_bytes, stream>>>(mg, mi, args);
   }
-  wgrad_umma_chunk_kernel<<<g.grid, kWgChunkThreads, g.smem_bytes, stream>>>(mg, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (g.splits > 1) {

@@ -146,6 +146,7 @@ def test_bprop_data_tf32x3_full_size_sampled_and_refusals():
     assert e.value.status == mx.NOT_SUPPORTED
 
 
+@pytest.mark.parametrize("pair", [-1, 1])
 @pytest.mark.parametrize("splits", [0, 1, 3])
 @pytest.mark.parametrize("shape", [
     (64, 14, 9, 40, 96, 3, 1, 1, 1.0),        # 28 channels x 9 taps per tile, two channel blocks
@@ -155,10 +156,12 @@ def test_bprop_data_tf32x3_full_size_sampled_and_refusals():
     (64, 12, 10, 16, 132, 3, 2, 1, 1.0),      # filters not a multiple of 128, stride 2
     (96, 10, 6, 8, 256, 4, 1, 3, -1.0),       # two filter blocks; 96 images = three 128-byte rows
 ], ids=lambda s: "x".join(str(v) for v in s))
-def test_bprop_filter_tf32x3(shape, splits, monkeypatch):
+def test_bprop_filter_tf32x3(shape, splits, pair, monkeypatch):
     """Filter gradient in the three-product mode (the three products as one reduction over
     three times the images, accumulated in chunks) against the gradient oracle at the exact
-    kernel's bar; same-signed operands, forced split counts."""
+    kernel's bar; same-signed operands, forced split counts, one-SM (pair = -1) and two-SM
+    tiles (pair = 1, forced also where the planner would not take them)."""
+    monkeypatch.setenv("MAXDNN_WGRAD_PAIR", str(pair))
     if splits:
         monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
     Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
