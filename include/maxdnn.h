@@ -223,10 +223,12 @@ maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float
                                        const float* filt, float* out, void* workspace,
                                        size_t workspace_bytes, void* cuda_stream);
 /* The gradient with respect to the maps (the adjoint defined under "Backward propagation"
- * below) in the same three-product mode, stride 1 only: the FPROP of dout with the flipped,
- * transposed filter bank, run through the kernels of maxdnn_conv_fprop_tf32x3.  dout / filt /
- * din are the fp32 tensors; workspace and errors as there (NOT_SUPPORTED: stride > 1, pad >
- * Sk-1, or what the TF32 kernel refuses for the transposed problem, whose filter count is Nc). */
+ * below) in the same three-product mode: the FPROP of dout with the flipped, transposed
+ * filter bank (stride 1) or, class by class, with its sub-filter banks (stride > 1: the
+ * residue classes of maxdnn_conv_bprop_data, side by side on the library's streams), run
+ * through the kernels of maxdnn_conv_fprop_tf32x3.  dout / filt / din are the fp32 tensors;
+ * workspace and errors as there (NOT_SUPPORTED: stride 1 with pad > Sk-1, or what the TF32
+ * kernel refuses for the transposed problem, whose filter count is Nc). */
 maxdnn_status maxdnn_conv_bprop_data_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
 maxdnn_status maxdnn_conv_bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout,
                                             const float* filt, float* din, void* workspace,

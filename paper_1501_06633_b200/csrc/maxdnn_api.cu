@@ -523,7 +523,7 @@ maxdnn_status dgrad_plan_check(const ConvDims& fd, maxdnn_kernel_kind kind, int 
 // once) and, for the fp32 kernel, its dense result (together: one din), each rounded up
 // to 256 bytes.
 struct DgradStridedPlan {
-  size_t ft_bytes, sub_bytes;
+  size_t ft_bytes, sub_bytes, pre_bytes;
 };
 
 inline size_t dgrad_class_ft_bytes(const ConvDims& d, const DgradAxis& ah, const DgradAxis& aw,
@@ -538,31 +538,37 @@ inline bool dgrad_class_live(const DgradAxis& ah, const DgradAxis& aw, int Ho, i
   return ah.J > 0 && aw.J > 0 && ah.n > 0 && aw.n > 0 && ah.crop < Ho && aw.crop < Wo;
 }
 
-maxdnn_status plan_dgrad_strided(const ConvDims& d, maxdnn_kernel_kind kind, DgradStridedPlan* p) {
+// x3 (three-product TF32 mode, kind = TF32): the gradient is split once into [hi; hi; lo]
+// along its channels (pre_bytes, ahead of everything else in the workspace) and every class's
+// bank is followed by its split [hi; lo; hi] (four times the bank in all).
+maxdnn_status plan_dgrad_strided(const ConvDims& d, maxdnn_kernel_kind kind, DgradStridedPlan* p,
+                                 bool x3 = false) {
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   p->ft_bytes = p->sub_bytes = 0;
+  p->pre_bytes = x3 ? round256((size_t)3 * d.No * Ho * Wo * d.Nb * 4) : 0;
   for (int rh = 0; rh < d.stride_h; ++rh)
     for (int rw = 0; rw < d.stride_w; ++rw) {
       const DgradAxis ah = dgrad_axis(rh, d.Skh, d.stride_h, d.pad_h, d.Hi);
       const DgradAxis aw = dgrad_axis(rw, d.Skw, d.stride_w, d.pad_w, d.Wi);
       if (!dgrad_class_live(ah, aw, Ho, Wo)) continue;
-      p->ft_bytes += dgrad_class_ft_bytes(d, ah, aw, eb);
+      p->ft_bytes += dgrad_class_ft_bytes(d, ah, aw, eb) * (x3 ? 4 : 1);
       if (kind == MAXDNN_KERNEL_FP32) p->sub_bytes += dgrad_class_sub_bytes(d, ah, aw);
     }
   return MAXDNN_OK;
 }
 
+
 maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, const void* dout,
                                  const void* filt, float* din, void* ws, size_t ws_bytes,
-                                 cudaStream_t stream) {
+                                 cudaStream_t stream, bool x3 = false) {
   const size_t eb = kind == MAXDNN_KERNEL_BF16 ? 2 : 4;
   DgradStridedPlan p;
-  maxdnn_status st = plan_dgrad_strided(d, kind, &p);
+  maxdnn_status st = plan_dgrad_strided(d, kind, &p, x3);
   if (st != MAXDNN_OK) return st;
-  if (ws_bytes < p.ft_bytes + p.sub_bytes) return MAXDNN_INVALID_VALUE;
+  if (ws_bytes < p.pre_bytes + p.ft_bytes + p.sub_bytes) return MAXDNN_INVALID_VALUE;
   if (d.Nb % 4 != 0) return MAXDNN_NOT_SUPPORTED;
   DeviceState* ds = nullptr;
   st = device_state(&ds);
@@ -571,8 +577,17 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
   int32_t Ho, Wo;
   check_dims(d, &Ho, &Wo);
   const int sh = d.stride_h, sw = d.stride_w;
-  uint8_t* ft_next = static_cast<uint8_t*>(ws);
+  uint8_t* ft_next = static_cast<uint8_t*>(ws) + p.pre_bytes;
   uint8_t* sub_next = ft_next + p.ft_bytes;
+  if (x3) {
+    // the gradient as [hi; hi; lo] along its channels, once, ahead of the fork
+    const size_t n4 = (size_t)d.No * Ho * Wo * d.Nb / 4;
+    tf32_split3_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, stream>>>(
+        static_cast<const float4*>(dout), static_cast<float4*>(ws), n4, 0x4u);
+    if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    dout = ws;
+  }
   // Positions that no tap reaches (a class without taps, or whose window lies outside
   // dout) must read zero: clear din first if there is such a class.
   bool all_covered = true;
@@ -605,7 +620,7 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
       const DgradAxis aw = dgrad_axis(rw, d.Skw, sw, d.pad_w, d.Wi);
       if (!dgrad_class_live(ah, aw, Ho, Wo)) continue;
       uint8_t* w_ft = ft_next;
-      ft_next += dgrad_class_ft_bytes(d, ah, aw, eb);
+      ft_next += dgrad_class_ft_bytes(d, ah, aw, eb) * (x3 ? 4 : 1);
       float* w_sub = reinterpret_cast<float*>(sub_next);
       if (!direct) sub_next += dgrad_class_sub_bytes(d, ah, aw);
       const int lane = class_index++ % 4;
@@ -645,6 +660,19 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
         fd.out_y_stride = (int64_t)sh * d.Wi * d.Nb;
         fd.out_o_stride = (int64_t)d.Hi * d.Wi * d.Nb;
         float* dst = din + ((size_t)ah.first * d.Wi + aw.first) * d.Nb;
+        if (x3) {
+          // the class's bank as [hi; lo; hi] along its channels (the gradient's filters),
+          // then the chunked TF32 kernels on the problem with 3 No channels
+          const size_t n4 = (size_t)d.No * ah.J * aw.J * d.Nc / 4;
+          float* w_ft3 = reinterpret_cast<float*>(w_ft + dgrad_class_ft_bytes(d, ah, aw, eb));
+          tf32_split3_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(
+              reinterpret_cast<const float4*>(w_ft), reinterpret_cast<float4*>(w_ft3), n4, 0x2u);
+          if (cudaGetLastError() != cudaSuccess) { result = MAXDNN_CUDA_ERROR; break; }
+          g_launches.fetch_add(1, std::memory_order_relaxed);
+          fd.Nc = 3 * d.No;
+          result = fprop_umma(fd, 4, src, w_ft3, dst, cs, env_or("MAXDNN_X3_CHUNK_ROWS", 768));
+          continue;
+        }
         result = fprop_umma(fd, (int)eb, src, w_ft, dst, cs);
         continue;
       }
@@ -1013,6 +1041,17 @@ maxdnn_status dgrad_tf32x3_desc(const maxdnn_conv_desc* desc, maxdnn_conv_desc* 
 
 maxdnn_status bprop_data_tf32x3(const maxdnn_conv_desc* desc, const float* dout, const float* filt,
                                 float* din, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  if (!desc) return MAXDNN_INVALID_VALUE;
+  if (desc->stride > 1) {
+    // the residue classes of maxdnn_conv_bprop_data, each through the chunked kernels
+    maxdnn_status st0 = check_desc(desc, nullptr, nullptr);
+    if (st0 != MAXDNN_OK) return st0;
+    if (!dout || !filt || !din || !ws) return MAXDNN_INVALID_VALUE;
+    if (!aligned16(dout) || !aligned16(filt) || !aligned16(din) || !aligned16(ws))
+      return MAXDNN_INVALID_VALUE;
+    return bprop_data_strided(dims_from(*desc), MAXDNN_KERNEL_TF32, dout, filt, din, ws, ws_bytes,
+                              stream, true);
+  }
   maxdnn_conv_desc t;
   size_t ft_bytes = 0, a = 0, b = 0;
   maxdnn_status st = dgrad_tf32x3_desc(desc, &t, &ft_bytes);
@@ -1446,7 +1485,16 @@ maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float
 }
 
 maxdnn_status maxdnn_conv_bprop_data_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
-  if (!bytes) return MAXDNN_INVALID_VALUE;
+  if (!bytes || !desc) return MAXDNN_INVALID_VALUE;
+  if (desc->stride > 1) {
+    maxdnn_status st0 = check_desc(desc, nullptr, nullptr);
+    if (st0 != MAXDNN_OK) return st0;
+    DgradStridedPlan p;
+    st0 = plan_dgrad_strided(dims_from(*desc), MAXDNN_KERNEL_TF32, &p, true);
+    if (st0 != MAXDNN_OK) return st0;
+    *bytes = p.pre_bytes + p.ft_bytes + p.sub_bytes;
+    return MAXDNN_OK;
+  }
   maxdnn_conv_desc t;
   size_t ft_bytes = 0, a = 0, b = 0;
   maxdnn_status st = dgrad_tf32x3_desc(desc, &t, &ft_bytes);

@@ -141,9 +141,35 @@ def test_bprop_data_tf32x3_full_size_sampled_and_refusals():
                                          alpha=w.alpha)[0] for p in pts]
     scale = max(abs(v) for v in vals)
     assert max(abs(float(got[p]) - v) for p, v in zip(pts, vals)) <= TOL_X3 * scale
-    with pytest.raises(mx.MaxdnnError) as e:        # stride 2: not in this mode
-        mx.conv_bprop_data_tf32x3_workspace(mx.ConvDesc.make(64, 56, 56, 128, 256, 3, 2, 1, 1.0))
+    with pytest.raises(mx.MaxdnnError) as e:        # pad > Sk - 1 at stride 1: no transposed FPROP
+        mx.conv_bprop_data_tf32x3_workspace(mx.ConvDesc.make(64, 16, 16, 32, 32, 3, 1, 3, 1.0))
     assert e.value.status == mx.NOT_SUPPORTED
+
+
+@pytest.mark.parametrize("shape", [
+    (64, 15, 11, 32, 64, 3, 2, 1, 1.0),       # classes with 2x2, 2x1, 1x2, 1x1 taps
+    (64, 16, 12, 32, 32, 2, 2, 0, 0.5),       # filter = stride: one tap per class
+    (64, 23, 19, 32, 64, 7, 4, 3, 1.0),       # stride 4: sixteen classes
+    (64, 14, 14, 32, 32, 2, 3, 0, 1.0),       # stride > filter: a class without taps stays zero
+    (32, 13, 10, 64, 96, 3, 2, 2, -1.0),      # pad = Sk - 1: a class whose window skips a row of dout
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_bprop_data_tf32x3_strided(shape):
+    """Stride > 1: every residue class through the chunked kernels (the gradient split once,
+    each class's sub-filter bank split after its transform), at the exact kernel's bar."""
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    w = wl.Workload("x3s", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
+                    ("uniform", 0.0, 1.0), 4800 + Sk)
+    _, filt = wl.make_inputs(w)
+    dout = np.abs(wl.make_dout(w))
+    d = mx.ConvDesc.make(*w.dims)
+    ws = torch.empty(mx.conv_bprop_data_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
+    mx.conv_bprop_data_tf32x3(d, torch.from_numpy(dout).cuda(), torch.from_numpy(filt).cuda(), din, ws)
+    assert mx.last_device_status() == mx.OK
+    ref = oracle.conv_bprop_data(dout, filt, (Hi, Wi), stride=stride, pad=pad, alpha=alpha)
+    got = din.cpu().numpy().reshape(ref.shape)
+    assert np.isfinite(got).all()
+    assert float(np.max(np.abs(got.astype(np.float64) - ref))) / float(np.max(np.abs(ref))) <= TOL_X3
 
 
 @pytest.mark.parametrize("pair", [-1, 1])
