@@ -202,6 +202,7 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   MAXDNN_FFMA_CASE(128, 128, 8, 8, 6)
   MAXDNN_FFMA_CASE(96, 128, 6, 8, 8)
   MAXDNN_FFMA_CASE(64, 128, 4, 8, 10)
+  MAXDNN_FFMA_CASE(64, 256, 4, 16, 14)
   MAXDNN_FFMA_CASE(32, 128, 2, 8, 12)
 #undef MAXDNN_FFMA_CASE
   return MAXDNN_NOT_SUPPORTED;
