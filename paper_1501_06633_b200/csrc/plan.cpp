@@ -92,7 +92,7 @@ static void fill_geom(const ConvDims& d, int32_t Ho, int32_t Wo, ConvGeom* g) {
 struct FfmaShape { int m, cols; double cost; };
 static const FfmaShape kFfmaShapes[] = {
     {128, 256, 0.97}, {256, 128, 0.99}, {128, 128, 1.00}, {96, 128, 1.10},
-    {96, 256, 1.12},  {64, 128, 1.18},  {64, 256, 1.11},  {32, 128, 1.50},
+    {96, 256, 1.12},  {64, 128, 1.18},  {64, 256, 1.05},  {32, 128, 1.50},
 };
 
 static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* n) {
