@@ -479,8 +479,12 @@ maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int for
       const int units = pair ? sm_count / 2 : sm_count;
       const double cost = (double)ceil_div(gc.n_tiles, units) * (gc.tile_px * gc.tile_n + 128) *
                           (pair ? 0.9 : 1.0);
-      // a narrower tile must promise at least 5 % (its steps carry fewer MMAs)
-      if (!have || cost < (ci == 0 ? best - 1e-9 : 0.95 * best)) {
+      // a narrower tile must promise at least 5 % where its K steps are short (measured:
+      // 27 x 27, 64 channels, tf32, four MMAs per step: 192-column pair tiles 9 % slower
+      // than the model's 2.8 % gain), 1 % where they are long (96 channels, 15 MMAs: 4 % faster)
+      const int mmas = gc.kwc * (gc.kc / (32 / elem_bytes));
+      const double bar = mmas >= 12 ? 0.99 : 0.95;
+      if (!have || cost < (ci == 0 ? best - 1e-9 : bar * best)) {
         best = cost;
         have = true;
         *g = gc;
