@@ -109,3 +109,47 @@ def test_strided_map_gradient_forks_and_joins(kernel):
     assert mx.last_device_status() == mx.OK
     got = total.cpu().numpy().reshape(ref.shape)
     assert float(np.max(np.abs(got - ref))) <= tol * scale
+
+
+def test_strided_map_gradient_from_two_host_threads():
+    """Two host threads, each with its own stream and buffers, call the strided map gradient
+    (which borrows the library's side streams and events) at the same time: the fork / join
+    sequences must not mix."""
+    import threading
+    shapes = [(64, 15, 11, 32, 64, 3, 2, 1, 1.0), (64, 23, 19, 32, 64, 7, 4, 3, 1.0)]
+    cases = []
+    for i, s in enumerate(shapes):
+        w = wl.Workload("mt", *s, ("uniform", -1.0, 1.0), ("uniform", -1.0, 1.0), 5100 + i)
+        _, filt = wl.make_inputs(w)
+        dout = wl.make_dout(w)
+        d = mx.ConvDesc.make(*w.dims)
+        ref = oracle.conv_bprop_data(dout, filt, (w.Hi, w.Wi), stride=w.stride, pad=w.pad, alpha=w.alpha)
+        cases.append((d, torch.from_numpy(dout).cuda(), torch.from_numpy(filt).cuda(), ref,
+                      torch.empty(mx.conv_bprop_data_workspace(d), dtype=torch.uint8, device="cuda"),
+                      torch.empty(mx.conv_in_elems(d), device="cuda")))
+    for c in cases:                                      # one-time set-up on this thread
+        mx.conv_bprop_data(c[0], c[1], c[2], c[5], c[4])
+    torch.cuda.synchronize()
+    errs = []
+
+    def worker(tid):
+        torch.cuda.set_device(0)
+        st = torch.cuda.Stream()
+        d, g, f, ref, ws, din = cases[tid]
+        for it in range(40):
+            with torch.cuda.stream(st):
+                din.fill_(float("nan"))
+                mx.conv_bprop_data(d, g, f, din, ws, stream=st)
+                got = din.cpu().numpy().reshape(ref.shape)
+            e = float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref)))
+            if not e <= 1e-5:
+                errs.append((tid, it, e))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errs, errs[:3]
+    assert mx.last_device_status() == mx.OK
