@@ -8,7 +8,11 @@
 One step = one FPROP convolution of the named workload (patch gather, inner
 product, alpha scaling and store — one kernel launch) on synthetic seeded
 inputs.  Prints ONE JSON line on rank 0.  Throughput is the paper's FLOP count
-C = 2 Nb Wo Ho (Nc Sk^2 + 1) No (Section 2) divided by time.
+C = 2 Nb Wo Ho (Nc Sk^2 + 1) No (Section 2) divided by time.  The default is the
+largest single-GPU layer (large3x3) through the exact fp32 kernel (the paper's
+arithmetic); the same line carries, under "tensor_cores", the TF32 and BF16
+tensor-core kernels on the same layer, each with its own time, clocks and
+roofline.
 """
 from __future__ import annotations
 
@@ -51,12 +55,16 @@ def parse_args():
     p.add_argument("--steps", type=int, default=300)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="first11x11s4", choices=wl.ORDER + wl.TABLE1_ORDER)
+    p.add_argument("--workload", default="large3x3", choices=wl.ORDER + wl.TABLE1_ORDER)
     p.add_argument("--kernel", default="fp32", choices=["fp32", "tf32", "bf16", "tf32x3"])
     p.add_argument("--op", default="fprop", choices=["fprop", "dgrad", "wgrad"],
                    help="fprop (the headline path) or one of its two adjoints (BPROP)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-tensor", action="store_true",
+                   help="skip the tensor-core kernels timed beside the fp32 headline")
+    p.add_argument("--min-seconds", type=float, default=0.6,
+                   help="length of the extra 'sustained' region behind the clock record")
     p.add_argument("--cpu-seconds", type=float, default=12.0,
                    help="target wall time of the CPU-baseline sample")
     return p.parse_args()
@@ -112,6 +120,22 @@ def oracle_sample(w, target_seconds):
     dt = time.perf_counter() - t0
     fl = flops(w, rows, Wo) * repeats
     return fl / dt / 1e12, dt, rows, Ho, repeats, oracle.num_threads()
+
+
+def oracle_single_thread_tiny():
+    """The oracle on ONE thread on the small config: the per-core rate behind `cores`."""
+    import oracle
+    w = wl.WORKLOADS["tiny3x3"]
+    inp, filt = wl.make_inputs(w)
+    Ho = (w.Hi + 2 * w.pad - w.Sk) // w.stride + 1
+    oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, nthreads=1)
+    reps, t0 = 0, time.perf_counter()
+    while reps < 3 or time.perf_counter() - t0 < 0.5:
+        oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha, nthreads=1)
+        reps += 1
+    dt = time.perf_counter() - t0
+    return {"value": flops(w, Ho, Ho) * reps / dt / 1e12, "unit": UNIT, "cores": 1,
+            "sample": "tiny3x3 whole x %d passes" % reps}
 
 
 def oracle_sample_bprop(w, op, target_seconds):
@@ -280,6 +304,206 @@ def whole_job_tflops(flops_per_rank, world, ms_step):
 # ----------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------
+def measure_tf32_peak():
+    """Dense TF32 throughput of the library GEMM on this GPU (the roofline's denominator for
+    the TF32 kernel): torch.matmul 8192^3 with TF32 enabled, best of 10, CUDA events."""
+    import torch
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        n = 8192
+        a = torch.randn(n, n, device="cuda")
+        b = torch.randn(n, n, device="cuda")
+        c = torch.empty(n, n, device="cuda")
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        best = None
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch.matmul(a, b, out=c)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+
+
+def peak_for(kernel, peaks, peaks_kind, sm_count, tf32_measured=None):
+    """(peak TFLOP/s, bound, where the number comes from) of one kernel kind."""
+    sm_max = float(peaks.get("sm_max_mhz") or 1965.0)
+    if kernel == "fp32":
+        # FP32 CUDA-core peak, Section 3.3's form: 2 FLOPs x 128 cores x SMs x clock
+        return (2.0 * 128 * sm_count * sm_max * 1e6 / 1e12, "alu",
+                "2*128*%d SMs*%.0f MHz (max SM clock, %s)" % (sm_count, sm_max, peaks_kind))
+    bf16 = float(peaks["bf16_tflops"])
+    if kernel == "bf16":
+        return bf16, "tensor", "cuBLAS bf16 burst (%s)" % peaks_kind
+    half = 0.5 * bf16
+    if tf32_measured is None:
+        peak, note = half, "half of cuBLAS bf16 burst (%s) = %.0f; tf32 GEMM not measured" % (peaks_kind, half)
+    else:
+        peak = max(half, tf32_measured)
+        note = ("larger of: torch.matmul 8192^3 tf32 best of 10, measured in this run = %.0f; half of "
+                "cuBLAS bf16 burst (%s) = %.0f" % (tf32_measured, peaks_kind, half))
+    if kernel == "tf32x3":
+        return peak / 3.0, "tensor", note + "; / 3 (three TF32 products per product counted)"
+    return peak, "tensor", note
+
+
+class Arm:
+    """One kernel kind on one workload and operation: device buffers (rotated so that no step
+    finds its operands in L2) and the call that runs one step."""
+
+    def __init__(self, mx, w, kernel, op, rank, world):
+        import torch
+        self.torch, self.mx, self.w, self.kernel, self.op, self.world = torch, mx, w, kernel, op, world
+        x3 = kernel == "tf32x3"            # three TF32 products: fp32 buffers, its own entry points
+        kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16,
+                "tf32x3": mx.KERNEL_TF32}[kernel]
+        self.kind, self.x3 = kind, x3
+        d = self.d = mx.ConvDesc.make(*w.dims)
+        self.nbytes, self.Ho, self.Wo = workload_bytes(w, kernel, op)
+        self.C = mx.conv_flops(d)          # the same bilinear form: all three operations cost C
+        assert self.C == flops(w, self.Ho, self.Wo)
+        # Each rank holds its own batch shard (same recipe, its own seed); neither FPROP nor
+        # the map gradient needs an exchange between shards; the filter gradient of a sharded
+        # batch is summed over ranks (all-reduce, inside the timed step).
+        inp, filt = shard_inputs(w, rank)
+        dout = wl.make_dout(w, seed_offset=rank) if op != "fprop" else None
+        n_sets = self.n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / self.nbytes)))
+        if kernel == "bf16":
+            to_host = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).reshape(-1)
+            as_op = lambda t: t.view(torch.bfloat16)
+        else:
+            to_host = lambda a: torch.from_numpy(a).reshape(-1)
+            as_op = lambda t: t
+        # operands: (big streamed operand, second operand); result: fp32
+        if op == "fprop":
+            h_a, h_b, n_res = to_host(inp), to_host(filt), mx.conv_out_elems(d)
+        elif op == "dgrad":
+            h_a, h_b, n_res = to_host(dout), to_host(filt), mx.conv_in_elems(d)
+        else:
+            h_a, h_b, n_res = to_host(inp), to_host(dout), mx.conv_filt_elems(d)
+        self.h_a, self.h_b, self.n_res = h_a.pin_memory(), h_b.pin_memory(), n_res
+        self.d_as = [self.h_a.cuda() for _ in range(n_sets)]
+        self.d_bs = [self.h_b.cuda() for _ in range(n_sets if op == "wgrad" else 2)]
+        self.d_res = [torch.empty(n_res, dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+        ws = None
+        if op == "dgrad":
+            ws = torch.empty(mx.conv_bprop_data_workspace(d, kind), dtype=torch.uint8, device="cuda")
+        elif op == "wgrad":
+            ws = torch.empty(max(16, mx.conv_bprop_filter_workspace(d, kind)), dtype=torch.uint8,
+                             device="cuda")
+        fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
+                 mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
+        # one call of the operation: run(a, b, r, workspace, stream)
+        if x3:
+            size_fn, call_fn = {
+                "fprop": (mx.conv_fprop_tf32x3_workspace, mx.conv_fprop_tf32x3),
+                "dgrad": (mx.conv_bprop_data_tf32x3_workspace, mx.conv_bprop_data_tf32x3),
+                "wgrad": (mx.conv_bprop_filter_tf32x3_workspace, mx.conv_bprop_filter_tf32x3)}[op]
+            ws = torch.empty(max(16, size_fn(d)), dtype=torch.uint8, device="cuda")
+            self.run = lambda a, b, r, wsp, stream=None: call_fn(d, a, b, r, wsp, stream=stream)
+        elif op == "fprop":
+            self.run = lambda a, b, r, wsp, stream=None: fprop(d, as_op(a), as_op(b), r, stream=stream)
+        elif op == "dgrad":
+            self.run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_data(
+                d, as_op(a), as_op(b), r, wsp, kind, stream=stream)
+        else:
+            self.run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_filter(
+                d, as_op(a), as_op(b), r, wsp, kind, stream=stream)
+        self.ws = ws
+
+    def step(self, i):
+        a, b, r = self.d_as[i % self.n_sets], self.d_bs[i % len(self.d_bs)], self.d_res[i % self.n_sets]
+        self.run(a, b, r, self.ws)
+        if self.op == "wgrad":
+            sum_gradient_over_ranks(r, self.world)      # NCCL all-reduce over the batch shards
+
+    def barrier(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def timed(self, steps, warmup, local_rank):
+        """W warm-up steps, then EXACTLY `steps` steps between two events, a barrier and a
+        synchronize on both sides.  Returns (ms of the region, clock record, launches)."""
+        torch, mx = self.torch, self.mx
+        for i in range(max(3, warmup)):
+            self.step(i)
+        self.barrier()
+        sampler = ClockSampler(local_rank)
+        launches0 = mx.launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.start()
+        self.barrier()
+        ev0.record()
+        for i in range(steps):
+            self.step(i)
+        ev1.record()
+        self.barrier()
+        clocks = sampler.stop()
+        launches = mx.launch_count() - launches0
+        if mx.last_device_status() != mx.OK:
+            raise SystemExit("a kernel reported a timed-out wait; results are not valid")
+        return ev0.elapsed_time(ev1), clocks, launches
+
+    def per_launch(self, n):
+        """Events around each of `n` steps: (median ms, best ms)."""
+        torch = self.torch
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(n)]
+        self.barrier()
+        for i, (e0, e1) in enumerate(evs):
+            e0.record()
+            self.step(i)
+            e1.record()
+        self.barrier()
+        ms = sorted(e0.elapsed_time(e1) for e0, e1 in evs)
+        return float(np.median(ms)), float(ms[0])
+
+    def sustained(self, steps, seconds, local_rank):
+        """The timed loop repeated until at least `seconds` have passed: a region long enough
+        for the clock record (NVML samples every 2 ms) to mean something."""
+        torch = self.torch
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        self.barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        done = 0
+        ev0.record()
+        while True:
+            for i in range(steps):
+                self.step(i)
+            done += steps
+            torch.cuda.current_stream().synchronize()
+            if time.perf_counter() - t0 >= seconds or done >= 200000:
+                break
+        ev1.record()
+        self.barrier()
+        clocks = sampler.stop()
+        return ev0.elapsed_time(ev1) / done, done, clocks
+
+
+def roofline_of(arm, ms_step, peak, bound, peak_note, peaks):
+    per_gpu = arm.C / (ms_step * 1e-3) / 1e12
+    t_compute = arm.C / (peak * 1e12)
+    t_hbm = arm.nbytes / (float(peaks["hbm_gbs"]) * 1e9)
+    return {
+        "bound": bound, "achieved": per_gpu, "peak": peak, "unit": "TFLOP/s", "frac": per_gpu / peak,
+        "traffic": NCU_TRAFFIC_BYTES.get((arm.w.name, arm.kernel)) if arm.op == "fprop" else None,
+        "peak_source": peak_note,
+        "roofline_time_us": max(t_compute, t_hbm) * 1e6,
+        "frac_of_roofline_time": max(t_compute, t_hbm) / (ms_step * 1e-3),
+        "achieved_hbm_gbs": arm.nbytes / (ms_step * 1e-3) / 1e9,
+    }
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -295,95 +519,34 @@ def run_ours(args):
 
     peaks, peaks_kind = load_peaks()
     w = wl.ALL[args.workload]
-    x3 = args.kernel == "tf32x3"            # three TF32 products: fp32 buffers, its own entry points
-    kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16,
-            "tf32x3": mx.KERNEL_TF32}[args.kernel]
-    d = mx.ConvDesc.make(*w.dims)
     op = args.op
-    nbytes, Ho, Wo = workload_bytes(w, args.kernel, op)
-    C = mx.conv_flops(d)          # the same bilinear form: all three operations cost C
-    assert C == flops(w, Ho, Wo)
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    arm = Arm(mx, w, args.kernel, op, rank, world)
+    d, C, n_sets, nbytes = arm.d, arm.C, arm.n_sets, arm.nbytes
+    x3, kind = arm.x3, arm.kind
 
-    # Each rank holds its own batch shard (same recipe, its own seed); neither FPROP nor
-    # the map gradient needs an exchange between shards; the filter gradient of a sharded
-    # batch is summed over ranks (all-reduce, inside the timed step).  Buffer
-    # sets are rotated so that no step finds its operands in L2.
-    inp, filt = shard_inputs(w, rank)
-    dout = wl.make_dout(w, seed_offset=rank) if op != "fprop" else None
-    n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / nbytes)))
-    bf16 = args.kernel == "bf16"
-    if bf16:
-        to_host = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).reshape(-1)
-        as_op = lambda t: t.view(torch.bfloat16)
-    else:
-        to_host = lambda a: torch.from_numpy(a).reshape(-1)
-        as_op = lambda t: t
-    # operands: (big streamed operand, second operand); result: fp32
-    if op == "fprop":
-        h_a, h_b, n_res = to_host(inp), to_host(filt), mx.conv_out_elems(d)
-    elif op == "dgrad":
-        h_a, h_b, n_res = to_host(dout), to_host(filt), mx.conv_in_elems(d)
-    else:
-        h_a, h_b, n_res = to_host(inp), to_host(dout), mx.conv_filt_elems(d)
-    h_a, h_b = h_a.pin_memory(), h_b.pin_memory()
-    d_as = [h_a.cuda() for _ in range(n_sets)]
-    d_bs = [h_b.cuda() for _ in range(n_sets if op == "wgrad" else 2)]
-    d_res = [torch.empty(n_res, dtype=torch.float32, device="cuda") for _ in range(n_sets)]
-    ws = None
-    if op == "dgrad":
-        ws = torch.empty(mx.conv_bprop_data_workspace(d, kind), dtype=torch.uint8, device="cuda")
-    elif op == "wgrad":
-        ws = torch.empty(max(16, mx.conv_bprop_filter_workspace(d, kind)), dtype=torch.uint8,
-                         device="cuda")
-    fprop = {mx.KERNEL_FP32: mx.conv_fprop, mx.KERNEL_TF32: mx.conv_fprop_tf32,
-             mx.KERNEL_BF16: mx.conv_fprop_bf16}[kind]
-    # one call of the operation: run(a, b, r, workspace, stream)
-    if x3:
-        size_fn, call_fn = {
-            "fprop": (mx.conv_fprop_tf32x3_workspace, mx.conv_fprop_tf32x3),
-            "dgrad": (mx.conv_bprop_data_tf32x3_workspace, mx.conv_bprop_data_tf32x3),
-            "wgrad": (mx.conv_bprop_filter_tf32x3_workspace, mx.conv_bprop_filter_tf32x3)}[op]
-        ws = torch.empty(max(16, size_fn(d)), dtype=torch.uint8, device="cuda")
-        run = lambda a, b, r, wsp, stream=None: call_fn(d, a, b, r, wsp, stream=stream)
-    elif op == "fprop":
-        run = lambda a, b, r, wsp, stream=None: fprop(d, as_op(a), as_op(b), r, stream=stream)
-    elif op == "dgrad":
-        run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_data(d, as_op(a), as_op(b), r, wsp, kind,
-                                                                   stream=stream)
-    else:
-        run = lambda a, b, r, wsp, stream=None: mx.conv_bprop_filter(d, as_op(a), as_op(b), r, wsp, kind,
-                                                                     stream=stream)
+    ms_total, clocks, launches = arm.timed(args.steps, args.warmup, local_rank)
 
-    def step(i):
-        a, b, r = d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets]
-        run(a, b, r, ws)
-        if op == "wgrad":
-            sum_gradient_over_ranks(r, world)      # NCCL all-reduce over the batch shards
+    # the same launches one by one (median / best beside the batch mean), then a region of
+    # at least --min-seconds for the clock record
+    pl_median, pl_best = arm.per_launch(max(3, min(args.steps, 50)))
+    sus_ms, sus_steps, sus_clocks = arm.sustained(max(1, args.steps), args.min_seconds, local_rank)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(max(3, args.warmup)):
-        step(i)
-    barrier()
-
-    sampler = ClockSampler(local_rank)
-    launches0 = mx.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.start()
-    barrier()
-    ev0.record()
-    for i in range(args.steps):
-        step(i)
-    ev1.record()
-    barrier()
-    clocks = sampler.stop()
-    launches = mx.launch_count() - launches0
-    ms_total = ev0.elapsed_time(ev1)
-    if mx.last_device_status() != mx.OK:
-        raise SystemExit("a kernel reported a timed-out wait; results are not valid")
+    # Section 3.3's efficiency counts processor clocks: elapsed SM cycles measured inside the
+    # kernel (maximum over its CTAs), fp32 FPROP only
+    kernel_clock = None
+    if args.kernel == "fp32" and op == "fprop":
+        mx.set_option("KERNEL_CLOCK", 1)
+        cyc = []
+        for i in range(5):
+            arm.step(i)
+            cyc.append(mx.last_kernel_clock())
+        mx.unset_option("KERNEL_CLOCK")
+        cyc.sort()
+        c_cycles, c_ns = cyc[len(cyc) // 2]
+        if c_cycles > 0 and c_ns > 0:
+            kernel_clock = {"sm_cycles": c_cycles, "ns": c_ns, "sm_mhz": c_cycles / c_ns * 1e3,
+                            "ce_cycles": C / (2.0 * 128 * sm_count * c_cycles)}
 
     # end to end from pinned host buffers: host -> device copies of both operands, the
     # kernel(s), device -> host copy of the result, every step.  FPROP goes through
@@ -392,8 +555,10 @@ def run_ours(args):
     # so that one step's result copy (device -> host) overlaps the next step's operand
     # copies (host -> device): the link is full duplex.  Every step still moves all its
     # bytes; the single-stream figure is reported beside it.
+    h_a, h_b, n_res = arm.h_a, arm.h_b, arm.n_res
+    d_as, d_bs, d_res, ws, run = arm.d_as, arm.d_bs, arm.d_res, arm.ws, arm.run
+    barrier = arm.barrier
     h_outs = [torch.empty(n_res, dtype=torch.float32).pin_memory() for _ in range(2)]
-    h_in, h_f, h_out = h_a, h_b, h_outs[0]
     streams = [torch.cuda.Stream(), torch.cuda.Stream()]
 
     def e2e_step(k, stream):
@@ -429,32 +594,43 @@ def run_ours(args):
 
     e2e_ms_single = time_e2e(1)
     e2e_ms = time_e2e(2)
+    if mx.last_device_status() != mx.OK:
+        raise SystemExit("a kernel reported a timed-out wait; results are not valid")
 
-    # Beside the default (exact fp32) line: the same workload through the three-product TF32
-    # entry point, which holds the exact kernel's accuracy bar on the tensor cores — reported
-    # as an extra object, outside every timed region above.
-    also = None
-    if world == 1 and args.kernel == "fp32" and op == "fprop":
-        try:
-            ws3 = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
-            n3 = max(1, min(args.steps, 100))
-            for i in range(3):
-                mx.conv_fprop_tf32x3(d, d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets], ws3)
-            torch.cuda.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record()
-            for i in range(n3):
-                mx.conv_fprop_tf32x3(d, d_as[i % n_sets], d_bs[i % len(d_bs)], d_res[i % n_sets], ws3)
-            a1.record()
-            torch.cuda.synchronize()
-            if mx.last_device_status() == mx.OK:
-                ms3 = a0.elapsed_time(a1) / n3
-                also = {"kernel": "tf32x3", "value": whole_job_tflops(C, 1, ms3), "unit": UNIT,
-                        "ms_per_step": ms3, "steps": n3,
-                        "note": "three TF32 products, K summed in chunks: tested to the exact kernel's "
-                                "bar (1e-5 of the largest output)"}
-        except mx.MaxdnnError:
-            also = None                     # a shape the tensor-core kernels do not take
+    # Beside the exact fp32 headline: the same workload on the tensor cores (TF32 and BF16
+    # operands, fp32 accumulate), each timed like the headline — W warm-ups, then the same
+    # number of steps between two events — with its own clock record and roofline.
+    tensor = None
+    tf32_measured = None
+    if world == 1 and op == "fprop" and args.kernel in ("fp32", "tf32", "tf32x3"):
+        tf32_measured = measure_tf32_peak()
+    if world == 1 and args.kernel == "fp32" and op == "fprop" and not args.no_tensor:
+        del arm.d_as, arm.d_bs, arm.d_res
+        d_as = d_bs = d_res = None
+        torch.cuda.empty_cache()
+        tensor = {}
+        for k in ("tf32", "bf16"):
+            try:
+                t_arm = Arm(mx, w, k, "fprop", rank, world)
+                t_ms, t_clocks, t_launches = t_arm.timed(args.steps, args.warmup, local_rank)
+                t_med, t_best = t_arm.per_launch(max(3, min(args.steps, 50)))
+                s_ms, s_steps, s_clocks = t_arm.sustained(max(1, args.steps), args.min_seconds, local_rank)
+            except mx.MaxdnnError as e:
+                tensor[k] = {"unavailable": str(e)}       # a shape this kernel does not take
+                continue
+            t_step = t_ms / args.steps
+            peak, bound, note = peak_for(k, peaks, peaks_kind, sm_count, tf32_measured)
+            tensor[k] = {
+                "value": whole_job_tflops(C, 1, t_step), "unit": UNIT, "ms_per_step": t_step,
+                "steps": args.steps, "warmup": max(3, args.warmup), "gpu_launches": int(t_launches),
+                "per_launch": {"median_ms": t_med, "best_ms": t_best},
+                "sustained": {"ms_per_step": s_ms, "steps": s_steps, "value": whole_job_tflops(C, 1, s_ms),
+                              "clocks": s_clocks},
+                "clocks": t_clocks,
+                "roofline": roofline_of(t_arm, t_step, peak, bound, note, peaks),
+            }
+            del t_arm
+            torch.cuda.empty_cache()
 
     ms_total, e2e_ms, e2e_ms_single = max_over_ranks([ms_total, e2e_ms, e2e_ms_single], "cuda", world)
     ms_step = ms_total / args.steps
@@ -462,25 +638,7 @@ def run_ours(args):
     e2e_value = whole_job_tflops(C, world, e2e_ms / e2e_steps)
 
     if rank == 0:
-        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
-        sm_max = float(peaks.get("sm_max_mhz") or clocks.get("sm_max_mhz") or 1965.0)
-        per_gpu = C / (ms_step * 1e-3) / 1e12
-        if args.kernel == "fp32":
-            # FP32 CUDA-core peak, Section 3.3's form: 2 FLOPs x 128 cores x SMs x clock
-            peak, bound = 2.0 * 128 * sm_count * sm_max * 1e6 / 1e12, "alu"
-            peak_note = "2*128*%d SMs*%.0f MHz (max SM clock, %s)" % (sm_count, sm_max, peaks_kind)
-        else:
-            bf16 = float(peaks["bf16_tflops"])
-            peak = bf16 if args.kernel == "bf16" else bf16 * (1.1 / 2.25)
-            if x3:
-                peak /= 3.0          # three TF32 products per product of the paper's count
-            bound = "tensor"
-            peak_note = ("cuBLAS bf16 burst (%s)" % peaks_kind) if args.kernel == "bf16" else \
-                ("cuBLAS bf16 burst (%s) x nominal tf32/bf16 ratio 1.1/2.25" % peaks_kind)
-            if x3:
-                peak_note += " / 3 (three TF32 products per product counted)"
-        t_compute = C / (peak * 1e12)
-        t_hbm = nbytes / (float(peaks["hbm_gbs"]) * 1e9)
+        peak, bound, peak_note = peak_for(args.kernel, peaks, peaks_kind, sm_count, tf32_measured)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
@@ -497,26 +655,29 @@ def run_ours(args):
                                 "batch shards, no collective"),
             },
             "clocks": clocks,
+            "per_launch": {"median_ms": pl_median, "best_ms": pl_best,
+                           "best_value": whole_job_tflops(C, world, pl_best)},
+            "sustained": {"ms_per_step": sus_ms, "steps": sus_steps,
+                          "value": whole_job_tflops(C, world, sus_ms), "clocks": sus_clocks,
+                          "note": "the timed loop repeated for at least %.1f s" % args.min_seconds},
             "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps, "streams": 2,
                     "value_single_stream": whole_job_tflops(C, world, e2e_ms_single / e2e_steps),
-                    "h2d_bytes_per_step": int(h_in.numel() * h_in.element_size()
-                                              + h_f.numel() * h_f.element_size()),
-                    "d2h_bytes_per_step": int(h_out.numel() * 4)},
+                    "h2d_bytes_per_step": int(h_a.numel() * h_a.element_size()
+                                              + h_b.numel() * h_b.element_size()),
+                    "d2h_bytes_per_step": int(n_res * 4)},
             "gpu_launches": int(launches),
-            "roofline": {
-                "bound": bound, "achieved": per_gpu, "peak": peak, "unit": "TFLOP/s",
-                "frac": per_gpu / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.kernel)) if op == "fprop" else None,
-                "peak_source": peak_note,
-                "roofline_time_us": max(t_compute, t_hbm) * 1e6,
-                "frac_of_roofline_time": max(t_compute, t_hbm) / (ms_step * 1e-3),
-                "achieved_hbm_gbs": nbytes / (ms_step * 1e-3) / 1e9,
-            },
+            "roofline": roofline_of(arm, ms_step, peak, bound, peak_note, peaks),
         }
-        if also is not None:
-            line["same_accuracy_on_tensor_cores"] = also
-        if clocks.get("sm_mhz"):
+        if (clocks.get("samples") or 0) < 50:
+            line["clocks"]["note"] = ("fewer than 50 clock samples in the %d-step region; see "
+                                      "sustained.clocks" % args.steps)
+        if tensor is not None:
+            line["tensor_cores"] = tensor
+        if kernel_clock is not None:
             # the paper's clock-independent efficiency: C / (2*128*SMs*elapsed SM cycles)
+            line["roofline"]["ce_cycles"] = kernel_clock["ce_cycles"]
+            line["roofline"]["kernel_clock"] = kernel_clock
+        if clocks.get("sm_mhz"):
             cycles = ms_step * 1e-3 * clocks["sm_mhz"] * 1e6
             line["roofline"]["ce_at_sampled_clock"] = C / (2.0 * 128 * sm_count * cycles)
         if world == 1 and not args.no_cpu_baseline and op != "fprop":
@@ -529,7 +690,8 @@ def run_ours(args):
             line["cpu_baseline"] = {
                 "value": tf, "unit": UNIT, "cores": threads, "kind": "oracle",
                 "sample": "%d of %d output rows of %s x %d passes, %.1f s" % (rows, Ho_, w.name,
-                                                                            reps, secs)}
+                                                                            reps, secs),
+                "single_thread_tiny3x3": oracle_single_thread_tiny()}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

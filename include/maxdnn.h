@@ -33,11 +33,16 @@
  *     Calls enqueue work and return; they never synchronise the stream.
  *   - Errors are return codes; nothing throws or aborts.  A call that returns
  *     an error other than MAXDNN_CUDA_ERROR has launched nothing.
- *   - The library keeps one small per-device status word (device memory,
+ *   - The library keeps one small per-device status block (device memory,
  *     allocated on the first fprop call on that device — make that first call
- *     outside any stream capture).  Kernels give every internal wait an
- *     iteration limit; a wait that runs out records a code there instead of
- *     hanging.  maxdnn_last_device_status() reads it.
+ *     outside any stream capture).  Kernels give every internal wait a time
+ *     limit; a wait that runs out records a code there instead of hanging and
+ *     the kernel ends normally with an invalid result.  The code is STICKY: it
+ *     stays until maxdnn_last_device_status() reads (and clears) it, whatever
+ *     is launched in between, so one query after a batch of calls tells whether
+ *     any of them gave up.  It does not disturb later launches: every launch
+ *     carries its own number, and only a give-up of the same launch makes its
+ *     other waits leave early.
  *   - There is no CPU fallback: without an sm_100 device the fprop calls fail
  *     with MAXDNN_NOT_SUPPORTED / MAXDNN_CUDA_ERROR.
  */
@@ -91,11 +96,11 @@ uint64_t maxdnn_conv_filt_elems(const maxdnn_conv_desc* desc);
 uint64_t maxdnn_conv_out_elems(const maxdnn_conv_desc* desc);
 
 /*
- * The address-generation stage (Section 3.2: pixel / channel offsets of the
- * patch are precomputed so that the three nested loops over channels, rows
- * and columns of a patch become one loop over a table).  Here one table entry
- * ("K step") names a box of patch rows that one TMA transfer stages into
- * shared memory, and the matching box of filter-matrix rows.
+ * The address-generation stage (Section 3.2's precomputed offset table: the
+ * walk over a patch is a single pass over table entries, with no index
+ * arithmetic left in the loop).  Here one table entry ("K step") names a box
+ * of patch rows that one TMA transfer stages into shared memory, and the
+ * matching box of filter-matrix rows.
  */
 typedef struct maxdnn_kstep {
   int16_t c0;   /* first channel of the box */
@@ -179,24 +184,31 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
  * library holds those 256 bytes until the process exits).
  *
  * Same arguments, layouts, result and NOT_SUPPORTED cases as maxdnn_conv_fprop
- * (the same kernel runs; the result is bitwise the same).  In addition:
+ * (the same plan and kernel — tile options included — so the result is bitwise
+ * the same).  In addition:
  *   - A problem whose kernel would need more than the 256 bytes of built-in
  *     scratch is refused with MAXDNN_NOT_SUPPORTED and nothing is launched.
- *     (The fp32 kernel needs 4 bytes for every descriptor it supports today.)
+ *     (The fp32 kernel needs 8 bytes for every descriptor it supports today;
+ *     plans that need a workspace in global memory are never chosen here.)
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and sets kernel
  *     attributes; make that first call before any stream capture begins.
- *   - All calls on a device share the one block, and each call clears the word
- *     it uses (a memset enqueued on `cuda_stream` ahead of the kernel).  Two
- *     calls whose work overlaps on the GPU — different streams, no ordering
- *     between them — therefore race on it; order them, or use
- *     maxdnn_conv_fprop for one of them.
- *   - A bounded wait that runs out still ends the kernel instead of hanging it,
- *     but this entry point has no way to hand that code back:
+ *   - All calls on a device share the one block, which keeps what earlier
+ *     calls left in it.  Nothing in it has to start at zero (a launch compares
+ *     the block with its own launch number), so no clearing is enqueued; but
+ *     two calls whose work overlaps on the GPU — different streams, no ordering
+ *     between them — race on it: if both give up a wait, only one code
+ *     survives, and one of them may take its full time limit to end.  Order
+ *     them, or use maxdnn_conv_fprop for one of them.
+ *   - A bounded wait that runs out ends the kernel instead of hanging it and
+ *     leaves its code in the built-in block:
+ *     maxdnn_last_device_status_noalloc() reads and clears it (a 4-byte copy to
+ *     the host and, after a failure, a 4-byte memset: no allocation either).
  *     maxdnn_last_device_status() reports on maxdnn_conv_fprop's block only.
  */
 maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const float* in,
                                         const float* filt, float* out, void* cuda_stream);
+maxdnn_status maxdnn_last_device_status_noalloc(void* cuda_stream);
 
 /*
  * FPROP with fp32-level accuracy on the tensor cores (three-product TF32): every fp32
@@ -215,8 +227,8 @@ maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const floa
  * paper has no counterpart (its kernel is an fp32 CUDA-core kernel).  Accuracy: the exact
  * kernel's class — measured 1e-6 .. 3e-6 of the largest output against the fp64 oracle for
  * K = 144 .. 9216 (exact fp32 kernel: 5e-7 .. 4e-6; plain TF32: 7e-4) — at about four
- * times the exact kernel's speed on 3x3 / 5x5 layers.  (MAXDNN_X3_CHUNK_ROWS=0 in the
- * environment selects the one-accumulator path: 2-3 % faster, error about 1e-8 K.)
+ * times the exact kernel's speed on 3x3 / 5x5 layers.  (Option X3_CHUNK_ROWS = 0 selects
+ * the one-accumulator path: 2-3 % faster, error about 1e-8 K.)
  */
 maxdnn_status maxdnn_conv_fprop_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes);
 maxdnn_status maxdnn_conv_fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in,
@@ -356,9 +368,45 @@ maxdnn_status maxdnn_conv_bprop_filter(const maxdnn_conv_desc* desc, maxdnn_kern
                                        void* cuda_stream);
 
 /* Synchronises `cuda_stream`, then reads and clears the current device's
- * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside a
- * kernel ran out; its output is not valid) or MAXDNN_CUDA_ERROR. */
+ * status word.  MAXDNN_OK, MAXDNN_DEVICE_TIMEOUT (a bounded wait inside some
+ * kernel launched since the last query ran out; that kernel's output is not
+ * valid) or MAXDNN_CUDA_ERROR. */
 maxdnn_status maxdnn_last_device_status(void* cuda_stream);
+
+/*
+ * Section 3.3 measures efficiency in processor clocks.  With option KERNEL_CLOCK set to 1,
+ * maxdnn_conv_fprop has every CTA of its kernel measure its own elapsed SM cycles
+ * (clock64) and nanoseconds (%globaltimer) from its first instruction to its last store,
+ * and keeps the maxima over the CTAs of the LATEST launch in the status block (a memset of
+ * those two words is enqueued ahead of the kernel).  This call synchronises `cuda_stream`
+ * and returns them: sm_cycles / nanoseconds is the SM clock the kernel ran at, and
+ * C / (2 * 128 * SMs * sm_cycles) the paper's clock-independent efficiency.  Both are 0 if
+ * the option was off.  32-bit counters: kernels of up to about two seconds.
+ */
+maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanoseconds,
+                                       void* cuda_stream);
+
+/*
+ * Tuning and test options (ablations and tests; none is needed in normal use; the
+ * paper has no counterpart).  An option is a named integer, "unset" by default.  `name`
+ * is one of FFMA_TILE_M, FFMA_COLS (pin the fp32 kernel's tile: filters 32/64/96/128/256,
+ * columns 128/256), FFMA_KH (filter rows per K step of few-channel layers), FFMA_STREAMK
+ * (0: never split tail tiles along K), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM
+ * tiles), UMMA_MERGE, UMMA_STAGE_KB, UMMA_COLS, WGRAD_SPLITS, WGRAD_PAIR, SM_COUNT (SM
+ * count for host-only workspace queries), X3_CHUNK_ROWS, DEBUG_STATUS, KERNEL_CLOCK (see
+ * maxdnn_last_kernel_clock), FFMA_LANES (0: 16-byte operand loads in the fp32 kernel), and
+ * TEST_MISSING_ARRIVAL (test hook: CTA 0's "full" barriers expect an arrival that
+ * never comes, so a bounded wait runs out).  The environment variable MAXDNN_<name>
+ * gives an option its initial value; the environment is read once, at the first use of
+ * any option in the process, never during a call.  TEST_MISSING_ARRIVAL has no
+ * environment variable: only maxdnn_set_option can switch it on.  Setting an option
+ * discards cached plans.  INVALID_VALUE for an unknown name.  Thread-safe; a call that is
+ * planning concurrently sees either the old or the new value.
+ */
+maxdnn_status maxdnn_set_option(const char* name, int32_t value);
+maxdnn_status maxdnn_unset_option(const char* name);
+maxdnn_status maxdnn_get_option(const char* name, int32_t* value, int32_t* is_set);
+void maxdnn_reset_options(void);   /* every option back to what the environment gave */
 
 /* How many kernels this library has launched in this process (all devices). */
 uint64_t maxdnn_launch_count(void);

@@ -15,7 +15,8 @@ __all__ = [
     "library_path", "load_library", "status_string", "conv_out_dims", "conv_flops",
     "conv_in_elems", "conv_filt_elems", "conv_out_elems", "conv_plan_query", "conv_fprop",
     "conv_fprop_tf32", "conv_fprop_bf16", "conv_fprop_host", "conv_fprop_noalloc",
-    "last_device_status",
+    "last_device_status", "last_device_status_noalloc",
+    "set_option", "unset_option", "get_option", "reset_options", "last_kernel_clock",
     "launch_count", "fprop_status", "EXPORTED_SYMBOLS",
     "conv_fprop_tf32x3_workspace", "conv_fprop_tf32x3",
     "conv_bprop_data_tf32x3_workspace", "conv_bprop_data_tf32x3",
@@ -45,6 +46,8 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv_bprop_filter_tf32x3_workspace", "maxdnn_conv_bprop_filter_tf32x3",
     "maxdnn_conv2_bprop_data_workspace", "maxdnn_conv2_bprop_data",
     "maxdnn_conv2_bprop_filter_workspace", "maxdnn_conv2_bprop_filter",
+    "maxdnn_last_device_status_noalloc", "maxdnn_set_option", "maxdnn_unset_option",
+    "maxdnn_get_option", "maxdnn_reset_options", "maxdnn_last_kernel_clock",
 ]
 
 
@@ -169,6 +172,18 @@ def load_library():
                                              ctypes.c_size_t, vp]
     lib.maxdnn_last_device_status.restype = ctypes.c_int
     lib.maxdnn_last_device_status.argtypes = [vp]
+    lib.maxdnn_last_device_status_noalloc.restype = ctypes.c_int
+    lib.maxdnn_last_device_status_noalloc.argtypes = [vp]
+    lib.maxdnn_set_option.restype = ctypes.c_int
+    lib.maxdnn_set_option.argtypes = [ctypes.c_char_p, ctypes.c_int32]
+    lib.maxdnn_unset_option.restype = ctypes.c_int
+    lib.maxdnn_unset_option.argtypes = [ctypes.c_char_p]
+    lib.maxdnn_get_option.restype = ctypes.c_int
+    lib.maxdnn_get_option.argtypes = [ctypes.c_char_p, P(ctypes.c_int32), P(ctypes.c_int32)]
+    lib.maxdnn_last_kernel_clock.restype = ctypes.c_int
+    lib.maxdnn_last_kernel_clock.argtypes = [P(ctypes.c_uint32), P(ctypes.c_uint32), vp]
+    lib.maxdnn_reset_options.restype = None
+    lib.maxdnn_reset_options.argtypes = []
     lib.maxdnn_launch_count.restype = ctypes.c_uint64
     lib.maxdnn_launch_count.argtypes = []
     _lib = lib
@@ -532,6 +547,44 @@ def conv_bprop_filter(desc: ConvDesc, inp, dout, dfilt, workspace, kind: int = K
 
 def last_device_status(stream=None) -> int:
     return int(load_library().maxdnn_last_device_status(_stream_ptr(stream)))
+
+
+def last_device_status_noalloc(stream=None) -> int:
+    return int(load_library().maxdnn_last_device_status_noalloc(_stream_ptr(stream)))
+
+
+def set_option(name: str, value: int) -> None:
+    st = load_library().maxdnn_set_option(name.encode(), int(value))
+    if st != OK:
+        raise MaxdnnError(st, "maxdnn_set_option(%s)" % name)
+
+
+def unset_option(name: str) -> None:
+    st = load_library().maxdnn_unset_option(name.encode())
+    if st != OK:
+        raise MaxdnnError(st, "maxdnn_unset_option(%s)" % name)
+
+
+def get_option(name: str):
+    """(value, is_set) of a tuning option."""
+    v, isset = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = load_library().maxdnn_get_option(name.encode(), ctypes.byref(v), ctypes.byref(isset))
+    if st != OK:
+        raise MaxdnnError(st, "maxdnn_get_option(%s)" % name)
+    return int(v.value), bool(isset.value)
+
+
+def last_kernel_clock(stream=None):
+    """(sm_cycles, nanoseconds) of the latest fp32 FPROP launch made with option KERNEL_CLOCK."""
+    c, ns = ctypes.c_uint32(0), ctypes.c_uint32(0)
+    st = load_library().maxdnn_last_kernel_clock(ctypes.byref(c), ctypes.byref(ns), _stream_ptr(stream))
+    if st != OK:
+        raise MaxdnnError(st, "maxdnn_last_kernel_clock")
+    return int(c.value), int(ns.value)
+
+
+def reset_options() -> None:
+    load_library().maxdnn_reset_options()
 
 
 def launch_count() -> int:

@@ -159,7 +159,7 @@ struct WgradArgs {
   WgradGeom g;
   float* dfilt;        // result when g.splits == 1
   float* partial;      // [splits][Nc Sk^2][No] otherwise
-  uint32_t* status;
+  WaitCtx wc;          // status block and this launch's epoch (see ptx_util.cuh)
 };
 
 // Which (tile, split, reduction step) comes next; the copy-issuing lane and the
@@ -239,7 +239,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   const uint32_t tx_bytes = (uint32_t)(g.box_o + g.rows) * 128u;
   auto produce = [&]() {
     if (!p_ok || pc.done(g)) return;
-    if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+    if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
       p_ok = false;
       return;
     }
@@ -295,7 +295,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
     for (int s = 0; s < n_steps; ++s) {
       if (issuer) produce();
       __syncwarp();
-      if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+      if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
         ok = false;
         break;
       }

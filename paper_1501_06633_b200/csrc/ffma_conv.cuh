@@ -35,13 +35,79 @@ __host__ __device__ constexpr int ffma_order(int mr, int nr) {
 struct FfmaArgs {
   ConvGeom g;
   float* out;
-  uint32_t* status;
+  WaitCtx wc;          // status block and this launch's epoch (see ptx_util.cuh)
   // Test hook for the bounded waits: if non-zero, CTA 0 initialises its "full" barriers
   // to expect one arrival more than they will ever get, so the consumers' first wait
   // runs out and the kernel reports kDevTimeoutFull instead of hanging.
   uint32_t test_missing_arrival;
+  // Non-zero: every CTA adds its elapsed SM cycles and nanoseconds (first instruction to
+  // last store) to words 2 and 3 of the status block with atomicMax — the elapsed
+  // processor clocks of Section 3.3's efficiency formula, measured inside the kernel.
+  uint32_t clock_stamp;
+  // Split tail (g.sk_tiles > 0): one slot of tile_m x tile_cols partial sums per CTA, and
+  // one flag word per CTA that receives this launch's epoch when the slot is complete.
+  float* sk_partial;
+  uint32_t* sk_flags;
   KStepTable table;
 };
+
+// ---------------------------------------------------------------------------------------
+// Work items.  A CTA walks whole tiles first (static round-robin over [tile_begin,
+// sk_first)), then its share of the SPLIT TAIL: the last sk_tiles tiles, fewer than the
+// grid has CTAs, would leave SMs idle for a whole tile's time, so their K steps — sk_tiles x
+// n_ksteps of them, numbered tile by tile — are dealt out evenly, CTA i taking the
+// contiguous range [i U / G, (i + 1) U / G).  A range is shorter than one tile, so it covers
+// the end of one tile and / or the beginning of the next.  The CTA whose range holds a
+// tile's LAST K step finishes that tile: it adds the partial sums that the lower-numbered
+// CTAs holding the tile's earlier steps wrote to their slots, in CTA order (a fixed order:
+// results are bitwise reproducible), then scales and stores.  Every CTA does its
+// contributing piece before its finishing piece, so a finisher waits only for CTAs with
+// lower numbers, which never wait for it.
+// ---------------------------------------------------------------------------------------
+enum FfmaItemKind : int { kItemWhole = 0, kItemContribute = 1, kItemFinish = 2 };
+
+struct FfmaItem {
+  int tile, s0, s1, kind;
+};
+
+// K-step range of CTA `cta` in the split tail: units [u0, u1) of sk_units.
+__device__ __forceinline__ void sk_range(const ConvGeom& g, int cta, int grid, int& u0, int& u1) {
+  u0 = (int)(((long long)cta * g.sk_units) / grid);
+  u1 = (int)(((long long)(cta + 1) * g.sk_units) / grid);
+}
+
+// The k-th item of this CTA, or false when there is none.
+__device__ __forceinline__ bool ffma_item(const ConvGeom& g, int k, FfmaItem& it) {
+  const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
+  const int first = g.tile_begin + cta;
+  const int n_whole = first < g.sk_first ? (g.sk_first - first + grid - 1) / grid : 0;
+  if (k < n_whole) {
+    it.tile = first + k * grid; it.s0 = 0; it.s1 = g.n_ksteps; it.kind = kItemWhole;
+    return true;
+  }
+  if (g.sk_tiles <= 0) return false;
+  int u0, u1;
+  sk_range(g, cta, grid, u0, u1);
+  if (u1 <= u0) return false;
+  const int n = g.n_ksteps;
+  const int ta = u0 / n;                       // tile (within the tail) where the range starts
+  const int a0 = u0 - ta * n;
+  const bool two = u1 > (ta + 1) * n;          // the range runs on into tile ta + 1
+  int piece = k - n_whole;
+  if (two) {
+    if (piece == 0) {                          // contribution to the next tile first
+      it.tile = g.sk_first + ta + 1; it.s0 = 0; it.s1 = u1 - (ta + 1) * n; it.kind = kItemContribute;
+      return true;
+    }
+    --piece;
+  }
+  if (piece != 0) return false;
+  it.tile = g.sk_first + ta;
+  it.s0 = a0;
+  it.s1 = two ? n : u1 - ta * n;
+  it.kind = it.s1 < n ? kItemContribute : (a0 == 0 ? kItemWhole : kItemFinish);
+  return true;
+}
 
 template <int MR, int NR>
 struct Frag {
@@ -49,18 +115,34 @@ struct Frag {
   float4 b[NR / 4];
 };
 
+// One 8-byte shared-memory load.  Written as an instruction of its own so that two
+// neighbouring ones are not fused into a 16-byte load: next to a stream of packed
+// multiply-adds a 16-byte load costs about 1.3 issue cycles, an 8-byte load about 0.1
+// (measured: the microbenchmark in ubench_fp32.cu).
+__device__ __forceinline__ float2 lds64(const float* p) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(smem_u32(p)));
+  return v;
+}
+
 // Thread (to, tn) of the 16 x 16 consumer grid reads, from row `a_row` of the staged
 // filter box, MR values (float4 groups 64 filters apart, or float2 groups 32 apart)
 // and, from the staged patch row, NR values (float4 groups 64 columns apart).
-template <int MR, int NR, bool FIXED>
+// W64: every group of four is fetched by two 8-byte loads instead of one 16-byte load.
+template <int MR, int NR, bool FIXED, bool W64>
 __device__ __forceinline__ void load_frag(Frag<MR, NR>& f, const float* a_row,
                                           const float* const (&b_row)[NR / 4], int b_off) {
   if constexpr (MR % 4 == 0) {
 #pragma unroll
     for (int q = 0; q < MR / 4; ++q) {
-      const float4 v = *reinterpret_cast<const float4*>(a_row + q * 64);
-      f.a[2 * q] = make_float2(v.x, v.y);
-      f.a[2 * q + 1] = make_float2(v.z, v.w);
+      if constexpr (W64) {
+        f.a[2 * q] = lds64(a_row + q * 64);
+        f.a[2 * q + 1] = lds64(a_row + q * 64 + 2);
+      } else {
+        const float4 v = *reinterpret_cast<const float4*>(a_row + q * 64);
+        f.a[2 * q] = make_float2(v.x, v.y);
+        f.a[2 * q + 1] = make_float2(v.z, v.w);
+      }
     }
   } else {
 #pragma unroll
@@ -68,10 +150,13 @@ __device__ __forceinline__ void load_frag(Frag<MR, NR>& f, const float* a_row,
   }
 #pragma unroll
   for (int h = 0; h < NR / 4; ++h) {
-    if constexpr (FIXED)
-      f.b[h] = *reinterpret_cast<const float4*>(b_row[0] + b_off + 64 * h);
-    else
-      f.b[h] = *reinterpret_cast<const float4*>(b_row[h] + b_off);
+    const float* src = FIXED ? b_row[0] + b_off + 64 * h : b_row[h] + b_off;
+    if constexpr (W64) {
+      const float2 lo = lds64(src), hi = lds64(src + 2);
+      f.b[h] = make_float4(lo.x, lo.y, hi.x, hi.y);
+    } else {
+      f.b[h] = *reinterpret_cast<const float4*>(src);
+    }
   }
 }
 
@@ -110,14 +195,17 @@ __device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR 
   }
 }
 
-// Producer state: which (tile, K step) is loaded next, into which ring stage.
+// Producer state: which (item, K step) is loaded next, into which ring stage.
 struct FfmaProducer {
-  int tile, step, stage;
+  int item, step, step_end, stage;   // step_end <= step: no work left
   uint32_t phase;
   int o0, n0, h0, w0;
 
-  __device__ __forceinline__ void set_tile(const ConvGeom& g, int mt) {
-    int r = tile;
+  __device__ __forceinline__ void set_item(const ConvGeom& g, int mt) {
+    FfmaItem it;
+    if (!ffma_item(g, item, it)) { step = 0; step_end = -1; return; }
+    step = it.s0; step_end = it.s1;
+    int r = it.tile;
     const int ob = r % g.o_blocks; r /= g.o_blocks;
     const int nch = r % g.n_chunks; r /= g.n_chunks;
     const int xr = r % g.x_runs;
@@ -129,13 +217,12 @@ struct FfmaProducer {
   }
 
   __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
-    tile = g.tile_begin + blockIdx.x;
-    step = 0; stage = 0; phase = 0;
+    item = 0; stage = 0; phase = 0;
     o0 = n0 = h0 = w0 = 0;
-    if (tile < g.tile_end) set_tile(g, mt);
+    set_item(g, mt);
   }
 
-  __device__ __forceinline__ bool has_work(const ConvGeom& g) const { return tile < g.tile_end; }
+  __device__ __forceinline__ bool has_work(const ConvGeom&) const { return step < step_end; }
 
   // Waits for the ring slot, issues the copies of one K step, advances.
   template <bool BACKOFF>
@@ -144,8 +231,8 @@ struct FfmaProducer {
                                         uint32_t full_bar, uint32_t empty_bar, int mt) {
     const ConvGeom& g = args.g;
     const uint32_t eb = empty_bar + 8u * stage;
-    const bool ok = BACKOFF ? mbar_wait_backoff(eb, phase ^ 1u, args.status, kDevTimeoutEmpty)
-                            : mbar_wait(eb, phase ^ 1u, args.status, kDevTimeoutEmpty);
+    const bool ok = BACKOFF ? mbar_wait_backoff(eb, phase ^ 1u, args.wc, kDevTimeoutEmpty)
+                            : mbar_wait(eb, phase ^ 1u, args.wc, kDevTimeoutEmpty);
     if (!ok) return false;
     const maxdnn_kstep ks = args.table.s[step];
     const uint32_t fb = full_bar + 8u * stage;
@@ -159,10 +246,9 @@ struct FfmaProducer {
       w += g.stride_w;
     }
     if (++stage == g.stages) { stage = 0; phase ^= 1u; }
-    if (++step == g.n_ksteps) {
-      step = 0;
-      tile += gridDim.x;
-      if (tile < g.tile_end) set_tile(g, mt);
+    if (++step == step_end) {
+      ++item;
+      set_item(g, mt);
     }
     return true;
   }
@@ -177,9 +263,27 @@ struct FfmaProducer {
   }
 };
 
+// Bounded wait for a peer CTA's "slot complete" flag (split tail).
+__device__ __noinline__ bool wait_peer_flag(const uint32_t* flag, uint32_t epoch, const WaitCtx& wc) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      uint32_t v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+      if (v == epoch) return true;
+      __nanosleep(100);
+    }
+    if (globaltimer_ns() - t0 > kWaitBudgetNs) break;
+    if (launch_gave_up(wc)) break;
+  }
+  record_give_up(wc, kDevTimeoutPeer);
+  return false;
+}
+
 #define MAXDNN_ROW(R) a_ptr + (R) * Mt, b_ptr, (R) * b_pitch
 
-template <int MR, int NR, bool FIXED>
+template <int MR, int NR, bool FIXED, bool W64>
 __global__ void __launch_bounds__(ffma_threads(MR, NR), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
@@ -200,9 +304,16 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const uint32_t bar_off = b_off + (uint32_t)stages * g.b_stage_bytes;
   const uint32_t full_bar = base + bar_off;          // stages x 8 bytes
   const uint32_t empty_bar = full_bar + 8u * stages; // stages x 8 bytes
+  const uint32_t sk_bar = empty_bar + 8u * stages;   // split tail: "every warp stored its partial sums"
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  long long stamp_cycles = 0;
+  uint64_t stamp_ns = 0;
+  if (args.clock_stamp != 0 && threadIdx.x == 0) {
+    stamp_cycles = clock64();
+    stamp_ns = globaltimer_ns();
+  }
 
   if (threadIdx.x == 0) {
     const uint32_t extra = (args.test_missing_arrival != 0 && blockIdx.x == 0) ? 1u : 0u;
@@ -210,12 +321,12 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       mbar_init(full_bar + 8u * s, 1 + extra);
       mbar_init(empty_bar + 8u * s, kFfmaConsumerWarps);
     }
+    mbar_init(sk_bar, kFfmaConsumerWarps);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
   __syncthreads();
 
-  const int n_ksteps = g.n_ksteps;
   const int rows = g.rows;
 
   if constexpr (!INLINE) {
@@ -279,7 +390,9 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   uint32_t phase = 0;
   bool ok = true;
 
-  for (int tile = g.tile_begin + blockIdx.x; tile < g.tile_end && ok; tile += gridDim.x) {
+  FfmaItem item;
+  for (int item_no = 0; ok && ffma_item(g, item_no, item); ++item_no) {
+    const int tile = item.tile;
     float2 P[MR / 2][NR / 2], Q[MR / 2][NR / 2];
 #pragma unroll
     for (int i = 0; i < MR / 2; ++i)
@@ -290,7 +403,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
 
     Frag<MR, NR> f0, f1;
-    ok = mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull);
+    ok = mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull);
     if (!ok) break;
     const float* a_ptr;
     const float* b_ptr[NH];
@@ -301,9 +414,9 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       for (int h = 0; h < NH; ++h) b_ptr[h] = bs + b_elem[h];
     };
     point_at_stage(stage);
-    load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(0));
+    load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(0));
 
-    for (int s = 0; s < n_ksteps; ++s) {
+    for (int s = item.s0; s < item.s1; ++s) {
       if constexpr (INLINE) {
         // Refill the slot this CTA finished two steps ago (every warp has released it
         // by now, so the wait does not hold warp 0 back) with the K step that is
@@ -320,13 +433,13 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       int r = 0;
 #pragma unroll 1
       for (; r + 4 < rows; r += 4) {
-        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(1));
         fma_block<MR, NR>(f0, P, Q);
-        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(2));
+        load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(2));
         fma_block<MR, NR>(f1, P, Q);
-        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(3));
+        load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(3));
         fma_block<MR, NR>(f0, P, Q);
-        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(4));
+        load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(4));
         fma_block<MR, NR>(f1, P, Q);
         a_ptr += 4 * Mt;
 #pragma unroll
@@ -334,9 +447,9 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
 #pragma unroll 1
       for (; rows - r > 2; r += 2) {   // 3 or 4 rows left: two of them here
-        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(1));
         fma_block<MR, NR>(f0, P, Q);
-        load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(2));
+        load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(2));
         fma_block<MR, NR>(f1, P, Q);
         a_ptr += 2 * Mt;
 #pragma unroll
@@ -344,24 +457,24 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       const bool two_left = (rows - r == 2);
       if (two_left) {
-        load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(1));
+        load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(1));
         fma_block<MR, NR>(f0, P, Q);
       }
       // The last row of this stage is in f1 (two_left) or f0.  Prefetch row 0 of
       // the next stage into the other buffer before computing it.
       const int cur_stage = stage;
       if (++stage == stages) { stage = 0; phase ^= 1u; }
-      const bool more = s + 1 < n_ksteps;
+      const bool more = s + 1 < item.s1;
       if (more) {
-        ok = mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull);
+        ok = mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull);
         if (!ok) break;
         point_at_stage(stage);
       }
       if (two_left) {
-        if (more) load_frag<MR, NR, FIXED>(f0, MAXDNN_ROW(0));
+        if (more) load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(0));
         fma_block<MR, NR>(f1, P, Q);
       } else {
-        if (more) load_frag<MR, NR, FIXED>(f1, MAXDNN_ROW(0));
+        if (more) load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(0));
         fma_block<MR, NR>(f0, P, Q);
         f0 = f1;
       }
@@ -369,6 +482,58 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       if (lane == 0) mbar_arrive(empty_bar + 8u * cur_stage);
     }
     if (!ok) break;
+
+    // ------------------------------------------------- split tail: partial sums
+    // A slot holds a thread's accumulators as float4 {P.x, P.y, Q.x, Q.y}, element
+    // [pair index][thread], so that a warp's store of one pair index is one 512-byte run.
+    constexpr int kPairs = (MR / 2) * (NR / 2);
+    if (item.kind == kItemContribute) {
+      float4* slot = reinterpret_cast<float4*>(args.sk_partial) +
+                     (size_t)blockIdx.x * (kPairs * 256) + threadIdx.x;
+#pragma unroll
+      for (int i = 0; i < MR / 2; ++i)
+#pragma unroll
+        for (int j = 0; j < NR / 2; ++j)
+          __stcg(slot + (i * (NR / 2) + j) * 256, make_float4(P[i][j].x, P[i][j].y, Q[i][j].x, Q[i][j].y));
+      __threadfence();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sk_bar);
+      if (threadIdx.x == 0) {
+        // every consumer warp has stored and fenced: publish the slot under this launch's epoch
+        if (mbar_wait(sk_bar, 0, args.wc, kDevTimeoutPeer))
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(args.sk_flags + blockIdx.x),
+                       "r"(args.wc.epoch) : "memory");
+      }
+      continue;
+    }
+    if (item.kind == kItemFinish) {
+      // the CTAs below this one whose ranges hold the tile's earlier K steps, in order
+      const int grid = (int)gridDim.x;
+      const int first_unit = (tile - g.sk_first) * g.n_ksteps;
+      int j = (int)(((long long)first_unit * grid) / g.sk_units);
+      int u0, u1;
+      sk_range(g, j, grid, u0, u1);
+      while (j > 0 && u0 > first_unit) { --j; sk_range(g, j, grid, u0, u1); }
+      while (u1 <= first_unit) { ++j; sk_range(g, j, grid, u0, u1); }
+      for (; j < (int)blockIdx.x && ok; ++j) {
+        sk_range(g, j, grid, u0, u1);
+        if (u1 <= u0) continue;                      // a CTA without a share
+        bool ready = true;
+        if (lane == 0) ready = wait_peer_flag(args.sk_flags + j, args.wc.epoch, args.wc);
+        ready = __shfl_sync(0xffffffffu, ready ? 1 : 0, 0) != 0;
+        if (!ready) { ok = false; break; }
+        const float4* slot = reinterpret_cast<const float4*>(args.sk_partial) +
+                             (size_t)j * (kPairs * 256) + threadIdx.x;
+#pragma unroll
+        for (int i = 0; i < MR / 2; ++i)
+#pragma unroll
+          for (int jj = 0; jj < NR / 2; ++jj) {
+            const float4 v = __ldcg(slot + (i * (NR / 2) + jj) * 256);
+            P[i][jj].x += v.x; P[i][jj].y += v.y; Q[i][jj].x += v.z; Q[i][jj].y += v.w;
+          }
+      }
+      if (!ok) break;
+    }
 
     // ---------------------------------------------------------- epilogue
     // alpha scaling and store; for a fixed filter a quarter-warp writes one full
@@ -411,6 +576,10 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   if constexpr (INLINE) {
     if (warp == 0 && lane == 0 && !(ok && prod_ok)) prod.drain(g, full_bar);
+  }
+  if (args.clock_stamp != 0 && threadIdx.x == 0 && args.wc.status) {
+    atomicMax(args.wc.status + 2, (uint32_t)(clock64() - stamp_cycles));
+    atomicMax(args.wc.status + 3, (uint32_t)(globaltimer_ns() - stamp_ns));
   }
 }
 #undef MAXDNN_ROW

@@ -28,15 +28,19 @@ struct DeviceState {
   bool ready = false;
   bool sm100 = false;
   int sm_count = 0;
-  uint32_t* status = nullptr;   // one word of device memory
-  bool ffma_attr[16] = {};
-  bool umma_attr[4] = {false, false, false, false};
-  bool wgrad_attr = false;
-  bool umma_chunk_attr = false;
-  bool umma_pair_chunk_attr = false;
-  bool wgrad_chunk_attr = false;
-  bool wgrad_pair_chunk_attr = false;
-  bool wgrad_umma_attr[4] = {false, false, false, false};
+  uint32_t* status = nullptr;   // the status block in device memory (see WaitCtx)
+  std::atomic<uint32_t> epoch{0};   // number of the latest launch that reports into it
+  // "dynamic shared memory limit raised" flags, one per kernel instance: set once under
+  // attr_mu, read without it afterwards
+  std::mutex attr_mu;
+  std::atomic<bool> ffma_attr[32];
+  std::atomic<bool> umma_attr[4];
+  std::atomic<bool> wgrad_attr;
+  std::atomic<bool> umma_chunk_attr;
+  std::atomic<bool> umma_pair_chunk_attr;
+  std::atomic<bool> wgrad_chunk_attr;
+  std::atomic<bool> wgrad_pair_chunk_attr;
+  std::atomic<bool> wgrad_umma_attr[4];
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
   cudaStream_t aux[3] = {nullptr, nullptr, nullptr};
@@ -46,8 +50,30 @@ struct DeviceState {
 };
 
 std::mutex g_mu;
-DeviceState g_dev[kMaxDevices];
+DeviceState g_dev[kMaxDevices];      // static storage: every flag starts false, every epoch 0
 std::atomic<uint64_t> g_launches{0};
+
+// Raises a kernel's dynamic shared-memory limit once per device.
+template <class Kern>
+maxdnn_status ensure_smem_attr(DeviceState* ds, std::atomic<bool>* done, Kern kern) {
+  if (done->load(std::memory_order_acquire)) return MAXDNN_OK;
+  std::lock_guard<std::mutex> lk(ds->attr_mu);
+  if (done->load(std::memory_order_relaxed)) return MAXDNN_OK;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  done->store(true, std::memory_order_release);
+  return MAXDNN_OK;
+}
+
+// The status block and a fresh epoch for one launch (never 0: word 1 of a cleared block).
+WaitCtx next_wait_ctx(DeviceState* ds) {
+  uint32_t e = ds->epoch.fetch_add(1, std::memory_order_relaxed) + 1;
+  if (e == 0) e = ds->epoch.fetch_add(1, std::memory_order_relaxed) + 1;
+  return WaitCtx{ds->status, e};
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -121,13 +147,8 @@ size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int env_int(const char* name) {
-  const char* v = getenv(name);
-  return v ? atoi(v) : 0;
-}
-
 // What a forward plan depends on: the problem, the device's SM count and the tuning
-// switches read from the environment.  A call that repeats the previous call's key on the
+// options (their generation number: any change of any option retires every cached plan).  A call that repeats the previous call's key on the
 // same thread keeps the previous plan (planning costs 1.5-4 us, a third of the host time of
 // a call; small layers are launch-bound).
 struct PlanKey {   // trivial: cleared with memset so that padding compares equal
@@ -135,11 +156,6 @@ struct PlanKey {   // trivial: cleared with memset so that padding compares equa
   int32_t v[8];
   bool valid;
 };
-
-int env_or(const char* name, int unset) {
-  const char* v = getenv(name);
-  return v ? atoi(v) : unset;
-}
 
 bool same_plan_key(const PlanKey& a, const PlanKey& b) {
   return a.valid && b.valid && memcmp(&a.d, &b.d, sizeof(ConvDims)) == 0 &&
@@ -169,18 +185,11 @@ struct PlanCache {
   }
 };
 
-template <int MR, int NR, bool FIXED>
+template <int MR, int NR, bool FIXED, bool W64>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
-  auto kern = ffma_conv_kernel<MR, NR, FIXED>;
-  if (!ds->ffma_attr[slot]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-    ds->ffma_attr[slot] = true;
-  }
+  auto kern = ffma_conv_kernel<MR, NR, FIXED, W64>;
+  if (ensure_smem_attr(ds, &ds->ffma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   kern<<<args.g.grid, ffma_threads(MR, NR), args.g.smem_bytes, stream>>>(mf, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -192,10 +201,15 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
                             const FfmaArgs& args, cudaStream_t stream) {
   const ConvGeom& g = args.g;
   const bool fx = g.fixed_pitch != 0;
+  const bool w64 = option(OPT_FFMA_LANES, 1) != 0;   // 8-byte operand loads (0: 16-byte loads)
 #define MAXDNN_FFMA_CASE(M, C, MR, NR, SLOT)                                             \
-  if (g.tile_m == (M) && g.tile_cols == (C))                                             \
-    return fx ? launch_ffma<MR, NR, true>(ds, (SLOT), mf, mi, args, stream)              \
-              : launch_ffma<MR, NR, false>(ds, (SLOT) + 1, mf, mi, args, stream);
+  if (g.tile_m == (M) && g.tile_cols == (C)) {                                           \
+    if (w64)                                                                             \
+      return fx ? launch_ffma<MR, NR, true, true>(ds, (SLOT) + 16, mf, mi, args, stream) \
+                : launch_ffma<MR, NR, false, true>(ds, (SLOT) + 17, mf, mi, args, stream); \
+    return fx ? launch_ffma<MR, NR, true, false>(ds, (SLOT), mf, mi, args, stream)       \
+              : launch_ffma<MR, NR, false, false>(ds, (SLOT) + 1, mf, mi, args, stream); \
+  }
   MAXDNN_FFMA_CASE(256, 128, 16, 8, 0)
   MAXDNN_FFMA_CASE(128, 256, 8, 16, 2)
   MAXDNN_FFMA_CASE(96, 256, 6, 16, 4)
@@ -226,20 +240,26 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   memset(&key, 0, sizeof(key));
   key.d = cd;
   key.v[0] = ds->sm_count;
-  key.v[1] = env_int("MAXDNN_FFMA_TILE_M");
-  key.v[2] = env_int("MAXDNN_FFMA_COLS");
+  key.v[1] = (int32_t)options_generation();
   key.valid = true;
   int slot = cache.find(key);
   if (slot < 0) {
     slot = cache.take();
-    st = plan_ffma(cd, ds->sm_count, key.v[1], key.v[2], &cache.args[slot].g, &cache.args[slot].table);
+    st = plan_ffma(cd, ds->sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS),
+                   &cache.args[slot].g, &cache.args[slot].table);
     if (st != MAXDNN_OK) return st;
     cache.key[slot] = key;
   }
   FfmaArgs& args = cache.args[slot];
   args.out = out;
-  args.status = ds->status;
-  args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see FfmaArgs
+  args.wc = next_wait_ctx(ds);
+  args.test_missing_arrival = (uint32_t)option(OPT_TEST_MISSING_ARRIVAL);   // see FfmaArgs
+  args.clock_stamp = (uint32_t)option(OPT_KERNEL_CLOCK);
+  if (args.clock_stamp != 0 &&
+      cudaMemsetAsync(ds->status + 2, 0, 8, stream) != cudaSuccess) {   // this launch's maxima
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
   const ConvGeom& g = args.g;
 
   CUtensorMap mf, mi;
@@ -277,14 +297,7 @@ maxdnn_status launch_umma_pair(DeviceState* ds, const CUtensorMap& mf, const CUt
                                const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
   auto kern = umma_pair_conv_kernel<BF16>;
   const int slot = BF16 ? 3 : 2;
-  if (!ds->umma_attr[slot]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-    ds->umma_attr[slot] = true;
-  }
+  if (ensure_smem_attr(ds, &ds->umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
   cfg.blockDim = dim3(kUmmaThreads, 1, 1);
@@ -308,14 +321,7 @@ maxdnn_status launch_umma_pair(DeviceState* ds, const CUtensorMap& mf, const CUt
 maxdnn_status launch_umma_chunk(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
                                 const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
   auto kern = umma_chunk_conv_kernel;
-  if (!ds->umma_chunk_attr) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-    ds->umma_chunk_attr = true;
-  }
+  if (ensure_smem_attr(ds, &ds->umma_chunk_attr, kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   kern<<<args.g.grid, kUmmaChunkThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -326,14 +332,7 @@ maxdnn_status launch_umma_pair_chunk(DeviceState* ds, const CUtensorMap& mf, con
                                      const CUtensorMap& mo, const UmmaArgs& args,
                                      cudaStream_t stream) {
   auto kern = umma_pair_chunk_conv_kernel;
-  if (!ds->umma_pair_chunk_attr) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-    ds->umma_pair_chunk_attr = true;
-  }
+  if (ensure_smem_attr(ds, &ds->umma_pair_chunk_attr, kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
   cfg.blockDim = dim3(kUmmaChunkThreads, 1, 1);
@@ -359,14 +358,7 @@ maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensor
                           const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
   auto kern = umma_conv_kernel<BF16>;
   const int slot = BF16 ? 1 : 0;
-  if (!ds->umma_attr[slot]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-    ds->umma_attr[slot] = true;
-  }
+  if (ensure_smem_attr(ds, &ds->umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   kern<<<args.g.grid, kUmmaThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -393,17 +385,13 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   key.d = cd;
   key.v[0] = ds->sm_count;
   key.v[1] = elem_bytes;
-  key.v[2] = env_int("MAXDNN_UMMA_KC");
-  key.v[3] = env_int("MAXDNN_UMMA_PAIR");
-  key.v[4] = env_or("MAXDNN_UMMA_MERGE", -12345);
-  key.v[5] = env_or("MAXDNN_UMMA_STAGE_KB", -12345);
-  key.v[6] = env_or("MAXDNN_UMMA_COLS", -12345);
+  key.v[2] = (int32_t)options_generation();
   key.valid = true;
   int slot = cache.find(key);
   if (slot < 0) {
     slot = cache.take();
-    st = plan_umma(cd, elem_bytes, ds->sm_count, key.v[2], key.v[3], &cache.args[slot].g,
-                   &cache.args[slot].table);
+    st = plan_umma(cd, elem_bytes, ds->sm_count, option(OPT_UMMA_KC), option(OPT_UMMA_PAIR),
+                   &cache.args[slot].g, &cache.args[slot].table);
     if (st != MAXDNN_OK) return st;
     cache.key[slot] = key;
   }
@@ -412,11 +400,11 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
   const uint64_t eb = (uint64_t)elem_bytes;
   const uint32_t atom = 128u / (uint32_t)elem_bytes;
   const bool bf16 = elem_bytes == 2;
-  args.status = ds->status;
+  args.wc = next_wait_ctx(ds);
   args.atom = atom;
   args.umma_k = 32u / (uint32_t)elem_bytes;
   args.is_bf16 = bf16 ? 1u : 0u;
-  args.test_missing_arrival = (uint32_t)env_int("MAXDNN_TEST_MISSING_ARRIVAL");   // see UmmaArgs
+  args.test_missing_arrival = (uint32_t)option(OPT_TEST_MISSING_ARRIVAL);   // see UmmaArgs
   // Staged layouts: filters [group of 32/64][kw][channel][128 B], patches
   // [pixel][image group][channel][128 B].
   args.lbo_a_bytes = (uint32_t)(g.kwc * g.kc) * 128u;
@@ -514,9 +502,9 @@ maxdnn_status dgrad_plan_check(const ConvDims& fd, maxdnn_kernel_kind kind, int 
   static thread_local ConvGeom g;
   static thread_local KStepTable t;
   if (kind == MAXDNN_KERNEL_FP32)
-    return plan_ffma(fd, sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
-  return plan_umma(fd, kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, env_int("MAXDNN_UMMA_KC"),
-                   env_int("MAXDNN_UMMA_PAIR"), &g, &t);
+    return plan_ffma(fd, sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS), &g, &t);
+  return plan_umma(fd, kind == MAXDNN_KERNEL_BF16 ? 2 : 4, sm_count, option(OPT_UMMA_KC),
+                   option(OPT_UMMA_PAIR), &g, &t);
 }
 
 // Workspace of the strided map gradient.  The classes run side by side, so each has its
@@ -578,6 +566,31 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
   int32_t Ho, Wo;
   check_dims(d, &Ho, &Wo);
   const int sh = d.stride_h, sw = d.stride_w;
+  // The FPROP that computes one residue class (dense result; the caller adds output pitches).
+  auto class_dims = [&](const DgradAxis& ah, const DgradAxis& aw) {
+    ConvDims fd;
+    fd.Nb = d.Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = x3 ? 3 * d.No : d.No;
+    fd.No = d.Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
+    fd.pad_w = aw.pad; fd.pad_h = ah.pad; fd.alpha = d.alpha;
+    fd.in_h_stride = (int64_t)Wo * d.Nb;
+    fd.in_c_stride = (int64_t)Ho * Wo * d.Nb;
+    fd.Ho_given = ah.n; fd.Wo_given = aw.n;
+    fd.out_x_stride = fd.out_y_stride = fd.out_o_stride = 0;
+    return fd;
+  };
+  // Nothing is launched unless every class has a plan (its FPROP has No' = Nc filters: the
+  // 16-byte row rule can refuse it) and the split kernels cover whole 16-byte groups.
+  if (x3 && (((size_t)d.No * Ho * Wo * d.Nb) % 4 != 0 || 3 * (int64_t)d.No > 32767))
+    return MAXDNN_NOT_SUPPORTED;
+  for (int rh = 0; rh < sh; ++rh)
+    for (int rw = 0; rw < sw; ++rw) {
+      const DgradAxis ah = dgrad_axis(rh, d.Skh, sh, d.pad_h, d.Hi);
+      const DgradAxis aw = dgrad_axis(rw, d.Skw, sw, d.pad_w, d.Wi);
+      if (!dgrad_class_live(ah, aw, Ho, Wo)) continue;
+      if (x3 && ((size_t)d.No * ah.J * aw.J * d.Nc) % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+      st = dgrad_plan_check(class_dims(ah, aw), kind, ds->sm_count);
+      if (st != MAXDNN_OK) return st;
+    }
   uint8_t* ft_next = static_cast<uint8_t*>(ws) + p.pre_bytes;
   uint8_t* sub_next = ft_next + p.ft_bytes;
   if (x3) {
@@ -633,14 +646,7 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
           aux_used[lane - 1] = true;
         }
       }
-      ConvDims fd;
-      fd.Nb = d.Nb; fd.Wi = Wo - aw.crop; fd.Hi = Ho - ah.crop; fd.Nc = d.No;
-      fd.No = d.Nc; fd.Skw = aw.J; fd.Skh = ah.J; fd.stride_w = fd.stride_h = 1;
-      fd.pad_w = aw.pad; fd.pad_h = ah.pad; fd.alpha = d.alpha;
-      fd.in_h_stride = (int64_t)Wo * d.Nb;
-      fd.in_c_stride = (int64_t)Ho * Wo * d.Nb;
-      fd.Ho_given = ah.n; fd.Wo_given = aw.n;
-      fd.out_x_stride = fd.out_y_stride = fd.out_o_stride = 0;
+      ConvDims fd = class_dims(ah, aw);
       const dim3 grid((unsigned)ceil_div(d.No, 32), (unsigned)ceil_div(d.Nc, 32),
                       (unsigned)(ah.J * aw.J));
       const dim3 block(32, 8);
@@ -670,8 +676,7 @@ maxdnn_status bprop_data_strided(const ConvDims& d, maxdnn_kernel_kind kind, con
               reinterpret_cast<const float4*>(w_ft), reinterpret_cast<float4*>(w_ft3), n4, 0x2u);
           if (cudaGetLastError() != cudaSuccess) { result = MAXDNN_CUDA_ERROR; break; }
           g_launches.fetch_add(1, std::memory_order_relaxed);
-          fd.Nc = 3 * d.No;
-          result = fprop_umma(fd, 4, src, w_ft3, dst, cs, env_or("MAXDNN_X3_CHUNK_ROWS", 768));
+          result = fprop_umma(fd, 4, src, w_ft3, dst, cs, option(OPT_X3_CHUNK_ROWS, 768));
           continue;
         }
         result = fprop_umma(fd, (int)eb, src, w_ft, dst, cs);
@@ -779,8 +784,8 @@ maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const voi
   static thread_local WgradArgs fargs;
   static thread_local WgradUmmaArgs uargs;
   WgradGeom& g = tensor ? uargs.g : fargs.g;
-  st = plan_wgrad(d, tensor ? eb : 0, ds->sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
-                  env_int("MAXDNN_WGRAD_PAIR"));
+  st = plan_wgrad(d, tensor ? eb : 0, ds->sm_count, option(OPT_WGRAD_SPLITS), &g,
+                  option(OPT_WGRAD_PAIR));
   if (st != MAXDNN_OK) return st;
   const size_t kno = (size_t)g.Nc * g.Skh * g.Skw * g.No;
   const size_t need = g.splits > 1 ? (size_t)g.splits * kno * 4 : 0;
@@ -812,20 +817,13 @@ maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const voi
   if (!tensor) {
     fargs.dfilt = dfilt;
     fargs.partial = static_cast<float*>(ws);
-    fargs.status = ds->status;
-    if (!ds->wgrad_attr) {
-      if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               227 * 1024) != cudaSuccess) {
-        cudaGetLastError();
-        return MAXDNN_CUDA_ERROR;
-      }
-      ds->wgrad_attr = true;
-    }
+    fargs.wc = next_wait_ctx(ds);
+    if (ensure_smem_attr(ds, &ds->wgrad_attr, wgrad_kernel) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
     wgrad_kernel<<<g.grid, kWgThreads, g.smem_bytes, stream>>>(mg, mi, fargs);
   } else {
     uargs.dfilt = dfilt;
     uargs.partial = static_cast<float*>(ws);
-    uargs.status = ds->status;
+    uargs.wc = next_wait_ctx(ds);
     uargs.atom = chunk;
     const uint32_t fmt = bf16 ? 1u : 2u;
     const uint32_t n_mma = (uint32_t)g.n_mma;
@@ -835,14 +833,7 @@ maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const voi
     const int slot = (bf16 ? 1 : 0) + (g.pair ? 2 : 0);
     if (g.pair) {
       auto kern = bf16 ? wgrad_umma_pair_kernel<true> : wgrad_umma_pair_kernel<false>;
-      if (!ds->wgrad_umma_attr[slot]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess) {
-          cudaGetLastError();
-          return MAXDNN_CUDA_ERROR;
-        }
-        ds->wgrad_umma_attr[slot] = true;
-      }
+      if (ensure_smem_attr(ds, &ds->wgrad_umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
       cfg.blockDim = dim3(kWgUmmaThreads, 1, 1);
@@ -861,14 +852,7 @@ maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const voi
       }
     } else {
       auto kern = bf16 ? wgrad_umma_kernel<true> : wgrad_umma_kernel<false>;
-      if (!ds->wgrad_umma_attr[slot]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess) {
-          cudaGetLastError();
-          return MAXDNN_CUDA_ERROR;
-        }
-        ds->wgrad_umma_attr[slot] = true;
-      }
+      if (ensure_smem_attr(ds, &ds->wgrad_umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
       kern<<<g.grid, kWgUmmaThreads, g.smem_bytes, stream>>>(mg, mi, uargs);
     }
   }
@@ -1018,7 +1002,7 @@ maxdnn_status fprop_tf32x3(const maxdnn_conv_desc* desc, const float* in, const 
   g_launches.fetch_add(2, std::memory_order_relaxed);
   // A fresh accumulator about every 768 rows of the split problem's K (256 of the
   // original): the accumulator's truncation then acts on short partial sums only.
-  const int chunk_rows = env_or("MAXDNN_X3_CHUNK_ROWS", 768);
+  const int chunk_rows = option(OPT_X3_CHUNK_ROWS, 768);
   if (chunk_rows > 0) return fprop_umma(dims_from(d3), 4, w_in, w_filt, out, stream, chunk_rows);
   return fprop_umma(&d3, 4, w_in, w_filt, out, stream);
 }
@@ -1101,7 +1085,7 @@ maxdnn_status plan_wgrad_x3(const maxdnn_conv_desc* desc, int sm_count, WgradX3P
   p->dout_bytes = round256((size_t)desc->No * Ho * Wo * 2 * desc->Nb * 4);
   static thread_local WgradGeom scratch;
   WgradGeom* gg = g ? g : &scratch;
-  st = plan_wgrad(p->d3, 4, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), gg, env_int("MAXDNN_WGRAD_PAIR"));
+  st = plan_wgrad(p->d3, 4, sm_count, option(OPT_WGRAD_SPLITS), gg, option(OPT_WGRAD_PAIR));
   if (st != MAXDNN_OK) return st;
   const size_t kno = (size_t)desc->Nc * desc->Sk * desc->Sk * desc->No;
   p->partial_bytes = gg->splits > 1 ? (size_t)gg->splits * kno * 4 : 0;
@@ -1161,23 +1145,16 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
   }
   args.dfilt = dfilt;
   args.partial = w_part;
-  args.status = ds->status;
+  args.wc = next_wait_ctx(ds);
   args.atom = 32u;
   // a fresh accumulator every 24 reduction steps: 768 terms of the tripled reduction
-  const int cs = env_or("MAXDNN_X3_CHUNK_ROWS", 768) / 32;
+  const int cs = option(OPT_X3_CHUNK_ROWS, 768) / 32;
   args.chunk_steps = (uint32_t)(cs < 1 ? 1 : cs);
   args.x3_per_part = (uint32_t)(desc->Nb / 32);
   args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) |
                (((g.pair ? 256u : 128u) >> 4) << 24);
   if (g.pair) {
-    if (!ds->wgrad_pair_chunk_attr) {
-      if (cudaFuncSetAttribute(wgrad_umma_pair_chunk_kernel,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
-        cudaGetLastError();
-        return MAXDNN_CUDA_ERROR;
-      }
-      ds->wgrad_pair_chunk_attr = true;
-    }
+    if (ensure_smem_attr(ds, &ds->wgrad_pair_chunk_attr, wgrad_umma_pair_chunk_kernel) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
     cfg.blockDim = dim3(kWgChunkThreads, 1, 1);
@@ -1195,14 +1172,7 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
       return MAXDNN_CUDA_ERROR;
     }
   } else {
-    if (!ds->wgrad_chunk_attr) {
-      if (cudaFuncSetAttribute(wgrad_umma_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               227 * 1024) != cudaSuccess) {
-        cudaGetLastError();
-        return MAXDNN_CUDA_ERROR;
-      }
-      ds->wgrad_chunk_attr = true;
-    }
+    if (ensure_smem_attr(ds, &ds->wgrad_chunk_attr, wgrad_umma_chunk_kernel) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
     wgrad_umma_chunk_kernel<<<g.grid, kWgChunkThreads, g.smem_bytes, stream>>>(mg, mi, args);
   }
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
@@ -1227,8 +1197,9 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
 constexpr size_t kStaticScratchBytes = 256;
 static __device__ __align__(256) uint32_t g_static_scratch[kStaticScratchBytes / sizeof(uint32_t)];
 
-// Scratch the fp32 kernel needs for a plan: one status word today.
-size_t ffma_scratch_bytes(const ConvGeom&) { return sizeof(uint32_t); }
+// Scratch the fp32 kernel needs for a plan: the two words of the status block (first code
+// recorded; epoch of the latest launch that gave up).
+size_t ffma_scratch_bytes(const ConvGeom&) { return 2 * sizeof(uint32_t); }
 
 DeviceState g_static_dev[kMaxDevices];   // `status` points into g_static_scratch of that device
 
@@ -1284,12 +1255,15 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
   static thread_local FfmaArgs args;
-  st = plan_ffma(dims_from(*desc), ds->sm_count, 0, 0, &args.g, &args.table);
+  // the plan of maxdnn_conv_fprop for this problem (tile options included)
+  st = plan_ffma(dims_from(*desc), ds->sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS),
+                 &args.g, &args.table);
   if (st != MAXDNN_OK) return st;
   if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
   args.out = out;
-  args.status = ds->status;
-  args.test_missing_arrival = 0;
+  args.wc = next_wait_ctx(ds);
+  args.test_missing_arrival = (uint32_t)option(OPT_TEST_MISSING_ARRIVAL);
+  args.clock_stamp = 0;
   const ConvGeom& g = args.g;
 
   CUtensorMap mf, mi;
@@ -1311,13 +1285,28 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
-  // The block is shared by every call and keeps what the last call left: the word
-  // the kernel tests must read zero when it starts.
-  if (cudaMemsetAsync(ds->status, 0, ffma_scratch_bytes(g), stream) != cudaSuccess) {
+  // The block is shared by every call and keeps what earlier calls left.  Nothing in it
+  // has to start at zero: word 0 is only ever written by a wait that ran out and is
+  // cleared by maxdnn_last_device_status_noalloc; word 1 is compared with this launch's
+  // epoch, which no earlier launch had.
+  return dispatch_ffma(ds, mf, mi, args, stream);
+}
+
+// Waits for the stream, reads word 0 of the device's status block and clears it if set.
+// No allocation: a 4-byte copy into host memory and, after a failure, a 4-byte memset.
+maxdnn_status read_and_clear_status(DeviceState* ds, cudaStream_t stream) {
+  uint32_t word = 0;
+  if (cudaStreamSynchronize(stream) != cudaSuccess ||
+      cudaMemcpy(&word, ds->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
-  return dispatch_ffma(ds, mf, mi, args, stream);
+  if (word != 0) {
+    if (option(OPT_DEBUG_STATUS)) fprintf(stderr, "maxdnn: device status word 0x%x\n", word);
+    cudaMemset(ds->status, 0, 4);
+    return MAXDNN_DEVICE_TIMEOUT;
+  }
+  return MAXDNN_OK;
 }
 
 }  // namespace
@@ -1381,10 +1370,10 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   static thread_local KStepTable t;
   switch (kind) {
     case MAXDNN_KERNEL_FP32:
-      st = plan_ffma(dims_from(*desc), sm_count, env_int("MAXDNN_FFMA_TILE_M"), env_int("MAXDNN_FFMA_COLS"), &g, &t);
+      st = plan_ffma(dims_from(*desc), sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS), &g, &t);
       break;
-    case MAXDNN_KERNEL_TF32: st = plan_umma(dims_from(*desc), 4, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
-    case MAXDNN_KERNEL_BF16: st = plan_umma(dims_from(*desc), 2, sm_count, env_int("MAXDNN_UMMA_KC"), env_int("MAXDNN_UMMA_PAIR"), &g, &t); break;
+    case MAXDNN_KERNEL_TF32: st = plan_umma(dims_from(*desc), 4, sm_count, option(OPT_UMMA_KC), option(OPT_UMMA_PAIR), &g, &t); break;
+    case MAXDNN_KERNEL_BF16: st = plan_umma(dims_from(*desc), 2, sm_count, option(OPT_UMMA_KC), option(OPT_UMMA_PAIR), &g, &t); break;
     default: return MAXDNN_INVALID_VALUE;
   }
   if (st != MAXDNN_OK) return st;
@@ -1515,7 +1504,7 @@ maxdnn_status maxdnn_conv_bprop_data_tf32x3(const maxdnn_conv_desc* desc, const 
 
 maxdnn_status maxdnn_conv_bprop_filter_tf32x3_workspace(const maxdnn_conv_desc* desc, size_t* bytes) {
   if (!bytes) return MAXDNN_INVALID_VALUE;
-  int sm = env_int("MAXDNN_SM_COUNT");
+  int sm = option(OPT_SM_COUNT);
   if (sm <= 0) {
     DeviceState* ds = nullptr;
     const maxdnn_status st = device_state(&ds);
@@ -1575,7 +1564,7 @@ maxdnn_status maxdnn_conv_bprop_data(const maxdnn_conv_desc* desc, maxdnn_kernel
 static maxdnn_status bprop_filter_workspace(const maxdnn::ConvDims& d, maxdnn_kernel_kind kind,
                                             size_t* bytes) {
   if (!bytes || !kind_ok(kind)) return MAXDNN_INVALID_VALUE;
-  int sm_count = env_int("MAXDNN_SM_COUNT");   // planning without a device (tests)
+  int sm_count = option(OPT_SM_COUNT);   // planning without a device (tests)
   if (sm_count <= 0) {
     DeviceState* ds = nullptr;
     const maxdnn_status st = device_state(&ds);
@@ -1584,8 +1573,8 @@ static maxdnn_status bprop_filter_workspace(const maxdnn::ConvDims& d, maxdnn_ke
   }
   WgradGeom g;
   const int eb = kind == MAXDNN_KERNEL_FP32 ? 0 : (kind == MAXDNN_KERNEL_BF16 ? 2 : 4);
-  const maxdnn_status st = plan_wgrad(d, eb, sm_count, env_int("MAXDNN_WGRAD_SPLITS"), &g,
-                                      env_int("MAXDNN_WGRAD_PAIR"));
+  const maxdnn_status st = plan_wgrad(d, eb, sm_count, option(OPT_WGRAD_SPLITS), &g,
+                                      option(OPT_WGRAD_PAIR));
   if (st != MAXDNN_OK) return st;
   *bytes = g.splits > 1 ? (size_t)g.splits * g.Nc * g.Skh * g.Skw * g.No * 4 : 0;
   return MAXDNN_OK;
@@ -1644,24 +1633,44 @@ maxdnn_status maxdnn_last_device_status(void* cuda_stream) {
   maxdnn_status st = device_state(&ds);
   if (st != MAXDNN_OK) return st;
   if (!ds->status) return MAXDNN_NOT_SUPPORTED;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  uint32_t word = 0;
-  if (cudaStreamSynchronize(stream) != cudaSuccess ||
-      cudaMemcpy(&word, ds->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
-    cudaGetLastError();
-    return MAXDNN_CUDA_ERROR;
-  }
-  if (word != 0) {
-    if (getenv("MAXDNN_DEBUG_STATUS")) fprintf(stderr, "maxdnn: device status word 0x%x\n", word);
-    cudaMemset(ds->status, 0, 4);
-    return MAXDNN_DEVICE_TIMEOUT;
-  }
-  return MAXDNN_OK;
+  return read_and_clear_status(ds, static_cast<cudaStream_t>(cuda_stream));
 }
 
 maxdnn_status maxdnn_conv_fprop_noalloc(const maxdnn_conv_desc* desc, const float* in,
                                         const float* filt, float* out, void* cuda_stream) {
   return fprop_fp32_noalloc(desc, in, filt, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_last_device_status_noalloc(void* cuda_stream) {
+  DeviceState* ds = nullptr;
+  maxdnn_status st = static_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->status) return MAXDNN_NOT_SUPPORTED;
+  return read_and_clear_status(ds, static_cast<cudaStream_t>(cuda_stream));
+}
+
+maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanoseconds,
+                                       void* cuda_stream) {
+  DeviceState* ds = nullptr;
+  maxdnn_status st = device_state(&ds);
+  if (st != MAXDNN_OK) return st;
+  if (!ds->status || !sm_cycles || !nanoseconds) return MAXDNN_INVALID_VALUE;
+  uint32_t w[2] = {0, 0};
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess ||
+      cudaMemcpy(w, ds->status + 2, 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
+  *sm_cycles = w[0];
+  *nanoseconds = w[1];
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_set_option(const char* name, int32_t value) { return set_option(name, value); }
+maxdnn_status maxdnn_unset_option(const char* name) { return unset_option(name); }
+void maxdnn_reset_options(void) { reset_options(); }
+maxdnn_status maxdnn_get_option(const char* name, int32_t* value, int32_t* is_set) {
+  return get_option(name, value, is_set);
 }
 
 uint64_t maxdnn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -4,7 +4,95 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 namespace maxdnn {
+
+// ---------------------------------------------------------------------------
+// Options: a small table of named integers (see plan.h).
+// ---------------------------------------------------------------------------
+namespace {
+const char* const kOptionNames[OPT_COUNT] = {
+    "FFMA_TILE_M", "FFMA_COLS", "FFMA_LANES", "FFMA_KH", "FFMA_STREAMK",
+    "UMMA_KC", "UMMA_PAIR", "UMMA_MERGE", "UMMA_STAGE_KB", "UMMA_COLS",
+    "WGRAD_SPLITS", "WGRAD_PAIR", "SM_COUNT", "X3_CHUNK_ROWS", "DEBUG_STATUS",
+    "KERNEL_CLOCK", "TEST_MISSING_ARRIVAL"};
+struct OptionSlot {
+  std::atomic<int32_t> value{0};
+  std::atomic<bool> set{false};
+};
+OptionSlot g_opt[OPT_COUNT];
+std::once_flag g_opt_once;
+std::atomic<uint32_t> g_opt_gen{1};
+
+void load_options_from_env() {
+  for (int i = 0; i < OPT_COUNT; ++i) {
+    g_opt[i].set.store(false);
+    g_opt[i].value.store(0);
+    if (i == OPT_TEST_MISSING_ARRIVAL) continue;      // never from the environment
+    char name[64] = "MAXDNN_";
+    strncat(name, kOptionNames[i], sizeof(name) - 8);
+    if (const char* v = getenv(name)) {
+      g_opt[i].value.store(atoi(v));
+      g_opt[i].set.store(true);
+    }
+  }
+}
+void ensure_options() { std::call_once(g_opt_once, load_options_from_env); }
+int find_option(const char* name) {
+  if (!name) return -1;
+  if (strncmp(name, "MAXDNN_", 7) == 0) name += 7;
+  for (int i = 0; i < OPT_COUNT; ++i)
+    if (strcmp(name, kOptionNames[i]) == 0) return i;
+  return -1;
+}
+}  // namespace
+
+bool option_is_set(OptionId id) {
+  ensure_options();
+  return g_opt[id].set.load(std::memory_order_relaxed);
+}
+int option(OptionId id, int unset_value) {
+  ensure_options();
+  return g_opt[id].set.load(std::memory_order_relaxed) ? g_opt[id].value.load(std::memory_order_relaxed)
+                                                       : unset_value;
+}
+maxdnn_status set_option(const char* name, int value) {
+  ensure_options();
+  const int i = find_option(name);
+  if (i < 0) return MAXDNN_INVALID_VALUE;
+  g_opt[i].value.store(value);
+  g_opt[i].set.store(true);
+  g_opt_gen.fetch_add(1);
+  return MAXDNN_OK;
+}
+maxdnn_status unset_option(const char* name) {
+  ensure_options();
+  const int i = find_option(name);
+  if (i < 0) return MAXDNN_INVALID_VALUE;
+  g_opt[i].set.store(false);
+  g_opt[i].value.store(0);
+  g_opt_gen.fetch_add(1);
+  return MAXDNN_OK;
+}
+maxdnn_status get_option(const char* name, int32_t* value, int32_t* is_set) {
+  ensure_options();
+  const int i = find_option(name);
+  if (i < 0) return MAXDNN_INVALID_VALUE;
+  if (value) *value = g_opt[i].value.load();
+  if (is_set) *is_set = g_opt[i].set.load() ? 1 : 0;
+  return MAXDNN_OK;
+}
+void reset_options() {
+  ensure_options();
+  load_options_from_env();
+  g_opt_gen.fetch_add(1);
+}
+uint32_t options_generation() {
+  ensure_options();
+  return g_opt_gen.load(std::memory_order_relaxed);
+}
 
 maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo) {
   if (!d) return MAXDNN_INVALID_VALUE;
@@ -265,8 +353,7 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   // 21 in bf16).
   const bool few = d.Nc < umma_k0 ||
                    (d.Nc < 2 * umma_k0 && 3 * d.Nc < 2 * align_up(d.Nc, umma_k0));
-  const bool merged = few && d.Skw > 1 && !pair && force_kc == 0 &&
-                      !(getenv("MAXDNN_UMMA_MERGE") && atoi(getenv("MAXDNN_UMMA_MERGE")) < 0);
+  const bool merged = few && d.Skw > 1 && !pair && force_kc == 0 && option(OPT_UMMA_MERGE, 0) >= 0;
   if (merged) {
     best_nn = atom;
     best_T = max_cols / atom < Wo ? max_cols / atom : Wo;
@@ -318,7 +405,7 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   // at least 9 (bf16) / 12 (tf32) MMAs (measured on the 3x3 / 5x5 layers); otherwise one
   // tap per step and 48 KB stages (four or more stages).
   int stage_budget = kwc > 1 ? 96 * 1024 : 48 * 1024;
-  if (const char* e = getenv("MAXDNN_UMMA_STAGE_KB")) { const int v = atoi(e); if (v >= 16 && v <= 96) stage_budget = v * 1024; }
+  if (option_is_set(OPT_UMMA_STAGE_KB)) { const int v = option(OPT_UMMA_STAGE_KB); if (v >= 16 && v <= 96) stage_budget = v * 1024; }
   auto stage_bytes = [&](int c) {
     return (kwc * 128 + (kwc > 1 ? (px_cta + kwc - 1) * g->cta_n : cols)) * c * elem_bytes;
   };
@@ -339,7 +426,7 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
   int kc = pick_kc();
   const int min_mmas = elem_bytes == 2 ? 9 : 12;
   if (kwc > 1 && (kwc * (kc / umma_k) < min_mmas || stage_bytes(kc) > stage_budget) &&
-      !getenv("MAXDNN_UMMA_STAGE_KB")) {
+      !option_is_set(OPT_UMMA_STAGE_KB)) {
     kwc = 1;
     stage_budget = 48 * 1024;
     kc = pick_kc();
@@ -375,7 +462,7 @@ static maxdnn_status plan_umma_as(const ConvDims& d, int elem_bytes, int sm_coun
     const int b_rows1 = merged_strip ? strip_w * box_c * (g->cta_n / atom) : cols / atom * rows1;
     int khc = 1;   // filter rows per step: stages of at most 40 KB (a deep ring beat longer steps)
     while (kw_parts == 1 && khc < d.Skh && (128 / atom * rows1 + b_rows1) * 128 * (khc + 1) <= 40 * 1024) ++khc;
-    if (const char* e = getenv("MAXDNN_UMMA_MERGE")) { const int v = atoi(e); if (v >= 1 && v <= d.Skh && kw_parts == 1) khc = v; }
+    if (option_is_set(OPT_UMMA_MERGE)) { const int v = option(OPT_UMMA_MERGE); if (v >= 1 && v <= d.Skh && kw_parts == 1) khc = v; }
     if (box_kw > 256 || rows1 * khc > 1024) return MAXDNN_NOT_SUPPORTED;
     // with the strip the rows of one filter row are contiguous in both operands, the
     // filter rows of a step are not (strip_w vs box_kw columns apart): kc counts the
@@ -455,8 +542,8 @@ maxdnn_status plan_umma(const ConvDims& d, int elem_bytes, int sm_count, int for
   // pin a choice.
   int cols_list[3] = {256, 192, 128};
   int n_cols = 3;
-  if (const char* e = getenv("MAXDNN_UMMA_COLS")) {
-    const int v = atoi(e);
+  if (option_is_set(OPT_UMMA_COLS)) {
+    const int v = option(OPT_UMMA_COLS);
     if (v >= 32 && v <= 256 && v % 32 == 0) { cols_list[0] = v; n_cols = 1; }
   }
   static thread_local ConvGeom gc;

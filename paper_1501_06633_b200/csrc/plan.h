@@ -11,6 +11,25 @@ namespace maxdnn {
 
 constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel parameters
 
+// Tuning and test switches (ablations, tests; none is needed in normal use).  Each has a
+// name; its value is "unset" until maxdnn_set_option gives it one.  The environment
+// variable MAXDNN_<NAME> supplies the initial value, read ONCE, at the first use of any
+// option in the process — never on the path of a call.  TEST_MISSING_ARRIVAL is the
+// exception: it has no environment variable and can only be set through the C ABI.
+enum OptionId : int {
+  OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_LANES, OPT_FFMA_KH, OPT_FFMA_STREAMK,
+  OPT_UMMA_KC, OPT_UMMA_PAIR, OPT_UMMA_MERGE, OPT_UMMA_STAGE_KB, OPT_UMMA_COLS,
+  OPT_WGRAD_SPLITS, OPT_WGRAD_PAIR, OPT_SM_COUNT, OPT_X3_CHUNK_ROWS, OPT_DEBUG_STATUS,
+  OPT_KERNEL_CLOCK, OPT_TEST_MISSING_ARRIVAL, OPT_COUNT
+};
+bool option_is_set(OptionId id);
+int option(OptionId id, int unset_value = 0);          // the value, or unset_value
+maxdnn_status set_option(const char* name, int value); // name without the MAXDNN_ prefix
+maxdnn_status unset_option(const char* name);
+maxdnn_status get_option(const char* name, int32_t* value, int32_t* is_set);
+void reset_options();                                  // back to the values the environment gave
+uint32_t options_generation();                         // changes whenever an option changes
+
 // The operation with per-axis filter size, stride and padding (Section 2 has one of each:
 // the public square descriptor maps to Skw = Skh = Sk and so on).
 struct ConvDims {
@@ -62,6 +81,9 @@ struct ConvGeom {
   int32_t grid;
   int32_t smem_bytes;
   int32_t Skh, stride_h, pad_h;                       // the h-axis filter size, stride, padding
+  // fp32 kernel, split tail: tiles [sk_first, tile_end) are computed by all CTAs together,
+  // their sk_units = sk_tiles x n_ksteps K steps dealt out evenly (0 tiles: no split)
+  int32_t sk_first, sk_tiles, sk_units;
 };
 
 struct KStepTable {
@@ -74,8 +96,17 @@ inline int align_up(int a, int b) { return ceil_div(a, b) * b; }
 maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo);
 
 // FFMA kernel plan.  force_tile_m / force_cols > 0 pin the tile shape (ablations).
+// allow_split: the caller can provide the workspace of a split tail (see ffma_split_bytes).
 maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
-                        ConvGeom* g, KStepTable* t);
+                        ConvGeom* g, KStepTable* t, bool allow_split = false);
+
+// Workspace of the fp32 kernel's split tail for any plan on `sm_count` SMs: one slot of
+// partial sums per CTA (the largest tile has 32768 columns x filters), then one flag per CTA.
+constexpr size_t kFfmaSplitSlotBytes = 32768 * 4;
+inline size_t ffma_split_flags_offset(int sm_count) { return (size_t)sm_count * kFfmaSplitSlotBytes; }
+inline size_t ffma_split_bytes(int sm_count) {
+  return ffma_split_flags_offset(sm_count) + (((size_t)sm_count * 4 + 255) & ~(size_t)255);
+}
 
 // Tensor-core kernel plan (elem_bytes 4 = TF32, 2 = BF16).
 // force_pair: 0 = choose, 1 = two-SM tiles (256 filters per CTA pair), -1 = one-SM tiles.

@@ -15,6 +15,7 @@ enum DeviceCode : uint32_t {
   kDevTimeoutAccum = 0x300,   // epilogue waited for an accumulator that never completed
   kDevTimeoutAccFree = 0x400, // MMA issuer waited for an accumulator that was never drained
   kDevTimeoutDrain = 0x500,   // exit path: a copy in flight did not land in time
+  kDevTimeoutPeer = 0x600,    // split tail: another CTA's partial sums never arrived
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -60,12 +61,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Where a wait that ran out reports, and how the other waits of the SAME launch learn of
+// it.  `status` points to the device's status block: word 0 keeps the first code any
+// launch recorded until the host reads it (sticky); word 1 holds the `epoch` — a number the
+// host gives every launch — of the latest launch in which a wait gave up.  A wait leaves
+// early only when word 1 equals its own launch's epoch, so a code left behind by an
+// earlier launch never cuts a healthy launch's waits short.
+struct WaitCtx {
+  uint32_t* status;
+  uint32_t epoch;
+};
+
 // Wait budget of every spin in these kernels: 2 s of wall clock, checked every
 // 256 failed polls.  A wait that runs out records `code` and returns false; the
 // caller then leaves its loops and the kernel ends normally.
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;
 
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t* status,
+__device__ __forceinline__ bool launch_gave_up(const WaitCtx& wc) {
+  return wc.status && reinterpret_cast<volatile uint32_t*>(wc.status)[1] == wc.epoch;
+}
+
+__device__ __forceinline__ void record_give_up(const WaitCtx& wc, uint32_t code) {
+  if (!wc.status) return;
+  atomicCAS(wc.status, 0u, code);
+  atomicExch(wc.status + 1, wc.epoch);
+}
+
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx& wc,
                                             uint32_t code) {
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
@@ -73,16 +95,16 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint3
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (globaltimer_ns() - t0 > kWaitBudgetNs) break;
-    if (status && *reinterpret_cast<volatile uint32_t*>(status) != 0) break;  // someone gave up
+    if (launch_gave_up(wc)) break;   // another wait of this launch ran out
   }
-  if (status) atomicCAS(status, 0u, code);
+  record_give_up(wc, code);
   return false;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc,
                                           uint32_t code) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, status, code);
+  return mbar_wait_slow(bar, parity, wc, code);
 }
 
 // Exit-path wait after another wait ran out: copies already issued land within
@@ -100,7 +122,7 @@ __device__ __noinline__ void mbar_wait_grace(uint32_t bar, uint32_t parity) {
 // Producer-side wait: sleeps between polls, so that a warp waiting for a ring slot
 // does not take issue slots from the arithmetic warps of its scheduler.  Same 2 s
 // budget as mbar_wait.
-__device__ __noinline__ bool mbar_wait_sleep_slow(uint32_t bar, uint32_t parity, uint32_t* status,
+__device__ __noinline__ bool mbar_wait_sleep_slow(uint32_t bar, uint32_t parity, const WaitCtx& wc,
                                                   uint32_t code) {
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
@@ -112,16 +134,16 @@ __device__ __noinline__ bool mbar_wait_sleep_slow(uint32_t bar, uint32_t parity,
       if (mbar_try_wait(bar, parity)) return true;
     }
     if (globaltimer_ns() - t0 > kWaitBudgetNs) break;
-    if (status && *reinterpret_cast<volatile uint32_t*>(status) != 0) break;
+    if (launch_gave_up(wc)) break;
   }
-  if (status) atomicCAS(status, 0u, code);
+  record_give_up(wc, code);
   return false;
 }
 
-__device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, uint32_t* status,
+__device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, const WaitCtx& wc,
                                                   uint32_t code) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_sleep_slow(bar, parity, status, code);
+  return mbar_wait_sleep_slow(bar, parity, wc, code);
 }
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {

@@ -40,7 +40,7 @@ struct UmmaArgs {
   uint32_t is_bf16;
   uint32_t test_missing_arrival;   // test hook: CTA 0's full barriers expect an arrival that never comes
   uint32_t chunk_steps;            // chunked kernel only: K steps per TMEM accumulator
-  uint32_t* status;
+  WaitCtx wc;          // status block and this launch's epoch (see ptx_util.cuh)
   KStepTable table;
 };
 
@@ -254,7 +254,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
-          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
             ok = false;
             break;
           }
@@ -306,7 +306,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       for (int tile = blockIdx.x; tile < g.n_tiles && ok; tile += gridDim.x, ++it) {
         const int acc = it & 1;
         const uint32_t acc_par = ((uint32_t)(it >> 1) & 1u) ^ 1u;
-        if (!mbar_wait(acce_bar + 8u * acc, acc_par, args.status, kDevTimeoutAccFree)) {
+        if (!mbar_wait(acce_bar + 8u * acc, acc_par, args.wc, kDevTimeoutAccFree)) {
           ok = false;
           break;
         }
@@ -314,7 +314,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
         uint32_t accumulate = 0;
         for (int s = 0; s < n_ksteps; ++s) {
-          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+          if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
             ok = false;
             break;
           }
@@ -353,7 +353,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       // Exit path: every MMA issued so far has finished before TMEM is released.
       if (elect_one()) tcgen05_commit(done_bar);
-      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+      mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -377,7 +377,7 @@ umma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const int o0 = ob * kUmmaM + q * 32;
       const int n0 = nch * g.tile_n;
       const int x0 = xr * g.tile_px;
-      if (!mbar_wait(accf_bar + 8u * acc, acc_par, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, acc_par, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }

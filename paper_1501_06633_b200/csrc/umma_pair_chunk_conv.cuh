@@ -64,7 +64,7 @@ __device__ __noinline__ void pair_chunk_epilogue_role(const CUtensorMap& map_out
     float tot[128];
     for (int c = 0; c < chunks_per_tile && ok; ++c, ++chunk) {
       const uint32_t acc = chunk & 1u;
-      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }
@@ -220,7 +220,7 @@ umma_pair_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
-          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
             ok = false;
             break;
           }
@@ -272,7 +272,7 @@ umma_pair_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         // chunk loop around the plain kernel's step loop (see umma_chunk_conv_kernel)
         for (int s0 = 0; s0 < n_ksteps && ok; s0 += chunk_steps, ++chunk) {
           const uint32_t acc = chunk & 1u;
-          if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.status,
+          if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.wc,
                          kDevTimeoutAccFree)) {
             ok = false;
             break;
@@ -282,7 +282,7 @@ umma_pair_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           const int s1 = s0 + chunk_steps < n_ksteps ? s0 + chunk_steps : n_ksteps;
           uint32_t accumulate = 0;
           for (int s = s0; s < s1; ++s) {
-            if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+            if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
               ok = false;
               break;
             }
@@ -319,7 +319,7 @@ umma_pair_chunk_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       // Exit path: every MMA issued so far has finished before TMEM is released.
       if (elect_one()) tcgen05_commit_pair(done_bar, 1);
-      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+      mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
     }
   } else {
     // ------------------------------------------------------------ epilogue

@@ -206,7 +206,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         maxdnn_kstep ks = args.table.s[0];
         for (int s = 0; s < n_ksteps; ++s) {
           const maxdnn_kstep ks_next = args.table.s[s + 1 < n_ksteps ? s + 1 : 0];
-          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+          if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
             ok = false;
             break;
           }
@@ -256,7 +256,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       for (int tile = pair; tile < g.n_tiles && ok; tile += n_pairs, ++it) {
         const int acc = it & 1;
         const uint32_t acc_par = ((uint32_t)(it >> 1) & 1u) ^ 1u;
-        if (!mbar_wait(acce_bar + 8u * acc, acc_par, args.status, kDevTimeoutAccFree)) {
+        if (!mbar_wait(acce_bar + 8u * acc, acc_par, args.wc, kDevTimeoutAccFree)) {
           ok = false;
           break;
         }
@@ -264,7 +264,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
         uint32_t accumulate = 0;
         for (int s = 0; s < n_ksteps; ++s) {
-          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+          if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
             ok = false;
             break;
           }
@@ -300,7 +300,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       // Exit path: every MMA issued so far has finished before TMEM is released.
       if (elect_one()) tcgen05_commit_pair(done_bar, 1);
-      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+      mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -324,7 +324,7 @@ umma_pair_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       const int o0 = ob * 2 * kUmmaM + (int)rank * kUmmaM + q * 32;
       const int n0 = nch * g.tile_n;
       const int x0 = xr * g.tile_px;
-      if (!mbar_wait(accf_bar + 8u * acc, acc_par, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, acc_par, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }

@@ -34,7 +34,7 @@ struct WgradUmmaArgs {
   uint32_t x3_per_part;   // chunked kernel only: reduction steps (groups of 32 images) per product part
   float* dfilt;
   float* partial;
-  uint32_t* status;
+  WaitCtx wc;          // status block and this launch's epoch (see ptx_util.cuh)
 };
 
 template <bool BF16>
@@ -109,7 +109,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t phase = 0;
     bool ok = true;
     while (ok && !pc.done(g)) {
-      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
         ok = false;
         break;
       }
@@ -147,7 +147,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       const int n_steps = cc.r_end - cc.r;
       // the epilogue has drained this accumulator (used two items ago)
       const uint32_t acc = it & 1u;
-      if (!mbar_wait(acce_bar + 8u * acc, ((it >> 1) & 1u) ^ 1u, args.status, kDevTimeoutAccFree)) {
+      if (!mbar_wait(acce_bar + 8u * acc, ((it >> 1) & 1u) ^ 1u, args.wc, kDevTimeoutAccFree)) {
         ok = false;
         break;
       }
@@ -155,7 +155,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       const uint32_t d_tmem = tmem_base + acc * 256u;
       uint32_t accumulate = 0;
       for (int s = 0; s < n_steps; ++s) {
-        if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+        if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
           ok = false;
           break;
         }
@@ -182,7 +182,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
       ++it;
     }
     if (elect_one()) tcgen05_commit(done_bar);
-    mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+    mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
   } else {
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
@@ -195,7 +195,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_dout,
     const float scale = direct ? g.alpha : 1.0f;
     while (ok && !cc.done(g)) {
       const uint32_t acc = it & 1u;
-      if (!mbar_wait(accf_bar + 8u * acc, (it >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, (it >> 1) & 1u, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }

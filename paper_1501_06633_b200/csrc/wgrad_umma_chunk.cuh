@@ -38,7 +38,7 @@ __device__ __noinline__ void wgrad_chunk_epilogue_role(const WgradUmmaArgs& args
     float tot[128];
     for (int c = 0; c < n_chunks && ok; ++c, ++chunk) {
       const uint32_t acc = chunk & 1u;
-      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }
@@ -150,7 +150,7 @@ wgrad_umma_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t phase = 0;
     bool ok = true;
     while (ok && !pc.done(g)) {
-      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
         ok = false;
         break;
       }
@@ -197,7 +197,7 @@ wgrad_umma_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
       // chunk loop around the plain kernel's step loop: a fresh accumulator per chunk
       for (int s0 = 0; s0 < n_steps && ok; s0 += chunk_steps, ++chunk) {
         const uint32_t acc = chunk & 1u;
-        if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.status, kDevTimeoutAccFree)) {
+        if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.wc, kDevTimeoutAccFree)) {
           ok = false;
           break;
         }
@@ -206,7 +206,7 @@ wgrad_umma_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
         const int s1 = s0 + chunk_steps < n_steps ? s0 + chunk_steps : n_steps;
         uint32_t accumulate = 0;
         for (int s = s0; s < s1; ++s) {
-          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+          if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
             ok = false;
             break;
           }
@@ -234,7 +234,7 @@ wgrad_umma_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
       cc.start(g, cc.item + (int)gridDim.x);
     }
     if (elect_one()) tcgen05_commit(done_bar);
-    mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+    mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
   } else {
     // ------------------------------------------------------------ epilogue
     wgrad_chunk_epilogue_role(args, row_tab, accf_bar, acce_bar, tmem_base, warp, lane);

@@ -101,7 +101,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t phase = 0;
     bool ok = true;
     while (ok && !pc.done(g)) {
-      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
         ok = false;
         break;
       }
@@ -138,7 +138,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
       while (ok && !cc.done(g)) {
         const int n_steps = cc.r_end - cc.r;
         const uint32_t acc = it & 1u;
-        if (!mbar_wait(acce_bar + 8u * acc, ((it >> 1) & 1u) ^ 1u, args.status, kDevTimeoutAccFree)) {
+        if (!mbar_wait(acce_bar + 8u * acc, ((it >> 1) & 1u) ^ 1u, args.wc, kDevTimeoutAccFree)) {
           ok = false;
           break;
         }
@@ -146,7 +146,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
         const uint32_t d_tmem = tmem_base + acc * 256u;
         uint32_t accumulate = 0;
         for (int s = 0; s < n_steps; ++s) {
-          if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+          if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
             ok = false;
             break;
           }
@@ -173,7 +173,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
         ++it;
       }
       if (elect_one()) tcgen05_commit_pair(done_bar, 1);
-      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+      mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
     }
   } else {
     // ------------------------------------------------------------ epilogue (both CTAs)
@@ -187,7 +187,7 @@ wgrad_umma_pair_kernel(const __grid_constant__ CUtensorMap map_dout,
     const float scale = direct ? g.alpha : 1.0f;
     while (ok && !cc.done(g)) {
       const uint32_t acc = it & 1u;
-      if (!mbar_wait(accf_bar + 8u * acc, (it >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, (it >> 1) & 1u, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }

@@ -31,7 +31,7 @@ __device__ __noinline__ void wgrad_pair_chunk_epilogue_role(const WgradUmmaArgs&
     float tot[128];
     for (int c = 0; c < n_chunks && ok; ++c, ++chunk) {
       const uint32_t acc = chunk & 1u;
-      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.status, kDevTimeoutAccum)) {
+      if (!mbar_wait(accf_bar + 8u * acc, (chunk >> 1) & 1u, args.wc, kDevTimeoutAccum)) {
         ok = false;
         break;
       }
@@ -157,7 +157,7 @@ wgrad_umma_pair_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
     uint32_t phase = 0;
     bool ok = true;
     while (ok && !pc.done(g)) {
-      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.status, kDevTimeoutEmpty)) {
+      if (!mbar_wait(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
         ok = false;
         break;
       }
@@ -201,7 +201,7 @@ wgrad_umma_pair_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
         const int n_steps = cc.r_end - cc.r;
         for (int s0 = 0; s0 < n_steps && ok; s0 += chunk_steps, ++chunk) {
           const uint32_t acc = chunk & 1u;
-          if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.status, kDevTimeoutAccFree)) {
+          if (!mbar_wait(acce_bar + 8u * acc, ((chunk >> 1) & 1u) ^ 1u, args.wc, kDevTimeoutAccFree)) {
             ok = false;
             break;
           }
@@ -210,7 +210,7 @@ wgrad_umma_pair_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
           const int s1 = s0 + chunk_steps < n_steps ? s0 + chunk_steps : n_steps;
           uint32_t accumulate = 0;
           for (int s = s0; s < s1; ++s) {
-            if (!mbar_wait(full_bar + 8u * stage, phase, args.status, kDevTimeoutFull)) {
+            if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
               ok = false;
               break;
             }
@@ -238,7 +238,7 @@ wgrad_umma_pair_chunk_kernel(const __grid_constant__ CUtensorMap map_dout,
         cc.start(g, cc.item + n_pairs);
       }
       if (elect_one()) tcgen05_commit_pair(done_bar, 1);
-      mbar_wait(done_bar, 0, args.status, kDevTimeoutDrain);
+      mbar_wait(done_bar, 0, args.wc, kDevTimeoutDrain);
     }
   } else {
     // ------------------------------------------------------------ epilogue (both CTAs)

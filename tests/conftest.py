@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _options_back_to_default():
+    """A test may pin tuning options (maxdnn_set_option); none survives into the next test."""
+    yield
+    try:
+        import paper_1501_06633_b200 as mx
+        mx.reset_options()
+    except (ImportError, OSError, AttributeError):
+        pass

@@ -128,7 +128,7 @@ WGRAD_SHAPES = [
 @pytest.mark.parametrize("shape", WGRAD_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
 def test_bprop_filter(shape, splits, monkeypatch):
     if splits:
-        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+        mx.set_option("WGRAD_SPLITS", splits)
     w, inp, filt, dout = make(shape, 1700 + shape[5])
     d = mx.ConvDesc.make(*w.dims)
     need = mx.conv_bprop_filter_workspace(d)
@@ -165,9 +165,9 @@ def test_bprop_filter_tensor_cores(shape, splits, pair, kernel, monkeypatch):
         pytest.skip("a row of bf16 images must be a multiple of 16 bytes")
     if pair == 1 and shape[3] == 3 and shape[5] == 11:
         pytest.skip("one channel per tile (121 taps): nothing to split between two CTAs")
-    monkeypatch.setenv("MAXDNN_WGRAD_PAIR", str(pair))
+    mx.set_option("WGRAD_PAIR", pair)
     if splits:
-        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+        mx.set_option("WGRAD_SPLITS", splits)
     w, inp, filt, dout = make(shape, 2600 + shape[5])
     d = mx.ConvDesc.make(*w.dims)
     need = mx.conv_bprop_filter_workspace(d, KIND[kernel])

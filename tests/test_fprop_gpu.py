@@ -94,14 +94,14 @@ def test_edge_shapes_fp32(shape):
     check_fp32(w)
 
 
-@pytest.mark.parametrize("tile_m,cols", [(32, 128), (64, 128), (96, 128), (128, 128), (256, 128),
+@pytest.mark.parametrize("tile_m,cols", [(32, 128), (64, 128), (96, 128), (128, 128), (256, 128), (64, 256),
                                          (96, 256), (128, 256)])
 @pytest.mark.parametrize("stride", [1, 2])
 def test_every_tile_shape(tile_m, cols, stride, monkeypatch):
     """Every kernel instance (register block, producer placement, one box per stage
     or one per pixel) on a shape with ragged filter, image and pixel tails."""
-    monkeypatch.setenv("MAXDNN_FFMA_TILE_M", str(tile_m))
-    monkeypatch.setenv("MAXDNN_FFMA_COLS", str(cols))
+    mx.set_option("FFMA_TILE_M", tile_m)
+    mx.set_option("FFMA_COLS", cols)
     w = wl.Workload("tiles", 64, 11, 8, 24, 296, 3, stride, 1, 1.0, ("uniform", -1.0, 1.0),
                     ("uniform", -1.0, 1.0), 99)
     d = mx.ConvDesc.make(*w.dims)

@@ -217,7 +217,7 @@ def test_few_channel_layers_merge_filter_columns_into_k(kernel, shape, khc, monk
     """Layers with fewer channels than the MMA's K take K steps that span all filter columns
     (and khc filter rows) of a few channels; surplus K rows are out-of-bounds zeros."""
     if khc:
-        monkeypatch.setenv("MAXDNN_UMMA_MERGE", str(khc))
+        mx.set_option("UMMA_MERGE", khc)
     Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha = shape
     w = wl.Workload("merged", Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha, ("uniform", -1.0, 1.0),
                     ("uniform", -1.0, 1.0), 8800 + Sk)
@@ -246,7 +246,7 @@ def test_few_channel_layers_merge_filter_columns_into_k(kernel, shape, khc, monk
 def test_two_sm_tiles(kernel, shape, monkeypatch):
     """The two-SM variant (256 filters per CTA pair, cta_group::2 MMAs), taken only on
     request, against the oracle."""
-    monkeypatch.setenv("MAXDNN_UMMA_PAIR", "1")
+    mx.set_option("UMMA_PAIR", 1)
     Nb, Wi, Hi, Nc, No, Sk, st, pad, alpha = shape
     if kernel == "bf16" and Nb % 64 != 0:
         pytest.skip("bf16 tiles hold whole groups of 64 images")

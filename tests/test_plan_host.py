@@ -190,7 +190,7 @@ def test_table1_shapes_give_the_printed_output_sizes_and_have_plans():
 def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     """Host-side planning of the backward entry points (no device needed: the SM count
     is given)."""
-    monkeypatch.setenv("MAXDNN_SM_COUNT", "148")
+    mx.set_option("SM_COUNT", 148)
     d = mx.ConvDesc.make(128, 27, 27, 96, 256, 5, 1, 2, 1.0)
     assert mx.conv_bprop_data_workspace(d, mx.KERNEL_FP32) == 96 * 25 * 256 * 4
     assert mx.conv_bprop_data_workspace(d, mx.KERNEL_BF16) == 96 * 25 * 256 * 2
@@ -214,7 +214,7 @@ def test_bprop_workspace_sizes_and_refusals(monkeypatch):
     big = mx.ConvDesc.make(128, 12, 12, 1024, 1024, 3, 1, 1, 1.0)   # 592 tiles: 4 whole waves
     assert mx.conv_bprop_filter_workspace(big) == 0
     assert mx.conv_bprop_filter_workspace(d, mx.KERNEL_BF16) % kno == 0     # 10 channels x 25 taps per tile
-    monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", "5")
+    mx.set_option("WGRAD_SPLITS", 5)
     assert mx.conv_bprop_filter_workspace(d) == 5 * kno
     with pytest.raises(mx.MaxdnnError) as e:
         mx.conv_bprop_filter_workspace(mx.ConvDesc.make(30, 16, 16, 8, 8, 3, 1, 1, 1.0))   # Nb % 4

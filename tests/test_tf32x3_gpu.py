@@ -63,7 +63,7 @@ def test_tf32x3_small(shape):
 def test_tf32x3_both_chunked_kernels(shape, pair, monkeypatch):
     """The chunked kernel on one-SM tiles (pair = -1) and on two-SM tiles (pair = 1, forced
     also where the planner would not take them), against the oracle at the exact kernel's bar."""
-    monkeypatch.setenv("MAXDNN_UMMA_PAIR", str(pair))
+    mx.set_option("UMMA_PAIR", pair)
     Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
     w = wl.Workload("x3p", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
                     ("uniform", 0.0, 1.0), 4500 + Nc)          # same-signed terms: the hard case
@@ -85,7 +85,7 @@ def test_tf32x3_full_size_sampled(name, chunked, monkeypatch):
     if not chunked:
         if name not in ("mid5x5", "overfeat_L5"):
             pytest.skip("one-accumulator path: two layers are enough")
-        monkeypatch.setenv("MAXDNN_X3_CHUNK_ROWS", "0")
+        mx.set_option("X3_CHUNK_ROWS", 0)
         tol = max(5e-5, 1.2e-8 * w.Nc * w.Sk * w.Sk)      # overfeat_L5: K = 9216
     inp, filt = wl.make_inputs(w)
     got = run(w, inp, filt)
@@ -187,9 +187,9 @@ def test_bprop_filter_tf32x3(shape, splits, pair, monkeypatch):
     three times the images, accumulated in chunks) against the gradient oracle at the exact
     kernel's bar; same-signed operands, forced split counts, one-SM (pair = -1) and two-SM
     tiles (pair = 1, forced also where the planner would not take them)."""
-    monkeypatch.setenv("MAXDNN_WGRAD_PAIR", str(pair))
+    mx.set_option("WGRAD_PAIR", pair)
     if splits:
-        monkeypatch.setenv("MAXDNN_WGRAD_SPLITS", str(splits))
+        mx.set_option("WGRAD_SPLITS", splits)
     Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
     w = wl.Workload("x3w", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", 0.0, 1.0),
                     ("uniform", 0.0, 1.0), 4700 + Nc)

@@ -36,12 +36,12 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(kernel, kind,
     out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
     assert mx.last_device_status() == mx.OK
 
-    monkeypatch.setenv("MAXDNN_TEST_MISSING_ARRIVAL", "1")     # CTA 0 waits for an arrival that never comes
+    mx.set_option("TEST_MISSING_ARRIVAL", 1)     # CTA 0 waits for an arrival that never comes
     assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # the launch itself succeeds
     assert mx.last_device_status() == mx.DEVICE_TIMEOUT               # ...the kernel gave up waiting
     assert mx.last_device_status() == mx.OK                           # reading clears the word
 
-    monkeypatch.delenv("MAXDNN_TEST_MISSING_ARRIVAL")
+    mx.unset_option("TEST_MISSING_ARRIVAL")
     assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK          # same context, next call
     assert mx.last_device_status() == mx.OK
     ref = oracle.conv_fprop(ref_in, ref_f, stride=w.stride, pad=w.pad, alpha=w.alpha)
@@ -61,11 +61,11 @@ def test_chunked_kernel_wait_runs_out_and_the_context_survives(No, monkeypatch):
     ws = torch.empty(mx.conv_fprop_tf32x3_workspace(d), dtype=torch.uint8, device="cuda")
     out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
     assert mx.last_device_status() == mx.OK
-    monkeypatch.setenv("MAXDNN_TEST_MISSING_ARRIVAL", "1")
+    mx.set_option("TEST_MISSING_ARRIVAL", 1)
     mx.conv_fprop_tf32x3(d, x, f, out, ws)
     assert mx.last_device_status() == mx.DEVICE_TIMEOUT
     assert mx.last_device_status() == mx.OK
-    monkeypatch.delenv("MAXDNN_TEST_MISSING_ARRIVAL")
+    mx.unset_option("TEST_MISSING_ARRIVAL")
     mx.conv_fprop_tf32x3(d, x, f, out, ws)
     assert mx.last_device_status() == mx.OK
     ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha)
