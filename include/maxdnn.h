@@ -120,7 +120,19 @@ typedef struct maxdnn_plan_info {
   int32_t n_tiles;     /* tiles in the whole problem */
   int32_t grid;        /* persistent CTAs launched */
   int32_t smem_bytes;  /* dynamic shared memory per CTA */
+  int32_t tile_cols;   /* columns the kernel instance is built for (fp32: 128 or 256) */
+  int32_t pair;        /* tensor kernels: 1 = two-SM tiles of 256 filters */
+  int32_t split_tiles; /* fp32 kernel: tiles of the last, partly filled wave whose K steps
+                          are dealt out over all CTAs (0 = every tile on one CTA) */
 } maxdnn_plan_info;
+
+/* One unit of a CTA's work in the fp32 kernel: K steps [s0, s1) of `tile`.  kind 0: the
+ * whole tile; 1: a contribution of partial sums to a tile of the split tail; 2: the piece
+ * that holds the tile's last K step, adds the other CTAs' partial sums in CTA order and
+ * stores the tile. */
+typedef struct maxdnn_work_item {
+  int32_t tile, s0, s1, kind;
+} maxdnn_work_item;
 
 /* Host-only: fills *info and, if steps != NULL, up to max_steps table entries
  * (HOST memory, caller-owned).  Needs no GPU when sm_count > 0 is given
@@ -129,6 +141,17 @@ typedef struct maxdnn_plan_info {
 maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel_kind kind,
                                      int32_t sm_count, maxdnn_plan_info* info,
                                      maxdnn_kstep* steps, int32_t max_steps);
+
+/* Host-only: the work items of CTA `cta` in the fp32 kernel's plan for `desc` on
+ * `sm_count` SMs, in the order the CTA walks them (the paper's kernel gives every block
+ * one output coordinate, Section 3.2; here persistent CTAs walk lists of tiles, and the
+ * last, partly filled wave of tiles may be split along K — maxdnn_conv_fprop does that
+ * whenever the stream's workspace is available; maxdnn_conv_plan_query reports the same
+ * plan).  Writes up to max_items items (HOST memory) and their number to *n_items.
+ * INVALID_VALUE for a cta outside the plan's grid. */
+maxdnn_status maxdnn_conv_plan_items(const maxdnn_conv_desc* desc, int32_t sm_count, int32_t cta,
+                                     maxdnn_work_item* items, int32_t max_items,
+                                     int32_t* n_items);
 
 /*
  * FPROP with exact fp32 arithmetic (Sections 3.1-3.2: register-blocked
@@ -377,8 +400,9 @@ maxdnn_status maxdnn_last_device_status(void* cuda_stream);
  * Section 3.3 measures efficiency in processor clocks.  With option KERNEL_CLOCK set to 1,
  * maxdnn_conv_fprop has every CTA of its kernel measure its own elapsed SM cycles
  * (clock64) and nanoseconds (%globaltimer) from its first instruction to its last store,
- * and keeps the maxima over the CTAs of the LATEST launch in the status block (a memset of
- * those two words is enqueued ahead of the kernel).  This call synchronises `cuda_stream`
+ * and keeps the maxima over the CTAs of the LATEST call in the status block (a memset of
+ * those words is enqueued ahead of the kernel; a plan that runs its split tail as a second
+ * kernel reports the sum of the two kernels' maxima).  This call synchronises `cuda_stream`
  * and returns them: sm_cycles / nanoseconds is the SM clock the kernel ran at, and
  * C / (2 * 128 * SMs * sm_cycles) the paper's clock-independent efficiency.  Both are 0 if
  * the option was off.  32-bit counters: kernels of up to about two seconds.
@@ -394,7 +418,7 @@ maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanosecond
  * (0: never split tail tiles along K), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM
  * tiles), UMMA_MERGE, UMMA_STAGE_KB, UMMA_COLS, WGRAD_SPLITS, WGRAD_PAIR, SM_COUNT (SM
  * count for host-only workspace queries), X3_CHUNK_ROWS, DEBUG_STATUS, KERNEL_CLOCK (see
- * maxdnn_last_kernel_clock), FFMA_LANES (0: 16-byte operand loads in the fp32 kernel), and
+ * maxdnn_last_kernel_clock), and
  * TEST_MISSING_ARRIVAL (test hook: CTA 0's "full" barriers expect an arrival that
  * never comes, so a bounded wait runs out).  The environment variable MAXDNN_<name>
  * gives an option its initial value; the environment is read once, at the first use of

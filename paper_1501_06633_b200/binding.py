@@ -10,7 +10,7 @@ import os
 from typing import Optional
 
 __all__ = [
-    "MaxdnnError", "ConvDesc", "PlanInfo", "KStep", "KERNEL_FP32", "KERNEL_TF32", "KERNEL_BF16",
+    "MaxdnnError", "ConvDesc", "PlanInfo", "KStep", "WorkItem", "conv_plan_items", "KERNEL_FP32", "KERNEL_TF32", "KERNEL_BF16",
     "OK", "INVALID_VALUE", "NOT_SUPPORTED", "CUDA_ERROR", "DEVICE_TIMEOUT",
     "library_path", "load_library", "status_string", "conv_out_dims", "conv_flops",
     "conv_in_elems", "conv_filt_elems", "conv_out_elems", "conv_plan_query", "conv_fprop",
@@ -48,6 +48,7 @@ EXPORTED_SYMBOLS = [
     "maxdnn_conv2_bprop_filter_workspace", "maxdnn_conv2_bprop_filter",
     "maxdnn_last_device_status_noalloc", "maxdnn_set_option", "maxdnn_unset_option",
     "maxdnn_get_option", "maxdnn_reset_options", "maxdnn_last_kernel_clock",
+    "maxdnn_conv_plan_items",
 ]
 
 
@@ -93,13 +94,22 @@ class KStep(ctypes.Structure):
 class PlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "Ho", "Wo", "tile_m", "tile_px", "tile_n", "kc", "kwc", "n_ksteps", "stages", "n_tiles",
-        "grid", "smem_bytes")]
+        "grid", "smem_bytes", "tile_cols", "pair", "split_tiles")]
+
+
+class WorkItem(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("tile", "s0", "s1", "kind")]
 
 
 _lib = None
 
 
 def library_path() -> str:
+    """The in-tree library, or the file named by the environment variable MAXDNN_LIBRARY
+    (another build of the same sources, e.g. with different compile-time switches)."""
+    override = os.environ.get("MAXDNN_LIBRARY")
+    if override:
+        return override
     return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmaxdnn.so")
 
 
@@ -127,6 +137,9 @@ def load_library():
     lib.maxdnn_conv_plan_query.restype = ctypes.c_int
     lib.maxdnn_conv_plan_query.argtypes = [P(ConvDesc), ctypes.c_int, ctypes.c_int32, P(PlanInfo),
                                            P(KStep), ctypes.c_int32]
+    lib.maxdnn_conv_plan_items.restype = ctypes.c_int
+    lib.maxdnn_conv_plan_items.argtypes = [P(ConvDesc), ctypes.c_int32, ctypes.c_int32, P(WorkItem),
+                                           ctypes.c_int32, P(ctypes.c_int32)]
     for name in ("maxdnn_conv_fprop", "maxdnn_conv_fprop_tf32", "maxdnn_conv_fprop_bf16",
                  "maxdnn_conv_fprop_noalloc"):
         getattr(lib, name).restype = ctypes.c_int
@@ -230,6 +243,15 @@ def conv_plan_query(desc: ConvDesc, kind: int = KERNEL_FP32, sm_count: int = 148
                                                  ctypes.byref(info), steps, 1024),
            "maxdnn_conv_plan_query")
     return info, [steps[i] for i in range(info.n_ksteps)]
+
+
+def conv_plan_items(desc: ConvDesc, cta: int, sm_count: int = 148):
+    """The work items [(tile, s0, s1, kind)...] of one CTA of the fp32 kernel's plan."""
+    items = (WorkItem * 4096)()
+    n = ctypes.c_int32(0)
+    _check(load_library().maxdnn_conv_plan_items(ctypes.byref(desc), int(sm_count), int(cta), items,
+                                                 4096, ctypes.byref(n)), "maxdnn_conv_plan_items")
+    return [(items[i].tile, items[i].s0, items[i].s1, items[i].kind) for i in range(min(n.value, 4096))]
 
 
 def _stream_ptr(stream) -> Optional[int]:

@@ -41,7 +41,7 @@ struct FfmaArgs {
   // runs out and the kernel reports kDevTimeoutFull instead of hanging.
   uint32_t test_missing_arrival;
   // Non-zero: every CTA adds its elapsed SM cycles and nanoseconds (first instruction to
-  // last store) to words 2 and 3 of the status block with atomicMax — the elapsed
+  // last store) to words 2 and 3 (split-tail kernel: 4 and 5) of the status block with atomicMax — the elapsed
   // processor clocks of Section 3.3's efficiency formula, measured inside the kernel.
   uint32_t clock_stamp;
   // Split tail (g.sk_tiles > 0): one slot of tile_m x tile_cols partial sums per CTA, and
@@ -64,49 +64,10 @@ struct FfmaArgs {
 // contributing piece before its finishing piece, so a finisher waits only for CTAs with
 // lower numbers, which never wait for it.
 // ---------------------------------------------------------------------------------------
-enum FfmaItemKind : int { kItemWhole = 0, kItemContribute = 1, kItemFinish = 2 };
-
-struct FfmaItem {
-  int tile, s0, s1, kind;
-};
-
-// K-step range of CTA `cta` in the split tail: units [u0, u1) of sk_units.
-__device__ __forceinline__ void sk_range(const ConvGeom& g, int cta, int grid, int& u0, int& u1) {
-  u0 = (int)(((long long)cta * g.sk_units) / grid);
-  u1 = (int)(((long long)(cta + 1) * g.sk_units) / grid);
-}
-
-// The k-th item of this CTA, or false when there is none.
+// The item arithmetic itself (ffma_item_at, sk_range) lives in plan.h so that the host can
+// list a CTA's items too.
 __device__ __forceinline__ bool ffma_item(const ConvGeom& g, int k, FfmaItem& it) {
-  const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
-  const int first = g.tile_begin + cta;
-  const int n_whole = first < g.sk_first ? (g.sk_first - first + grid - 1) / grid : 0;
-  if (k < n_whole) {
-    it.tile = first + k * grid; it.s0 = 0; it.s1 = g.n_ksteps; it.kind = kItemWhole;
-    return true;
-  }
-  if (g.sk_tiles <= 0) return false;
-  int u0, u1;
-  sk_range(g, cta, grid, u0, u1);
-  if (u1 <= u0) return false;
-  const int n = g.n_ksteps;
-  const int ta = u0 / n;                       // tile (within the tail) where the range starts
-  const int a0 = u0 - ta * n;
-  const bool two = u1 > (ta + 1) * n;          // the range runs on into tile ta + 1
-  int piece = k - n_whole;
-  if (two) {
-    if (piece == 0) {                          // contribution to the next tile first
-      it.tile = g.sk_first + ta + 1; it.s0 = 0; it.s1 = u1 - (ta + 1) * n; it.kind = kItemContribute;
-      return true;
-    }
-    --piece;
-  }
-  if (piece != 0) return false;
-  it.tile = g.sk_first + ta;
-  it.s0 = a0;
-  it.s1 = two ? n : u1 - ta * n;
-  it.kind = it.s1 < n ? kItemContribute : (a0 == 0 ? kItemWhole : kItemFinish);
-  return true;
+  return ffma_item_at(g, (int)gridDim.x, (int)blockIdx.x, k, it);
 }
 
 template <int MR, int NR>
@@ -195,17 +156,27 @@ __device__ __forceinline__ void fma_block(const Frag<MR, NR>& f, float2 (&P)[MR 
   }
 }
 
-// Producer state: which (item, K step) is loaded next, into which ring stage.
+// Producer state: which K step of which tile is loaded next, into which ring stage.  The
+// whole-tile kernel (SPLIT = false) walks tiles tile_begin + CTA, + grid, ... below tile_end,
+// all K steps of each; the split-tail kernel walks this CTA's work items.
+template <bool SPLIT>
 struct FfmaProducer {
-  int item, step, step_end, stage;   // step_end <= step: no work left
-  uint32_t phase;
+  int item, step, step_end, stage;   // item: tile number (whole tiles) or item number (split)
+  uint32_t phase;                    // step_end <= step: no work left
   int o0, n0, h0, w0;
 
   __device__ __forceinline__ void set_item(const ConvGeom& g, int mt) {
-    FfmaItem it;
-    if (!ffma_item(g, item, it)) { step = 0; step_end = -1; return; }
-    step = it.s0; step_end = it.s1;
-    int r = it.tile;
+    int r;
+    if constexpr (SPLIT) {
+      FfmaItem it;
+      if (!ffma_item(g, item, it)) { step = 0; step_end = -1; return; }
+      step = it.s0; step_end = it.s1;
+      r = it.tile;
+    } else {
+      if (item >= g.tile_end) { step = 0; step_end = -1; return; }
+      step = 0; step_end = g.n_ksteps;
+      r = item;
+    }
     const int ob = r % g.o_blocks; r /= g.o_blocks;
     const int nch = r % g.n_chunks; r /= g.n_chunks;
     const int xr = r % g.x_runs;
@@ -217,7 +188,8 @@ struct FfmaProducer {
   }
 
   __device__ __forceinline__ void init(const ConvGeom& g, int mt) {
-    item = 0; stage = 0; phase = 0;
+    item = SPLIT ? 0 : g.tile_begin + (int)blockIdx.x;
+    stage = 0; phase = 0;
     o0 = n0 = h0 = w0 = 0;
     set_item(g, mt);
   }
@@ -247,7 +219,7 @@ struct FfmaProducer {
     }
     if (++stage == g.stages) { stage = 0; phase ^= 1u; }
     if (++step == step_end) {
-      ++item;
+      item += SPLIT ? 1 : (int)gridDim.x;
       set_item(g, mt);
     }
     return true;
@@ -281,9 +253,15 @@ __device__ __noinline__ bool wait_peer_flag(const uint32_t* flag, uint32_t epoch
   return false;
 }
 
+
+
 #define MAXDNN_ROW(R) a_ptr + (R) * Mt, b_ptr, (R) * b_pitch
 
-template <int MR, int NR, bool FIXED, bool W64>
+// SPLIT = false: whole tiles [tile_begin, tile_end).  SPLIT = true: this CTA's pieces of the
+// split tail (launched after the whole-tile kernel on the same stream; work items as if
+// tile_begin were the first split tile).  Operands come by 8-byte loads for the blocks of
+// 16 columns and by 16-byte loads for the others (which is faster was measured per block).
+template <int MR, int NR, bool FIXED, bool SPLIT>
 __global__ void __launch_bounds__(ffma_threads(MR, NR), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
@@ -292,6 +270,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   constexpr int Nt = 16 * NR;           // columns per tile
   constexpr int NH = NR / 4;            // float4 column groups per thread
   constexpr bool INLINE = ffma_inline_producer(MR, NR);
+  constexpr bool W64 = NR == 16;
   extern __shared__ uint8_t smem_raw[];
   const ConvGeom& g = args.g;
 
@@ -321,7 +300,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       mbar_init(full_bar + 8u * s, 1 + extra);
       mbar_init(empty_bar + 8u * s, kFfmaConsumerWarps);
     }
-    mbar_init(sk_bar, kFfmaConsumerWarps);
+    if constexpr (SPLIT) mbar_init(sk_bar, kFfmaConsumerWarps);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -335,7 +314,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       if (lane == 0) {
         prefetch_tensormap(&map_filt);
         prefetch_tensormap(&map_in);
-        FfmaProducer p;
+        FfmaProducer<SPLIT> p;
         p.init(g, Mt);
         bool ok = true;
         while (ok && p.has_work(g))
@@ -348,14 +327,16 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   }
 
   // -------------------------------------------------------------- consumers
-  FfmaProducer prod;          // used by warp 0 only, and only when INLINE
+  // Producer state of the INLINE variants (registers: kept in shared memory it cost the
+  // large blocks 3 %, the loads sitting in warp 0's instruction stream).
+  FfmaProducer<SPLIT> prod;
   bool prod_ok = true;
-  prod.init(g, Mt);
   if constexpr (INLINE) {
     if (warp == 0) {
       if (lane == 0) {
         prefetch_tensormap(&map_filt);
         prefetch_tensormap(&map_in);
+        prod.init(g, Mt);
         for (int s = 0; s + 2 < stages && prod_ok && prod.has_work(g); ++s)
           prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off, base + b_off,
                                                full_bar, empty_bar, Mt);
@@ -369,20 +350,27 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   const int tn = wn * 8 + (lane & 7);    // 0..15 along the column axis
   const int a_elem = (MR % 4 == 0) ? 4 * to : 2 * to;
 
-  // This thread's groups of four columns -> (pixel, image) and smem offset.
+  // Offset (in floats, inside a stage) of this thread's groups of four columns.  Group h is
+  // column 4 tn + 64 h of the tile = (pixel, image) (col / tile_n, col % tile_n); with one box
+  // per stage the columns of a row are contiguous, else a pixel's box starts b_slot_bytes
+  // after its neighbour's.  (The epilogue recomputes pixel and image from the column.)
   const int used_cols = g.tile_px * g.tile_n;
-  int col_px[NH], col_n[NH];
   uint32_t b_elem[NH];
+  // (pixel, image) of each group: kept in registers by the small blocks, recomputed in the
+  // epilogue by the large ones, which have no registers to spare
+  int col_px[INLINE ? 1 : NH], col_n[INLINE ? 1 : NH];
 #pragma unroll
   for (int h = 0; h < NH; ++h) {
     const int col = 4 * tn + 64 * h;
-    const bool live = col < used_cols;
-    col_px[h] = live ? col / g.tile_n : -1;
-    col_n[h] = live ? col % g.tile_n : 0;
+    if constexpr (!INLINE) {
+      col_px[h] = col < used_cols ? col / g.tile_n : -1;
+      col_n[h] = col < used_cols ? col % g.tile_n : 0;
+    }
     if (FIXED)
       b_elem[h] = (uint32_t)col;
     else
-      b_elem[h] = live ? (uint32_t)(col_px[h] * (g.b_slot_bytes >> 2) + col_n[h]) : 0u;
+      b_elem[h] = col < used_cols
+                      ? (uint32_t)((col / g.tile_n) * (g.b_slot_bytes >> 2) + col % g.tile_n) : 0u;
   }
   const int b_pitch = FIXED ? Nt : g.tile_n;   // floats between patch rows
 
@@ -390,9 +378,11 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   uint32_t phase = 0;
   bool ok = true;
 
-  FfmaItem item;
-  for (int item_no = 0; ok && ffma_item(g, item_no, item); ++item_no) {
-    const int tile = item.tile;
+  // One work item: K steps [s0, s1) of `tile` into fresh accumulators, then what its kind
+  // asks for.  The instance with SPLIT = false is the whole-tile one (all K steps, plain
+  // epilogue): none of the split tail's code or state is part of it, so the loop that walks
+  // whole tiles is compiled exactly as a kernel without a split tail would be.
+  auto run_item = [&](const int tile, const int s0, const int s1, const int kind) {
     float2 P[MR / 2][NR / 2], Q[MR / 2][NR / 2];
 #pragma unroll
     for (int i = 0; i < MR / 2; ++i)
@@ -404,7 +394,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
     Frag<MR, NR> f0, f1;
     ok = mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull);
-    if (!ok) break;
+    if (!ok) return;
     const float* a_ptr;
     const float* b_ptr[NH];
     auto point_at_stage = [&](int st) {
@@ -416,7 +406,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     point_at_stage(stage);
     load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(0));
 
-    for (int s = item.s0; s < item.s1; ++s) {
+    for (int s = s0; s < s1; ++s) {
       if constexpr (INLINE) {
         // Refill the slot this CTA finished two steps ago (every warp has released it
         // by now, so the wait does not hold warp 0 back) with the K step that is
@@ -464,7 +454,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       // the next stage into the other buffer before computing it.
       const int cur_stage = stage;
       if (++stage == stages) { stage = 0; phase ^= 1u; }
-      const bool more = s + 1 < item.s1;
+      const bool more = s + 1 < s1;
       if (more) {
         ok = mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull);
         if (!ok) break;
@@ -481,58 +471,64 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar + 8u * cur_stage);
     }
-    if (!ok) break;
+    if (!ok) return;
 
-    // ------------------------------------------------- split tail: partial sums
-    // A slot holds a thread's accumulators as float4 {P.x, P.y, Q.x, Q.y}, element
-    // [pair index][thread], so that a warp's store of one pair index is one 512-byte run.
-    constexpr int kPairs = (MR / 2) * (NR / 2);
-    if (item.kind == kItemContribute) {
-      float4* slot = reinterpret_cast<float4*>(args.sk_partial) +
-                     (size_t)blockIdx.x * (kPairs * 256) + threadIdx.x;
-#pragma unroll
-      for (int i = 0; i < MR / 2; ++i)
-#pragma unroll
-        for (int j = 0; j < NR / 2; ++j)
-          __stcg(slot + (i * (NR / 2) + j) * 256, make_float4(P[i][j].x, P[i][j].y, Q[i][j].x, Q[i][j].y));
-      __threadfence();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(sk_bar);
-      if (threadIdx.x == 0) {
-        // every consumer warp has stored and fenced: publish the slot under this launch's epoch
-        if (mbar_wait(sk_bar, 0, args.wc, kDevTimeoutPeer))
-          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(args.sk_flags + blockIdx.x),
-                       "r"(args.wc.epoch) : "memory");
-      }
-      continue;
-    }
-    if (item.kind == kItemFinish) {
-      // the CTAs below this one whose ranges hold the tile's earlier K steps, in order
-      const int grid = (int)gridDim.x;
-      const int first_unit = (tile - g.sk_first) * g.n_ksteps;
-      int j = (int)(((long long)first_unit * grid) / g.sk_units);
-      int u0, u1;
-      sk_range(g, j, grid, u0, u1);
-      while (j > 0 && u0 > first_unit) { --j; sk_range(g, j, grid, u0, u1); }
-      while (u1 <= first_unit) { ++j; sk_range(g, j, grid, u0, u1); }
-      for (; j < (int)blockIdx.x && ok; ++j) {
-        sk_range(g, j, grid, u0, u1);
-        if (u1 <= u0) continue;                      // a CTA without a share
-        bool ready = true;
-        if (lane == 0) ready = wait_peer_flag(args.sk_flags + j, args.wc.epoch, args.wc);
-        ready = __shfl_sync(0xffffffffu, ready ? 1 : 0, 0) != 0;
-        if (!ready) { ok = false; break; }
-        const float4* slot = reinterpret_cast<const float4*>(args.sk_partial) +
-                             (size_t)j * (kPairs * 256) + threadIdx.x;
+    if constexpr (SPLIT) {
+      // ----------------------------------------------- split tail: partial sums
+      // A slot holds a thread's accumulators as float4 {P.x, P.y, Q.x, Q.y}, element
+      // [pair index][thread], so that a warp's store of one pair index is one 512-byte run.
+      constexpr int kPairs = (MR / 2) * (NR / 2);
+      if (kind == kItemContribute) {
+        float4* slot = reinterpret_cast<float4*>(args.sk_partial) +
+                       (size_t)blockIdx.x * (kPairs * 256) + threadIdx.x;
 #pragma unroll
         for (int i = 0; i < MR / 2; ++i)
 #pragma unroll
-          for (int jj = 0; jj < NR / 2; ++jj) {
-            const float4 v = __ldcg(slot + (i * (NR / 2) + jj) * 256);
-            P[i][jj].x += v.x; P[i][jj].y += v.y; Q[i][jj].x += v.z; Q[i][jj].y += v.w;
-          }
+          for (int j = 0; j < NR / 2; ++j)
+            __stcg(slot + (i * (NR / 2) + j) * 256,
+                   make_float4(P[i][j].x, P[i][j].y, Q[i][j].x, Q[i][j].y));
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sk_bar);
+        if (threadIdx.x == 0) {
+          // every consumer warp has stored and fenced: publish the slot under this launch's epoch
+          if (mbar_wait(sk_bar, 0, args.wc, kDevTimeoutPeer))
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(args.sk_flags + blockIdx.x),
+                         "r"(args.wc.epoch) : "memory");
+        }
+        return;
       }
-      if (!ok) break;
+      if (kind == kItemFinish) {
+        // the CTAs below this one whose ranges hold the tile's earlier K steps, in order
+        const int grid = (int)gridDim.x;
+        const int first_unit = (tile - g.sk_first) * g.n_ksteps;
+        int j = (int)(((long long)first_unit * grid) / g.sk_units);
+        int u0, u1;
+        sk_range(g, j, grid, &u0, &u1);
+        while (j > 0 && u0 > first_unit) { --j; sk_range(g, j, grid, &u0, &u1); }
+        while (u1 <= first_unit) { ++j; sk_range(g, j, grid, &u0, &u1); }
+        for (; j < (int)blockIdx.x && ok; ++j) {
+          sk_range(g, j, grid, &u0, &u1);
+          if (u1 <= u0) continue;                      // a CTA without a share
+          bool ready = true;
+          if (lane == 0) ready = wait_peer_flag(args.sk_flags + j, args.wc.epoch, args.wc);
+          ready = __shfl_sync(0xffffffffu, ready ? 1 : 0, 0) != 0;
+          __syncwarp();          // lane 0's acquire orders the other lanes' reads of the slot
+          if (!ready) { ok = false; break; }
+          const float4* slot = reinterpret_cast<const float4*>(args.sk_partial) +
+                               (size_t)j * (kPairs * 256) + threadIdx.x;
+#pragma unroll
+          for (int i = 0; i < MR / 2; ++i)
+#pragma unroll
+            for (int jj = 0; jj < NR / 2; ++jj) {
+              const float4 v = __ldcg(slot + (i * (NR / 2) + jj) * 256);
+              P[i][jj].x += v.x; P[i][jj].y += v.y; Q[i][jj].x += v.z; Q[i][jj].y += v.w;
+              // at most four loads in flight: the accumulators leave no room for more
+              if ((jj & 3) == 3) asm volatile("" ::: "memory");
+            }
+        }
+        if (!ok) return;
+      }
     }
 
     // ---------------------------------------------------------- epilogue
@@ -557,9 +553,18 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         const int i2 = i >> 1, ia = i & 1;
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-          const int x = x0 + col_px[h];
-          const int n = n0 + col_n[h];
-          if (col_px[h] < 0 || x >= g.Wo || n >= g.Nb) continue;
+          int x, n;
+          if constexpr (INLINE) {
+            const int col = 4 * tn + 64 * h;
+            if (col >= used_cols) continue;
+            x = x0 + col / g.tile_n;
+            n = n0 + col % g.tile_n;
+          } else {
+            if (col_px[h] < 0) continue;
+            x = x0 + col_px[h];
+            n = n0 + col_n[h];
+          }
+          if (x >= g.Wo || n >= g.Nb) continue;
           float4 v;
           // columns 4h .. 4h+3 of this row: j = 2*j2 + jb with j2 = 2h, 2h+1
           v.x = ia == 0 ? P[i2][2 * h].x : Q[i2][2 * h].y;
@@ -572,14 +577,24 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         }
       }
     }
+  };
+
+  if constexpr (SPLIT) {
+    FfmaItem item;
+    for (int k = 0; ok && ffma_item(g, k, item); ++k)
+      run_item(item.tile, item.s0, item.s1, item.kind);
+  } else {
+    const int n_ksteps = g.n_ksteps;
+    for (int tile = g.tile_begin + blockIdx.x; tile < g.tile_end && ok; tile += gridDim.x)
+      run_item(tile, 0, n_ksteps, (int)kItemWhole);
   }
 
   if constexpr (INLINE) {
     if (warp == 0 && lane == 0 && !(ok && prod_ok)) prod.drain(g, full_bar);
   }
   if (args.clock_stamp != 0 && threadIdx.x == 0 && args.wc.status) {
-    atomicMax(args.wc.status + 2, (uint32_t)(clock64() - stamp_cycles));
-    atomicMax(args.wc.status + 3, (uint32_t)(globaltimer_ns() - stamp_ns));
+    atomicMax(args.wc.status + (SPLIT ? 4 : 2), (uint32_t)(clock64() - stamp_cycles));
+    atomicMax(args.wc.status + (SPLIT ? 5 : 3), (uint32_t)(globaltimer_ns() - stamp_ns));
   }
 }
 #undef MAXDNN_ROW

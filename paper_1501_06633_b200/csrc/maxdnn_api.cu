@@ -43,6 +43,13 @@ struct DeviceState {
   std::atomic<bool> wgrad_umma_attr[4];
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
+  // Workspaces of the fp32 kernel's split tail, one per stream that has used one (work on
+  // one stream runs in order, so its launches can share a workspace; launches on different
+  // streams may overlap and must not).  Allocated on a stream's first such call.
+  struct SplitWs { cudaStream_t stream; void* ptr; };
+  SplitWs split_ws[8] = {};
+  int n_split_ws = 0;
+  std::mutex split_mu;
   cudaStream_t aux[3] = {nullptr, nullptr, nullptr};
   cudaEvent_t ev_fork = nullptr;
   cudaEvent_t ev_join[3] = {nullptr, nullptr, nullptr};
@@ -66,6 +73,34 @@ maxdnn_status ensure_smem_attr(DeviceState* ds, std::atomic<bool>* done, Kern ke
   }
   done->store(true, std::memory_order_release);
   return MAXDNN_OK;
+}
+
+// The split-tail workspace of `stream` on this device, or null when there is none and none
+// can be had now: the stream is being captured (no allocation inside a capture), all eight
+// slots belong to other streams, or the allocation fails.  The caller then plans without a
+// split.
+void* split_workspace(DeviceState* ds, cudaStream_t stream) {
+  std::lock_guard<std::mutex> lk(ds->split_mu);
+  for (int i = 0; i < ds->n_split_ws; ++i)
+    if (ds->split_ws[i].stream == stream) return ds->split_ws[i].ptr;
+  if (ds->n_split_ws >= 8) return nullptr;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (cap != cudaStreamCaptureStatusNone) return nullptr;
+  void* p = nullptr;
+  const size_t bytes = ffma_split_bytes(ds->sm_count);
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  // flags start at 0; a launch's epoch is never 0
+  if (cudaMemset(static_cast<uint8_t*>(p) + ffma_split_flags_offset(ds->sm_count), 0,
+                 bytes - ffma_split_flags_offset(ds->sm_count)) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(p);
+    return nullptr;
+  }
+  ds->split_ws[ds->n_split_ws].stream = stream;
+  ds->split_ws[ds->n_split_ws].ptr = p;
+  ++ds->n_split_ws;
+  return p;
 }
 
 // The status block and a fresh epoch for one launch (never 0: word 1 of a cleared block).
@@ -185,10 +220,10 @@ struct PlanCache {
   }
 };
 
-template <int MR, int NR, bool FIXED, bool W64>
+template <int MR, int NR, bool FIXED, bool SPLIT>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
-  auto kern = ffma_conv_kernel<MR, NR, FIXED, W64>;
+  auto kern = ffma_conv_kernel<MR, NR, FIXED, SPLIT>;
   if (ensure_smem_attr(ds, &ds->ffma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   kern<<<args.g.grid, ffma_threads(MR, NR), args.g.smem_bytes, stream>>>(mf, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
@@ -196,19 +231,19 @@ maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, cons
   return MAXDNN_OK;
 }
 
-// Picks the kernel instance built for the plan's tile shape.
+// Picks the kernel instance built for the plan's tile shape: the whole-tile kernel, or
+// (split) the kernel that computes the split tail.
 maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
-                            const FfmaArgs& args, cudaStream_t stream) {
+                            const FfmaArgs& args, cudaStream_t stream, bool split = false) {
   const ConvGeom& g = args.g;
   const bool fx = g.fixed_pitch != 0;
-  const bool w64 = option(OPT_FFMA_LANES, 1) != 0;   // 8-byte operand loads (0: 16-byte loads)
-#define MAXDNN_FFMA_CASE(M, C, MR, NR, SLOT)                                             \
-  if (g.tile_m == (M) && g.tile_cols == (C)) {                                           \
-    if (w64)                                                                             \
-      return fx ? launch_ffma<MR, NR, true, true>(ds, (SLOT) + 16, mf, mi, args, stream) \
+#define MAXDNN_FFMA_CASE(M, C, MR, NR, SLOT)                                               \
+  if (g.tile_m == (M) && g.tile_cols == (C)) {                                             \
+    if (split)                                                                             \
+      return fx ? launch_ffma<MR, NR, true, true>(ds, (SLOT) + 16, mf, mi, args, stream)   \
                 : launch_ffma<MR, NR, false, true>(ds, (SLOT) + 17, mf, mi, args, stream); \
-    return fx ? launch_ffma<MR, NR, true, false>(ds, (SLOT), mf, mi, args, stream)       \
-              : launch_ffma<MR, NR, false, false>(ds, (SLOT) + 1, mf, mi, args, stream); \
+    return fx ? launch_ffma<MR, NR, true, false>(ds, (SLOT), mf, mi, args, stream)         \
+              : launch_ffma<MR, NR, false, false>(ds, (SLOT) + 1, mf, mi, args, stream);   \
   }
   MAXDNN_FFMA_CASE(256, 128, 16, 8, 0)
   MAXDNN_FFMA_CASE(128, 256, 8, 16, 2)
@@ -220,6 +255,27 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   MAXDNN_FFMA_CASE(32, 128, 2, 8, 12)
 #undef MAXDNN_FFMA_CASE
   return MAXDNN_NOT_SUPPORTED;
+}
+
+// The one or two launches of a plan: whole tiles, then (if the plan splits its last wave)
+// the split tail on the same stream.  `args` is modified (tile range) and restored.
+maxdnn_status launch_ffma_plan(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
+                               FfmaArgs& args, cudaStream_t stream) {
+  ConvGeom& g = args.g;
+  if (g.sk_tiles <= 0) return dispatch_ffma(ds, mf, mi, args, stream);
+  const int32_t begin = g.tile_begin, end = g.tile_end;
+  maxdnn_status st = MAXDNN_OK;
+  if (g.sk_first > begin) {
+    g.tile_end = g.sk_first;
+    st = dispatch_ffma(ds, mf, mi, args, stream);
+    g.tile_end = end;
+  }
+  if (st == MAXDNN_OK) {
+    g.tile_begin = g.sk_first;         // the split kernel's items start at the first split tile
+    st = dispatch_ffma(ds, mf, mi, args, stream, true);
+    g.tile_begin = begin;
+  }
+  return st;
 }
 
 maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt, float* out,
@@ -235,28 +291,35 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
   if (st != MAXDNN_OK) return st;
   if (!ds->sm100) return MAXDNN_NOT_SUPPORTED;
 
+  // A plan may split its tail wave along K when this stream has (or can get) a workspace.
+  void* split_ws = option(OPT_FFMA_STREAMK, 1) != 0 ? split_workspace(ds, stream) : nullptr;
   static thread_local PlanCache<FfmaArgs> cache;   // 4 KB tables: kept off the stack
   PlanKey key;
   memset(&key, 0, sizeof(key));
   key.d = cd;
   key.v[0] = ds->sm_count;
   key.v[1] = (int32_t)options_generation();
+  key.v[2] = split_ws != nullptr;
   key.valid = true;
   int slot = cache.find(key);
   if (slot < 0) {
     slot = cache.take();
     st = plan_ffma(cd, ds->sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS),
-                   &cache.args[slot].g, &cache.args[slot].table);
+                   &cache.args[slot].g, &cache.args[slot].table, split_ws != nullptr);
     if (st != MAXDNN_OK) return st;
     cache.key[slot] = key;
   }
   FfmaArgs& args = cache.args[slot];
   args.out = out;
+  args.sk_partial = static_cast<float*>(split_ws);
+  args.sk_flags = split_ws ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(split_ws) +
+                                                         ffma_split_flags_offset(ds->sm_count))
+                           : nullptr;
   args.wc = next_wait_ctx(ds);
   args.test_missing_arrival = (uint32_t)option(OPT_TEST_MISSING_ARRIVAL);   // see FfmaArgs
   args.clock_stamp = (uint32_t)option(OPT_KERNEL_CLOCK);
   if (args.clock_stamp != 0 &&
-      cudaMemsetAsync(ds->status + 2, 0, 8, stream) != cudaSuccess) {   // this launch's maxima
+      cudaMemsetAsync(ds->status + 2, 0, 16, stream) != cudaSuccess) {   // this call's maxima
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
@@ -283,7 +346,7 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
-  return dispatch_ffma(ds, mf, mi, args, stream);
+  return launch_ffma_plan(ds, mf, mi, args, stream);
 }
 
 maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const float* filt,
@@ -1261,6 +1324,8 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
   if (st != MAXDNN_OK) return st;
   if (ffma_scratch_bytes(args.g) > kStaticScratchBytes) return MAXDNN_NOT_SUPPORTED;
   args.out = out;
+  args.sk_partial = nullptr;       // no workspace here: the plan never splits its tail
+  args.sk_flags = nullptr;
   args.wc = next_wait_ctx(ds);
   args.test_missing_arrival = (uint32_t)option(OPT_TEST_MISSING_ARRIVAL);
   args.clock_stamp = 0;
@@ -1370,7 +1435,8 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   static thread_local KStepTable t;
   switch (kind) {
     case MAXDNN_KERNEL_FP32:
-      st = plan_ffma(dims_from(*desc), sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS), &g, &t);
+      st = plan_ffma(dims_from(*desc), sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS), &g, &t,
+                     true);
       break;
     case MAXDNN_KERNEL_TF32: st = plan_umma(dims_from(*desc), 4, sm_count, option(OPT_UMMA_KC), option(OPT_UMMA_PAIR), &g, &t); break;
     case MAXDNN_KERNEL_BF16: st = plan_umma(dims_from(*desc), 2, sm_count, option(OPT_UMMA_KC), option(OPT_UMMA_PAIR), &g, &t); break;
@@ -1381,8 +1447,39 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   info->tile_m = g.tile_m; info->tile_px = g.tile_px; info->tile_n = g.tile_n;
   info->kc = g.kc; info->kwc = g.kwc; info->n_ksteps = g.n_ksteps; info->stages = g.stages;
   info->n_tiles = g.n_tiles; info->grid = g.grid; info->smem_bytes = g.smem_bytes;
+  info->tile_cols = g.tile_cols; info->pair = g.pair;
+  info->split_tiles = kind == MAXDNN_KERNEL_FP32 ? g.sk_tiles : 0;
   if (steps)
     for (int i = 0; i < g.n_ksteps && i < max_steps; ++i) steps[i] = t.s[i];
+  return MAXDNN_OK;
+}
+
+maxdnn_status maxdnn_conv_plan_items(const maxdnn_conv_desc* desc, int32_t sm_count, int32_t cta,
+                                     maxdnn_work_item* items, int32_t max_items,
+                                     int32_t* n_items) {
+  if (!desc || !n_items || (max_items > 0 && !items)) return MAXDNN_INVALID_VALUE;
+  maxdnn_status st = check_desc(desc, nullptr, nullptr);
+  if (st != MAXDNN_OK) return st;
+  if (sm_count <= 0) {
+    DeviceState* ds = nullptr;
+    st = device_state(&ds);
+    if (st != MAXDNN_OK) return st;
+    sm_count = ds->sm_count;
+  }
+  static thread_local ConvGeom g;
+  static thread_local KStepTable t;
+  st = plan_ffma(dims_from(*desc), sm_count, option(OPT_FFMA_TILE_M), option(OPT_FFMA_COLS), &g, &t, true);
+  if (st != MAXDNN_OK) return st;
+  if (cta < 0 || cta >= g.grid) return MAXDNN_INVALID_VALUE;
+  int n = 0;
+  FfmaItem it;
+  while (ffma_item_at(g, g.grid, cta, n, it)) {
+    if (n < max_items) {
+      items[n].tile = it.tile; items[n].s0 = it.s0; items[n].s1 = it.s1; items[n].kind = it.kind;
+    }
+    ++n;
+  }
+  *n_items = n;
   return MAXDNN_OK;
 }
 
@@ -1655,14 +1752,14 @@ maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanosecond
   maxdnn_status st = device_state(&ds);
   if (st != MAXDNN_OK) return st;
   if (!ds->status || !sm_cycles || !nanoseconds) return MAXDNN_INVALID_VALUE;
-  uint32_t w[2] = {0, 0};
+  uint32_t w[4] = {0, 0, 0, 0};   // whole-tile kernel, split-tail kernel
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess ||
-      cudaMemcpy(w, ds->status + 2, 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaMemcpy(w, ds->status + 2, 16, cudaMemcpyDeviceToHost) != cudaSuccess) {
     cudaGetLastError();
     return MAXDNN_CUDA_ERROR;
   }
-  *sm_cycles = w[0];
-  *nanoseconds = w[1];
+  *sm_cycles = w[0] + w[2];
+  *nanoseconds = w[1] + w[3];
   return MAXDNN_OK;
 }
 

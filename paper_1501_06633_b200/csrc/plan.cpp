@@ -14,7 +14,7 @@ namespace maxdnn {
 // ---------------------------------------------------------------------------
 namespace {
 const char* const kOptionNames[OPT_COUNT] = {
-    "FFMA_TILE_M", "FFMA_COLS", "FFMA_LANES", "FFMA_KH", "FFMA_STREAMK",
+    "FFMA_TILE_M", "FFMA_COLS", "FFMA_KH", "FFMA_STREAMK",
     "UMMA_KC", "UMMA_PAIR", "UMMA_MERGE", "UMMA_STAGE_KB", "UMMA_COLS",
     "WGRAD_SPLITS", "WGRAD_PAIR", "SM_COUNT", "X3_CHUNK_ROWS", "DEBUG_STATUS",
     "KERNEL_CLOCK", "TEST_MISSING_ARRIVAL"};
@@ -214,8 +214,49 @@ static double pick_columns(const ConvDims& d, int Wo, int cols, int* nn_out, int
   return best_eff;
 }
 
+// K step of the fp32 kernel: kc channels of one filter tap, or (few channels) kc channels
+// of a whole filter row of Skw taps.
+static void ffma_kstep(const ConvDims& d, int* kc_out, int* kwc_out) {
+  int kc, kwc;
+  if (d.Nc >= 8) {
+    kwc = 1;
+    const int kc_max = 32;
+    kc = kc_max;
+    int best_pad = 1 << 30;
+    for (int c = kc_max; c >= 8; c -= 4) {
+      const int padded = ceil_div(d.Nc, c) * c;
+      if (padded < best_pad) { best_pad = padded; kc = c; }
+    }
+  } else {
+    kwc = d.Skw;
+    kc = 40 / d.Skw;
+    if (kc < 1) kc = 1;
+    if (kc > d.Nc) kc = d.Nc;
+  }
+  *kc_out = kc;
+  *kwc_out = kwc;
+}
+
+// Time of `tiles` tiles on `units` persistent CTAs, in tile times.  Without a split the
+// last, partly filled wave costs a whole tile time.  With the tail split along K (see
+// ffma_conv.cuh) it costs its share R / units plus the fix-up: every CTA writes or reads
+// back partial sums (a tile's accumulators: about 16 K rows' worth of time per slot) and a
+// finisher adds about units / R slots one after the other.
+static double ffma_waves(int64_t tiles, int units, int k_rows_per_tile, bool allow_split,
+                         bool* split_out) {
+  const int64_t W = tiles / units, R = tiles % units;
+  *split_out = false;
+  if (R == 0) return (double)W;
+  const double whole = (double)(W + 1);
+  if (!allow_split || k_rows_per_tile < 64) return whole;
+  const double slot = 16.0 / (double)k_rows_per_tile;
+  const double split = (double)W + (double)R / units + 0.03 + slot * (1.0 + (double)units / (double)R);
+  if (split < whole - 0.03) { *split_out = true; return split; }
+  return whole;
+}
+
 maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
-                        ConvGeom* g, KStepTable* t) {
+                        ConvGeom* g, KStepTable* t, bool allow_split) {
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
@@ -225,9 +266,14 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
   fill_geom(d, Ho, Wo, g);
 
-  // Tile shape: fewest SM-time units over whole waves of persistent CTAs.
+  // Tile shape: fewest SM-time units over the waves of persistent CTAs.
   double best_t = 1e300;
   int best_m = 0, best_cols = 0, best_nn = 0, best_T = 0;
+  bool best_split = false;
+  int kc0, kwc0;
+  ffma_kstep(d, &kc0, &kwc0);
+  const int k_rows = ceil_div(d.Nc, kc0) * kc0 * d.Skw * d.Skh;
+  if (option(OPT_FFMA_STREAMK, 1) == 0) allow_split = false;
   for (const FfmaShape& sh : kFfmaShapes) {
     if (force_tile_m > 0 && sh.m != force_tile_m) continue;
     if (force_cols > 0 && sh.cols != force_cols) continue;
@@ -236,9 +282,12 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
     pick_columns(d, Wo, sh.cols, &nn, &T);
     if (force_cols <= 0 && sh.cols > 128 && nn * T <= 128) continue;   // would not fill it
     const int64_t tiles = (int64_t)ceil_div(d.No, sh.m) * ceil_div(Wo, T) * Ho * ceil_div(d.Nb, nn);
-    const int64_t waves = (tiles + sm_count - 1) / sm_count;
-    const double tm = (double)waves * sh.m * sh.cols * sh.cost;
-    if (tm < best_t - 1e-9) { best_t = tm; best_m = sh.m; best_cols = sh.cols; best_nn = nn; best_T = T; }
+    bool split = false;
+    const double waves = ffma_waves(tiles, sm_count, k_rows, allow_split && tiles > sm_count, &split);
+    const double tm = waves * sh.m * sh.cols * sh.cost;
+    if (tm < best_t - 1e-9) {
+      best_t = tm; best_m = sh.m; best_cols = sh.cols; best_nn = nn; best_T = T; best_split = split;
+    }
   }
   if (best_m == 0) return MAXDNN_NOT_SUPPORTED;
   g->tile_m = best_m;
@@ -256,24 +305,9 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
 
   // K step: kc channels of one filter tap, or (few channels) kc channels of a
   // whole filter row of Sk taps.
-  int kc, kwc;
+  int kc = kc0, kwc = kwc0;
   // Tiles whose first consumer warp issues the copies keep one ring slot as slack.
   const bool inline_producer = (best_m / 16) * (best_cols / 16) >= 96;
-  if (d.Nc >= 8) {
-    kwc = 1;
-    const int kc_max = 32;
-    kc = kc_max;
-    int best_pad = 1 << 30;
-    for (int c = kc_max; c >= 8; c -= 4) {
-      const int padded = ceil_div(d.Nc, c) * c;
-      if (padded < best_pad) { best_pad = padded; kc = c; }
-    }
-  } else {
-    kwc = d.Skw;
-    kc = 40 / d.Skw;
-    if (kc < 1) kc = 1;
-    if (kc > d.Nc) kc = d.Nc;
-  }
   int n = 0;
   build_table(d, kc, kwc, t, &n);
   while (n > kMaxKSteps && kwc == 1 && kc < 256) {   // very deep filters: larger boxes
@@ -310,6 +344,18 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   g->stages = stages;
   g->smem_bytes = stages * stage + 1024;   // + barriers, + slack for alignment
   g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
+  // Split tail: the tiles of the last, partly filled wave (every K step of the table is
+  // dealt out, so the share of a CTA must be at least two steps).
+  g->sk_first = g->n_tiles;
+  g->sk_tiles = 0;
+  g->sk_units = 0;
+  const int tail = g->n_tiles % g->grid;
+  if (best_split && g->n_tiles > g->grid && tail > 0 && (int64_t)tail * n >= 2 * (int64_t)g->grid &&
+      (size_t)best_m * best_cols * 4 <= kFfmaSplitSlotBytes) {
+    g->sk_tiles = tail;
+    g->sk_first = g->n_tiles - tail;
+    g->sk_units = tail * n;
+  }
   return MAXDNN_OK;
 }
 

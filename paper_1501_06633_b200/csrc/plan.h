@@ -17,7 +17,7 @@ constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel pa
 // option in the process — never on the path of a call.  TEST_MISSING_ARRIVAL is the
 // exception: it has no environment variable and can only be set through the C ABI.
 enum OptionId : int {
-  OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_LANES, OPT_FFMA_KH, OPT_FFMA_STREAMK,
+  OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_KH, OPT_FFMA_STREAMK,
   OPT_UMMA_KC, OPT_UMMA_PAIR, OPT_UMMA_MERGE, OPT_UMMA_STAGE_KB, OPT_UMMA_COLS,
   OPT_WGRAD_SPLITS, OPT_WGRAD_PAIR, OPT_SM_COUNT, OPT_X3_CHUNK_ROWS, OPT_DEBUG_STATUS,
   OPT_KERNEL_CLOCK, OPT_TEST_MISSING_ARRIVAL, OPT_COUNT
@@ -89,6 +89,57 @@ struct ConvGeom {
 struct KStepTable {
   maxdnn_kstep s[kMaxKSteps];
 };
+
+#ifdef __CUDACC__
+#define MAXDNN_HD __host__ __device__ __forceinline__
+#else
+#define MAXDNN_HD inline
+#endif
+
+// Work items of the fp32 kernel (see ffma_conv.cuh): a whole tile, a contribution of
+// partial sums to a tile of the split tail, or the piece that finishes such a tile.
+enum FfmaItemKind : int { kItemWhole = 0, kItemContribute = 1, kItemFinish = 2 };
+struct FfmaItem {
+  int tile, s0, s1, kind;    // K steps [s0, s1) of `tile`
+};
+
+// K-step range of CTA `cta` in the split tail: units [u0, u1) of sk_units.
+MAXDNN_HD void sk_range(const ConvGeom& g, int cta, int grid, int* u0, int* u1) {
+  *u0 = (int)(((long long)cta * g.sk_units) / grid);
+  *u1 = (int)(((long long)(cta + 1) * g.sk_units) / grid);
+}
+
+// The k-th item of CTA `cta` of a grid of `grid` CTAs, or false when there is none.
+MAXDNN_HD bool ffma_item_at(const ConvGeom& g, int grid, int cta, int k, FfmaItem& it) {
+  const int first = g.tile_begin + cta;
+  const int n_whole = first < g.sk_first ? (g.sk_first - first + grid - 1) / grid : 0;
+  if (k < n_whole) {
+    it.tile = first + k * grid; it.s0 = 0; it.s1 = g.n_ksteps; it.kind = kItemWhole;
+    return true;
+  }
+  if (g.sk_tiles <= 0) return false;
+  int u0, u1;
+  sk_range(g, cta, grid, &u0, &u1);
+  if (u1 <= u0) return false;
+  const int n = g.n_ksteps;
+  const int ta = u0 / n;                       // tile (within the tail) where the range starts
+  const int a0 = u0 - ta * n;
+  const bool two = u1 > (ta + 1) * n;          // the range runs on into tile ta + 1
+  int piece = k - n_whole;
+  if (two) {
+    if (piece == 0) {                          // the contribution to the next tile comes first
+      it.tile = g.sk_first + ta + 1; it.s0 = 0; it.s1 = u1 - (ta + 1) * n; it.kind = kItemContribute;
+      return true;
+    }
+    --piece;
+  }
+  if (piece != 0) return false;
+  it.tile = g.sk_first + ta;
+  it.s0 = a0;
+  it.s1 = two ? n : u1 - ta * n;
+  it.kind = it.s1 < n ? kItemContribute : (a0 == 0 ? kItemWhole : kItemFinish);
+  return true;
+}
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int align_up(int a, int b) { return ceil_div(a, b) * b; }

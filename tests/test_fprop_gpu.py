@@ -110,6 +110,48 @@ def test_every_tile_shape(tile_m, cols, stride, monkeypatch):
     check_fp32(w)
 
 
+SPLIT = [
+    # shapes whose plan splits the last wave of tiles along K (more tiles than CTAs, a
+    # partly filled last wave), with the tile shape pinned so that every register block's
+    # partial-sum path runs: (dims, tile_m, cols)
+    ((128, 15, 13, 32, 128, 3, 1, 1, 1.0), 0, 0),
+    ((64, 24, 17, 24, 256, 3, 1, 1, 0.5), 0, 0),
+    ((128, 14, 12, 40, 200, 5, 1, 2, 1.0), 0, 0),
+    ((128, 16, 10, 64, 128, 3, 1, 1, 1.0), 0, 0),
+    ((128, 16, 10, 24, 96, 3, 1, 1, 1.0), 32, 128),
+    ((128, 16, 12, 24, 192, 3, 1, 1, 1.0), 96, 128),
+    ((128, 20, 18, 24, 256, 3, 1, 1, 1.0), 256, 128),
+    ((64, 40, 18, 40, 128, 3, 1, 1, 1.0), 128, 256),
+    ((64, 80, 36, 40, 64, 3, 2, 1, 1.0), 64, 256),
+    ((64, 40, 36, 16, 96, 3, 1, 1, 1.0), 96, 256),
+    ((128, 63, 59, 3, 96, 11, 4, 0, 1.0), 96, 128),
+]
+
+
+@pytest.mark.parametrize("dims,tile_m,cols", SPLIT, ids=lambda v: "x".join(str(x) for x in v)
+                         if isinstance(v, tuple) else str(v))
+def test_split_tail_fp32(dims, tile_m, cols):
+    """The tail wave split along K: contributions through the workspace, finishers adding
+    them in CTA order — against the oracle, and bitwise equal from run to run."""
+    if tile_m:
+        mx.set_option("FFMA_TILE_M", tile_m)
+        mx.set_option("FFMA_COLS", cols)
+    w = wl.Workload("split", *dims, ("uniform", -1.0, 1.0), ("uniform", -1.0, 1.0), 321)
+    d = mx.ConvDesc.make(*w.dims)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    info, _ = mx.conv_plan_query(d, mx.KERNEL_FP32, sms)
+    assert info.split_tiles > 0, "this shape is meant to have a split tail"
+    inp, filt = wl.make_inputs(w)
+    a = check_fp32(w, inp, filt)
+    b = run_fp32(w, inp, filt)
+    np.testing.assert_array_equal(a, b)
+    # and the same problem with the split switched off
+    mx.set_option("FFMA_STREAMK", 0)
+    info, _ = mx.conv_plan_query(d, mx.KERNEL_FP32, sms)
+    assert info.split_tiles == 0
+    check_fp32(w, inp, filt)
+
+
 def test_special_values_fp32():
     """Delta filter reproduces the map bit for bit; permuting filters permutes the output."""
     rng = np.random.default_rng(5)

@@ -234,3 +234,61 @@ def test_ragged_workspace_sizes():
     assert mx.conv_fprop_ragged_workspace(mx.ConvDesc.make(32, 14, 9, 16, 64, 3, 1, 1, 1.0)) == 0
     assert mx.conv_fprop_ragged_workspace(mx.ConvDesc.make(32, 14, 9, 16, 64, 3, 1, 1, 1.0),
                                           mx.KERNEL_BF16) > 0          # bf16 wants 64 images
+
+
+# ---------------------------------------------------------------------------
+# Split tail of the fp32 kernel: the K steps of the last, partly filled wave of tiles are
+# dealt out over all CTAs.  Host-only check of the work-item lists.
+# ---------------------------------------------------------------------------
+SPLIT_SHAPES = [wl.ALL[n].dims for n in ("first11x11s4", "mid5x5", "wide3x3", "large3x3",
+                                         "alexnet_conv4", "overfeat_L2", "overfeat_L5")] + [
+    (64, 20, 10, 64, 128, 3, 1, 1, 1.0),      # 200 tiles of 128 x 128 (or fewer, larger)
+    (128, 13, 13, 40, 96, 3, 1, 1, 1.0),
+    (32, 30, 30, 24, 64, 5, 2, 2, 1.0),
+]
+
+
+@pytest.mark.parametrize("dims", SPLIT_SHAPES, ids=lambda s: "x".join(str(v) for v in s))
+@pytest.mark.parametrize("sm_count", [148, 132, 7])
+def test_split_tail_items_cover_every_k_step_once(dims, sm_count):
+    d = mx.ConvDesc.make(*dims)
+    info, _ = mx.conv_plan_query(d, mx.KERNEL_FP32, sm_count)
+    n = info.n_ksteps
+    seen = {}                      # (tile, step) -> cta
+    finisher, contributors = {}, {}
+    for cta in range(info.grid):
+        items = mx.conv_plan_items(d, cta, sm_count)
+        kinds = [k for (_, _, _, k) in items]
+        assert kinds.count(1) <= 1 and kinds.count(2) <= 1
+        if 1 in kinds and 2 in kinds:
+            assert kinds.index(1) < kinds.index(2)          # contribute first, then finish
+        whole_done = False
+        for tile, s0, s1, kind in items:
+            assert 0 <= tile < info.n_tiles and 0 <= s0 < s1 <= n
+            if kind == 0:
+                assert (s0, s1) == (0, n) and not whole_done or tile >= info.n_tiles - info.split_tiles
+            else:
+                whole_done = True                           # split pieces come after whole tiles
+                assert tile >= info.n_tiles - info.split_tiles
+            if kind == 1:
+                assert s1 < n
+                contributors.setdefault(tile, []).append(cta)
+            if kind == 2:
+                assert s1 == n and s0 > 0
+                assert tile not in finisher
+                finisher[tile] = cta
+            for s in range(s0, s1):
+                assert (tile, s) not in seen, "K step computed twice"
+                seen[(tile, s)] = cta
+    assert len(seen) == info.n_tiles * n, "a K step is missing"
+    for tile, ctas in contributors.items():
+        assert tile in finisher, "partial sums nobody collects"
+        assert max(ctas) < finisher[tile]                   # a finisher waits for lower CTAs only
+        # the contributors are exactly the CTAs between the first one and the finisher that
+        # have a share at all: their steps are contiguous and ascend with the CTA number
+        steps = [(min(s for (t, s), c in seen.items() if t == tile and c == cta), cta) for cta in ctas]
+        assert steps == sorted(steps) and [c for _, c in steps] == sorted(ctas)
+    for tile in finisher:
+        assert tile in contributors
+    if info.split_tiles:
+        assert 0 < info.split_tiles < info.grid
