@@ -122,6 +122,8 @@ typedef struct maxdnn_plan_info {
   int32_t smem_bytes;  /* dynamic shared memory per CTA */
   int32_t tile_cols;   /* columns the kernel instance is built for (fp32: 128 or 256) */
   int32_t pair;        /* tensor kernels: 1 = two-SM tiles of 256 filters */
+  int32_t khc;         /* filter rows per K step (fp32 few-channel plans: a box spans khc rows,
+                          clipped at the filter's last row) */
   int32_t split_tiles; /* fp32 kernel: tiles of the last, partly filled wave whose K steps
                           are dealt out over all CTAs (0 = every tile on one CTA) */
 } maxdnn_plan_info;
@@ -415,7 +417,7 @@ maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanosecond
  * paper has no counterpart).  An option is a named integer, "unset" by default.  `name`
  * is one of FFMA_TILE_M, FFMA_COLS (pin the fp32 kernel's tile: filters 32/64/96/128/256,
  * columns 128/256), FFMA_KH (filter rows per K step of few-channel layers), FFMA_STREAMK
- * (0: never split tail tiles along K), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM
+ * (0: never split tail tiles along K; 2: always, whatever the model says), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM
  * tiles), UMMA_MERGE, UMMA_STAGE_KB, UMMA_COLS, WGRAD_SPLITS, WGRAD_PAIR, SM_COUNT (SM
  * count for host-only workspace queries), X3_CHUNK_ROWS, DEBUG_STATUS, KERNEL_CLOCK (see
  * maxdnn_last_kernel_clock), and

@@ -94,7 +94,7 @@ class KStep(ctypes.Structure):
 class PlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "Ho", "Wo", "tile_m", "tile_px", "tile_n", "kc", "kwc", "n_ksteps", "stages", "n_tiles",
-        "grid", "smem_bytes", "tile_cols", "pair", "split_tiles")]
+        "grid", "smem_bytes", "tile_cols", "pair", "khc", "split_tiles")]
 
 
 class WorkItem(ctypes.Structure):

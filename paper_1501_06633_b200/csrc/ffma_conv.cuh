@@ -209,11 +209,13 @@ struct FfmaProducer {
     const maxdnn_kstep ks = args.table.s[step];
     const uint32_t fb = full_bar + 8u * stage;
     mbar_arrive_expect_tx(fb, (uint32_t)(g.a_box_bytes + g.b_boxes * g.b_box_bytes));
-    tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, o0, ks.kw0, ks.kh, ks.c0);
+    // boxes are (o | n, kw | w, c, kh | h): filter rows outermost, so that the rows of a short
+    // last step are the leading rows of its box
+    tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, o0, ks.kw0, ks.c0, ks.kh);
     uint32_t dst = b_base + (uint32_t)stage * g.b_stage_bytes;
     int w = w0 + ks.kw0;
     for (int t = 0; t < g.b_boxes; ++t) {
-      tma_load_4d(dst, map_in, fb, n0, w, h0 + ks.kh, ks.c0);
+      tma_load_4d(dst, map_in, fb, n0, w, ks.c0, h0 + ks.kh);
       dst += g.b_slot_bytes;
       w += g.stride_w;
     }
@@ -306,7 +308,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   }
   __syncthreads();
 
-  const int rows = g.rows;
+  const int rows_full = g.rows;
 
   if constexpr (!INLINE) {
     if (warp == kFfmaConsumerWarps) {
@@ -420,6 +422,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
       }
       // f0 holds row 0 of this stage.  Four rows per iteration while the row
       // after the block is still inside the stage.
+      const int rows = s < g.short_from ? rows_full : g.rows_short;
       int r = 0;
 #pragma unroll 1
       for (; r + 4 < rows; r += 4) {

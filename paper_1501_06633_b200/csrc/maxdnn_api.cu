@@ -327,21 +327,21 @@ maxdnn_status fprop_fp32(const ConvDims& cd, const float* in, const float* filt,
 
   CUtensorMap mf, mi;
   {
-    // filter bank as (o, kw, kh, c)
-    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Skh, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skw * g.No * 4,
-                             (uint64_t)g.Skh * g.Skw * g.No * 4};
-    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    // filter bank as (o, kw, c, kh): a box lands as [kh][c][kw][o]
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Nc, (uint64_t)g.Skh};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skh * g.Skw * g.No * 4,
+                             (uint64_t)g.Skw * g.No * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, (uint32_t)g.kc, (uint32_t)g.box_kh};
     st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
   {
-    // maps as (n, w, h, c)
-    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    // maps as (n, w, c, h): a box lands as [h][c][w][n]
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Nc, (uint64_t)g.Hi};
     const uint64_t hs = dims_in_h(g, cd.in_h_stride), cs = dims_in_c(g, cd.in_c_stride);
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, hs * 4, cs * 4};
-    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, cs * 4, hs * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, (uint32_t)g.kc, (uint32_t)g.box_kh};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
@@ -1333,19 +1333,19 @@ maxdnn_status fprop_fp32_noalloc(const maxdnn_conv_desc* desc, const float* in, 
 
   CUtensorMap mf, mi;
   {
-    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Skh, (uint64_t)g.Nc};
-    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skw * g.No * 4,
-                             (uint64_t)g.Skh * g.Skw * g.No * 4};
-    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, 1u, (uint32_t)g.kc};
+    const uint64_t dims[4] = {(uint64_t)g.No, (uint64_t)g.Skw, (uint64_t)g.Nc, (uint64_t)g.Skh};
+    const uint64_t str[3] = {(uint64_t)g.No * 4, (uint64_t)g.Skh * g.Skw * g.No * 4,
+                             (uint64_t)g.Skw * g.No * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_m, (uint32_t)g.kwc, (uint32_t)g.kc, (uint32_t)g.box_kh};
     st = encode_map(&mf, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, filt, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Hi, (uint64_t)g.Nc};
+    const uint64_t dims[4] = {(uint64_t)g.Nb, (uint64_t)g.Wi, (uint64_t)g.Nc, (uint64_t)g.Hi};
     const uint64_t hs = dims_in_h(g, 0), cs = dims_in_c(g, 0);
-    const uint64_t str[3] = {(uint64_t)g.Nb * 4, hs * 4, cs * 4};
-    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, 1u, (uint32_t)g.kc};
+    const uint64_t str[3] = {(uint64_t)g.Nb * 4, cs * 4, hs * 4};
+    const uint32_t box[4] = {(uint32_t)g.tile_n, (uint32_t)g.b_box_w, (uint32_t)g.kc, (uint32_t)g.box_kh};
     st = encode_map(&mi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, in, dims, str, box,
                     CU_TENSOR_MAP_SWIZZLE_NONE);
     if (st != MAXDNN_OK) return st;
@@ -1447,7 +1447,7 @@ maxdnn_status maxdnn_conv_plan_query(const maxdnn_conv_desc* desc, maxdnn_kernel
   info->tile_m = g.tile_m; info->tile_px = g.tile_px; info->tile_n = g.tile_n;
   info->kc = g.kc; info->kwc = g.kwc; info->n_ksteps = g.n_ksteps; info->stages = g.stages;
   info->n_tiles = g.n_tiles; info->grid = g.grid; info->smem_bytes = g.smem_bytes;
-  info->tile_cols = g.tile_cols; info->pair = g.pair;
+  info->tile_cols = g.tile_cols; info->pair = g.pair; info->khc = g.box_kh;
   info->split_tiles = kind == MAXDNN_KERNEL_FP32 ? g.sk_tiles : 0;
   if (steps)
     for (int i = 0; i < g.n_ksteps && i < max_steps; ++i) steps[i] = t.s[i];

@@ -183,9 +183,9 @@ static const FfmaShape kFfmaShapes[] = {
     {96, 256, 1.12},  {64, 128, 1.18},  {64, 256, 1.05},  {32, 128, 1.50},
 };
 
-static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* n) {
+static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* n, int khc = 1) {
   int k = 0;
-  for (int kh = 0; kh < d.Skh; ++kh)
+  for (int kh = 0; kh < d.Skh; kh += khc)
     for (int kw0 = 0; kw0 < d.Skw; kw0 += kwc)
       for (int c0 = 0; c0 < d.Nc; c0 += kc) {
         if (k < kMaxKSteps) {
@@ -216,8 +216,8 @@ static double pick_columns(const ConvDims& d, int Wo, int cols, int* nn_out, int
 
 // K step of the fp32 kernel: kc channels of one filter tap, or (few channels) kc channels
 // of a whole filter row of Skw taps.
-static void ffma_kstep(const ConvDims& d, int* kc_out, int* kwc_out) {
-  int kc, kwc;
+static void ffma_kstep(const ConvDims& d, int* kc_out, int* kwc_out, int* khc_out) {
+  int kc, kwc, khc = 1;
   if (d.Nc >= 8) {
     kwc = 1;
     const int kc_max = 32;
@@ -232,9 +232,17 @@ static void ffma_kstep(const ConvDims& d, int* kc_out, int* kwc_out) {
     kc = 40 / d.Skw;
     if (kc < 1) kc = 1;
     if (kc > d.Nc) kc = d.Nc;
+    // Several filter rows per step where one row is short (33 K rows for 11 x 11 x 3): every
+    // step costs the consumers a barrier round trip and loop tails, a third of the
+    // instructions on that layer.  About 100 rows per step (two ring stages) measured best.
+    khc = 100 / (kc * kwc);
+    if (option_is_set(OPT_FFMA_KH)) khc = option(OPT_FFMA_KH);
+    if (khc < 1) khc = 1;
+    if (khc > d.Skh) khc = d.Skh;
   }
   *kc_out = kc;
   *kwc_out = kwc;
+  *khc_out = khc;
 }
 
 // Time of `tiles` tiles on `units` persistent CTAs, in tile times.  Without a split the
@@ -248,7 +256,9 @@ static double ffma_waves(int64_t tiles, int units, int k_rows_per_tile, bool all
   *split_out = false;
   if (R == 0) return (double)W;
   const double whole = (double)(W + 1);
-  if (!allow_split || k_rows_per_tile < 64) return whole;
+  if (!allow_split) return whole;
+  if (option(OPT_FFMA_STREAMK, 1) == 2) { *split_out = true; return whole - 0.5; }   // forced (tests)
+  if (k_rows_per_tile < 512) return whole;   // short sums: the fix-up eats the gain
   const double slot = 16.0 / (double)k_rows_per_tile;
   const double split = (double)W + (double)R / units + 0.03 + slot * (1.0 + (double)units / (double)R);
   if (split < whole - 0.03) { *split_out = true; return split; }
@@ -270,8 +280,8 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   double best_t = 1e300;
   int best_m = 0, best_cols = 0, best_nn = 0, best_T = 0;
   bool best_split = false;
-  int kc0, kwc0;
-  ffma_kstep(d, &kc0, &kwc0);
+  int kc0, kwc0, khc0;
+  ffma_kstep(d, &kc0, &kwc0, &khc0);
   const int k_rows = ceil_div(d.Nc, kc0) * kc0 * d.Skw * d.Skh;
   if (option(OPT_FFMA_STREAMK, 1) == 0) allow_split = false;
   for (const FfmaShape& sh : kFfmaShapes) {
@@ -306,16 +316,29 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   // K step: kc channels of one filter tap, or (few channels) kc channels of a
   // whole filter row of Sk taps.
   int kc = kc0, kwc = kwc0;
+  int khc = khc0;
+  // two ring stages must fit (three where a consumer warp issues the copies)
+  const int min_stages = (best_m / 16) * (best_cols / 16) >= 96 ? 3 : 2;
+  while (khc > 1 && min_stages * kc * kwc * khc * (best_m + best_cols) * 4 > 200 * 1024) --khc;
   // Tiles whose first consumer warp issues the copies keep one ring slot as slack.
   const bool inline_producer = (best_m / 16) * (best_cols / 16) >= 96;
   int n = 0;
-  build_table(d, kc, kwc, t, &n);
+  build_table(d, kc, kwc, t, &n, khc);
   while (n > kMaxKSteps && kwc == 1 && kc < 256) {   // very deep filters: larger boxes
     kc *= 2;
     build_table(d, kc, kwc, t, &n);
   }
   if (n > kMaxKSteps) return MAXDNN_NOT_SUPPORTED;
-  g->kc = kc; g->kwc = kwc; g->rows = kc * kwc; g->n_ksteps = n;
+  g->kc = kc; g->kwc = kwc; g->box_kh = khc; g->rows = kc * kwc * khc; g->n_ksteps = n;
+  // The steps of the last group of filter rows are short when khc does not divide Skh
+  // (the boxes' surplus filter rows are zeros; the consumers skip them).
+  g->short_from = n;
+  g->rows_short = g->rows;
+  if (d.Skh % khc != 0) {
+    const int per_group = n / ceil_div(d.Skh, khc);
+    g->short_from = n - per_group;
+    g->rows_short = kc * kwc * (d.Skh % khc);
+  }
 
   g->a_box_bytes = g->rows * g->tile_m * 4;
   g->a_stage_bytes = g->a_box_bytes;
@@ -344,13 +367,13 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   g->stages = stages;
   g->smem_bytes = stages * stage + 1024;   // + barriers, + slack for alignment
   g->grid = g->n_tiles < sm_count ? g->n_tiles : sm_count;
-  // Split tail: the tiles of the last, partly filled wave (every K step of the table is
-  // dealt out, so the share of a CTA must be at least two steps).
+  // Split tail: the tiles of the last, partly filled wave (whole K steps of the table are
+  // dealt out, so there must be at least one for every CTA).
   g->sk_first = g->n_tiles;
   g->sk_tiles = 0;
   g->sk_units = 0;
   const int tail = g->n_tiles % g->grid;
-  if (best_split && g->n_tiles > g->grid && tail > 0 && (int64_t)tail * n >= 2 * (int64_t)g->grid &&
+  if (best_split && g->n_tiles > g->grid && tail > 0 && (int64_t)tail * n >= (int64_t)g->grid &&
       (size_t)best_m * best_cols * 4 <= kFfmaSplitSlotBytes) {
     g->sk_tiles = tail;
     g->sk_first = g->n_tiles - tail;

@@ -84,6 +84,9 @@ struct ConvGeom {
   // fp32 kernel, split tail: tiles [sk_first, tile_end) are computed by all CTAs together,
   // their sk_units = sk_tiles x n_ksteps K steps dealt out evenly (0 tiles: no split)
   int32_t sk_first, sk_tiles, sk_units;
+  // fp32 kernel: K steps from short_from on hold rows_short rows (the last group of filter
+  // rows of a few-channel plan whose box_kh rows per step do not divide the filter height)
+  int32_t short_from, rows_short;
 };
 
 struct KStepTable {

@@ -280,3 +280,28 @@ def test_full_size_sampled_strided_bprop_data(kernel):
     scale = max(abs(v) for v, _ in vals)
     for p, (v, a) in zip(pts, vals):
         assert abs(float(got[p]) - v) <= 1e-5 * scale, p
+
+
+@pytest.mark.parametrize("kind", [mx.KERNEL_FP32, mx.KERNEL_TF32, mx.KERNEL_BF16, "tf32x3"])
+def test_unsupported_strided_map_gradient_launches_nothing(kind):
+    """A strided map gradient whose per-class sub-problems have no plan (their 'filters' are
+    the layer's channels: 3 here, against the 16-byte row rule) is refused before anything
+    is enqueued: no memset, no split, no transform kernel."""
+    d = mx.ConvDesc.make(64, 23, 23, 3, 32, 5, 2, 1)
+    Ho, Wo = mx.conv_out_dims(d)
+    bf16 = kind == mx.KERNEL_BF16
+    dt = torch.bfloat16 if bf16 else torch.float32
+    dout = torch.zeros(32 * Ho * Wo * 64, dtype=dt, device="cuda")
+    filt = torch.zeros(mx.conv_filt_elems(d), dtype=dt, device="cuda")
+    din = torch.full((mx.conv_in_elems(d),), 7.0, dtype=torch.float32, device="cuda")
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    before = mx.launch_count()
+    with pytest.raises(mx.MaxdnnError) as e:
+        if kind == "tf32x3":
+            mx.conv_bprop_data_tf32x3(d, dout, filt, din, ws)
+        else:
+            mx.conv_bprop_data(d, dout, filt, din, ws, kind)
+    assert e.value.status == mx.NOT_SUPPORTED
+    assert mx.launch_count() == before
+    torch.cuda.synchronize()
+    assert bool((din == 7.0).all())           # not cleared, not written

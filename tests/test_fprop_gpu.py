@@ -123,8 +123,9 @@ SPLIT = [
     ((128, 20, 18, 24, 256, 3, 1, 1, 1.0), 256, 128),
     ((64, 40, 18, 40, 128, 3, 1, 1, 1.0), 128, 256),
     ((64, 80, 36, 40, 64, 3, 2, 1, 1.0), 64, 256),
+    ((64, 40, 18, 40, 64, 3, 1, 1, 1.0), 64, 256),
     ((64, 40, 36, 16, 96, 3, 1, 1, 1.0), 96, 256),
-    ((128, 63, 59, 3, 96, 11, 4, 0, 1.0), 96, 128),
+    ((128, 55, 83, 3, 96, 11, 4, 0, 1.0), 96, 128),      # 11 filter rows in steps of 2: a short last step
 ]
 
 
@@ -133,6 +134,7 @@ SPLIT = [
 def test_split_tail_fp32(dims, tile_m, cols):
     """The tail wave split along K: contributions through the workspace, finishers adding
     them in CTA order — against the oracle, and bitwise equal from run to run."""
+    mx.set_option("FFMA_STREAMK", 2)       # split whenever there is a tail, whatever its length
     if tile_m:
         mx.set_option("FFMA_TILE_M", tile_m)
         mx.set_option("FFMA_COLS", cols)
@@ -150,6 +152,22 @@ def test_split_tail_fp32(dims, tile_m, cols):
     info, _ = mx.conv_plan_query(d, mx.KERNEL_FP32, sms)
     assert info.split_tiles == 0
     check_fp32(w, inp, filt)
+
+
+@pytest.mark.parametrize("khc", [1, 2, 3, 5, 7])
+@pytest.mark.parametrize("dims", [
+    (128, 31, 27, 3, 96, 11, 4, 0, 1.0),     # one pixel per tile: one box per stage
+    (16, 23, 19, 3, 12, 7, 2, 3, 0.5),       # several pixels per tile: one box per pixel; apron
+    (32, 12, 9, 5, 40, 5, 1, 2, 1.0),        # channels in two blocks (3 + 2), stride 1
+], ids=lambda s: "x".join(str(v) for v in s))
+def test_filter_rows_per_k_step(dims, khc):
+    """Few-channel layers take several filter rows per K step; where their number does not
+    divide the filter height the last step is short."""
+    mx.set_option("FFMA_KH", khc)
+    w = wl.Workload("khc", *dims, ("uniform", -1.0, 1.0), ("uniform", -1.0, 1.0), 77)
+    info, _ = mx.conv_plan_query(mx.ConvDesc.make(*w.dims), mx.KERNEL_FP32, 148)
+    assert info.kwc == w.Sk and 1 <= info.khc <= khc
+    check_fp32(w)
 
 
 def test_special_values_fp32():
@@ -173,10 +191,14 @@ def test_run_to_run_bitwise_identical():
     np.testing.assert_array_equal(a, b)
 
 
-@pytest.mark.parametrize("name", ["first11x11s4", "mid5x5", "wide3x3", "large3x3"])
+# every workload at the size and in the launch configuration that the benchmark times
+FULL_SIZE_FP32 = ["first11x11s4", "mid5x5", "wide3x3", "large3x3"] + wl.TABLE1_ORDER
+
+
+@pytest.mark.parametrize("name", FULL_SIZE_FP32)
 def test_full_size_sampled_fp32(name):
     """Benchmark sizes: a band of full output rows plus random single outputs."""
-    w = wl.WORKLOADS[name]
+    w = wl.ALL[name]
     inp, filt = wl.make_inputs(w)
     got = run_fp32(w, inp, filt)
     Ho, Wo = got.shape[1:3]

@@ -83,7 +83,7 @@ def emulate_fp32_plan(w, inp, filt, sm_count=148):
     d = mx.ConvDesc.make(*w.dims)
     info, steps = mx.conv_plan_query(d, mx.KERNEL_FP32, sm_count)
     Ho, Wo = info.Ho, info.Wo
-    Mt, T, Nn, kc, kwc = info.tile_m, info.tile_px, info.tile_n, info.kc, info.kwc
+    Mt, T, Nn, kc, kwc, khc = info.tile_m, info.tile_px, info.tile_n, info.kc, info.kwc, info.khc
     o_blocks = -(-w.No // Mt)
     n_chunks = -(-w.Nb // Nn)
     x_runs = -(-Wo // T)
@@ -93,7 +93,7 @@ def emulate_fp32_plan(w, inp, filt, sm_count=148):
     # every (c, kh, kw) is covered by exactly one table entry
     seen = np.zeros((w.Nc, w.Sk, w.Sk), dtype=np.int32)
     for s in steps:
-        seen[s.c0:s.c0 + kc, s.kh, s.kw0:s.kw0 + kwc] += 1
+        seen[s.c0:s.c0 + kc, s.kh:s.kh + khc, s.kw0:s.kw0 + kwc] += 1   # (clipped at the last row)
         assert s.kw0 + kwc <= w.Sk, "a box must not run past the filter row"
     assert np.all(seen == 1)
     out = np.full((w.No, Ho, Wo, w.Nb), np.nan)
@@ -105,10 +105,10 @@ def emulate_fp32_plan(w, inp, filt, sm_count=148):
         o0, n0, x0 = ob * Mt, nch * Nn, xr * T
         acc = np.zeros((Mt, T, Nn))
         for s in steps:
-            A = box(filt, (s.c0, s.kh, s.kw0, o0), (kc, 1, kwc, Mt))           # [c][1][kw][o]
+            A = box(filt, (s.c0, s.kh, s.kw0, o0), (kc, khc, kwc, Mt))         # [c][kh][kw][o]
             for t in range(T):
                 Bx = box(inp, (s.c0, y * w.stride - w.pad + s.kh,
-                               (x0 + t) * w.stride - w.pad + s.kw0, n0), (kc, 1, kwc, Nn))
+                               (x0 + t) * w.stride - w.pad + s.kw0, n0), (kc, khc, kwc, Nn))
                 acc[:, t, :] += np.einsum("ckwo,ckwn->on", A, Bx)
         for t in range(T):
             if x0 + t >= Wo:
@@ -292,3 +292,72 @@ def test_split_tail_items_cover_every_k_step_once(dims, sm_count):
         assert tile in contributors
     if info.split_tiles:
         assert 0 < info.split_tiles < info.grid
+
+
+# ---------------------------------------------------------------------------
+# Every kernel instance and plan kind that the planner picks for a benchmarked workload
+# must be one that a GPU parity test runs.  The GPU tests' parameter lists are read here
+# (planning needs no GPU) and compared with the plans of all fifteen workloads.
+# ---------------------------------------------------------------------------
+def plan_signature(dims, kind, sms=148):
+    d = mx.ConvDesc.make(*dims)
+    info, _ = mx.conv_plan_query(d, kind, sms)
+    Nb, Wi, Hi, Nc, No, Sk, stride, pad, _ = dims
+    if kind == mx.KERNEL_FP32:
+        one_box = info.tile_px * info.tile_n == info.tile_cols and \
+            (info.tile_px == 1 or (stride == 1 and info.kwc == 1))
+        return ("fp32", info.tile_m, info.tile_cols, one_box, info.kwc > 1, info.khc > 1,
+                info.split_tiles > 0)
+    few = Nc < (8 if kind == mx.KERNEL_TF32 else 16)
+    return ("tf32" if kind == mx.KERNEL_TF32 else "bf16", info.pair, info.tile_px * info.tile_n,
+            few, info.kwc > 1, stride > 1)
+
+
+def test_every_benchmarked_plan_is_one_a_gpu_parity_test_runs():
+    import test_fprop_gpu as tf
+    import test_fprop_tensor_gpu as tt
+    # full-size cases: the GPU tests run exactly these workloads (sampled against the oracle)
+    fp32_full = set(tf.FULL_SIZE_FP32)
+    tensor_full = set(tt.FULL_SIZE_TENSOR) | {("large3x3", "tf32"), ("large3x3", "bf16")}
+    for name in wl.ORDER + wl.TABLE1_ORDER:
+        w = wl.ALL[name]
+        if name != "tiny3x3":
+            assert name in fp32_full, name
+            for k in ("tf32", "bf16"):
+                assert (name, k) in tensor_full, (name, k)
+    # and, beyond running the same workload: the same KIND of plan is also compared with the
+    # oracle element by element at a reduced size (all outputs, canary strips)
+    reduced = set()
+    for name, kw in tf.TABLE1_REDUCED.items():
+        reduced.add(plan_signature(wl.TABLE1[name].scaled(**kw).dims, mx.KERNEL_FP32))
+    for name, kw in [("first11x11s4", dict(Nb=128, Wi=51, Hi=43, No=96)),
+                     ("mid5x5", dict(Nb=128, Wi=9, Hi=7, Nc=96, No=256)),
+                     ("wide3x3", dict(Nb=128, Wi=6, Hi=5, Nc=256, No=384)),
+                     ("large3x3", dict(Nb=64, Wi=14, Hi=9, Nc=128, No=256))]:
+        reduced.add(plan_signature(wl.WORKLOADS[name].scaled(**kw).dims, mx.KERNEL_FP32))
+    reduced.add(plan_signature(wl.WORKLOADS["tiny3x3"].dims, mx.KERNEL_FP32))
+    try:
+        for tile_m, cols in [(32, 128), (64, 128), (96, 128), (128, 128), (256, 128), (64, 256),
+                             (96, 256), (128, 256)]:
+            for stride in (1, 2):
+                mx.set_option("FFMA_TILE_M", tile_m)
+                mx.set_option("FFMA_COLS", cols)
+                reduced.add(plan_signature((64, 11, 8, 24, 296, 3, stride, 1, 1.0), mx.KERNEL_FP32))
+        for dims, tile_m, cols in tf.SPLIT:
+            mx.reset_options()
+            mx.set_option("FFMA_STREAMK", 2)
+            if tile_m:
+                mx.set_option("FFMA_TILE_M", tile_m)
+                mx.set_option("FFMA_COLS", cols)
+            reduced.add(plan_signature(dims, mx.KERNEL_FP32))
+    finally:
+        mx.reset_options()
+    missing = []
+    for name in wl.ORDER + wl.TABLE1_ORDER:
+        sig = plan_signature(wl.ALL[name].dims, mx.KERNEL_FP32)
+        # which filter rows / columns a step spans is a property of the shape, not a kernel
+        # instance: match on (tile, one box per stage?, split?)
+        key = (sig[1], sig[2], sig[3], sig[6])
+        if key not in {(r[1], r[2], r[3], r[6]) for r in reduced}:
+            missing.append((name, sig))
+    assert not missing, "full-size fp32 plans without a reduced-size parity case: %r" % missing

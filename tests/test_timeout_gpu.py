@@ -71,3 +71,27 @@ def test_chunked_kernel_wait_runs_out_and_the_context_survives(No, monkeypatch):
     ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha)
     got = out.cpu().numpy().reshape(ref.shape)
     assert float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref))) <= 1e-5
+
+
+@pytest.mark.parametrize("kernel,kind", [("fp32", mx.KERNEL_FP32), ("bf16", mx.KERNEL_BF16)])
+def test_a_stale_timeout_code_does_not_disturb_later_launches(kernel, kind):
+    """The status word is sticky until it is read.  A launch that follows a timed-out one
+    WITHOUT the word having been read must still be exact: its waits leave early only for
+    a give-up of their own launch (each launch carries its own number)."""
+    w = wl.WORKLOADS["large3x3"].scaled(Nb=64, Wi=12, Hi=8, Nc=64, No=128)
+    d = mx.ConvDesc.make(*w.dims)
+    d_in, d_f, ref_in, ref_f = _tensors(w, kernel)
+    bad = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    out = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    assert mx.last_device_status() == mx.OK
+    mx.set_option("TEST_MISSING_ARRIVAL", 1)
+    assert mx.fprop_status(d, d_in, d_f, bad, kind) == mx.OK       # this one gives up
+    mx.unset_option("TEST_MISSING_ARRIVAL")
+    for _ in range(3):                                                  # these must not
+        assert mx.fprop_status(d, d_in, d_f, out, kind) == mx.OK
+    torch.cuda.synchronize()
+    ref = oracle.conv_fprop(ref_in, ref_f, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    got = out.cpu().numpy().reshape(ref.shape)
+    assert float(np.max(np.abs(got - ref))) / float(np.max(np.abs(ref))) <= 1e-5
+    assert mx.last_device_status() == mx.DEVICE_TIMEOUT               # the code is still there
+    assert mx.last_device_status() == mx.OK

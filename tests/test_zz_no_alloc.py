@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_1501_06633_b200 as mx
 from paper_1501_06633_b200 import workloads as wl
 
@@ -29,7 +30,7 @@ def both_entry_points(w, seed_offset):
     mx.conv_fprop(d, d_in, d_f, ref)
     assert mx.last_device_status() == mx.OK
     mx.conv_fprop_noalloc(d, d_in, d_f, got)
-    torch.cuda.synchronize()
+    assert mx.last_device_status_noalloc() == mx.OK
     return got.cpu().numpy(), ref.cpu().numpy()
 
 
@@ -45,6 +46,47 @@ def test_noalloc_entry_point_matches_fprop_twice_in_a_row():
     # and once more on the first shape: the shared block carries nothing over
     got, ref = both_entry_points(shapes[0], seed_offset=7)
     np.testing.assert_allclose(got, ref, rtol=0, atol=TOL_FP32 * float(np.max(np.abs(ref))))
+
+
+def test_noalloc_entry_point_against_the_oracle_and_without_allocating():
+    """The same call checked against the CPU oracle, with the device's free memory unchanged
+    across it (the first call on the device included, if this test runs in a fresh process)."""
+    w = wl.WORKLOADS["tiny3x3"]
+    inp, filt = wl.make_inputs(w)
+    d = mx.ConvDesc.make(*w.dims)
+    d_in, d_f = torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda()
+    got = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    mx.conv_fprop_noalloc(d, d_in, d_f, got)
+    assert mx.last_device_status_noalloc() == mx.OK
+    assert torch.cuda.mem_get_info()[0] == free_before
+    ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    g = got.cpu().numpy().reshape(ref.shape)
+    err = float(np.max(np.abs(g.astype(np.float64) - ref))) / float(np.max(np.abs(ref)))
+    assert err <= TOL_FP32
+
+
+def test_noalloc_entry_point_reports_a_wait_that_ran_out():
+    """Its kernel reports into the built-in block, which has its own status query: a bounded
+    wait that runs out (test hook: an arrival that never comes) is seen there and only there,
+    and the next call is exact again."""
+    w = wl.WORKLOADS["tiny3x3"]
+    inp, filt = wl.make_inputs(w)
+    d = mx.ConvDesc.make(*w.dims)
+    d_in, d_f = torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda()
+    got = torch.zeros(mx.conv_out_elems(d), dtype=torch.float32, device="cuda")
+    assert mx.last_device_status_noalloc() == mx.OK and mx.last_device_status() == mx.OK
+    mx.set_option("TEST_MISSING_ARRIVAL", 1)
+    mx.conv_fprop_noalloc(d, d_in, d_f, got)
+    mx.unset_option("TEST_MISSING_ARRIVAL")
+    mx.conv_fprop_noalloc(d, d_in, d_f, got)           # queued behind it, status not read yet
+    assert mx.last_device_status() == mx.OK            # the cudaMalloc'd block saw nothing
+    assert mx.last_device_status_noalloc() == mx.DEVICE_TIMEOUT
+    assert mx.last_device_status_noalloc() == mx.OK    # reading clears it
+    ref = oracle.conv_fprop(inp, filt, stride=w.stride, pad=w.pad, alpha=w.alpha)
+    g = got.cpu().numpy().reshape(ref.shape)
+    assert float(np.max(np.abs(g - ref))) / float(np.max(np.abs(ref))) <= TOL_FP32
 
 
 def test_noalloc_entry_point_rejects_what_fprop_rejects():
