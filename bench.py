@@ -61,6 +61,9 @@ def parse_args():
                    help="fprop (the headline path) or one of its two adjoints (BPROP)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--nb", type=int, default=0,
+                   help="override the workload's minibatch (a count that is not a multiple of 4 "
+                        "goes through maxdnn_conv_fprop_ragged)")
     p.add_argument("--no-tensor", action="store_true",
                    help="skip the tensor-core kernels timed beside the fp32 headline")
     p.add_argument("--min-seconds", type=float, default=0.6,
@@ -364,6 +367,7 @@ class Arm:
         kind = {"fp32": mx.KERNEL_FP32, "tf32": mx.KERNEL_TF32, "bf16": mx.KERNEL_BF16,
                 "tf32x3": mx.KERNEL_TF32}[kernel]
         self.kind, self.x3 = kind, x3
+        self.ragged = op == "fprop" and kernel == "fp32" and bool(w.Nb % 4 or w.No % 4)
         d = self.d = mx.ConvDesc.make(*w.dims)
         self.nbytes, self.Ho, self.Wo = workload_bytes(w, kernel, op)
         self.C = mx.conv_flops(d)          # the same bilinear form: all three operations cost C
@@ -407,6 +411,12 @@ class Arm:
                 "wgrad": (mx.conv_bprop_filter_tf32x3_workspace, mx.conv_bprop_filter_tf32x3)}[op]
             ws = torch.empty(max(16, size_fn(d)), dtype=torch.uint8, device="cuda")
             self.run = lambda a, b, r, wsp, stream=None: call_fn(d, a, b, r, wsp, stream=stream)
+        elif op == "fprop" and kernel == "fp32" and (w.Nb % 4 or w.No % 4):
+            # counts outside the 16-byte row rule: the ragged entry point (fp32: in-kernel staging)
+            ws = torch.empty(max(16, mx.conv_fprop_ragged_workspace(d, kind)), dtype=torch.uint8,
+                             device="cuda")
+            self.run = lambda a, b, r, wsp, stream=None: mx.conv_fprop_ragged(d, a, b, r, wsp, kind,
+                                                                              stream=stream)
         elif op == "fprop":
             self.run = lambda a, b, r, wsp, stream=None: fprop(d, as_op(a), as_op(b), r, stream=stream)
         elif op == "dgrad":
@@ -519,6 +529,8 @@ def run_ours(args):
 
     peaks, peaks_kind = load_peaks()
     w = wl.ALL[args.workload]
+    if args.nb > 0:
+        w = w.scaled(Nb=args.nb)
     op = args.op
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     arm = Arm(mx, w, args.kernel, op, rank, world)
@@ -563,7 +575,7 @@ def run_ours(args):
 
     def e2e_step(k, stream):
         a, b, r = d_as[k % n_sets], d_bs[k % len(d_bs)], d_res[k % n_sets]
-        if op == "fprop" and not x3:
+        if op == "fprop" and not x3 and not arm.ragged:
             mx.conv_fprop_host(d, kind, h_a, h_b, h_outs[k], a, b, r, stream=stream)
         else:
             with torch.cuda.stream(stream):

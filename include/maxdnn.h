@@ -287,13 +287,22 @@ maxdnn_status maxdnn_conv_bprop_filter_tf32x3(const maxdnn_conv_desc* desc, cons
 
 /*
  * FPROP for shapes the entry points above refuse because of the 16-byte row rule
- * (Nb or No not a multiple of 4 for fp32; of 32 / 64 and 32 for tf32 / bf16): the
- * maps and filters are copied into zero-padded staging tensors in the caller's
- * workspace (Nb, No rounded up), the matching kernel runs on the padded problem,
- * and the result is copied back without the padding.  Same arguments and result
- * as the matching entry point; `workspace` as for the backward entry points
- * below (size from maxdnn_conv_fprop_ragged_workspace; 0 when the shape needs no
- * padding, in which case the kernel runs directly on the caller's tensors).
+ * (Nb or No not a multiple of 4 for fp32; of 32 / 64 and 32 for tf32 / bf16).
+ * Two routes.  In-kernel (fp32 only): the kernel stages the ragged rows itself — four copy
+ * warps move the patch rows (and the filter rows, if No is ragged) into shared memory with
+ * 4- or 8-byte loads and stores, zeros for the apron and for the tails of Nb and No, in
+ * place of the bulk tensor copies, and the epilogue stores element by element — so no
+ * padded copy of any tensor is made and no workspace is needed.  Padded (every kind): the
+ * maps and filters are copied into zero-padded staging tensors in the
+ * caller's workspace (Nb, No rounded up), the matching kernel runs on the padded
+ * problem, and the result is copied back without the padding.  Same arguments and
+ * result as the matching entry point; `workspace` as for the backward entry points
+ * below (size from maxdnn_conv_fprop_ragged_workspace; 0 when none is needed: an aligned
+ * shape, which runs directly on the caller's tensors, or the in-kernel route).  The padded
+ * route is the default for every kind: measured, the copy warps of the in-kernel route cost
+ * the arithmetic warps more issue slots (12 % of a long-K layer's time, far more on a
+ * 3-channel layer) than the padded route's extra passes over maps and result cost memory
+ * time.  Option RAGGED_PADDED = -1 selects the in-kernel route for fp32.
  * The paper has no counterpart (Section 3.3 only notes that its kernel wants
  * multiples of 64 filters and 8 images for efficiency).
  */
@@ -420,7 +429,7 @@ maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanosecond
  * (0: never split tail tiles along K; 2: always, whatever the model says), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM
  * tiles), UMMA_MERGE, UMMA_STAGE_KB, UMMA_COLS, WGRAD_SPLITS, WGRAD_PAIR, SM_COUNT (SM
  * count for host-only workspace queries), X3_CHUNK_ROWS, DEBUG_STATUS, KERNEL_CLOCK (see
- * maxdnn_last_kernel_clock), and
+ * maxdnn_last_kernel_clock), RAGGED_PADDED (see maxdnn_conv_fprop_ragged), and
  * TEST_MISSING_ARRIVAL (test hook: CTA 0's "full" barriers expect an arrival that
  * never comes, so a bounded wait runs out).  The environment variable MAXDNN_<name>
  * gives an option its initial value; the environment is read once, at the first use of

@@ -23,8 +23,9 @@ namespace maxdnn {
 
 constexpr int kFfmaConsumerWarps = 8;
 __host__ __device__ constexpr bool ffma_inline_producer(int mr, int nr) { return mr * nr >= 96; }
-__host__ __device__ constexpr int ffma_threads(int mr, int nr) {
-  return (kFfmaConsumerWarps + (ffma_inline_producer(mr, nr) ? 0 : 1)) * 32;
+__host__ __device__ constexpr int ffma_threads(int mr, int nr, bool ragged = false) {
+  // ragged: four copy warps (two for patches, two for filters) that move the rows themselves
+  return (kFfmaConsumerWarps + (ragged ? 4 : ffma_inline_producer(mr, nr) ? 0 : 1)) * 32;
 }
 
 // Multiply-add order per register-block shape (see fma_block), from timings on B200.
@@ -49,6 +50,10 @@ struct FfmaArgs {
   float* sk_partial;
   uint32_t* sk_flags;
   KStepTable table;
+  // Ragged kernel only (Nb or No not a multiple of 4, which the bulk tensor copies cannot
+  // address): the tensors themselves, read by the copy warps with 4-byte asynchronous copies.
+  const float* in;
+  const float* filt;
 };
 
 // ---------------------------------------------------------------------------------------
@@ -257,22 +262,173 @@ __device__ __noinline__ bool wait_peer_flag(const uint32_t* flag, uint32_t epoch
 
 
 
+// ---------------------------------------------------------------------------------------
+// Ragged shapes.  A row of Nb images (or No filters) that is not a multiple of 16 bytes
+// cannot be the pitch of a bulk tensor copy.  The ragged kernel therefore stages the same
+// boxes with ordinary loads and shared-memory stores of 4 or 8 bytes (zeros for what lies
+// outside the tensors — the apron, the tails of Nb and No, surplus rows of a K step), made
+// by four copy warps: two for the patch rows, two for the filter rows, each arriving on the
+// stage's "full" barrier when its rows are written (4 arrivals per stage).  The
+// staged layout is the one-box-per-pixel layout of the bulk path, so the consumers are
+// unchanged; the epilogue stores element by element with bounds.
+// ---------------------------------------------------------------------------------------
+// VEC floats (4 or 8 bytes) of one lane: loaded from global memory (zeros if !valid; the
+// source is not read then) and stored to shared memory.
+template <int VEC> struct RaggedVal { float v[VEC]; };
+template <int VEC>
+__device__ __forceinline__ RaggedVal<VEC> ragged_ldg(const float* src, bool valid) {
+  RaggedVal<VEC> r;
+  if constexpr (VEC == 2) {
+    float2 t = make_float2(0.f, 0.f);
+    if (valid) t = __ldg(reinterpret_cast<const float2*>(src));
+    r.v[0] = t.x; r.v[1] = t.y;
+  } else {
+    r.v[0] = valid ? __ldg(src) : 0.f;
+  }
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ void ragged_sts(uint32_t dst, const RaggedVal<VEC>& r) {
+  if constexpr (VEC == 2)
+    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(r.v[0]), "f"(r.v[1]) : "memory");
+  else
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(r.v[0]) : "memory");
+}
+
+// One copy warp's whole life: every K step of every tile of this CTA.  PATCH: the patch
+// rows [pixel][kh][c][kw] of tile_n images each; else the filter rows [kh][c][kw] of MT
+// filters.  Two warps share each kind, each taking half of a box's channels.  The copy
+// warps compete with eight warps of packed multiply-adds for issue slots (those leave about
+// a tenth), so the loop over a box's channels is bare: one load, one shared-memory store and
+// two pointer increments per 32 x VEC floats, eight loads in flight per lane; everything
+// that depends on the pixel, the filter row or column is computed outside it.
+// (Asynchronous copies of 4 or 8 bytes were tried first and were no faster: the limit is
+// the instruction count of the copy warps, not the copy mechanism.)
+template <int MT, bool PATCH, int VEC>
+__device__ __forceinline__ void ragged_copy_loop(const FfmaArgs& args, int part, int parts,
+                                                 uint32_t stage_base, uint32_t stage_bytes,
+                                                 uint32_t full_bar, uint32_t empty_bar,
+                                                 const CUtensorMap* map_filt, uint32_t a_base) {
+  constexpr int kInFlight = 8;
+  const ConvGeom& g = args.g;
+  const int lane = threadIdx.x & 31;
+  const float* const tensor = PATCH ? args.in : args.filt;
+  const int len = PATCH ? g.tile_n : MT;                       // floats per staged row
+  const uint32_t row_bytes = 4u * (uint32_t)len;
+  const uint32_t c_pitch = row_bytes * (uint32_t)g.kwc;        // next channel in the stage
+  const size_t plane = PATCH ? (size_t)g.Hi * g.Wi * g.Nb : (size_t)g.Skh * g.Skw * g.No;
+  const int ci_lo = part * g.kc / parts, ci_hi = (part + 1) * g.kc / parts;   // this warp's channels
+  int stage = 0;
+  uint32_t phase = 0;
+  for (int tile = g.tile_begin + (int)blockIdx.x; tile < g.tile_end; tile += (int)gridDim.x) {
+    int r = tile;
+    const int ob = r % g.o_blocks; r /= g.o_blocks;
+    const int nch = r % g.n_chunks; r /= g.n_chunks;
+    const int xr = r % g.x_runs;
+    const int y = r / g.x_runs;
+    const int i0 = PATCH ? nch * g.tile_n : ob * MT;              // first image / filter
+    const int n_valid = min(len, (PATCH ? g.Nb : g.No) - i0);
+    const int x0 = xr * g.tile_px;
+    for (int s = 0; s < g.n_ksteps; ++s) {
+      if (!mbar_wait_backoff(empty_bar + 8u * stage, phase ^ 1u, args.wc, kDevTimeoutEmpty)) return;
+      const maxdnn_kstep ks = args.table.s[s];
+      const uint32_t dst0 = stage_base + (uint32_t)stage * stage_bytes;
+      const int c_valid = g.Nc - ks.c0;                            // channels of the box inside the tensor
+      if (map_filt != nullptr && lane == 0) {
+        // filter rows that the bulk tensor copy can address (No a multiple of 4): one copy,
+        // counted on the same barrier (this arrival is the barrier's fifth)
+        const uint32_t fb = full_bar + 8u * stage;
+        mbar_arrive_expect_tx(fb, (uint32_t)g.a_box_bytes);
+        tma_load_4d(a_base + (uint32_t)stage * g.a_stage_bytes, map_filt, fb, ob * MT, ks.kw0, ks.c0, ks.kh);
+      }
+      for (int t = 0; t < (PATCH ? g.tile_px : 1); ++t) {
+        for (int khi = 0; khi < g.box_kh; ++khi) {
+          for (int kwi = 0; kwi < g.kwc; ++kwi) {
+            // the row of channel c0 for this (pixel, filter row, filter column), and whether
+            // it lies inside the tensor
+            bool ok;
+            size_t off;
+            if constexpr (PATCH) {
+              const int h = y * g.stride_h - g.pad_h + ks.kh + khi;
+              const int w = (x0 + t) * g.stride_w - g.pad_w + ks.kw0 + kwi;
+              ok = ks.kh + khi < g.Skh && h >= 0 && h < g.Hi && w >= 0 && w < g.Wi;
+              off = ok ? (((size_t)ks.c0 * g.Hi + h) * g.Wi + w) * (size_t)g.Nb : 0;
+            } else {
+              const int kh = ks.kh + khi, kw = ks.kw0 + kwi;
+              ok = kh < g.Skh && kw < g.Skw;
+              off = ok ? (((size_t)ks.c0 * g.Skh + kh) * g.Skw + kw) * (size_t)g.No : 0;
+            }
+            const uint32_t d_row = dst0 + (PATCH ? (uint32_t)t * g.b_slot_bytes : 0u) +
+                                   (uint32_t)(khi * g.kc * g.kwc + kwi) * row_bytes;
+            for (int e = lane * VEC; e < len; e += 32 * VEC) {
+              const bool e_ok = ok && e < n_valid;
+              const float* src = tensor + (e_ok ? off + i0 + e + (size_t)ci_lo * plane : 0);
+              uint32_t dst = d_row + 4u * (uint32_t)e + (uint32_t)ci_lo * c_pitch;
+              for (int ci = ci_lo; ci < ci_hi; ci += kInFlight) {
+                RaggedVal<VEC> val[kInFlight];
+#pragma unroll
+                for (int j = 0; j < kInFlight; ++j)
+                  val[j] = ragged_ldg<VEC>(src + (e_ok ? j * plane : 0), e_ok && ci + j < c_valid);
+#pragma unroll
+                for (int j = 0; j < kInFlight; ++j)
+                  if (ci + j < ci_hi) ragged_sts<VEC>(dst + (uint32_t)j * c_pitch, val[j]);
+                if (e_ok) src += kInFlight * plane;
+                dst += (uint32_t)kInFlight * c_pitch;
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8u * stage);
+      if (++stage == g.stages) { stage = 0; phase ^= 1u; }
+    }
+  }
+}
+
+// 8-byte pieces where every row start and every row length allows it, else 4-byte ones.
+// With ragged filters (No not a multiple of 4) warps 0, 1 copy patches and 2, 3 filters;
+// else all four copy patches and lane 0 of the first also issues the filter boxes as bulk
+// tensor copies.
+template <int MT>
+__device__ __noinline__ void ragged_copy_warp(const FfmaArgs& args, int role, const CUtensorMap* map_filt,
+                                              uint32_t a_base, uint32_t b_base, uint32_t full_bar,
+                                              uint32_t empty_bar) {
+  const ConvGeom& g = args.g;
+  const bool filt_bulk = (g.No & 3) == 0;
+  const bool patch_role = filt_bulk || role < 2;
+  const int parts = filt_bulk ? 4 : 2, part = filt_bulk ? role : (role & 1);
+  const CUtensorMap* mf = (filt_bulk && role == 0) ? map_filt : nullptr;
+  if (patch_role) {
+    const bool pairs = ((g.Nb | g.tile_n) & 1) == 0 && (reinterpret_cast<uintptr_t>(args.in) & 7) == 0;
+    if (pairs) ragged_copy_loop<MT, true, 2>(args, part, parts, b_base, g.b_stage_bytes, full_bar, empty_bar, mf, a_base);
+    else ragged_copy_loop<MT, true, 1>(args, part, parts, b_base, g.b_stage_bytes, full_bar, empty_bar, mf, a_base);
+  } else {
+    const bool pairs = (g.No & 1) == 0 && (reinterpret_cast<uintptr_t>(args.filt) & 7) == 0;
+    if (pairs) ragged_copy_loop<MT, false, 2>(args, part, parts, a_base, g.a_stage_bytes, full_bar, empty_bar, nullptr, 0);
+    else ragged_copy_loop<MT, false, 1>(args, part, parts, a_base, g.a_stage_bytes, full_bar, empty_bar, nullptr, 0);
+  }
+}
+
 #define MAXDNN_ROW(R) a_ptr + (R) * Mt, b_ptr, (R) * b_pitch
 
 // SPLIT = false: whole tiles [tile_begin, tile_end).  SPLIT = true: this CTA's pieces of the
 // split tail (launched after the whole-tile kernel on the same stream; work items as if
 // tile_begin were the first split tile).  Operands come by 8-byte loads for the blocks of
 // 16 columns and by 16-byte loads for the others (which is faster was measured per block).
-template <int MR, int NR, bool FIXED, bool SPLIT>
-__global__ void __launch_bounds__(ffma_threads(MR, NR), 1)
+// RAGGED: the copy warps of ragged_copy_warp instead of bulk tensor copies, bounds-checked
+// element stores (whole tiles, one box per pixel only).
+template <int MR, int NR, bool FIXED, bool SPLIT, bool RAGGED = false>
+__global__ void __launch_bounds__(ffma_threads(MR, NR, RAGGED), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
                  const __grid_constant__ FfmaArgs args) {
   constexpr int Mt = 16 * MR;           // filters per tile
   constexpr int Nt = 16 * NR;           // columns per tile
   constexpr int NH = NR / 4;            // float4 column groups per thread
-  constexpr bool INLINE = ffma_inline_producer(MR, NR);
+  constexpr bool INLINE = ffma_inline_producer(MR, NR) && !RAGGED;
   constexpr bool W64 = NR == 16;
+  static_assert(!RAGGED || (!FIXED && !SPLIT && !ffma_inline_producer(MR, NR)), "ragged instances");
   extern __shared__ uint8_t smem_raw[];
   const ConvGeom& g = args.g;
 
@@ -299,7 +455,8 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   if (threadIdx.x == 0) {
     const uint32_t extra = (args.test_missing_arrival != 0 && blockIdx.x == 0) ? 1u : 0u;
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar + 8u * s, 1 + extra);
+      // ragged: four copy warps, and the lane that issues bulk filter copies where it can
+      mbar_init(full_bar + 8u * s, (RAGGED ? 4 + ((g.No & 3) == 0 ? 1 : 0) : 1) + extra);
       mbar_init(empty_bar + 8u * s, kFfmaConsumerWarps);
     }
     if constexpr (SPLIT) mbar_init(sk_bar, kFfmaConsumerWarps);
@@ -310,7 +467,14 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   const int rows_full = g.rows;
 
-  if constexpr (!INLINE) {
+  if constexpr (RAGGED) {
+    if (warp >= kFfmaConsumerWarps) {
+      if (threadIdx.x == kFfmaConsumerWarps * 32 && (g.No & 3) == 0) prefetch_tensormap(&map_filt);
+      ragged_copy_warp<Mt>(args, warp - kFfmaConsumerWarps, &map_filt, base + a_off, base + b_off,
+                           full_bar, empty_bar);
+      return;
+    }
+  } else if constexpr (!INLINE) {
     if (warp == kFfmaConsumerWarps) {
       // ---------------------------------------------------- producer warp
       if (lane == 0) {
@@ -576,7 +740,14 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
           v.w = ia == 0 ? Q[i2][2 * h + 1].x : P[i2][2 * h + 1].y;
           v.x *= alpha; v.y *= alpha; v.z *= alpha; v.w *= alpha;
           float* dst = args.out + (((size_t)o * g.Ho + y) * g.Wo + x) * (size_t)g.Nb + n;
-          __stcs(reinterpret_cast<float4*>(dst), v);
+          if constexpr (RAGGED) {       // rows of Nb floats start anywhere: element stores
+            __stcs(dst, v.x);
+            if (n + 1 < g.Nb) __stcs(dst + 1, v.y);
+            if (n + 2 < g.Nb) __stcs(dst + 2, v.z);
+            if (n + 3 < g.Nb) __stcs(dst + 3, v.w);
+          } else {
+            __stcs(reinterpret_cast<float4*>(dst), v);
+          }
         }
       }
     }

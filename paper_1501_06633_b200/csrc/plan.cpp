@@ -17,7 +17,7 @@ const char* const kOptionNames[OPT_COUNT] = {
     "FFMA_TILE_M", "FFMA_COLS", "FFMA_KH", "FFMA_STREAMK",
     "UMMA_KC", "UMMA_PAIR", "UMMA_MERGE", "UMMA_STAGE_KB", "UMMA_COLS",
     "WGRAD_SPLITS", "WGRAD_PAIR", "SM_COUNT", "X3_CHUNK_ROWS", "DEBUG_STATUS",
-    "KERNEL_CLOCK", "TEST_MISSING_ARRIVAL"};
+    "KERNEL_CLOCK", "RAGGED_PADDED", "TEST_MISSING_ARRIVAL"};
 struct OptionSlot {
   std::atomic<int32_t> value{0};
   std::atomic<bool> set{false};
@@ -202,7 +202,8 @@ static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* 
 static double pick_columns(const ConvDims& d, int Wo, int cols, int* nn_out, int* T_out) {
   int best_nn = 4, best_T = 1;
   double best_eff = -1.0;
-  for (int nn = (d.Nb < cols ? d.Nb : cols); nn >= 4; nn -= 4) {
+  const int nb4 = align_up(d.Nb, 4);       // (ragged counts: the tile's images round up)
+  for (int nn = (nb4 < cols ? nb4 : cols); nn >= 4; nn -= 4) {
     int T = cols / nn;
     if (T > Wo) T = Wo;
     const double eff =
@@ -266,15 +267,16 @@ static double ffma_waves(int64_t tiles, int units, int k_rows_per_tile, bool all
 }
 
 maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
-                        ConvGeom* g, KStepTable* t, bool allow_split) {
+                        ConvGeom* g, KStepTable* t, bool allow_split, bool ragged) {
   int32_t Ho, Wo;
   maxdnn_status st = check_dims(d, &Ho, &Wo);
   if (st != MAXDNN_OK) return st;
   st = common_limits(d, 4);
   if (st != MAXDNN_OK) return st;
-  if (d.Nb % 4 != 0 || d.No % 4 != 0) return MAXDNN_NOT_SUPPORTED;
+  if (!ragged && (d.Nb % 4 != 0 || d.No % 4 != 0)) return MAXDNN_NOT_SUPPORTED;
   if (sm_count <= 0) return MAXDNN_INVALID_VALUE;
   fill_geom(d, Ho, Wo, g);
+  if (ragged) allow_split = false;
 
   // Tile shape: fewest SM-time units over the waves of persistent CTAs.
   double best_t = 1e300;
@@ -287,6 +289,8 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   for (const FfmaShape& sh : kFfmaShapes) {
     if (force_tile_m > 0 && sh.m != force_tile_m) continue;
     if (force_cols > 0 && sh.cols != force_cols) continue;
+    // the ragged kernel is built for the blocks that leave room for two copy warps
+    if (ragged && (sh.cols != 128 || sh.m > 128 || sh.m == 96)) continue;
     if (force_tile_m <= 0 && sh.m > align_up(d.No, 32) && sh.m != 32) continue;
     int nn, T;
     pick_columns(d, Wo, sh.cols, &nn, &T);
@@ -344,7 +348,7 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   g->a_stage_bytes = g->a_box_bytes;
   // One box per stage whenever the tile's columns are one contiguous run of the map
   // (one pixel, or adjacent pixels of a stride-1 layer); else one box per pixel.
-  g->fixed_pitch = (g->tile_px * g->tile_n == g->tile_cols &&
+  g->fixed_pitch = (!ragged && g->tile_px * g->tile_n == g->tile_cols &&
                     (g->tile_px == 1 || (d.stride_w == 1 && kwc == 1))) ? 1 : 0;
   if (g->fixed_pitch) {
     g->b_boxes = 1;

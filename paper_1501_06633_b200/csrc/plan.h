@@ -20,7 +20,7 @@ enum OptionId : int {
   OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_KH, OPT_FFMA_STREAMK,
   OPT_UMMA_KC, OPT_UMMA_PAIR, OPT_UMMA_MERGE, OPT_UMMA_STAGE_KB, OPT_UMMA_COLS,
   OPT_WGRAD_SPLITS, OPT_WGRAD_PAIR, OPT_SM_COUNT, OPT_X3_CHUNK_ROWS, OPT_DEBUG_STATUS,
-  OPT_KERNEL_CLOCK, OPT_TEST_MISSING_ARRIVAL, OPT_COUNT
+  OPT_KERNEL_CLOCK, OPT_RAGGED_PADDED, OPT_TEST_MISSING_ARRIVAL, OPT_COUNT
 };
 bool option_is_set(OptionId id);
 int option(OptionId id, int unset_value = 0);          // the value, or unset_value
@@ -151,8 +151,9 @@ maxdnn_status check_desc(const maxdnn_conv_desc* d, int32_t* Ho, int32_t* Wo);
 
 // FFMA kernel plan.  force_tile_m / force_cols > 0 pin the tile shape (ablations).
 // allow_split: the caller can provide the workspace of a split tail (see ffma_split_bytes).
+// ragged: Nb and No need not be multiples of 4 (the kernel instance with copy warps).
 maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int force_cols,
-                        ConvGeom* g, KStepTable* t, bool allow_split = false);
+                        ConvGeom* g, KStepTable* t, bool allow_split = false, bool ragged = false);
 
 // Workspace of the fp32 kernel's split tail for any plan on `sm_count` SMs: one slot of
 // partial sums per CTA (the largest tile has 32768 columns x filters), then one flag per CTA.

@@ -227,6 +227,9 @@ def test_ragged_workspace_sizes():
     r256 = lambda b: (b + 255) // 256 * 256
     d = mx.ConvDesc.make(30, 14, 9, 16, 50, 3, 1, 1, 1.0)
     Ho, Wo = 9, 14
+    mx.set_option("RAGGED_PADDED", -1)
+    assert mx.conv_fprop_ragged_workspace(d, mx.KERNEL_FP32) == 0     # staged inside the kernel
+    mx.unset_option("RAGGED_PADDED")
     assert mx.conv_fprop_ragged_workspace(d, mx.KERNEL_FP32) == \
         r256(16 * 9 * 14 * 32 * 4) + r256(16 * 9 * 52 * 4) + r256(52 * Ho * Wo * 32 * 4)
     assert mx.conv_fprop_ragged_workspace(d, mx.KERNEL_BF16) == \

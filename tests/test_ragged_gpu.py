@@ -1,5 +1,6 @@
 """FPROP for minibatch / filter counts outside the 16-byte row rule of the bulk tensor
-copies, through zero-padded staging tensors, against the oracle."""
+copies — staged inside the fp32 kernel by copy warps, through zero-padded staging tensors
+for the tensor-core kernels (and for fp32 on request) — against the oracle."""
 import numpy as np
 import pytest
 import torch
@@ -16,6 +17,8 @@ TOL = {"fp32": 1e-5, "tf32": 5e-3, "bf16": 2e-2}
 SHAPES = [
     # Nb Wi Hi Nc No Sk stride pad alpha
     (30, 14, 9, 16, 50, 3, 1, 1, 1.0),       # both ragged
+    (62, 20, 13, 40, 130, 3, 1, 1, 1.0),     # several tiles of 128 filters, two pixels x 64 images
+    (150, 9, 7, 12, 70, 5, 1, 2, -1.0),      # two image chunks, the second ragged
     (7, 12, 12, 5, 3, 5, 2, 2, 0.5),         # tiny odd counts, stride 2
     (33, 23, 19, 3, 96, 11, 4, 0, 1.0),      # one image over a multiple of 32
     (64, 10, 8, 24, 45, 3, 1, 0, 1.0),       # only the filters ragged
@@ -23,10 +26,14 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("kernel", ["fp32", "tf32", "bf16"])
+@pytest.mark.parametrize("kernel", ["fp32", "fp32-padded", "tf32", "bf16"])
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(str(v) for v in s))
 def test_fprop_ragged(kernel, shape):
     Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha = shape
+    in_kernel = kernel == "fp32"
+    if kernel.startswith("fp32"):
+        mx.set_option("RAGGED_PADDED", -1 if in_kernel else 1)      # pin the route
+        kernel = "fp32"
     w = wl.Workload("ragged", Nb, Wi, Hi, Nc, No, Sk, stride, pad, alpha, ("uniform", -1.0, 1.0),
                     ("uniform", -1.0, 1.0), 5150 + Nb)
     inp, filt = wl.make_inputs(w)
@@ -36,8 +43,9 @@ def test_fprop_ragged(kernel, shape):
         st = mx.fprop_status(d, torch.from_numpy(inp).cuda(), torch.from_numpy(filt).cuda(), out0)
         assert st == mx.NOT_SUPPORTED                               # the plain entry point refuses
     need = mx.conv_fprop_ragged_workspace(d, KIND[kernel])
-    assert need > 0
-    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    assert (need == 0) if in_kernel else (need > 0)      # the fp32 kernel pads nothing
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    launches = mx.launch_count()
     if kernel == "bf16":
         to_dev = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
         r_in, r_f = wl.from_bf16_bits(wl.to_bf16_bits(inp)), wl.from_bf16_bits(wl.to_bf16_bits(filt))
@@ -47,6 +55,7 @@ def test_fprop_ragged(kernel, shape):
     out = torch.full((mx.conv_out_elems(d),), float("nan"), dtype=torch.float32, device="cuda")
     mx.conv_fprop_ragged(d, to_dev(inp), to_dev(filt), out, ws, KIND[kernel])
     assert mx.last_device_status() == mx.OK
+    assert mx.launch_count() - launches == (1 if in_kernel else 4)
     ref = oracle.conv_fprop(r_in, r_f, stride=stride, pad=pad, alpha=alpha)
     got = out.cpu().numpy().reshape(ref.shape)
     assert np.all(np.isfinite(got))
