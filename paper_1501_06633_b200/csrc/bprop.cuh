@@ -304,25 +304,25 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
       for (int q = 0; q < 8; ++q) {
         const uint8_t* sg = ss + g_base + (((uint32_t)q ^ o7) << 4);
         const uint8_t* sp = ss + p_base + (((uint32_t)q ^ t7) << 4);
-        float4 G[8], P[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          G[j] = *reinterpret_cast<const float4*>(sg + j * 2048);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          P[i] = *reinterpret_cast<const float4*>(sp + i * 2048);
         // first the even pair of r for all 64 results, then the odd pair: consecutive
-        // multiply-adds never depend on each other
+        // multiply-adds never depend on each other.  Each half is fetched by 8-byte loads of
+        // its own (16 operand registers live at a time instead of 64; beside a stream of
+        // packed multiply-adds an 8-byte load is nearly free, a 16-byte load is not).
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
+          float2 G[8], P[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            G[j] = lds64(sg + j * 2048 + half * 8);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            P[i] = lds64(sp + i * 2048 + half * 8);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float2 gj = half ? make_float2(G[j].z, G[j].w) : make_float2(G[j].x, G[j].y);
 #pragma unroll
             for (int ii = 0; ii < 8; ++ii) {
               const int i = (j & 1) ? 7 - ii : ii;
-              const float2 pi = half ? make_float2(P[i].z, P[i].w) : make_float2(P[i].x, P[i].y);
-              acc[i][j] = __ffma2_rn(pi, gj, acc[i][j]);
+              acc[i][j] = __ffma2_rn(P[i], G[j], acc[i][j]);
             }
           }
         }

@@ -81,16 +81,6 @@ struct Frag {
   float4 b[NR / 4];
 };
 
-// One 8-byte shared-memory load.  Written as an instruction of its own so that two
-// neighbouring ones are not fused into a 16-byte load: next to a stream of packed
-// multiply-adds a 16-byte load costs about 1.3 issue cycles, an 8-byte load about 0.1
-// (measured: the microbenchmark in ubench_fp32.cu).
-__device__ __forceinline__ float2 lds64(const float* p) {
-  float2 v;
-  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(smem_u32(p)));
-  return v;
-}
-
 // Thread (to, tn) of the 16 x 16 consumer grid reads, from row `a_row` of the staged
 // filter box, MR values (float4 groups 64 filters apart, or float2 groups 32 apart)
 // and, from the staged patch row, NR values (float4 groups 64 columns apart).

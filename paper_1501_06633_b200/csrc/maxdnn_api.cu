@@ -11,13 +11,7 @@
 #include "ffma_conv.cuh"
 #include "plan.h"
 #include "umma_conv.cuh"
-#include "umma_chunk_conv.cuh"
-#include "umma_pair_chunk_conv.cuh"
-#include "wgrad_umma_chunk.cuh"
-#include "wgrad_umma_pair_chunk.cuh"
-#include "umma_pair_conv.cuh"
 #include "wgrad_umma.cuh"
-#include "wgrad_umma_pair.cuh"
 
 namespace maxdnn {
 namespace {
@@ -34,13 +28,9 @@ struct DeviceState {
   // attr_mu, read without it afterwards
   std::mutex attr_mu;
   std::atomic<bool> ffma_attr[40];
-  std::atomic<bool> umma_attr[4];
+  std::atomic<bool> umma_attr[8];
   std::atomic<bool> wgrad_attr;
-  std::atomic<bool> umma_chunk_attr;
-  std::atomic<bool> umma_pair_chunk_attr;
-  std::atomic<bool> wgrad_chunk_attr;
-  std::atomic<bool> wgrad_pair_chunk_attr;
-  std::atomic<bool> wgrad_umma_attr[4];
+  std::atomic<bool> wgrad_umma_attr[8];
   // Side streams for the strided map gradient, whose residue classes are independent
   // launches: run side by side, the tail wave of one class overlaps the next class.
   // Workspaces of the fp32 kernel's split tail, one per stream that has used one (work on
@@ -377,76 +367,57 @@ maxdnn_status fprop_fp32(const maxdnn_conv_desc* desc, const float* in, const fl
   return fprop_fp32(dims_from(*desc), in, filt, out, stream);
 }
 
-template <bool BF16>
-maxdnn_status launch_umma_pair(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
-                               const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
-  auto kern = umma_pair_conv_kernel<BF16>;
-  const int slot = BF16 ? 3 : 2;
-  if (ensure_smem_attr(ds, &ds->umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
-  cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, mf, mi, mo, args) != cudaSuccess) {
-    cudaGetLastError();
-    return MAXDNN_CUDA_ERROR;
-  }
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return MAXDNN_OK;
-}
-
-maxdnn_status launch_umma_chunk(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
-                                const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
-  auto kern = umma_chunk_conv_kernel;
-  if (ensure_smem_attr(ds, &ds->umma_chunk_attr, kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-  kern<<<args.g.grid, kUmmaChunkThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
-  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return MAXDNN_OK;
-}
-
-maxdnn_status launch_umma_pair_chunk(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
-                                     const CUtensorMap& mo, const UmmaArgs& args,
-                                     cudaStream_t stream) {
-  auto kern = umma_pair_chunk_conv_kernel;
-  if (ensure_smem_attr(ds, &ds->umma_pair_chunk_attr, kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
-  cfg.blockDim = dim3(kUmmaChunkThreads, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, mf, mi, mo, args) != cudaSuccess) {
-    cudaGetLastError();
-    return MAXDNN_CUDA_ERROR;
-  }
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  return MAXDNN_OK;
-}
-
-template <bool BF16>
+// One launch of the tensor-core forward kernel: one-SM or two-SM tiles (a cluster of two
+// CTAs), K in one accumulator or summed in chunks.
+template <bool BF16, bool PAIR, bool CHUNK>
 maxdnn_status launch_umma(DeviceState* ds, const CUtensorMap& mf, const CUtensorMap& mi,
                           const CUtensorMap& mo, const UmmaArgs& args, cudaStream_t stream) {
-  auto kern = umma_conv_kernel<BF16>;
-  const int slot = BF16 ? 1 : 0;
+  auto kern = umma_conv_kernel<BF16, PAIR, CHUNK>;
+  const int slot = (BF16 ? 1 : 0) + (PAIR ? 2 : 0) + (CHUNK ? 4 : 0);
   if (ensure_smem_attr(ds, &ds->umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-  kern<<<args.g.grid, kUmmaThreads, args.g.smem_bytes, stream>>>(mf, mi, mo, args);
-  if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
+  cfg.blockDim = dim3(umma_threads(CHUNK), 1, 1);
+  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = PAIR ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, kern, mf, mi, mo, args) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
   g_launches.fetch_add(1, std::memory_order_relaxed);
+  return MAXDNN_OK;
+}
+
+// One launch of the tensor-core filter-gradient kernel.
+template <bool BF16, bool PAIR, bool CHUNK>
+maxdnn_status launch_wgrad_umma(DeviceState* ds, const CUtensorMap& mg, const CUtensorMap& mi,
+                                const WgradUmmaArgs& args, cudaStream_t stream) {
+  auto kern = wgrad_umma_kernel<BF16, PAIR, CHUNK>;
+  const int slot = (BF16 ? 1 : 0) + (PAIR ? 2 : 0) + (CHUNK ? 4 : 0);
+  if (ensure_smem_attr(ds, &ds->wgrad_umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)args.g.grid, 1, 1);
+  cfg.blockDim = dim3(wgrad_umma_threads(CHUNK), 1, 1);
+  cfg.dynamicSmemBytes = (size_t)args.g.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = PAIR ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, kern, mg, mi, args) != cudaSuccess) {
+    cudaGetLastError();
+    return MAXDNN_CUDA_ERROR;
+  }
   return MAXDNN_OK;
 }
 
@@ -559,14 +530,14 @@ maxdnn_status fprop_umma(const ConvDims& cd, int elem_bytes, const void* in, con
     if (bf16) return MAXDNN_INVALID_VALUE;
     const int steps = chunk_rows / g.rows;
     args.chunk_steps = (uint32_t)(steps < 1 ? 1 : steps);
-    return g.pair ? launch_umma_pair_chunk(ds, mf, mi, mo, args, stream)
-                  : launch_umma_chunk(ds, mf, mi, mo, args, stream);
+    return g.pair ? launch_umma<false, true, true>(ds, mf, mi, mo, args, stream)
+                  : launch_umma<false, false, true>(ds, mf, mi, mo, args, stream);
   }
   if (g.pair)
-    return bf16 ? launch_umma_pair<true>(ds, mf, mi, mo, args, stream)
-                : launch_umma_pair<false>(ds, mf, mi, mo, args, stream);
-  return bf16 ? launch_umma<true>(ds, mf, mi, mo, args, stream)
-              : launch_umma<false>(ds, mf, mi, mo, args, stream);
+    return bf16 ? launch_umma<true, true, false>(ds, mf, mi, mo, args, stream)
+                : launch_umma<false, true, false>(ds, mf, mi, mo, args, stream);
+  return bf16 ? launch_umma<true, false, false>(ds, mf, mi, mo, args, stream)
+              : launch_umma<false, false, false>(ds, mf, mi, mo, args, stream);
 }
 
 maxdnn_status fprop_umma(const maxdnn_conv_desc* desc, int elem_bytes, const void* in,
@@ -915,31 +886,13 @@ maxdnn_status bprop_filter(const ConvDims& d, maxdnn_kernel_kind kind, const voi
     const uint32_t m_mma = g.pair ? 256u : 128u;
     uargs.idesc = (1u << 4) | (fmt << 7) | (fmt << 10)      // fp32 accumulate, operand formats;
                   | ((n_mma >> 3) << 17) | ((m_mma >> 4) << 24);   // both operands K-major; N, M
-    const int slot = (bf16 ? 1 : 0) + (g.pair ? 2 : 0);
-    if (g.pair) {
-      auto kern = bf16 ? wgrad_umma_pair_kernel<true> : wgrad_umma_pair_kernel<false>;
-      if (ensure_smem_attr(ds, &ds->wgrad_umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
-      cfg.blockDim = dim3(kWgUmmaThreads, 1, 1);
-      cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
-      cfg.stream = stream;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = 2;
-      attr[0].val.clusterDim.y = 1;
-      attr[0].val.clusterDim.z = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      if (cudaLaunchKernelEx(&cfg, kern, mg, mi, uargs) != cudaSuccess) {
-        cudaGetLastError();
-        return MAXDNN_CUDA_ERROR;
-      }
-    } else {
-      auto kern = bf16 ? wgrad_umma_kernel<true> : wgrad_umma_kernel<false>;
-      if (ensure_smem_attr(ds, &ds->wgrad_umma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-      kern<<<g.grid, kWgUmmaThreads, g.smem_bytes, stream>>>(mg, mi, uargs);
-    }
+    if (g.pair)
+      st = bf16 ? launch_wgrad_umma<true, true, false>(ds, mg, mi, uargs, stream)
+                : launch_wgrad_umma<false, true, false>(ds, mg, mi, uargs, stream);
+    else
+      st = bf16 ? launch_wgrad_umma<true, false, false>(ds, mg, mi, uargs, stream)
+                : launch_wgrad_umma<false, false, false>(ds, mg, mi, uargs, stream);
+    if (st != MAXDNN_OK) return st;
   }
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -1255,28 +1208,9 @@ maxdnn_status bprop_filter_tf32x3(const maxdnn_conv_desc* desc, const float* in,
   args.x3_per_part = (uint32_t)(desc->Nb / 32);
   args.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (((uint32_t)g.n_mma >> 3) << 17) |
                (((g.pair ? 256u : 128u) >> 4) << 24);
-  if (g.pair) {
-    if (ensure_smem_attr(ds, &ds->wgrad_pair_chunk_attr, wgrad_umma_pair_chunk_kernel) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)g.grid, 1, 1);
-    cfg.blockDim = dim3(kWgChunkThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, wgrad_umma_pair_chunk_kernel, mg, mi, args) != cudaSuccess) {
-      cudaGetLastError();
-      return MAXDNN_CUDA_ERROR;
-    }
-  } else {
-    if (ensure_smem_attr(ds, &ds->wgrad_chunk_attr, wgrad_umma_chunk_kernel) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
-    wgrad_umma_chunk_kernel<<<g.grid, kWgChunkThreads, g.smem_bytes, stream>>>(mg, mi, args);
-  }
+  st = g.pair ? launch_wgrad_umma<false, true, true>(ds, mg, mi, args, stream)
+              : launch_wgrad_umma<false, false, true>(ds, mg, mi, args, stream);
+  if (st != MAXDNN_OK) return st;
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (g.splits > 1) {

@@ -179,6 +179,16 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* m, 
       : "memory");
 }
 
+// One 8-byte shared-memory load.  Written as an instruction of its own so that two
+// neighbouring ones are not fused into a 16-byte load: next to a stream of packed
+// multiply-adds a 16-byte load costs about 1.3 issue cycles, an 8-byte load about 0.1
+// (measured: the microbenchmark in ubench_fp32.cu).
+__device__ __forceinline__ float2 lds64(const void* p) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(smem_u32(p)));
+  return v;
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
