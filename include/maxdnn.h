@@ -209,8 +209,11 @@ maxdnn_status maxdnn_conv_fprop_host(const maxdnn_conv_desc* desc, maxdnn_kernel
  * library holds those 256 bytes until the process exits).
  *
  * Same arguments, layouts, result and NOT_SUPPORTED cases as maxdnn_conv_fprop
- * (the same plan and kernel — tile options included — so the result is bitwise
- * the same).  In addition:
+ * (the same kernel and tile choice, tile options included; bitwise the same
+ * result whenever maxdnn_conv_fprop's plan runs whole tiles only — where that
+ * plan splits its last wave along K, which needs a workspace, this entry point
+ * runs the last wave as whole tiles and the two results differ by rounding
+ * order).  In addition:
  *   - A problem whose kernel would need more than the 256 bytes of built-in
  *     scratch is refused with MAXDNN_NOT_SUPPORTED and nothing is launched.
  *     (The fp32 kernel needs 8 bytes for every descriptor it supports today;

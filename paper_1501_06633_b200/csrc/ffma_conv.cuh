@@ -30,7 +30,18 @@ __host__ __device__ constexpr int ffma_threads(int mr, int nr, bool ragged = fal
 
 // Multiply-add order per register-block shape (see fma_block), from timings on B200.
 __host__ __device__ constexpr int ffma_order(int mr, int nr) {
+#ifdef MAXDNN_ORDER_8x16
+  if (mr == 8 && nr == 16) return MAXDNN_ORDER_8x16;
+#endif
   return (mr == 16 && nr == 8) ? 0 : (mr == 6 && nr == 8) ? 2 : 1;
+}
+
+// Rows of K per iteration of the main loop, by register block and rows per K step.  The
+// 8 x 8 and 6 x 8 blocks gain 5-8 % from long iterations (16 rows for the 32-row steps of the
+// many-channel layers, 32 rows for the ~100-row steps of the few-channel layers); the blocks
+// of 128 accumulators lose 1.5 % with 8 rows, the 4 x 8 and 4 x 16 blocks 2-3 %, and keep 4.
+__host__ __device__ constexpr int ffma_long_block(int mr, int nr, bool long_steps) {
+  return ((mr == 8 || mr == 6) && nr == 8) ? (long_steps ? 32 : 16) : 4;
 }
 
 struct FfmaArgs {
@@ -214,12 +225,18 @@ struct FfmaProducer {
       dst += g.b_slot_bytes;
       w += g.stride_w;
     }
+    advance(g, mt);
+    return true;
+  }
+
+  // The state after one more K step has been issued (by this thread or by another one that
+  // keeps an identical copy of the state).
+  __device__ __forceinline__ void advance(const ConvGeom& g, int mt) {
     if (++stage == g.stages) { stage = 0; phase ^= 1u; }
     if (++step == step_end) {
       item += SPLIT ? 1 : (int)gridDim.x;
       set_item(g, mt);
     }
-    return true;
   }
 
   // After a failed wait: let every copy already issued land before the CTA's shared
@@ -408,7 +425,9 @@ __device__ __noinline__ void ragged_copy_warp(const FfmaArgs& args, int role, co
 // 16 columns and by 16-byte loads for the others (which is faster was measured per block).
 // RAGGED: the copy warps of ragged_copy_warp instead of bulk tensor copies, bounds-checked
 // element stores (whole tiles, one box per pixel only).
-template <int MR, int NR, bool FIXED, bool SPLIT, bool RAGGED = false>
+// LB: rows of K per iteration of the main loop (4, or more for the small register blocks:
+// see ffma_long_block).
+template <int MR, int NR, bool FIXED, bool SPLIT, bool RAGGED = false, int LB = 4>
 __global__ void __launch_bounds__(ffma_threads(MR, NR, RAGGED), 1)
 ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
                  const __grid_constant__ CUtensorMap map_in,
@@ -418,6 +437,8 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   constexpr int NH = NR / 4;            // float4 column groups per thread
   constexpr bool INLINE = ffma_inline_producer(MR, NR) && !RAGGED;
   constexpr bool W64 = NR == 16;
+  constexpr int kLongBlock = LB;   // rows per iteration of the first loop over a step's rows
+  static_assert(LB >= 4 && LB % 2 == 0, "rows per iteration");
   static_assert(!RAGGED || (!FIXED && !SPLIT && !ffma_inline_producer(MR, NR)), "ragged instances");
   extern __shared__ uint8_t smem_raw[];
   const ConvGeom& g = args.g;
@@ -487,17 +508,28 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   // large blocks 3 %, the loads sitting in warp 0's instruction stream).
   FfmaProducer<SPLIT> prod;
   bool prod_ok = true;
+  // The consumer warps take turns at the producer's job, one K step each, so that its
+  // instructions are spread over the four schedulers instead of slowing one of them (all
+  // the others end up waiting for that one).  Every thread keeps the producer's state and
+  // advances it once per K step; only lane 0 of the warp whose turn it is issues the copies.
+  int turn = 0;
   if constexpr (INLINE) {
-    if (warp == 0) {
-      if (lane == 0) {
-        prefetch_tensormap(&map_filt);
-        prefetch_tensormap(&map_in);
-        prod.init(g, Mt);
-        for (int s = 0; s + 2 < stages && prod_ok && prod.has_work(g); ++s)
+    prod.init(g, Mt);
+    if (warp == 0 && lane == 0) {
+      prefetch_tensormap(&map_filt);
+      prefetch_tensormap(&map_in);
+    }
+    for (int s = 0; s + 2 < stages && prod.has_work(g); ++s) {
+      if (warp == 0) {
+        if (lane == 0 && prod_ok)
           prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off, base + b_off,
                                                full_bar, empty_bar, Mt);
+        else
+          prod.advance(g, Mt);
+        __syncwarp();
+      } else {
+        prod.advance(g, Mt);
       }
-      __syncwarp();
     }
   }
 
@@ -567,17 +599,41 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
         // Refill the slot this CTA finished two steps ago (every warp has released it
         // by now, so the wait does not hold warp 0 back) with the K step that is
         // (stages - 2) ahead of the one being consumed.
-        if (warp == 0) {
-          if (lane == 0 && prod_ok && prod.has_work(g))
-            prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off,
-                                                 base + b_off, full_bar, empty_bar, Mt);
-          __syncwarp();
+        if (prod.has_work(g)) {
+          if (warp == turn) {
+            if (lane == 0 && prod_ok)
+              prod_ok = prod.template issue<false>(args, &map_filt, &map_in, base + a_off,
+                                                   base + b_off, full_bar, empty_bar, Mt);
+            else
+              prod.advance(g, Mt);
+            __syncwarp();
+          } else {
+            prod.advance(g, Mt);
+          }
         }
+        turn = (turn + 1) & 7;
       }
       // f0 holds row 0 of this stage.  Four rows per iteration while the row
       // after the block is still inside the stage.
       const int rows = s < g.short_from ? rows_full : g.rows_short;
       int r = 0;
+      if constexpr (kLongBlock > 4) {
+        // The small register blocks spend a larger share of their instructions on the
+        // loop itself: they take kLongBlock rows per iteration first.
+#pragma unroll 1
+        for (; r + kLongBlock < rows; r += kLongBlock) {
+#pragma unroll
+          for (int u = 0; u < kLongBlock; u += 2) {
+            load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(u + 1));
+            fma_block<MR, NR>(f0, P, Q);
+            load_frag<MR, NR, FIXED, W64>(f0, MAXDNN_ROW(u + 2));
+            fma_block<MR, NR>(f1, P, Q);
+          }
+          a_ptr += kLongBlock * Mt;
+#pragma unroll
+          for (int h = 0; h < NH; ++h) b_ptr[h] += kLongBlock * b_pitch;
+        }
+      }
 #pragma unroll 1
       for (; r + 4 < rows; r += 4) {
         load_frag<MR, NR, FIXED, W64>(f1, MAXDNN_ROW(1));
@@ -754,7 +810,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   }
 
   if constexpr (INLINE) {
-    if (warp == 0 && lane == 0 && !(ok && prod_ok)) prod.drain(g, full_bar);
+    if (lane == 0 && !(ok && prod_ok)) prod.drain(g, full_bar);
   }
   if (args.clock_stamp != 0 && threadIdx.x == 0 && args.wc.status) {
     atomicMax(args.wc.status + (SPLIT ? 4 : 2), (uint32_t)(clock64() - stamp_cycles));

@@ -27,7 +27,7 @@ struct DeviceState {
   // "dynamic shared memory limit raised" flags, one per kernel instance: set once under
   // attr_mu, read without it afterwards
   std::mutex attr_mu;
-  std::atomic<bool> ffma_attr[40];
+  std::atomic<bool> ffma_attr[80];
   std::atomic<bool> umma_attr[8];
   std::atomic<bool> wgrad_attr;
   std::atomic<bool> wgrad_umma_attr[8];
@@ -210,10 +210,10 @@ struct PlanCache {
   }
 };
 
-template <int MR, int NR, bool FIXED, bool SPLIT, bool RAGGED = false>
+template <int MR, int NR, bool FIXED, bool SPLIT, bool RAGGED = false, int LB = 4>
 maxdnn_status launch_ffma(DeviceState* ds, int slot, const CUtensorMap& mf, const CUtensorMap& mi,
                           const FfmaArgs& args, cudaStream_t stream) {
-  auto kern = ffma_conv_kernel<MR, NR, FIXED, SPLIT, RAGGED>;
+  auto kern = ffma_conv_kernel<MR, NR, FIXED, SPLIT, RAGGED, LB>;
   if (ensure_smem_attr(ds, &ds->ffma_attr[slot], kern) != MAXDNN_OK) return MAXDNN_CUDA_ERROR;
   kern<<<args.g.grid, ffma_threads(MR, NR, RAGGED), args.g.smem_bytes, stream>>>(mf, mi, args);
   if (cudaGetLastError() != cudaSuccess) return MAXDNN_CUDA_ERROR;
@@ -227,13 +227,21 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
                             const FfmaArgs& args, cudaStream_t stream, bool split = false) {
   const ConvGeom& g = args.g;
   const bool fx = g.fixed_pitch != 0;
+  // rows per iteration of the kernel's main loop: by block shape and step length
+  const bool long_steps = g.rows >= 64;
+#define MAXDNN_FFMA_LAUNCH(MR, NR, LB, SLOT)                                                        \
+  do {                                                                                              \
+    if (split)                                                                                      \
+      return fx ? launch_ffma<MR, NR, true, true, false, LB>(ds, (SLOT) + 16, mf, mi, args, stream)   \
+                : launch_ffma<MR, NR, false, true, false, LB>(ds, (SLOT) + 17, mf, mi, args, stream); \
+    return fx ? launch_ffma<MR, NR, true, false, false, LB>(ds, (SLOT), mf, mi, args, stream)       \
+              : launch_ffma<MR, NR, false, false, false, LB>(ds, (SLOT) + 1, mf, mi, args, stream); \
+  } while (0)
 #define MAXDNN_FFMA_CASE(M, C, MR, NR, SLOT)                                               \
   if (g.tile_m == (M) && g.tile_cols == (C)) {                                             \
-    if (split)                                                                             \
-      return fx ? launch_ffma<MR, NR, true, true>(ds, (SLOT) + 16, mf, mi, args, stream)   \
-                : launch_ffma<MR, NR, false, true>(ds, (SLOT) + 17, mf, mi, args, stream); \
-    return fx ? launch_ffma<MR, NR, true, false>(ds, (SLOT), mf, mi, args, stream)         \
-              : launch_ffma<MR, NR, false, false>(ds, (SLOT) + 1, mf, mi, args, stream);   \
+    if (ffma_long_block(MR, NR, true) != ffma_long_block(MR, NR, false) && long_steps)     \
+      MAXDNN_FFMA_LAUNCH(MR, NR, ffma_long_block(MR, NR, true), (SLOT) + 40);              \
+    MAXDNN_FFMA_LAUNCH(MR, NR, ffma_long_block(MR, NR, false), (SLOT));                    \
   }
   MAXDNN_FFMA_CASE(256, 128, 16, 8, 0)
   MAXDNN_FFMA_CASE(128, 256, 8, 16, 2)
@@ -244,6 +252,7 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   MAXDNN_FFMA_CASE(64, 256, 4, 16, 14)
   MAXDNN_FFMA_CASE(32, 128, 2, 8, 12)
 #undef MAXDNN_FFMA_CASE
+#undef MAXDNN_FFMA_LAUNCH
   return MAXDNN_NOT_SUPPORTED;
 }
 

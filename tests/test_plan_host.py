@@ -309,8 +309,12 @@ def plan_signature(dims, kind, sms=148):
     if kind == mx.KERNEL_FP32:
         one_box = info.tile_px * info.tile_n == info.tile_cols and \
             (info.tile_px == 1 or (stride == 1 and info.kwc == 1))
+        # rows of K per step >= 64: the 8 x 8 and 6 x 8 blocks then run the instance with the
+        # longer main-loop iterations
+        long_steps = info.kc * info.kwc * info.khc >= 64 and info.tile_cols == 128 and \
+            info.tile_m in (96, 128)
         return ("fp32", info.tile_m, info.tile_cols, one_box, info.kwc > 1, info.khc > 1,
-                info.split_tiles > 0)
+                info.split_tiles > 0, long_steps)
     few = Nc < (8 if kind == mx.KERNEL_TF32 else 16)
     return ("tf32" if kind == mx.KERNEL_TF32 else "bf16", info.pair, info.tile_px * info.tile_n,
             few, info.kwc > 1, stride > 1)
@@ -360,7 +364,7 @@ def test_every_benchmarked_plan_is_one_a_gpu_parity_test_runs():
         sig = plan_signature(wl.ALL[name].dims, mx.KERNEL_FP32)
         # which filter rows / columns a step spans is a property of the shape, not a kernel
         # instance: match on (tile, one box per stage?, split?)
-        key = (sig[1], sig[2], sig[3], sig[6])
-        if key not in {(r[1], r[2], r[3], r[6]) for r in reduced}:
+        key = (sig[1], sig[2], sig[3], sig[6], sig[7])
+        if key not in {(r[1], r[2], r[3], r[6], r[7]) for r in reduced}:
             missing.append((name, sig))
     assert not missing, "full-size fp32 plans without a reduced-size parity case: %r" % missing
