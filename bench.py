@@ -40,12 +40,15 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # under profiles/ (None = not captured).  Writes still sitting in L2 when the kernel ends
 # are not in these figures, which is why they are below the algorithmic bytes.
 NCU_TRAFFIC_BYTES = {
-    ("first11x11s4", "fp32"): int((79.32 + 94.30) * 1e6),
-    ("mid5x5", "fp32"): int((38.50 + 38.82) * 1e6),
-    ("large3x3", "fp32"): int((104.3 + 151.1) * 1e6),
-    ("large3x3", "bf16"): int((52.02 + 145.9) * 1e6),
-    ("large3x3", "tf32"): int((104.1 + 149.0) * 1e6),
-    ("mid5x5", "bf16"): int((19.17 + 37.48) * 1e6),
+    # fp32 plans with a split tail: both launches of a step (whole tiles + split tail)
+    ("first11x11s4", "fp32"): int((79.71 + 93.40) * 1e6),
+    ("mid5x5", "fp32"): int((34.39 + 22.83 + 12.10 + 0.49) * 1e6),
+    ("wide3x3", "fp32"): int((24.82 + 0.29 + 8.24 + 0.0) * 1e6),
+    ("large3x3", "fp32"): int((100.3 + 140.8 + 8.98 + 0.07) * 1e6),
+    ("large3x3", "bf16"): int((52.02 + 146.8) * 1e6),
+    ("large3x3", "tf32"): int((104.0 + 149.8) * 1e6),
+    ("mid5x5", "bf16"): int((19.17 + 37.60) * 1e6),
+    ("first11x11s4", "bf16"): int((39.67 + 89.99) * 1e6),
 }
 
 

@@ -22,7 +22,7 @@
 namespace maxdnn {
 
 constexpr int kFfmaConsumerWarps = 8;
-__host__ __device__ constexpr bool ffma_inline_producer(int mr, int nr) { return mr * nr >= 96; }
+__host__ __device__ constexpr bool ffma_inline_producer(int mr, int nr) { return mr * nr >= kFfmaInlineMinAcc; }
 __host__ __device__ constexpr int ffma_threads(int mr, int nr, bool ragged = false) {
   // ragged: four copy warps (two for patches, two for filters) that move the rows themselves
   return (kFfmaConsumerWarps + (ragged ? 4 : ffma_inline_producer(mr, nr) ? 0 : 1)) * 32;
@@ -30,9 +30,6 @@ __host__ __device__ constexpr int ffma_threads(int mr, int nr, bool ragged = fal
 
 // Multiply-add order per register-block shape (see fma_block), from timings on B200.
 __host__ __device__ constexpr int ffma_order(int mr, int nr) {
-#ifdef MAXDNN_ORDER_8x16
-  if (mr == 8 && nr == 16) return MAXDNN_ORDER_8x16;
-#endif
   return (mr == 16 && nr == 8) ? 0 : (mr == 6 && nr == 8) ? 2 : 1;
 }
 
@@ -439,7 +436,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
   constexpr bool W64 = NR == 16;
   constexpr int kLongBlock = LB;   // rows per iteration of the first loop over a step's rows
   static_assert(LB >= 4 && LB % 2 == 0, "rows per iteration");
-  static_assert(!RAGGED || (!FIXED && !SPLIT && !ffma_inline_producer(MR, NR)), "ragged instances");
+  static_assert(!RAGGED || (!FIXED && !SPLIT), "ragged instances");
   extern __shared__ uint8_t smem_raw[];
   const ConvGeom& g = args.g;
 

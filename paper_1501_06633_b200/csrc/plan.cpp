@@ -322,10 +322,9 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   int kc = kc0, kwc = kwc0;
   int khc = khc0;
   // two ring stages must fit (three where a consumer warp issues the copies)
-  const int min_stages = (best_m / 16) * (best_cols / 16) >= 96 ? 3 : 2;
+  const bool inline_producer = !ragged && (best_m / 16) * (best_cols / 16) >= kFfmaInlineMinAcc;
+  const int min_stages = inline_producer ? 3 : 2;
   while (khc > 1 && min_stages * kc * kwc * khc * (best_m + best_cols) * 4 > 200 * 1024) --khc;
-  // Tiles whose first consumer warp issues the copies keep one ring slot as slack.
-  const bool inline_producer = (best_m / 16) * (best_cols / 16) >= 96;
   int n = 0;
   build_table(d, kc, kwc, t, &n, khc);
   while (n > kMaxKSteps && kwc == 1 && kc < 256) {   // very deep filters: larger boxes

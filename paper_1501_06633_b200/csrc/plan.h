@@ -157,6 +157,10 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
 
 // Workspace of the fp32 kernel's split tail for any plan on `sm_count` SMs: one slot of
 // partial sums per CTA (the largest tile has 32768 columns x filters), then one flag per CTA.
+// Register blocks of at least this many accumulators have no producer warp: their consumer
+// warps take turns at issuing the copies (see ffma_conv.cuh), and their ring has >= 3 slots.
+// (Measured: the smaller blocks are 4-8 % slower without their producer warp.)
+constexpr int kFfmaInlineMinAcc = 96;
 constexpr size_t kFfmaSplitSlotBytes = 32768 * 4;
 inline size_t ffma_split_flags_offset(int sm_count) { return (size_t)sm_count * kFfmaSplitSlotBytes; }
 inline size_t ffma_split_bytes(int sm_count) {
