@@ -237,28 +237,34 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   uint32_t p_phase = 0;
   bool p_ok = true;
   const uint32_t tx_bytes = (uint32_t)(g.box_o + g.rows) * 128u;
-  auto produce = [&]() {
-    if (!p_ok || pc.done(g)) return;
-    if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
-      p_ok = false;
-      return;
+  // The eight warps take turns at issuing the copies, one reduction step each (a fixed
+  // issuing warp slows its scheduler, and the whole CTA runs at that scheduler's pace):
+  // every thread keeps the cursor and advances it once per step; lane 0 of the warp whose
+  // turn it is waits for the ring slot (free since two steps) and issues the two copies.
+  auto produce = [&](bool mine) {
+    if (pc.done(g)) return;
+    if (mine && p_ok) {
+      if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
+        p_ok = false;
+      } else {
+        const uint32_t fb = full_bar + 8u * p_stage;
+        const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
+        mbar_arrive_expect_tx(fb, tx_bytes);
+        tma_load_4d(dst, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
+        tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride_w - g.pad_w,
+                    pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc);
+      }
     }
-    const uint32_t fb = full_bar + 8u * p_stage;
-    const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
-    mbar_arrive_expect_tx(fb, tx_bytes);
-    tma_load_4d(dst, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
-    tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride_w - g.pad_w,
-                pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc);
     if (++p_stage == stages) { p_stage = 0; p_phase ^= 1u; }
     pc.advance(g, (int)gridDim.x);
   };
-  const bool issuer = (warp == 0 && lane == 0);
-  if (issuer) {
+  int turn = 0;
+  if (warp == 0 && lane == 0) {
     prefetch_tensormap(&map_dout);
     prefetch_tensormap(&map_in);
-    pc.start(g, blockIdx.x);
-    for (int s = 0; s + 2 < stages; ++s) produce();
   }
+  pc.start(g, blockIdx.x);
+  for (int s = 0; s + 2 < stages; ++s) produce(warp == 0 && lane == 0);
   __syncwarp();
 
   // ------------------------------------------------ arithmetic (all 8 warps)
@@ -293,7 +299,8 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
     const int n_steps = cc.r_end - cc.r;
 
     for (int s = 0; s < n_steps; ++s) {
-      if (issuer) produce();
+      produce(warp == turn && lane == 0);
+      turn = (turn + 1) & 7;
       __syncwarp();
       if (!mbar_wait(full_bar + 8u * stage, phase, args.wc, kDevTimeoutFull)) {
         ok = false;
@@ -359,7 +366,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   }
 
   // Exit path of the issuing lane after a wait ran out: let copies in flight land.
-  if (issuer && (!ok || !p_ok)) {
+  if (lane == 0 && (!ok || !p_ok)) {
     for (int s = 0; s < stages; ++s) {
       const uint32_t par = (s < p_stage) ? p_phase : (p_phase ^ 1u);
       mbar_wait_grace(full_bar + 8u * s, par);
