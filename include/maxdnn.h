@@ -163,6 +163,15 @@ maxdnn_status maxdnn_conv_plan_items(const maxdnn_conv_desc* desc, int32_t sm_co
  * tensor copies), Sk > 127, Nc > 32767, a map dimension that does not fit the
  * tensor-copy descriptor (>= 2^31 bytes in one row pitch), or a device that is
  * not sm_100.
+ * Memory the library owns: where the plan splits its last wave of tiles along K (see
+ * maxdnn_conv_plan_items) the partial sums go through a workspace of 128 KB per SM that
+ * the library allocates once per (device, stream) — on the first such call on that
+ * stream, never during stream capture (a capture on a stream that has no workspace yet
+ * runs whole tiles only; up to eight streams per device get one, later ones run whole
+ * tiles only).  The workspace belongs to the stream: launches on one stream are ordered
+ * and share it safely; a graph captured on stream S uses S's workspace, so its replays
+ * must not overlap each other or other fp32 FPROP work on S.  Results of the two plans
+ * differ by rounding order only; each is bitwise reproducible from run to run.
  */
 maxdnn_status maxdnn_conv_fprop(const maxdnn_conv_desc* desc, const float* in, const float* filt,
                                 float* out, void* cuda_stream);

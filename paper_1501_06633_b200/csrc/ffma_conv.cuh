@@ -33,10 +33,11 @@ __host__ __device__ constexpr int ffma_order(int mr, int nr) {
   return (mr == 16 && nr == 8) ? 0 : (mr == 6 && nr == 8) ? 2 : 1;
 }
 
-// Rows of K per iteration of the main loop, by register block and rows per K step.  The
-// 8 x 8 and 6 x 8 blocks gain 5-8 % from long iterations (16 rows for the 32-row steps of the
-// many-channel layers, 32 rows for the ~100-row steps of the few-channel layers); the blocks
-// of 128 accumulators lose 1.5 % with 8 rows, the 4 x 8 and 4 x 16 blocks 2-3 %, and keep 4.
+// Rows of K per iteration of the main loop, by register block and rows per K step
+// (long_steps: 96 rows and more).  The 8 x 8 and 6 x 8 blocks gain 5-8 % from long iterations
+// (16 rows for steps of 32 to 64 rows, 32 rows for the ~100-row steps; 12 to 30 rows measure
+// alike, 46 rows overflow the instruction cache: -10 %); the blocks of 128 accumulators lose
+// 1.5 % with 8 rows, the 4 x 8 and 4 x 16 blocks 2-3 %, and keep 4.
 __host__ __device__ constexpr int ffma_long_block(int mr, int nr, bool long_steps) {
   return ((mr == 8 || mr == 6) && nr == 8) ? (long_steps ? 32 : 16) : 4;
 }

@@ -228,7 +228,7 @@ maxdnn_status dispatch_ffma(DeviceState* ds, const CUtensorMap& mf, const CUtens
   const ConvGeom& g = args.g;
   const bool fx = g.fixed_pitch != 0;
   // rows per iteration of the kernel's main loop: by block shape and step length
-  const bool long_steps = g.rows >= 64;
+  const bool long_steps = g.rows >= 96;
 #define MAXDNN_FFMA_LAUNCH(MR, NR, LB, SLOT)                                                        \
   do {                                                                                              \
     if (split)                                                                                      \

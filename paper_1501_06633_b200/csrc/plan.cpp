@@ -14,7 +14,7 @@ namespace maxdnn {
 // ---------------------------------------------------------------------------
 namespace {
 const char* const kOptionNames[OPT_COUNT] = {
-    "FFMA_TILE_M", "FFMA_COLS", "FFMA_KH", "FFMA_STREAMK",
+    "FFMA_TILE_M", "FFMA_COLS", "FFMA_KH", "FFMA_KC", "FFMA_STREAMK",
     "UMMA_KC", "UMMA_PAIR", "UMMA_MERGE", "UMMA_STAGE_KB", "UMMA_COLS",
     "WGRAD_SPLITS", "WGRAD_PAIR", "SM_COUNT", "X3_CHUNK_ROWS", "DEBUG_STATUS",
     "KERNEL_CLOCK", "RAGGED_PADDED", "TEST_MISSING_ARRIVAL"};
@@ -177,11 +177,13 @@ static void fill_geom(const ConvDims& d, int32_t Ho, int32_t Wo, ConvGeom* g) {
 // Tile shapes the fp32 kernel is built for, with the relative cost per
 // multiply-accumulate measured for each on layers that fill the tile (smaller register
 // blocks spend a larger share of issue slots on operand loads; with 16 rows of K per loop
-// iteration the 8 x 8 block is level with the blocks of 128 accumulators).
+// iteration and K steps of 64 or 96 rows the 8 x 8 block is ahead of the blocks of 128
+// accumulators, whose rows of 1.5 KB leave room for steps of 32 to 48 rows only).
+constexpr int kFfmaSmemBudget = 224 * 1024;   // ring stages of a CTA (227 KB is the device's limit)
 struct FfmaShape { int m, cols; double cost; };
 static const FfmaShape kFfmaShapes[] = {
-    {128, 256, 1.000}, {256, 128, 1.005}, {128, 128, 1.012}, {96, 128, 1.08},
-    {96, 256, 1.06},   {64, 128, 1.23},   {64, 256, 1.125},  {32, 128, 2.10},
+    {128, 256, 1.000}, {256, 128, 1.010}, {128, 128, 0.980}, {96, 128, 1.025},
+    {96, 256, 1.09},   {64, 128, 1.165},  {64, 256, 1.063},  {32, 128, 2.03},
 };
 
 static void build_table(const ConvDims& d, int kc, int kwc, KStepTable* t, int* n, int khc = 1) {
@@ -218,11 +220,14 @@ static double pick_columns(const ConvDims& d, int Wo, int cols, int* nn_out, int
 
 // K step of the fp32 kernel: kc channels of one filter tap, or (few channels) kc channels
 // of a whole filter row of Skw taps.
-static void ffma_kstep(const ConvDims& d, int* kc_out, int* kwc_out, int* khc_out) {
+static void ffma_kstep(const ConvDims& d, int kc_max, int* kc_out, int* kwc_out, int* khc_out) {
   int kc, kwc, khc = 1;
   if (d.Nc >= 8) {
     kwc = 1;
-    const int kc_max = 32;
+    if (option_is_set(OPT_FFMA_KC)) {
+      const int v = option(OPT_FFMA_KC);
+      if (v >= 8 && v <= 128 && v % 4 == 0) kc_max = v;
+    }
     kc = kc_max;
     int best_pad = 1 << 30;
     for (int c = kc_max; c >= 8; c -= 4) {
@@ -284,7 +289,7 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
   int best_m = 0, best_cols = 0, best_nn = 0, best_T = 0;
   bool best_split = false;
   int kc0, kwc0, khc0;
-  ffma_kstep(d, &kc0, &kwc0, &khc0);
+  ffma_kstep(d, 32, &kc0, &kwc0, &khc0);
   const int k_rows = ceil_div(d.Nc, kc0) * kc0 * d.Skw * d.Skh;
   if (option(OPT_FFMA_STREAMK, 1) == 0) allow_split = false;
   for (const FfmaShape& sh : kFfmaShapes) {
@@ -323,12 +328,24 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
 
   // K step: kc channels of one filter tap, or (few channels) kc channels of a
   // whole filter row of Sk taps.
-  int kc = kc0, kwc = kwc0;
-  int khc = khc0;
   // two ring stages must fit (three where a consumer warp issues the copies)
   const bool inline_producer = !ragged && (best_m / 16) * (best_cols / 16) >= kFfmaInlineMinAcc;
   const int min_stages = inline_producer ? 3 : 2;
-  while (khc > 1 && min_stages * kc * kwc * khc * (best_m + best_cols) * 4 > 200 * 1024) --khc;
+  // Many-channel layers: as many channels per step as leave that many stages — every step
+  // costs the consumers a barrier round trip, pointer rebuilds and loop tails (about 200
+  // instructions per warp), so long steps pay: 128 x 128 tiles with 64- or 96-row steps run
+  // 2-3 % faster than with 32-row steps (and than the 128 x 256 tiles, whose 1.5 KB rows
+  // leave room for 48).  The ragged kernel keeps 32.
+  int kc_max = 32;
+  if (!ragged) {
+    kc_max = (kFfmaSmemBudget / (min_stages * (best_m + best_cols) * 4)) & ~3;
+    if (kc_max > 112) kc_max = 112;
+    if (kc_max < 32) kc_max = 32;
+  }
+  ffma_kstep(d, kc_max, &kc0, &kwc0, &khc0);
+  int kc = kc0, kwc = kwc0;
+  int khc = khc0;
+  while (khc > 1 && min_stages * kc * kwc * khc * (best_m + best_cols) * 4 > kFfmaSmemBudget) --khc;
   int n = 0;
   build_table(d, kc, kwc, t, &n, khc);
   while (n > kMaxKSteps && kwc == 1 && kc < 256) {   // very deep filters: larger boxes
@@ -367,8 +384,7 @@ maxdnn_status plan_ffma(const ConvDims& d, int sm_count, int force_tile_m, int f
     g->b_stage_bytes = g->b_slot_bytes * g->tile_px;
   }
   const int stage = g->a_stage_bytes + g->b_stage_bytes;
-  const int budget = 200 * 1024;
-  int stages = budget / stage;
+  int stages = kFfmaSmemBudget / stage;
   if (stages > 8) stages = 8;
   if (stages < (inline_producer ? 3 : 2)) return MAXDNN_NOT_SUPPORTED;
   g->stages = stages;

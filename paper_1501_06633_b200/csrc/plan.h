@@ -17,7 +17,7 @@ constexpr int kMaxKSteps = 1024;   // capacity of the table carried in kernel pa
 // option in the process — never on the path of a call.  TEST_MISSING_ARRIVAL is the
 // exception: it has no environment variable and can only be set through the C ABI.
 enum OptionId : int {
-  OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_KH, OPT_FFMA_STREAMK,
+  OPT_FFMA_TILE_M = 0, OPT_FFMA_COLS, OPT_FFMA_KH, OPT_FFMA_KC, OPT_FFMA_STREAMK,
   OPT_UMMA_KC, OPT_UMMA_PAIR, OPT_UMMA_MERGE, OPT_UMMA_STAGE_KB, OPT_UMMA_COLS,
   OPT_WGRAD_SPLITS, OPT_WGRAD_PAIR, OPT_SM_COUNT, OPT_X3_CHUNK_ROWS, OPT_DEBUG_STATUS,
   OPT_KERNEL_CLOCK, OPT_RAGGED_PADDED, OPT_TEST_MISSING_ARRIVAL, OPT_COUNT

@@ -117,7 +117,7 @@ SPLIT = [
     ((128, 15, 13, 32, 128, 3, 1, 1, 1.0), 0, 0),
     ((64, 24, 17, 24, 256, 3, 1, 1, 0.5), 0, 0),
     ((128, 14, 12, 40, 200, 5, 1, 2, 1.0), 0, 0),
-    ((128, 16, 10, 64, 128, 3, 1, 1, 1.0), 0, 0),
+    ((128, 16, 10, 128, 128, 3, 1, 1, 1.0), 0, 0),
     ((128, 16, 10, 24, 96, 3, 1, 1, 1.0), 32, 128),
     ((128, 16, 12, 24, 192, 3, 1, 1, 1.0), 96, 128),
     ((128, 20, 18, 24, 256, 3, 1, 1, 1.0), 256, 128),
@@ -126,6 +126,7 @@ SPLIT = [
     ((64, 40, 18, 40, 64, 3, 1, 1, 1.0), 64, 256),
     ((64, 40, 36, 16, 96, 3, 1, 1, 1.0), 96, 256),
     ((128, 55, 83, 3, 96, 11, 4, 0, 1.0), 96, 128),      # 11 filter rows in steps of 2: a short last step
+    ((128, 13, 9, 96, 256, 3, 1, 1, 1.0), 128, 128),     # 96 channels per step: the long-iteration instance
 ]
 
 
