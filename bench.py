@@ -42,9 +42,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     # fp32 plans with a split tail: both launches of a step (whole tiles + split tail)
     ("first11x11s4", "fp32"): int((79.71 + 93.40) * 1e6),
-    ("mid5x5", "fp32"): int((34.39 + 22.83 + 12.10 + 0.49) * 1e6),
-    ("wide3x3", "fp32"): int((24.82 + 0.29 + 8.24 + 0.0) * 1e6),
-    ("large3x3", "fp32"): int((100.3 + 140.8 + 8.98 + 0.07) * 1e6),
+    ("mid5x5", "fp32"): int((38.00 + 33.58 + 8.44 + 0.0) * 1e6),
+    ("wide3x3", "fp32"): int((24.82 + 0.21 + 8.24 + 0.0) * 1e6),
+    ("large3x3", "fp32"): int((104.0 + 151.3 + 3.21 + 0.0) * 1e6),
     ("large3x3", "bf16"): int((52.02 + 146.8) * 1e6),
     ("large3x3", "tf32"): int((104.0 + 149.8) * 1e6),
     ("mid5x5", "bf16"): int((19.17 + 37.60) * 1e6),
