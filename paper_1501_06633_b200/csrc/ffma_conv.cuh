@@ -14,7 +14,7 @@
 // The producer is a ninth warp when the register block leaves room for it
 // (registers are allocated per four warps, so nine warps cap a thread at 168).
 // Larger blocks (MR*NR >= 96) run with eight warps and 255 registers; there the
-// first consumer warp issues the copies itself, one K step per step it consumes.
+// consumer warps take turns at issuing the copies, one K step each.
 #pragma once
 #include "plan.h"
 #include "ptx_util.cuh"
@@ -503,7 +503,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
 
   // -------------------------------------------------------------- consumers
   // Producer state of the INLINE variants (registers: kept in shared memory it cost the
-  // large blocks 3 %, the loads sitting in warp 0's instruction stream).
+  // large blocks 3 %, the loads sitting in the consumers' instruction stream).
   FfmaProducer<SPLIT> prod;
   bool prod_ok = true;
   // The consumer warps take turns at the producer's job, one K step each, so that its
@@ -595,7 +595,7 @@ ffma_conv_kernel(const __grid_constant__ CUtensorMap map_filt,
     for (int s = s0; s < s1; ++s) {
       if constexpr (INLINE) {
         // Refill the slot this CTA finished two steps ago (every warp has released it
-        // by now, so the wait does not hold warp 0 back) with the K step that is
+        // by now, so the wait does not hold the issuing warp back) with the K step that is
         // (stages - 2) ahead of the one being consumed.
         if (prod.has_work(g)) {
           if (warp == turn) {
