@@ -154,6 +154,7 @@ unpad_inner_kernel(const float* __restrict__ src, float* __restrict__ dst, size_
 
 constexpr int kWgThreads = 256;               // 8 warps: 16 x 16 threads, 8 x 8 results each (stride 16)
 constexpr uint32_t kWgOperandBytes = 128 * 128;   // 128 rows x 32 floats
+constexpr int kWgSub = 2;                         // reduction steps per ring stage
 
 struct WgradArgs {
   WgradGeom g;
@@ -214,8 +215,10 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   // index mod 8), which needs 1024-byte aligned buffers.
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const int stages = g.stages;
-  const uint32_t stage_bytes = 2u * kWgOperandBytes;
+  // A ring stage holds kWgSub consecutive reduction steps (fewer at the end of an item): the
+  // consumers pay one barrier round trip and one producer turn per stage.
+  const int stages = g.stages / kWgSub;
+  const uint32_t stage_bytes = (uint32_t)kWgSub * 2u * kWgOperandBytes;
   const uint32_t full_bar = base + (uint32_t)stages * stage_bytes;
   const uint32_t empty_bar = full_bar + 8u * stages;
   const int warp = threadIdx.x >> 5;
@@ -243,20 +246,28 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
   // turn it is waits for the ring slot (free since two steps) and issues the two copies.
   auto produce = [&](bool mine) {
     if (pc.done(g)) return;
-    if (mine && p_ok) {
+    const int n_sub = (pc.r + 1 < pc.r_end) ? kWgSub : 1;   // a stage never spans two items
+    bool go = mine && p_ok;
+    const uint32_t fb = full_bar + 8u * p_stage;
+    const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
+    if (go) {
       if (!mbar_wait(empty_bar + 8u * p_stage, p_phase ^ 1u, args.wc, kDevTimeoutEmpty)) {
         p_ok = false;
+        go = false;
       } else {
-        const uint32_t fb = full_bar + 8u * p_stage;
-        const uint32_t dst = base + (uint32_t)p_stage * stage_bytes;
-        mbar_arrive_expect_tx(fb, tx_bytes);
-        tma_load_4d(dst, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
-        tma_load_4d(dst + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride_w - g.pad_w,
-                    pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc);
+        mbar_arrive_expect_tx(fb, (uint32_t)n_sub * tx_bytes);
       }
     }
+    for (int sub = 0; sub < n_sub; ++sub) {
+      if (go) {
+        const uint32_t d2 = dst + (uint32_t)sub * 2u * kWgOperandBytes;
+        tma_load_4d(d2, &map_dout, fb, pc.nc * 32, pc.x, pc.y, pc.ob * 128);
+        tma_load_4d(d2 + kWgOperandBytes, &map_in, fb, pc.nc * 32, pc.x * g.stride_w - g.pad_w,
+                    pc.y * g.stride_h - g.pad_h + pc.khb * g.bh, pc.cb * g.bc);
+      }
+      pc.advance(g, (int)gridDim.x);
+    }
     if (++p_stage == stages) { p_stage = 0; p_phase ^= 1u; }
-    pc.advance(g, (int)gridDim.x);
   };
   int turn = 0;
   if (warp == 0 && lane == 0) {
@@ -298,7 +309,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
     const int ob = cc.ob, cb = cc.cb, khb = cc.khb, split = cc.split;
     const int n_steps = cc.r_end - cc.r;
 
-    for (int s = 0; s < n_steps; ++s) {
+    for (int s = 0; s < n_steps; s += kWgSub) {
       produce(warp == turn && lane == 0);
       turn = (turn + 1) & 7;
       __syncwarp();
@@ -306,7 +317,10 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
         ok = false;
         break;
       }
-      const uint8_t* ss = base_ptr + (size_t)stage * stage_bytes;
+      const int n_sub = (s + 1 < n_steps) ? kWgSub : 1;
+#pragma unroll 1
+      for (int sub = 0; sub < n_sub; ++sub) {
+      const uint8_t* ss = base_ptr + (size_t)stage * stage_bytes + (size_t)sub * 2u * kWgOperandBytes;
       // Sixteen blocks per step: (16-byte chunk q, half of it): first the even pair of r for
       // all 64 results, then the odd pair, so consecutive multiply-adds never depend on each
       // other.  Operands come by 8-byte loads (beside a stream of packed multiply-adds an
@@ -337,6 +351,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dout, const __grid_constant
           }
         }
       }
+      }   // sub
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar + 8u * stage);
       if (++stage == stages) { stage = 0; phase ^= 1u; }
