@@ -36,9 +36,11 @@ __host__ __device__ constexpr int ffma_order(int mr, int nr) {
 // Rows of K per iteration of the main loop, by register block and rows per K step
 // (long_steps: 96 rows and more).  The 8 x 8 and 6 x 8 blocks gain 5-8 % from long iterations
 // (16 rows for steps of 32 to 64 rows, 32 rows for the ~100-row steps; 12 to 30 rows measure
-// alike, 46 rows overflow the instruction cache: -10 %); the blocks of 128 accumulators lose
-// 1.5 % with 8 rows, the 4 x 8 and 4 x 16 blocks 2-3 %, and keep 4.
+// alike, 46 rows overflow the instruction cache: -10 %); the 4 x 8 block gains 3.5 % from 32
+// rows on ~100-row steps and loses 2-3 % from long iterations on 32-row steps; the blocks of
+// 128 accumulators lose 1.5 % with 8 rows, the 4 x 16 block 2-3 %: those keep 4.
 __host__ __device__ constexpr int ffma_long_block(int mr, int nr, bool long_steps) {
+  if (mr == 4 && nr == 8) return long_steps ? 32 : 4;
   return ((mr == 8 || mr == 6) && nr == 8) ? (long_steps ? 32 : 16) : 4;
 }
 

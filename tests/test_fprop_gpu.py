@@ -159,6 +159,7 @@ def test_split_tail_fp32(dims, tile_m, cols):
 @pytest.mark.parametrize("dims", [
     (128, 31, 27, 3, 96, 11, 4, 0, 1.0),     # one pixel per tile: one box per stage
     (128, 31, 27, 3, 128, 11, 4, 0, 1.0),    # 128 filters: the 8 x 8 block on long steps
+    (128, 31, 27, 3, 64, 11, 4, 0, 1.0),     # 64 filters: the 4 x 8 block on long steps
     (16, 23, 19, 3, 12, 7, 2, 3, 0.5),       # several pixels per tile: one box per pixel; apron
     (32, 12, 9, 5, 40, 5, 1, 2, 1.0),        # channels in two blocks (3 + 2), stride 1
 ], ids=lambda s: "x".join(str(v) for v in s))

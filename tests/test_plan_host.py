@@ -309,10 +309,10 @@ def plan_signature(dims, kind, sms=148):
     if kind == mx.KERNEL_FP32:
         one_box = info.tile_px * info.tile_n == info.tile_cols and \
             (info.tile_px == 1 or (stride == 1 and info.kwc == 1))
-        # rows of K per step >= 96: the 8 x 8 and 6 x 8 blocks then run the instance with the
+        # rows of K per step >= 96: the 8 x 8, 6 x 8 and 4 x 8 blocks then run the instance with the
         # longer main-loop iterations
         long_steps = info.kc * info.kwc * info.khc >= 96 and info.tile_cols == 128 and \
-            info.tile_m in (96, 128)
+            info.tile_m in (64, 96, 128)
         return ("fp32", info.tile_m, info.tile_cols, one_box, info.kwc > 1, info.khc > 1,
                 info.split_tiles > 0, long_steps)
     few = Nc < (8 if kind == mx.KERNEL_TF32 else 16)
