@@ -437,9 +437,9 @@ maxdnn_status maxdnn_last_kernel_clock(uint32_t* sm_cycles, uint32_t* nanosecond
  * Tuning and test options (ablations and tests; none is needed in normal use; the
  * paper has no counterpart).  An option is a named integer, "unset" by default.  `name`
  * is one of FFMA_TILE_M, FFMA_COLS (pin the fp32 kernel's tile: filters 32/64/96/128/256,
- * columns 128/256), FFMA_KH (filter rows per K step of few-channel layers), FFMA_KC (most
- * channels per K step of many-channel layers, a multiple of 4 in 8..128; default: what the
- * tile's ring holds), FFMA_STREAMK (0: never split tail tiles along K; 2: always, whatever
+ * columns 128/256), FFMA_KH (filter rows per K step of few-channel layers), FFMA_KC (upper
+ * limit of the channels per K step of many-channel layers, a multiple of 4 in 8..128, below
+ * what the tile's ring would hold), FFMA_STREAMK (0: never split tail tiles along K; 2: always, whatever
  * the model says), UMMA_KC, UMMA_PAIR (1 two-SM / -1 one-SM tiles), UMMA_MERGE, UMMA_STAGE_KB, UMMA_COLS, WGRAD_SPLITS, WGRAD_PAIR, SM_COUNT (SM
  * count for host-only workspace queries), X3_CHUNK_ROWS, DEBUG_STATUS, KERNEL_CLOCK (see
  * maxdnn_last_kernel_clock), RAGGED_PADDED (see maxdnn_conv_fprop_ragged), and

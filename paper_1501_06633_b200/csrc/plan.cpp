@@ -226,7 +226,7 @@ static void ffma_kstep(const ConvDims& d, int kc_max, int* kc_out, int* kwc_out,
     kwc = 1;
     if (option_is_set(OPT_FFMA_KC)) {
       const int v = option(OPT_FFMA_KC);
-      if (v >= 8 && v <= 128 && v % 4 == 0) kc_max = v;
+      if (v >= 8 && v <= 128 && v % 4 == 0 && v < kc_max) kc_max = v;   // an upper limit
     }
     kc = kc_max;
     int best_pad = 1 << 30;

@@ -173,6 +173,24 @@ def test_filter_rows_per_k_step(dims, khc):
     check_fp32(w)
 
 
+@pytest.mark.parametrize("kc", [8, 20, 32, 64, 112])
+@pytest.mark.parametrize("dims,tile", [
+    ((128, 14, 9, 112, 128, 3, 1, 1, 1.0), (128, 128)),    # 8 x 8 block: steps of up to 112 rows
+    ((64, 20, 9, 96, 96, 3, 1, 1, 0.5), (96, 128)),        # 6 x 8 block, four pixels of 32 images
+    ((64, 24, 10, 72, 256, 3, 2, 1, 1.0), (128, 256)),     # 8 x 16 block: the ring caps the step at 48 rows
+], ids=lambda v: "x".join(str(x) for x in v))
+def test_channels_per_k_step(dims, tile, kc):
+    """Many-channel layers take as many channels per K step as the tile's ring allows; the
+    option pins an upper limit (the planner picks the divisor-friendly count below it)."""
+    mx.set_option("FFMA_KC", kc)
+    mx.set_option("FFMA_TILE_M", tile[0])
+    mx.set_option("FFMA_COLS", tile[1])
+    w = wl.Workload("kc", *dims, ("uniform", -1.0, 1.0), ("uniform", -1.0, 1.0), 99)
+    info, _ = mx.conv_plan_query(mx.ConvDesc.make(*w.dims), mx.KERNEL_FP32, 148)
+    assert info.kwc == 1 and info.kc <= kc and info.stages >= 2
+    check_fp32(w)
+
+
 def test_special_values_fp32():
     """Delta filter reproduces the map bit for bit; permuting filters permutes the output."""
     rng = np.random.default_rng(5)
